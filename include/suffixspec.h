@@ -1,0 +1,184 @@
+/*
+ * suffixspec: batched SuffixDecoding draft generation on one NVIDIA B200.
+ *
+ * C ABI.  Every pointer named d_* is DEVICE memory owned by the caller; every
+ * other pointer is HOST memory.  A store owns all of its device memory from
+ * sd_build() until sd_free().  Calls are asynchronous on `stream` (a
+ * cudaStream_t passed as void*, NULL = default stream) unless stated, and
+ * after sd_build() no call allocates device memory.
+ *
+ * Return value: SD_OK (0) or a negative SD_ERR_* code.  Nothing aborts, throws
+ * or traps.  Conditions that depend on device data (a request whose slot pool
+ * ran full, an empty slot) are reported per request in d_status and leave the
+ * store consistent.
+ *
+ * Limits: depth_cap <= 32, max_spec_cap <= 64, P <= depth_cap is not required
+ * (pattern lengths above depth_cap or above the context length never match).
+ */
+#ifndef SUFFIXSPEC_H
+#define SUFFIXSPEC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sd_store sd_store;
+
+enum {
+    SD_OK = 0,
+    SD_ERR_INVALID_ARG = -1,
+    SD_ERR_CUDA = -2,
+    SD_ERR_NOMEM = -3,
+    SD_ERR_CAPACITY = -4
+};
+
+/* per-request status bits (d_status of sd_speculate, sd_slot_info) */
+enum {
+    SD_STATUS_OK = 0,
+    SD_STATUS_BAD_SLOT = 1,       /* slot index out of range                         */
+    SD_STATUS_POOL_FULL = 2,      /* the slot's node pool or text buffer ran full;    */
+                                  /* its tree stopped growing at the last good token  */
+    SD_STATUS_GLOBAL_FULL = 4,    /* the global node pool ran full during an insert   */
+    SD_STATUS_BAD_TOKEN = 8       /* a token outside [0, V) was met; the tree stopped */
+                                  /* growing at the last good token                   */
+};
+
+/* sd_spec_params.flags */
+enum {
+    SD_FLAG_GLOBAL_ONLY = 1,      /* speculate from the global tree only              */
+    SD_FLAG_REQUEST_ONLY = 2,     /* speculate from the per-request tree only         */
+    SD_FLAG_LINEAR = 4            /* chain-only expansion ("Suffix (linear)")         */
+};
+
+typedef struct {
+    int32_t vocab;                /* V: token ids are in [0, V)                       */
+    int32_t depth_cap;            /* D: paths longer than D tokens are not stored     */
+    int32_t max_requests;         /* number of request slots                          */
+    int32_t max_req_tokens;       /* max prompt + generated tokens per slot           */
+    int32_t max_spec_cap;         /* M: row stride of the per-draft outputs, <= 64    */
+    int64_t global_extra_nodes;   /* node head-room for online inserts into the       */
+                                  /* global tree; < 0: library default                */
+    int64_t slot_pool_nodes;      /* node pool per slot; <= 0: library default        */
+                                  /* (2 * max_req_tokens * depth_cap)                 */
+} sd_build_params;
+
+typedef struct {
+    int32_t P;                    /* max pattern length                               */
+    double alpha;                 /* max speculation factor: MAX_SPEC(p) = alpha * p  */
+    int32_t max_spec;             /* cap on MAX_SPEC(p), <= max_spec_cap              */
+    uint32_t flags;               /* SD_FLAG_*                                        */
+} sd_spec_params;
+
+typedef struct {
+    int64_t global_nodes;         /* live nodes of the global tree                    */
+    int64_t global_pool_used;     /* node entries handed out (live + abandoned)       */
+    int64_t global_pool_cap;
+    int64_t global_tokens;        /* tokens inserted so far                           */
+    int64_t slot_pool_nodes;      /* node entries per slot                            */
+    int64_t device_bytes;         /* device memory owned by the store                 */
+    int32_t global_status;        /* SD_STATUS_GLOBAL_FULL or 0                       */
+} sd_stats_t;
+
+/*
+ * sd_build: create a store and build the GLOBAL suffix tree over a corpus of
+ * previous outputs in one offline step (Section 3, "Suffix Tree Construction").
+ * One node per token; the root-to-node path is a token string of at most
+ * depth_cap tokens that occurs in some sequence, and the node's count is its
+ * number of occurrences (COUNT as used by Eq. 1).  Strings do not cross
+ * sequence boundaries.  The tree is built on the GPU by a depth-capped suffix
+ * sort followed by adjacent-suffix LCPs.
+ *   d_corpus       int32[seq_offsets[n_seqs]]  tokens of all sequences, back to back
+ *   d_seq_offsets  int64[n_seqs + 1]           start of each sequence, ascending, [0] = 0
+ * n_seqs may be 0 (empty global tree; both pointers may then be NULL).
+ * Also allocates max_requests empty per-request trees.  Synchronises the stream.
+ * On success *out is the new store; on failure *out is NULL and nothing leaks.
+ * Errors: INVALID_ARG (NULL, limits, a corpus token outside [0, V), offsets not
+ * ascending), NOMEM (cudaMalloc failed), CUDA.
+ */
+int sd_build(const sd_build_params* params, const int32_t* d_corpus, const int64_t* d_seq_offsets,
+             int32_t n_seqs, void* stream, sd_store** out);
+
+/*
+ * sd_append: online update of the trees (Section 3, "Suffix Tree Construction":
+ * tokens of the ongoing request are added as they are generated; a finished
+ * request's output is added to the global tree).
+ * For item i in [0, n):
+ *   d_slot[i] >= 0 : append tokens d_tokens[d_offsets[i] .. d_offsets[i+1]) to the
+ *                    per-request tree (and stored context) of that slot; if
+ *                    d_reset[i] != 0 the slot is emptied first (new request, the
+ *                    tokens are its prompt).  A slot may appear at most once per call.
+ *   d_slot[i] == -1: insert the tokens as one whole sequence into the GLOBAL tree.
+ * After the call each tree equals the tree built from scratch over its text.
+ *   d_slot int32[n], d_offsets int64[n+1], d_tokens int32[d_offsets[n]],
+ *   d_reset uint8[n] or NULL (no resets).
+ * A slot whose pool or text buffer would overflow keeps its state from before
+ * the offending token and gets SD_STATUS_POOL_FULL (see sd_slot_info); a full
+ * global pool sets SD_STATUS_GLOBAL_FULL in sd_stats.  n == 0 is a no-op.
+ * Errors: INVALID_ARG, CUDA (launch failure).
+ */
+int sd_append(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* d_offsets,
+              const int32_t* d_tokens, const uint8_t* d_reset, void* stream);
+
+/*
+ * sd_speculate: GenerateCandidateTree of Algorithm 1 for n requests at once.
+ * For each request the context x_{1:t} is the slot's stored text.  For the
+ * global tree, then the per-request tree, and p = 1..P: MatchPattern walks the
+ * last p tokens; ExpandSpeculationTree grows the sub-tree greedily by the
+ * largest D(N) (Eq. 1, Eq. 2) up to min(floor(alpha * p), max_spec) draft nodes
+ * (Eq. 3; the match node itself is not a draft); SCORE (Eq. 4) is the sum of
+ * D over the draft nodes in the order added; the first tree with the strictly
+ * largest score wins.  Candidate ties: larger D, then smaller token id, then
+ * smaller index of the parent inside the speculation tree.  All scores are
+ * IEEE binary64: divide, multiply root-to-leaf, add in insertion order, no FMA.
+ * Outputs, row stride M = max_spec_cap, draft nodes in insertion order:
+ *   d_n_draft     int32[n]        number of draft nodes (0: no speculation)
+ *   d_tokens      int32[n][M]     token of each draft node, -1 beyond n_draft
+ *   d_parents     int32[n][M]     index of the parent draft node, -1 = child of the
+ *                                 match node (also -1 beyond n_draft)
+ *   d_positions   int32[n][M]     0-based sequence position t + depth - 1, -1 beyond
+ *   d_mask        uint32[n][M][(M+31)/32]  bit j of row i set iff j == i or j is an
+ *                                 ancestor of i (tree-attention mask), 0 beyond
+ *   d_chosen_tree int32[n]        0 global, 1 per-request, -1 none
+ *   d_chosen_p    int32[n]        pattern length of the chosen tree, 0 if none
+ *   d_score       double[n]       SCORE of the chosen tree, 0.0 if none
+ *   d_status      int32[n]        SD_STATUS_* of the request's slot
+ *   d_budget_cap  int32[n] or NULL: per-request cap on the draft size (< 0: none)
+ * Errors: INVALID_ARG (n > max_requests, max_spec > M, P < 1 ...), CUDA.
+ */
+int sd_speculate(sd_store* store, int32_t n, const int32_t* d_slot, const sd_spec_params* params,
+                 const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents,
+                 int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
+                 double* d_score, int32_t* d_status, void* stream);
+
+/*
+ * sd_query_counts: COUNT of arbitrary token paths (the quantity Eq. 1 divides),
+ * for checking a store against an independent implementation.
+ *   d_tree int32[n]: -1 global tree, else slot; path i is
+ *   d_paths[d_offsets[i] .. d_offsets[i+1]); d_counts int32[n] receives the count,
+ *   0 when the path is not in the tree (or is longer than depth_cap).
+ */
+int sd_query_counts(sd_store* store, int32_t n, const int32_t* d_tree, const int64_t* d_offsets,
+                    const int32_t* d_paths, int32_t* d_counts, void* stream);
+
+/*
+ * sd_slot_info: per-slot context length, live node count and status.
+ *   d_slot int32[n]; outputs int32[n] each, any may be NULL.
+ */
+int sd_slot_info(sd_store* store, int32_t n, const int32_t* d_slot, int32_t* d_len, int32_t* d_nodes,
+                 int32_t* d_status, void* stream);
+
+/* sd_stats: store-wide figures into HOST memory.  Synchronises the stream. */
+int sd_stats(sd_store* store, sd_stats_t* out, void* stream);
+
+/* sd_free: release a store (NULL is a no-op).  Synchronises the device. */
+void sd_free(sd_store* store);
+
+/* sd_strerror: static description of an SD_* return code. */
+const char* sd_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SUFFIXSPEC_H */

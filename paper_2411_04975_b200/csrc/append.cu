@@ -1,0 +1,201 @@
+// Online update of the suffix trees (Section 3, "Suffix Tree Construction": the
+// tokens of the ongoing request are added as they are generated, a finished
+// request's output is added to the global tree).
+//
+// One warp owns one tree for the duration of the kernel.  Appending token x at
+// context length t adds one occurrence to every string that ends at x and is at
+// most D tokens long: lane L extends the ACTIVE node of depth L (the node of
+// the last L tokens; lane 0 extends the root) by child x, creating it or
+// raising its count.  The 32 lanes work on 32 different parents at once.
+#include "common.cuh"
+
+namespace {
+
+struct TreeRef {
+    int4* ent;
+    int32_t* root;
+    int cap;                 // entries in the pool
+};
+
+__device__ __forceinline__ int* word(int4* e, int k) { return reinterpret_cast<int*>(e) + k; }
+
+// Inserts child x at sorted position `pos` into the child run of `parent`
+// (cb, n children, flags in w).  `fresh` > 0: the run is full and moves to
+// ent[fresh ...).  Returns the new child's entry index.
+__device__ int insert_child(int4* ent, int parent, int cb, int n, int pos, int x, int fresh, bool moves) {
+    const int4 ne = make_int4(x, 1, 0, 0);
+    int idx;
+    if (moves) {
+        for (int k = 0; k < pos; ++k) ent[fresh + k] = ent[cb + k];
+        ent[fresh + pos] = ne;
+        for (int k = pos; k < n; ++k) ent[fresh + k + 1] = ent[cb + k];
+        *word(&ent[parent], 2) = fresh;
+        idx = fresh + pos;
+    } else {
+        for (int k = n - 1; k >= pos; --k) ent[cb + k + 1] = ent[cb + k];
+        ent[cb + pos] = ne;
+        idx = cb + pos;
+    }
+    *word(&ent[parent], 3) = n + 1;               // dynamic run from now on (no RUN_STATIC)
+    return idx;
+}
+
+// All 32 lanes call.  `act` is this lane's active node of depth lane + 1 (-1: none);
+// on return it is the active node after x was appended.  `t` is the context length
+// before the append.  `used` / `live` are warp-uniform pool counters.
+// Returns false, changing nothing, if the pool cannot hold the new nodes.
+__device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, int& act, int& used, int& live) {
+    const unsigned FULL = 0xffffffffu;
+    const int parent = __shfl_up_sync(FULL, act, 1);            // node of depth `lane`
+    const bool valid = lane <= min(t, D - 1);
+    int found = -1, pos = 0, cb = 0, n = 0;
+    unsigned w = 0;
+    if (valid) {
+        if (lane == 0) {
+            found = tr.root[x];
+        } else {
+            const int4 pe = tr.ent[parent];
+            cb = pe.z; w = (unsigned)pe.w; n = (int)(w & RUN_COUNT_MASK);
+            int lo = 0, hi = n;
+            while (lo < hi) {                                    // at most 24 rounds: n < 2^24
+                const int mid = (lo + hi) >> 1;
+                if (tr.ent[cb + mid].x < x) lo = mid + 1; else hi = mid;
+            }
+            pos = lo;
+            if (pos < n && tr.ent[cb + pos].x == x) found = cb + pos;
+        }
+    }
+    const bool need = valid && found < 0;
+    int asz = 0;                                                 // fresh entries this lane needs
+    if (need) {
+        if (lane == 0) asz = 1;
+        else if ((uint32_t)n == sd_run_capacity(w)) asz = (int)sd_pow2ceil((uint32_t)n + 1u);
+    }
+    int inc = asz;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(FULL, inc, o);
+        if (lane >= o) inc += y;
+    }
+    const int total = __shfl_sync(FULL, inc, 31);
+    if ((long long)used + total > (long long)tr.cap) return false;
+    const int fresh = used + inc - asz;
+    used += total;
+
+    // A lane that moves entries of its run must not do so while the next lane edits the
+    // header of an entry inside that run (only possible when the last tokens repeat one
+    // token).  Then the inserts go one at a time, deepest first.
+    const int next_parent = __shfl_down_sync(FULL, parent, 1);
+    const int next_need = __shfl_down_sync(FULL, need ? 1 : 0, 1);
+    const bool clash = need && lane >= 1 && lane < 31 && next_need && next_parent >= cb && next_parent < cb + n;
+    const bool serial = __any_sync(FULL, clash);
+
+    if (valid && found >= 0) {
+        *word(&tr.ent[found], 1) += 1;
+        act = found;
+    }
+    if (!serial) {
+        if (need) {
+            if (lane == 0) {
+                tr.ent[fresh] = make_int4(x, 1, 0, 0);
+                tr.root[x] = fresh;
+                act = fresh;
+            } else {
+                act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, asz > 0);
+            }
+        }
+        __syncwarp();
+    } else {
+        for (int l = 31; l >= 0; --l) {
+            if (lane == l && need) {
+                if (lane == 0) {
+                    tr.ent[fresh] = make_int4(x, 1, 0, 0);
+                    tr.root[x] = fresh;
+                    act = fresh;
+                } else {
+                    act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, asz > 0);
+                }
+            }
+            __syncwarp();
+        }
+    }
+    if (!valid) act = -1;
+    live += __popc(__ballot_sync(FULL, need));
+    return true;
+}
+
+// Warp 0 of the grid inserts whole sequences into the global tree, one after the
+// other; warp i + 1 appends item i to its request slot.
+__global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_offsets,
+                              const int32_t* d_tokens, const uint8_t* d_reset) {
+    const int lane = threadIdx.x & 31;
+    const int warp = (int)((blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5);
+    if (warp > n) return;
+    if (warp == 0) {
+        TreeRef tr{sv.g_ent, sv.g_root, (int)sv.g_cap};
+        int used = sv.g_state->used, live = sv.g_state->live, status = sv.g_state->status;
+        long long tokens = sv.g_state->tokens;
+        bool any = false;
+        for (int i = 0; i < n; ++i) {
+            if (d_slot[i] != -1) continue;
+            any = true;
+            int act = -1;
+            const long long b = d_offsets[i], e = d_offsets[i + 1];
+            for (long long k = b; k < e && !(status & SD_STATUS_GLOBAL_FULL); ++k) {
+                const int x = d_tokens[k];
+                if (x < 0 || x >= sv.V) { status |= SD_STATUS_BAD_TOKEN; break; }
+                if (!append_token(tr, sv.D, x, (int)(k - b), lane, act, used, live)) {
+                    status |= SD_STATUS_GLOBAL_FULL;
+                    break;
+                }
+                ++tokens;
+            }
+        }
+        if (any && lane == 0) {
+            sv.g_state->used = used; sv.g_state->live = live; sv.g_state->status = status;
+            sv.g_state->tokens = tokens;
+        }
+        return;
+    }
+    const int i = warp - 1;
+    const int slot = d_slot[i];
+    if (slot < 0 || slot >= sv.R) return;
+    SlotState* ss = sv.s_state + slot;
+    int32_t* text = sv.s_text + (long long)slot * sv.T;
+    TreeRef tr{sv.s_ent + (long long)slot * sv.spn, sv.s_root + (long long)slot * sv.V, (int)sv.spn};
+    int len = ss->len, used = ss->used, live = ss->live, status = ss->status;
+    int act = lane < SD_MAX_DEPTH ? ss->active[lane] : -1;
+    if (d_reset && d_reset[i]) {
+        // forget the old tree: only root-table cells of tokens that occur can be set
+        for (int k = lane; k < len; k += 32) tr.root[text[k]] = -1;
+        __syncwarp();
+        len = 0; used = 0; live = 0; status = 0; act = -1;
+    }
+    const long long b = d_offsets[i], e = d_offsets[i + 1];
+    for (long long k = b; k < e && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)); ++k) {
+        const int x = d_tokens[k];
+        if (x < 0 || x >= sv.V) { status |= SD_STATUS_BAD_TOKEN; break; }
+        if (len >= sv.T || !append_token(tr, sv.D, x, len, lane, act, used, live)) {
+            status |= SD_STATUS_POOL_FULL;
+            break;
+        }
+        if (lane == 0) text[len] = x;
+        ++len;
+    }
+    ss->active[lane] = act;
+    if (lane == 0) { ss->len = len; ss->used = used; ss->live = live; ss->status = status; }
+}
+
+}  // namespace
+
+extern "C" int sd_append(sd_store* s, int32_t n, const int32_t* d_slot, const int64_t* d_offsets,
+                         const int32_t* d_tokens, const uint8_t* d_reset, void* stream) {
+    if (!s || n < 0) return SD_ERR_INVALID_ARG;
+    if (n == 0) return SD_OK;
+    if (!d_slot || !d_offsets) return SD_ERR_INVALID_ARG;
+    const int warps_per_block = 4;
+    const unsigned blocks = (unsigned)((n + 1 + warps_per_block - 1) / warps_per_block);
+    append_kernel<<<blocks, warps_per_block * 32, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset);
+    SD_CUDA_OK(cudaGetLastError());
+    return SD_OK;
+}

@@ -1,0 +1,552 @@
+// Offline build of the global suffix tree (Section 3, "Suffix Tree Construction")
+// on the GPU: depth-capped suffix sort by prefix doubling, adjacent-suffix LCPs,
+// then one pass per depth that lays the nodes down as sorted child runs.
+// Hand-written LSD radix sort and scans (no CUB / Thrust).
+#include <algorithm>
+#include <new>
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace {
+
+typedef unsigned long long u64;
+typedef long long i64;
+
+// ------------------------------------------------------------------ scan
+constexpr int SCAN_THREADS = 256;
+constexpr int SCAN_ITEMS = 8;
+constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
+
+struct LoadInt {
+    const int* p;
+    __device__ int operator()(i64 i) const { return p[i]; }
+};
+
+// Exclusive scan inside each tile of 2048 values f(i); tile totals go to sums[].
+template <class F>
+__global__ void scan_tiles_kernel(F f, i64 n, int* out, int* sums) {
+    __shared__ int wsum[SCAN_THREADS / 32];
+    const i64 base = (i64)blockIdx.x * SCAN_TILE + (i64)threadIdx.x * SCAN_ITEMS;
+    int v[SCAN_ITEMS];
+    int s = 0;
+#pragma unroll
+    for (int k = 0; k < SCAN_ITEMS; ++k) {
+        i64 idx = base + k;
+        v[k] = idx < n ? f(idx) : 0;
+        s += v[k];
+    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int inc = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    if (lane == 31) wsum[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+        int x = lane < SCAN_THREADS / 32 ? wsum[lane] : 0;
+        int xi = x;
+#pragma unroll
+        for (int o = 1; o < SCAN_THREADS / 32; o <<= 1) {
+            int y = __shfl_up_sync(0xffffffffu, xi, o);
+            if (lane >= o) xi += y;
+        }
+        if (lane < SCAN_THREADS / 32) wsum[lane] = xi - x;
+        if (lane == SCAN_THREADS / 32 - 1) sums[blockIdx.x] = xi;
+    }
+    __syncthreads();
+    int ex = wsum[w] + inc - s;
+#pragma unroll
+    for (int k = 0; k < SCAN_ITEMS; ++k) {
+        i64 idx = base + k;
+        if (idx < n) out[idx] = ex;
+        ex += v[k];
+    }
+}
+
+__global__ void scan_add_kernel(int* out, i64 n, const int* tile_offsets) {
+    const i64 base = (i64)blockIdx.x * SCAN_TILE;
+    const int add = tile_offsets[blockIdx.x];
+    for (int k = threadIdx.x; k < SCAN_TILE; k += SCAN_THREADS) {
+        i64 idx = base + k;
+        if (idx < n) out[idx] += add;
+    }
+}
+
+__global__ void copy_one_kernel(int* dst, const int* src) { *dst = *src; }
+
+inline i64 scan_tmp_ints(i64 n) {       // ints of scratch exclusive_scan() needs
+    i64 total = 0;
+    while (true) {
+        i64 nb = (n + SCAN_TILE - 1) / SCAN_TILE;
+        if (nb < 1) nb = 1;
+        total += (nb + 31) / 32 * 32;
+        if (nb == 1) break;
+        n = nb;
+    }
+    return total + 32;
+}
+
+// In-place exclusive scan of data[0..n); grand total to *total_out.
+void scan_in_place(int* data, i64 n, int* tmp, int* total_out, cudaStream_t st) {
+    i64 nb = (n + SCAN_TILE - 1) / SCAN_TILE;
+    if (nb < 1) nb = 1;
+    scan_tiles_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(LoadInt{data}, n, data, tmp);
+    if (nb == 1) {
+        copy_one_kernel<<<1, 1, 0, st>>>(total_out, tmp);
+    } else {
+        scan_in_place(tmp, nb, tmp + (nb + 31) / 32 * 32, total_out, st);
+        scan_add_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(data, n, tmp);
+    }
+}
+
+// out[i] = sum_{k<i} f(k) for i in [0, n]; out has n + 1 slots.
+template <class F>
+void exclusive_scan(F f, i64 n, int* out, int* tmp, cudaStream_t st) {
+    i64 nb = (n + SCAN_TILE - 1) / SCAN_TILE;
+    if (nb < 1) nb = 1;
+    scan_tiles_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(f, n, out, tmp);
+    if (nb == 1) {
+        copy_one_kernel<<<1, 1, 0, st>>>(out + n, tmp);
+    } else {
+        scan_in_place(tmp, nb, tmp + (nb + 31) / 32 * 32, out + n, st);
+        scan_add_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(out, n, tmp);
+    }
+}
+
+// ------------------------------------------------------------------ radix sort
+constexpr int RS_THREADS = 256;
+constexpr int RS_ITEMS = 8;
+constexpr int RS_TILE = RS_THREADS * RS_ITEMS;
+
+__global__ void rs_hist_kernel(const u64* keys, i64 n, int shift, int* hist, int nblk) {
+    __shared__ int h[256];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const i64 base = (i64)blockIdx.x * RS_TILE;
+    for (int k = threadIdx.x; k < RS_TILE; k += RS_THREADS) {
+        i64 idx = base + k;
+        if (idx < n) atomicAdd(&h[(int)((keys[idx] >> shift) & 255)], 1);
+    }
+    __syncthreads();
+    hist[(i64)threadIdx.x * nblk + blockIdx.x] = h[threadIdx.x];
+}
+
+// Stable scatter of one 8-bit digit.  offsets[d * nblk + b] is the first output
+// slot of digit d for tile b.
+__global__ void rs_scatter_kernel(const u64* keys_in, const uint32_t* vals_in, u64* keys_out,
+                                  uint32_t* vals_out, i64 n, int shift, const int* offsets, int nblk) {
+    __shared__ int warp_cnt[RS_THREADS / 32][256];
+    __shared__ int base[256];
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    base[tid] = offsets[(i64)tid * nblk + blockIdx.x];
+    const i64 tile0 = (i64)blockIdx.x * RS_TILE;
+    for (int r = 0; r < RS_ITEMS; ++r) {
+#pragma unroll
+        for (int ww = 0; ww < RS_THREADS / 32; ++ww) warp_cnt[ww][tid] = 0;
+        __syncthreads();
+        const i64 idx = tile0 + (i64)r * RS_THREADS + tid;
+        const bool valid = idx < n;
+        u64 key = 0;
+        uint32_t val = 0;
+        int digit = 256 + lane;                       // unique: matches nobody
+        if (valid) {
+            key = keys_in[idx];
+            val = vals_in[idx];
+            digit = (int)((key >> shift) & 255);
+        }
+        const unsigned peers = __match_any_sync(0xffffffffu, digit);
+        const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+        if (valid && rank_in_warp == 0) warp_cnt[w][digit] = __popc(peers);
+        __syncthreads();
+        {
+            int run = base[tid];
+#pragma unroll
+            for (int ww = 0; ww < RS_THREADS / 32; ++ww) {
+                int c = warp_cnt[ww][tid];
+                warp_cnt[ww][tid] = run;
+                run += c;
+            }
+            base[tid] = run;
+        }
+        __syncthreads();
+        if (valid) {
+            const int dst = warp_cnt[w][digit] + rank_in_warp;
+            keys_out[dst] = key;
+            vals_out[dst] = val;
+        }
+        __syncthreads();
+    }
+}
+
+struct SortBuffers {
+    u64* keys[2];
+    uint32_t* vals[2];
+    int* hist;        // 256 * nblk + 1
+    int* scan_tmp;
+};
+
+// Sorts by the bit ranges [0, bits_lo) and [32, 32 + bits_hi) of the key, LSD.
+// Input in buffer 0; returns the index of the buffer that holds the result.
+int radix_sort_pairs(SortBuffers& b, i64 n, int bits_lo, int bits_hi, cudaStream_t st) {
+    int cur = 0;
+    const int nblk = (int)((n + RS_TILE - 1) / RS_TILE);
+    if (nblk == 0) return 0;
+    int shifts[16];
+    int ns = 0;
+    for (int s = 0; s < bits_lo; s += 8) shifts[ns++] = s;
+    for (int s = 0; s < bits_hi; s += 8) shifts[ns++] = 32 + s;
+    for (int k = 0; k < ns; ++k) {
+        rs_hist_kernel<<<nblk, RS_THREADS, 0, st>>>(b.keys[cur], n, shifts[k], b.hist, nblk);
+        scan_in_place(b.hist, (i64)256 * nblk, b.scan_tmp, b.hist + (i64)256 * nblk, st);
+        rs_scatter_kernel<<<nblk, RS_THREADS, 0, st>>>(b.keys[cur], b.vals[cur], b.keys[cur ^ 1], b.vals[cur ^ 1],
+                                                       n, shifts[k], b.hist, nblk);
+        cur ^= 1;
+    }
+    return cur;
+}
+
+// ------------------------------------------------------------------ suffix order
+// end_pos[i]: one past the last token of the sequence that holds position i.
+__global__ void seq_end_kernel(const int64_t* seq_offsets, int n_seqs, i64 n, int* end_pos) {
+    i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    int lo = 0, hi = n_seqs;                          // largest s with seq_offsets[s] <= i
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (seq_offsets[mid] <= i) lo = mid; else hi = mid;
+    }
+    end_pos[i] = (int)seq_offsets[lo + 1];
+}
+
+// bad[0] != 0 when a token is outside [0, V) or the offsets do not ascend from 0
+__global__ void validate_kernel(const int32_t* tok, i64 n, int V, const int64_t* seq_offsets, int n_seqs, int* bad) {
+    i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n && (tok[i] < 0 || tok[i] >= V)) atomicOr(bad, 1);
+    if (i < n_seqs && seq_offsets[i] > seq_offsets[i + 1]) atomicOr(bad, 2);
+    if (i == 0 && seq_offsets[0] != 0) atomicOr(bad, 2);
+}
+
+__global__ void rank0_kernel(const int32_t* tok, i64 n, int* rank) {
+    i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) rank[i] = tok[i] + 1;                  // 0 is "past the end of the sequence"
+}
+
+// key = (rank of the first `off` tokens, rank of the next block) ; 0 pads short suffixes
+__global__ void make_keys_kernel(const int* ra, const int* rb, int off, const int* end_pos, i64 n, u64* keys,
+                                 uint32_t* vals) {
+    i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    unsigned second = (i + off < end_pos[i]) ? (unsigned)rb[i + off] : 0u;
+    keys[i] = ((u64)(unsigned)ra[i] << 32) | second;
+    vals[i] = (uint32_t)i;
+}
+
+struct KeyChange {
+    const u64* keys;
+    __device__ int operator()(i64 j) const { return j == 0 ? 1 : (keys[j] != keys[j - 1] ? 1 : 0); }
+};
+
+__global__ void assign_rank_kernel(const u64* keys, const uint32_t* vals, const int* ex, i64 n, int* rank_out) {
+    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    int flag = j == 0 ? 1 : (keys[j] != keys[j - 1] ? 1 : 0);
+    rank_out[vals[j]] = ex[j] + flag;                 // dense, 1-based
+}
+
+// lcp[j] = common prefix (capped) of sorted suffixes j-1 and j; len[j] = capped length of suffix j
+__global__ void lcp_kernel(const int32_t* tok, const uint32_t* sa, const int* end_pos, i64 n, int D, uint8_t* lcp,
+                           uint8_t* len) {
+    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    i64 b = sa[j];
+    int lb = min((i64)D, (i64)end_pos[b] - b);
+    len[j] = (uint8_t)lb;
+    int l = 0;
+    if (j > 0) {
+        i64 a = sa[j - 1];
+        int la = min((i64)D, (i64)end_pos[a] - a);
+        int m = min(la, lb);
+        while (l < m && tok[a + l] == tok[b + l]) ++l;
+    }
+    lcp[j] = (uint8_t)l;
+}
+
+// nodes per depth: suffix j opens one node at every depth in (lcp[j], len[j]]
+__global__ void level_hist_kernel(const uint8_t* lcp, const uint8_t* len, i64 n, unsigned long long* level_nodes) {
+    __shared__ int diff[SD_MAX_DEPTH + 2];
+    if (threadIdx.x < SD_MAX_DEPTH + 2) diff[threadIdx.x] = 0;
+    __syncthreads();
+    for (i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (i64)gridDim.x * blockDim.x) {
+        int a = lcp[j], b = len[j];
+        if (b > a) {
+            atomicAdd(&diff[a + 1], 1);
+            atomicAdd(&diff[b + 1], -1);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int d = 1; d <= SD_MAX_DEPTH; ++d) {
+            run += diff[d];
+            if (run) atomicAdd(&level_nodes[d], (unsigned long long)run);
+        }
+    }
+}
+
+struct OpensNode {            // suffix j opens a node at depth d
+    const uint8_t* lcp;
+    const uint8_t* len;
+    int d;
+    __device__ int operator()(i64 j) const { return (lcp[j] < d && d <= len[j]) ? 1 : 0; }
+};
+struct Boundary {             // suffix j differs from its predecessor within the first d tokens
+    const uint8_t* lcp;
+    int d;
+    __device__ int operator()(i64 j) const { return lcp[j] < d ? 1 : 0; }
+};
+
+__global__ void seg_pos_kernel(const uint8_t* lcp, int d, const int* bscan, i64 n, int* segpos) {
+    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j > n) return;
+    if (j == n) { segpos[bscan[n]] = (int)n; return; }
+    if (lcp[j] < d) segpos[bscan[j]] = (int)j;
+}
+
+// Lay down the depth-d nodes.  Nodes of one depth are numbered in suffix order, so
+// the children of a node are consecutive at depth d + 1 and sorted by token.
+__global__ void emit_level_kernel(const int32_t* tok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len,
+                                  i64 n, int d, int D, const int* r_d, const int* r_next, const int* bscan,
+                                  const int* segpos, i64 base_d, i64 base_next, int4* ent, int32_t* root) {
+    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    if (!(lcp[j] < d && d <= len[j])) return;
+    const int nb = segpos[bscan[j] + 1];              // first suffix past this node's range
+    int4 e;
+    e.x = tok[(i64)sa[j] + d - 1];
+    e.y = nb - (int)j;                                // every suffix in the range is an occurrence
+    int nc = 0, cb = 0;
+    if (d < D) {
+        nc = r_next[nb] - r_next[j];
+        if (nc > 0) cb = (int)(base_next + r_next[j]);
+    }
+    e.z = cb;
+    e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC) : 0;
+    const i64 idx = base_d + r_d[j];
+    ent[idx] = e;
+    if (d == 1) root[e.x] = (int)idx;
+}
+
+__global__ void init_global_state_kernel(GlobalState* g, int used, long long tokens) {
+    g->used = used; g->live = used; g->status = 0; g->pad = 0; g->tokens = tokens;
+}
+
+struct DeviceArena {          // temporaries of one build, released together
+    void* ptr[40];
+    int n = 0;
+    ~DeviceArena() { for (int i = 0; i < n; ++i) cudaFree(ptr[i]); }
+    template <class T> bool get(T** out, i64 count) {
+        void* p = nullptr;
+        if (count < 1) count = 1;
+        if (cudaMalloc(&p, (size_t)count * sizeof(T)) != cudaSuccess) { cudaGetLastError(); return false; }
+        ptr[n++] = p;
+        *out = (T*)p;
+        return true;
+    }
+};
+
+inline unsigned grid_for(i64 n, int threads) { return (unsigned)((n + threads - 1) / threads); }
+
+int bits_for(i64 maxval) {
+    int b = 1;
+    while ((1ll << b) <= maxval && b < 32) ++b;
+    return b;
+}
+
+}  // namespace
+
+template <class T>
+static bool store_alloc(sd_store* s, T** out, long long count) {
+    void* p = nullptr;
+    if (count < 1) count = 1;
+    if (cudaMalloc(&p, (size_t)count * sizeof(T)) != cudaSuccess) { cudaGetLastError(); return false; }
+    s->device_bytes += count * (long long)sizeof(T);
+    *out = (T*)p;
+    return true;
+}
+
+static void store_release(sd_store* s) {
+    if (!s) return;
+    cudaFree(s->g_ent); cudaFree(s->g_root); cudaFree(s->g_state);
+    cudaFree(s->s_ent); cudaFree(s->s_root); cudaFree(s->s_text); cudaFree(s->s_state);
+    cudaFree(s->j_score); cudaFree(s->j_n); cudaFree(s->j_tok); cudaFree(s->j_par);
+    delete s;
+}
+
+extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const int64_t* d_seq_offsets, int32_t n_seqs,
+                        void* stream, sd_store** out) {
+    if (!out) return SD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!p || p->vocab < 1 || p->depth_cap < 1 || p->depth_cap > SD_MAX_DEPTH || p->max_requests < 1 ||
+        p->max_req_tokens < 1 || p->max_spec_cap < 1 || p->max_spec_cap > SD_MAX_SPEC || n_seqs < 0)
+        return SD_ERR_INVALID_ARG;
+    if (n_seqs > 0 && (!d_corpus || !d_seq_offsets)) return SD_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    i64 N = 0;
+    if (n_seqs > 0) {
+        SD_CUDA_OK(cudaMemcpyAsync(&N, d_seq_offsets + n_seqs, sizeof(i64), cudaMemcpyDeviceToHost, st));
+        SD_CUDA_OK(cudaStreamSynchronize(st));
+        if (N < 0 || N >= (1ll << 31) - 2) return SD_ERR_INVALID_ARG;
+    }
+
+    sd_store* s = new (std::nothrow) sd_store();
+    if (!s) return SD_ERR_NOMEM;
+    memset(s, 0, sizeof(*s));
+    s->V = p->vocab; s->D = p->depth_cap; s->R = p->max_requests; s->T = p->max_req_tokens; s->M = p->max_spec_cap;
+    const int D = s->D;
+    s->spn = p->slot_pool_nodes > 0 ? p->slot_pool_nodes : 2ll * s->T * D;
+    if (s->spn >= (1ll << 31) - 2) { delete s; return SD_ERR_INVALID_ARG; }
+
+    const i64 jobs = (i64)s->R * 2 * D;
+    bool ok = store_alloc(s, &s->g_root, s->V) && store_alloc(s, &s->g_state, 1) &&
+              store_alloc(s, &s->s_ent, (i64)s->R * s->spn) && store_alloc(s, &s->s_root, (i64)s->R * s->V) &&
+              store_alloc(s, &s->s_text, (i64)s->R * s->T) && store_alloc(s, &s->s_state, s->R) &&
+              store_alloc(s, &s->j_score, jobs) && store_alloc(s, &s->j_n, jobs) &&
+              store_alloc(s, &s->j_tok, jobs * s->M) && store_alloc(s, &s->j_par, jobs * s->M);
+    if (!ok) { store_release(s); return SD_ERR_NOMEM; }
+    cudaError_t ce = cudaMemsetAsync(s->g_root, 0xFF, sizeof(int32_t) * (size_t)s->V, st);
+    if (ce == cudaSuccess) ce = cudaMemsetAsync(s->s_root, 0xFF, sizeof(int32_t) * (size_t)s->R * s->V, st);
+    if (ce == cudaSuccess) ce = cudaMemsetAsync(s->s_state, 0, sizeof(SlotState) * (size_t)s->R, st);
+    if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
+
+    i64 n_nodes = 0;
+    i64 level_base[SD_MAX_DEPTH + 2] = {0};
+    DeviceArena tmp;
+    SortBuffers sb;
+    int *end_pos = nullptr, *rank[8] = {nullptr}, *comb[2] = {nullptr, nullptr}, *ex = nullptr;
+    uint8_t *lcp = nullptr, *len = nullptr;
+    unsigned long long* level_nodes = nullptr;
+    const uint32_t* sa = nullptr;
+    const int T256 = 256;
+
+    if (N > 0) {
+        const int nblk = (int)((N + RS_TILE - 1) / RS_TILE);
+        int m = 0;
+        while ((2 << m) <= D) ++m;                    // 2^m <= D < 2^(m+1)
+        ok = tmp.get(&sb.keys[0], N) && tmp.get(&sb.keys[1], N) && tmp.get(&sb.vals[0], N) &&
+             tmp.get(&sb.vals[1], N) && tmp.get(&sb.hist, (i64)256 * nblk + 1) &&
+             tmp.get(&sb.scan_tmp, scan_tmp_ints(std::max<i64>((i64)256 * nblk, N + 1))) &&
+             tmp.get(&end_pos, N) && tmp.get(&ex, N + 1) && tmp.get(&lcp, N) && tmp.get(&len, N) &&
+             tmp.get(&level_nodes, SD_MAX_DEPTH + 2);
+        for (int k = 0; ok && k <= m; ++k) ok = tmp.get(&rank[k], N);
+        ok = ok && tmp.get(&comb[0], N) && tmp.get(&comb[1], N);
+        if (!ok) { store_release(s); return SD_ERR_NOMEM; }
+
+        {
+            int* bad = (int*)level_nodes;
+            int h_bad = 0;
+            ce = cudaMemsetAsync(bad, 0, sizeof(int), st);
+            validate_kernel<<<grid_for(std::max<i64>(N, n_seqs), T256), T256, 0, st>>>(d_corpus, N, s->V, d_seq_offsets,
+                                                                                      n_seqs, bad);
+            if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, st);
+            if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+            if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
+            if (h_bad) { store_release(s); return SD_ERR_INVALID_ARG; }
+        }
+        seq_end_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_seq_offsets, n_seqs, N, end_pos);
+        rank0_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, N, rank[0]);
+        int bits = bits_for(std::max<i64>(s->V, N) + 1);
+        int sorted = 0;
+        // rank[k] orders the first 2^k tokens of every suffix
+        auto round = [&](const int* ra, const int* rb, int off, int* rout) {
+            make_keys_kernel<<<grid_for(N, T256), T256, 0, st>>>(ra, rb, off, end_pos, N, sb.keys[0], sb.vals[0]);
+            sorted = radix_sort_pairs(sb, N, bits, bits, st);
+            if (rout) {
+                exclusive_scan(KeyChange{sb.keys[sorted]}, N, ex, sb.scan_tmp, st);
+                assign_rank_kernel<<<grid_for(N, T256), T256, 0, st>>>(sb.keys[sorted], sb.vals[sorted], ex, N, rout);
+            }
+        };
+        if (m == 0) {
+            round(rank[0], rank[0], 1 << 30, nullptr);        // D == 1: the first token alone
+        } else {
+            const bool pow2 = D == (1 << m);
+            for (int k = 0; k < m; ++k)
+                round(rank[k], rank[k], 1 << k, (pow2 && k == m - 1) ? nullptr : rank[k + 1]);
+            if (!pow2) {
+                // append the remaining binary digits of D, high to low
+                int cur_len = 1 << m, rem = D - cur_len, which = 0;
+                const int* cur = rank[m];
+                for (int b = m - 1; b >= 0; --b) {
+                    if (!(rem & (1 << b))) continue;
+                    rem -= 1 << b;
+                    int* dst = rem == 0 ? nullptr : comb[which];
+                    round(cur, rank[b], cur_len, dst);
+                    cur = dst;
+                    which ^= 1;
+                    cur_len += 1 << b;
+                }
+            }
+        }
+        sa = sb.vals[sorted];
+        lcp_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, sa, end_pos, N, D, lcp, len);
+        ce = cudaMemsetAsync(level_nodes, 0, sizeof(unsigned long long) * (SD_MAX_DEPTH + 2), st);
+        level_hist_kernel<<<(unsigned)std::min<i64>(grid_for(N, T256), 1184), T256, 0, st>>>(lcp, len, N, level_nodes);
+        unsigned long long h_level[SD_MAX_DEPTH + 2];
+        if (ce == cudaSuccess)
+            ce = cudaMemcpyAsync(h_level, level_nodes, sizeof(h_level), cudaMemcpyDeviceToHost, st);
+        if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+        if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
+        for (int d = 1; d <= D; ++d) { level_base[d] = n_nodes; n_nodes += (i64)h_level[d]; }
+        level_base[D + 1] = n_nodes;
+    }
+
+    i64 extra = p->global_extra_nodes >= 0 ? p->global_extra_nodes : std::max<i64>(1ll << 22, n_nodes);
+    s->g_cap = n_nodes + extra;
+    if (s->g_cap >= (1ll << 31) - 2) { store_release(s); return SD_ERR_INVALID_ARG; }
+    if (!store_alloc(s, &s->g_ent, s->g_cap)) { store_release(s); return SD_ERR_NOMEM; }
+
+    if (N > 0) {
+        int *r_a = nullptr, *r_b = nullptr, *bscan = nullptr, *segpos = nullptr;
+        ok = tmp.get(&r_a, N + 1) && tmp.get(&r_b, N + 1) && tmp.get(&segpos, N + 2);
+        bscan = ex;
+        if (!ok) { store_release(s); return SD_ERR_NOMEM; }
+        int* r_next = r_a;  // scan of depth d + 1 (unused at d == D)
+        int* r_cur = r_b;
+        for (int d = D; d >= 1; --d) {
+            exclusive_scan(OpensNode{lcp, len, d}, N, r_cur, sb.scan_tmp, st);
+            exclusive_scan(Boundary{lcp, d}, N, bscan, sb.scan_tmp, st);
+            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(lcp, d, bscan, N, segpos);
+            emit_level_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, sa, lcp, len, N, d, D, r_cur, r_next, bscan,
+                                                                 segpos, level_base[d], level_base[d + 1], s->g_ent,
+                                                                 s->g_root);
+            std::swap(r_cur, r_next);
+        }
+    }
+    init_global_state_kernel<<<1, 1, 0, st>>>(s->g_state, (int)n_nodes, N);
+    ce = cudaStreamSynchronize(st);
+    if (ce == cudaSuccess) ce = cudaGetLastError();
+    if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
+    *out = s;
+    return SD_OK;
+}
+
+extern "C" void sd_free(sd_store* s) {
+    if (!s) return;
+    cudaDeviceSynchronize();
+    store_release(s);
+}
+
+extern "C" const char* sd_strerror(int code) {
+    switch (code) {
+        case SD_OK: return "ok";
+        case SD_ERR_INVALID_ARG: return "invalid argument";
+        case SD_ERR_CUDA: return "CUDA runtime error";
+        case SD_ERR_NOMEM: return "out of device memory";
+        case SD_ERR_CAPACITY: return "capacity exceeded";
+        default: return "unknown error";
+    }
+}

@@ -1,0 +1,81 @@
+// Shared declarations of the suffixspec CUDA library (sm_100a).
+//
+// Node storage.  A tree node is a 16-byte ENTRY that lives inside its parent's
+// child run:
+//     x = token id          y = count (occurrences of the root-to-node path)
+//     z = index of the first entry of this node's own child run
+//     w = number of children (low 24 bits) | RUN_STATIC (bit 31)
+// A child run is a contiguous array of entries sorted by token id, so one
+// 16-byte load per child yields everything Eq. 1 needs (token, count) plus the
+// way down.  A run with n children built online has room for pow2ceil(n)
+// entries; a run laid down by the offline build is an exact fit (RUN_STATIC)
+// and moves to a roomier place on its first insert.  Depth-1 nodes are found
+// through a direct table root[token] -> entry index (-1: absent), so the root
+// needs no run of its own.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "suffixspec.h"
+
+#define SD_MAX_DEPTH 32
+#define SD_MAX_SPEC 64
+#define RUN_STATIC 0x80000000u
+#define RUN_COUNT_MASK 0x00FFFFFFu
+
+struct GlobalState {          // device-resident bookkeeping of the global tree
+    int32_t used;             // entries handed out
+    int32_t live;             // live nodes
+    int32_t status;           // SD_STATUS_GLOBAL_FULL or 0
+    int32_t pad;
+    long long tokens;         // tokens inserted
+};
+
+struct SlotState {            // device-resident bookkeeping of one request slot
+    int32_t len;              // context length t
+    int32_t used;             // entries handed out of the slot pool
+    int32_t live;             // live nodes
+    int32_t status;           // SD_STATUS_*
+    int32_t active[SD_MAX_DEPTH];   // active[d-1]: entry of the node for the last d tokens
+};
+
+struct sd_store {
+    int32_t V, D, R, T, M;
+    // global tree
+    int4* g_ent;
+    long long g_cap;
+    int32_t* g_root;          // [V]
+    GlobalState* g_state;
+    // per-request trees
+    int4* s_ent;              // [R][spn]
+    long long spn;
+    int32_t* s_root;          // [R][V]
+    int32_t* s_text;          // [R][T]
+    SlotState* s_state;       // [R]
+    // scratch of sd_speculate: one record per (request, tree, p) job
+    double* j_score;          // [R*2*D]
+    int32_t* j_n;             // [R*2*D]
+    int32_t* j_tok;           // [R*2*D][M]
+    int32_t* j_par;           // [R*2*D][M]
+    long long device_bytes;
+};
+
+__host__ __device__ inline uint32_t sd_pow2ceil(uint32_t n) {
+    uint32_t c = 1;
+    while (c < n) c <<= 1;
+    return c;
+}
+
+// Room of a child run that currently holds n children.
+__host__ __device__ inline uint32_t sd_run_capacity(uint32_t w) {
+    uint32_t n = w & RUN_COUNT_MASK;
+    if (n == 0) return 0;
+    return (w & RUN_STATIC) ? n : sd_pow2ceil(n);
+}
+
+#define SD_CUDA_OK(expr)                                   \
+    do {                                                   \
+        cudaError_t _e = (expr);                           \
+        if (_e != cudaSuccess) return SD_ERR_CUDA;         \
+    } while (0)

@@ -1,0 +1,233 @@
+"""GPU parity: the CUDA path against the CPU oracle, element by element, on the
+same seeded inputs, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def U():
+    import gpu_util
+    return gpu_util
+
+
+def _rand_seqs(rng, n, lo, hi, vocab):
+    return [rng.integers(0, vocab, size=int(rng.integers(lo, hi + 1))).astype(np.int32) for _ in range(n)]
+
+
+# ---------------------------------------------------------------- offline build (a1)
+@pytest.mark.parametrize("D", [1, 2, 3, 5, 8, 13, 32])
+@pytest.mark.parametrize("vocab", [2, 50])
+def test_build_counts_match_oracle(U, D, vocab):
+    rng = np.random.default_rng(D * 100 + vocab)
+    seqs = _rand_seqs(rng, 12, 0, 300, vocab) + [np.full(70, 1, dtype=np.int32)]
+    pr = U.Pair(seqs, vocab=vocab, D=D, n_slots=1, max_req_tokens=8)
+    pr.check_tree(-1)
+    # absent and over-long paths count 0
+    paths = [[vocab - 1] * (D + 1), [0] * min(D, 3) + [vocab - 1] * 0]
+    off, flat = U.ragged(paths)
+    got = pr.g.query_counts(U.dev_i32([-1, -1]), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat)).cpu().numpy()
+    assert got[0] == 0 and got[1] == pr.o.count(-1, paths[1])
+    pr.close()
+
+
+def test_build_spans_many_tiles_and_ragged_tail(U):
+    # > 2048-element sort/scan tiles, ragged last tile, repeated spans
+    from workload.generator import get_workload
+    w = get_workload("tiny")
+    corpus = w.corpus()
+    seqs = [corpus[i * 512:(i + 1) * 512] for i in range(64)]
+    seqs[-1] = seqs[-1][:301]
+    pr = U.Pair(seqs, vocab=32000, D=32, n_slots=1, max_req_tokens=8)
+    pr.check_tree(-1)
+    pr.close()
+
+
+def test_build_empty_corpus_and_bad_inputs(U):
+    import paper_2411_04975_b200 as sfx
+    pr = U.Pair([], vocab=10, D=4, n_slots=2, max_req_tokens=16)
+    assert pr.g.stats()["global_nodes"] == 0
+    got, _ = pr.check_speculate([0, 1], 4, 2.0, 8)
+    assert (got["n_draft"] == 0).all()
+    pr.close()
+    with pytest.raises(sfx.SuffixSpecError):       # token outside [0, V)
+        U.Pair([np.array([1, 2, 99], dtype=np.int32)], vocab=10, D=4, n_slots=1, max_req_tokens=8)
+    with pytest.raises(sfx.SuffixSpecError):       # depth cap beyond the limit
+        U.Pair([np.array([1, 2], dtype=np.int32)], vocab=10, D=33, n_slots=1, max_req_tokens=8)
+    with pytest.raises(sfx.SuffixSpecError):
+        U.Pair([np.array([1, 2], dtype=np.int32)], vocab=10, D=4, n_slots=1, max_req_tokens=8, M=65)
+
+
+# ---------------------------------------------------------------- online update (a2, a3, a4)
+@pytest.mark.parametrize("D", [1, 4, 32])
+@pytest.mark.parametrize("vocab", [1, 2, 40])
+def test_append_matches_oracle_after_every_batch(U, D, vocab):
+    rng = np.random.default_rng(7 * D + vocab)
+    n_slots = 5
+    pr = U.Pair(_rand_seqs(rng, 3, 5, 40, vocab), vocab=vocab, D=D, n_slots=n_slots, max_req_tokens=400)
+    # prompts (reset), one slot left empty
+    slots = [0, 1, 2, 3]
+    pr.append(slots, _rand_seqs(rng, 4, 0, 120, vocab), reset=[1, 1, 1, 1])
+    for s in range(n_slots):
+        pr.check_tree(s)
+    for step in range(6):
+        k = int(rng.integers(1, n_slots + 1))
+        slots = sorted(rng.choice(n_slots, size=k, replace=False).tolist())
+        toks = _rand_seqs(rng, k, 0, 9, vocab)
+        if step == 3:                               # long runs of one token (periodic tail)
+            toks = [np.full(40, vocab - 1, dtype=np.int32) for _ in slots]
+        pr.append(slots, toks)
+        for s in range(n_slots):
+            pr.check_tree(s)
+    # a new request reuses a slot
+    pr.append([1, 4], _rand_seqs(rng, 2, 30, 60, vocab), reset=[1, 0])
+    for s in (1, 4):
+        pr.check_tree(s)
+    pr.check_tree(-1)                               # the global tree was never touched
+    pr.close()
+
+
+@pytest.mark.parametrize("vocab", [2, 30])
+def test_global_online_insert(U, vocab):
+    rng = np.random.default_rng(vocab)
+    pr = U.Pair(_rand_seqs(rng, 6, 10, 200, vocab), vocab=vocab, D=8, n_slots=2, max_req_tokens=64)
+    for step in range(4):
+        seqs = _rand_seqs(rng, 3, 0, 90, vocab)
+        pr.append([-1, 0, -1, -1], [seqs[0], rng.integers(0, vocab, size=5).astype(np.int32), seqs[1], seqs[2]])
+        pr.check_tree(-1)
+        pr.check_tree(0)
+    assert pr.g.stats()["global_tokens"] == pr.o.count(-1, [0]) + sum(
+        pr.o.count(-1, [v]) for v in range(1, vocab))
+    pr.close()
+    # into an empty global tree
+    pr = U.Pair([], vocab=vocab, D=5, n_slots=1, max_req_tokens=8)
+    pr.append([-1, -1], _rand_seqs(rng, 2, 20, 50, vocab))
+    pr.check_tree(-1)
+    pr.close()
+
+
+def test_pool_overflow_is_reported_and_tree_stays_consistent(U):
+    rng = np.random.default_rng(3)
+    pr = U.Pair([], vocab=1000, D=8, n_slots=2, max_req_tokens=64, slot_pool_nodes=100)
+    toks = rng.integers(0, 1000, size=60).astype(np.int32)
+    off, flat = U.ragged([toks, toks[:5]])
+    pr.g.append(U.dev_i32([0, 1]), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat))
+    info = pr.g.slot_info(U.dev_i32([0, 1, 7]))
+    status = info["status"].cpu().numpy()
+    assert status[0] & 2 and status[1] == 0 and status[2] == 1
+    kept = int(info["len"][0])
+    assert 0 < kept < 60
+    pr.o.slot_append(0, toks[:kept]); pr.o.slot_append(1, toks[:5])
+    pr.check_tree(0); pr.check_tree(1)
+    out = pr.g.speculate(U.dev_i32([0, 1]), 4, 2.0, 8)
+    assert int(out["n_draft"][0]) == 0 and int(out["status"][0]) & 2
+    # text buffer limit
+    pr.g.append(U.dev_i32([1]), torch.as_tensor(np.array([0, 70]), device=U.DEV), U.dev_i32(np.arange(70) % 3))
+    assert int(pr.g.slot_info(U.dev_i32([1]))["status"][0]) & 2
+    # a token outside the vocabulary stops that slot only
+    pr.g.append(U.dev_i32([0]), torch.as_tensor(np.array([0, 2]), device=U.DEV), U.dev_i32([5, 1000]),
+                torch.ones(1, dtype=torch.uint8, device=U.DEV))
+    assert int(pr.g.slot_info(U.dev_i32([0]))["status"][0]) == 8
+    pr.close()
+
+
+# ---------------------------------------------------------------- speculate (a5 - a8)
+@pytest.mark.parametrize("seed", range(4))
+def test_speculate_small_vocab_stress(U, seed):
+    """Low-entropy text: wide child runs, many equal scores (tie rules), deep trees."""
+    rng = np.random.default_rng(40 + seed)
+    vocab = [2, 3, 6, 12][seed]
+    D = [32, 8, 16, 5][seed]
+    n_slots = 24
+    pr = U.Pair(_rand_seqs(rng, 20, 50, 400, vocab), vocab=vocab, D=D, n_slots=n_slots, max_req_tokens=300)
+    pr.append(list(range(n_slots)), _rand_seqs(rng, n_slots, 0, 200, vocab), reset=[1] * n_slots)
+    slots = list(range(n_slots))
+    for (P, alpha, ms) in [(8, 1.0, 8), (32, 2.0, 64), (40, 1.5, 33), (3, 0.5, 64), (16, 4.0, 64), (5, 8.0, 1)]:
+        for flags in (0, 1, 2, 4, 5, 6):
+            pr.check_speculate(slots, P, alpha, ms, flags)
+    bc = rng.integers(-1, 20, size=n_slots).astype(np.int32)
+    pr.check_speculate(slots, 16, 2.0, 64, 0, bc)
+    # subset of the batch, in another order
+    pr.check_speculate([5, 3, 17], 16, 2.0, 64)
+    pr.close()
+
+
+def test_speculate_tiny_config(U):
+    """BASELINE config 0 at full size."""
+    from workload.generator import get_workload
+    w = get_workload("tiny")
+    c = w.cfg
+    corpus = w.corpus()
+    seqs = [corpus[i * c.seq_len:(i + 1) * c.seq_len] for i in range(c.n_seqs)]
+    pr = U.Pair(seqs, vocab=c.vocab, D=c.depth_cap, n_slots=c.batch, max_req_tokens=c.prompt_len + 64, M=c.max_spec)
+    pr.append(list(range(c.batch)), w.prompts(), reset=[1] * c.batch)
+    got, want = pr.check_speculate(list(range(c.batch)), c.max_pattern, c.alpha, c.max_spec)
+    assert (got["n_draft"] > 0).any()
+    for s in range(c.batch):
+        pr.check_tree(s)
+    pr.close()
+
+
+def test_speculate_wide_runs(U):
+    """A match node with thousands of children (several 32-entry chunks, the
+    32-way search) and a bounded frontier much smaller than the run."""
+    rng = np.random.default_rng(5)
+    vocab = 5000
+    seqs = [np.stack([np.zeros(3000, dtype=np.int32), rng.integers(1, vocab, size=3000).astype(np.int32)],
+                     axis=1).reshape(-1)]
+    seqs += _rand_seqs(rng, 10, 100, 300, vocab)
+    pr = U.Pair(seqs, vocab=vocab, D=6, n_slots=4, max_req_tokens=700)
+    prompts = [np.concatenate([s[:600], [0]]).astype(np.int32) for s in (seqs[0], seqs[0][2:], seqs[1], seqs[2])]
+    pr.append([0, 1, 2, 3], prompts, reset=[1] * 4)
+    for (P, alpha, ms) in [(1, 64.0, 64), (4, 16.0, 64), (6, 2.0, 7)]:
+        pr.check_speculate([0, 1, 2, 3], P, alpha, ms)
+    for s in range(4):
+        pr.check_tree(s)
+    pr.check_tree(-1)
+    pr.close()
+
+
+def test_speculate_edge_cases(U):
+    import paper_2411_04975_b200 as sfx
+    rng = np.random.default_rng(1)
+    pr = U.Pair(_rand_seqs(rng, 4, 20, 60, 4), vocab=4, D=8, n_slots=3, max_req_tokens=64, M=40)
+    pr.append([0, 2], _rand_seqs(rng, 2, 10, 30, 4), reset=[1, 1])
+    # slot 1 is empty (t = 0): no pattern, no draft
+    got, _ = pr.check_speculate([0, 1, 2], 8, 2.0, 40)
+    assert got["n_draft"][1] == 0 and got["chosen_tree"][1] == -1
+    assert got["mask"].shape == (3, 40, 2)
+    # max_spec 0 and alpha 0: empty drafts everywhere
+    got, _ = pr.check_speculate([0, 2], 8, 2.0, 0)
+    assert (got["n_draft"] == 0).all()
+    got, _ = pr.check_speculate([0, 2], 8, 0.0, 40)
+    assert (got["n_draft"] == 0).all()
+    # out-of-range slot: status only
+    out = pr.g.speculate(U.dev_i32([0, 9]), 8, 2.0, 40)
+    assert int(out["status"][1]) == 1 and int(out["n_draft"][1]) == 0 and int(out["status"][0]) == 0
+    # argument errors are return codes
+    for bad in (dict(P=0), dict(max_spec=41), dict(flags=3), dict(alpha=float("nan"))):
+        kw = dict(P=8, alpha=2.0, max_spec=40, flags=0)
+        kw.update(bad)
+        with pytest.raises(sfx.SuffixSpecError):
+            pr.g.speculate(U.dev_i32([0]), kw["P"], kw["alpha"], kw["max_spec"], kw["flags"])
+    with pytest.raises(sfx.SuffixSpecError):
+        pr.g.speculate(U.dev_i32([0, 1, 2, 0]), 8, 2.0, 40)        # more requests than slots
+    # n = 0 is a no-op
+    pr.g.speculate(torch.zeros(0, dtype=torch.int32, device=U.DEV), 8, 2.0, 40)
+    pr.g.append(torch.zeros(0, dtype=torch.int32, device=U.DEV), torch.zeros(1, dtype=torch.int64, device=U.DEV),
+                torch.zeros(0, dtype=torch.int32, device=U.DEV))
+    pr.close()
+
+
+def test_speculate_is_deterministic(U):
+    rng = np.random.default_rng(2)
+    pr = U.Pair(_rand_seqs(rng, 10, 100, 300, 5), vocab=5, D=16, n_slots=16, max_req_tokens=256)
+    pr.append(list(range(16)), _rand_seqs(rng, 16, 50, 200, 5), reset=[1] * 16)
+    a = pr.g.speculate(U.dev_i32(list(range(16))), 16, 2.0, 64)
+    a = {k: v.clone() for k, v in a.items()}
+    b = pr.g.speculate(U.dev_i32(list(range(16))), 16, 2.0, 64)
+    for k in a:
+        assert torch.equal(a[k], b[k])
+    pr.close()

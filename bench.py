@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of batched SuffixDecoding draft generation on B200.
+
+A step is one decode step of the whole batch on the headline workload
+(config "large_batch": 4M-token global corpus, 256 requests with 4,096-token
+prompts): sd_speculate for every request, then sd_append of the tokens each
+request accepted in that step (a seeded schedule, mean 4 tokens, taken from the
+request's hidden continuation).  The global tree and the prompts are built
+before the timed region.  One JSON line is printed by rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workload.generator import accept_schedule, get_workload  # noqa: E402
+
+METRIC = "speculation trees/s at batch 256 (one sd_speculate + sd_append per step)"
+UNIT = "trees/s"
+OUT_BYTES_PER_REQ = 4 * 64 * 3 + 64 * 8 + 4 * 3 + 8          # tokens, parents, positions, mask, scalars
+FLUSH_BYTES = 256 << 20
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="large_batch")
+    ap.add_argument("--no-oracle", action="store_true", help="skip the CPU-oracle leg (profiling runs)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--oracle-samples", type=int, default=4)
+    ap.add_argument("--small", action="store_true", help="1/16 corpus, batch 32: quick functional run")
+    return ap.parse_args()
+
+
+def make_workload(args):
+    kw = {}
+    if args.small:
+        kw = dict(n_seqs=256, batch=32)
+    return get_workload(args.config, **kw)
+
+
+class StepInputs:
+    """Per-step append inputs for `n_steps` steps of `B` requests."""
+
+    def __init__(self, w, first_request, B, n_steps, prompts):
+        self.sched = accept_schedule(B, n_steps, seed_index=first_request)
+        total = self.sched.sum(axis=0)
+        self.cont = [w.continuation(first_request + i, prompts[i], length=int(total[i]) + 1) for i in range(B)]
+        self.cursor = np.zeros(B, dtype=np.int64)
+        self.max_total = int(total.max())
+        self.offsets, self.tokens, self.lists = [], [], []
+        for k in range(n_steps):
+            a = self.sched[k]
+            off = np.zeros(B + 1, dtype=np.int64)
+            off[1:] = np.cumsum(a)
+            lists = [self.cont[i][self.cursor[i]:self.cursor[i] + a[i]] for i in range(B)]
+            self.cursor += a
+            self.offsets.append(off)
+            self.lists.append(lists)
+            self.tokens.append(np.concatenate(lists).astype(np.int32))
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for j, n in enumerate(names) if any(len(r) >= 7 and r[3 + j] == "Active" for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def oracle_threads(B):
+    return max(1, min(os.cpu_count() or 1, B))
+
+
+# --------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2411_04975_b200 as sfx
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = make_workload(args)
+    c = w.cfg
+    B, K, W = c.batch, args.steps, args.warmup
+    Ke = 0 if args.no_e2e else K
+    We = 0 if args.no_e2e else min(W, 3)
+    n_steps = W + K + We + Ke
+    first = rank * B                                  # weak scaling: every rank has its own requests
+    prompts = [w.prompt(first + i) for i in range(B)]
+    steps = StepInputs(w, first, B, n_steps, prompts)
+
+    corpus = torch.as_tensor(w.corpus(), device=dev)
+    offsets = torch.as_tensor(w.corpus_offsets(), device=dev)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    store = sfx.SuffixStore(corpus, offsets, vocab=c.vocab, depth_cap=c.depth_cap, max_requests=B,
+                            max_req_tokens=c.prompt_len + steps.max_total + 8, max_spec_cap=c.max_spec)
+    torch.cuda.synchronize()
+    build_ms = (time.perf_counter() - t0) * 1e3
+    slots = torch.arange(B, dtype=torch.int32, device=dev)
+    poff = np.zeros(B + 1, dtype=np.int64)
+    poff[1:] = np.cumsum([len(p) for p in prompts])
+    t0 = time.perf_counter()
+    store.append(slots, torch.as_tensor(poff, device=dev), torch.as_tensor(np.concatenate(prompts), device=dev),
+                 torch.ones(B, dtype=torch.uint8, device=dev))
+    torch.cuda.synchronize()
+    prompt_ms = (time.perf_counter() - t0) * 1e3
+
+    d_off = [torch.as_tensor(o, device=dev) for o in steps.offsets[:W + K]]
+    d_tok = [torch.as_tensor(t, device=dev) for t in steps.tokens[:W + K]]
+    out = store.alloc_outputs(B)
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    def step(k):
+        store.speculate(slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
+        store.append(slots, d_off[k], d_tok[k])
+
+    n_samp = 0 if (args.no_oracle or world > 1) else max(1, min(args.oracle_samples, K))
+    sample_steps = sorted({W + (j * K) // n_samp for j in range(n_samp)}) if n_samp else []
+    saved = {}
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    for k in range(W):
+        flush.zero_()
+        step(k)
+    torch.cuda.synchronize()
+    if rank == 0:                                      # let the clock sampler come up
+        t_wait = time.perf_counter()
+        while not sampler.rows and time.perf_counter() - t_wait < 5.0:
+            time.sleep(0.05)
+        sampler.rows.clear()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    wall0 = time.perf_counter()
+    for j in range(K):
+        k = W + j
+        flush.zero_()                                  # L2 flush, outside the per-step events
+        ev[j][0].record()
+        store.speculate(slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
+        ev[j][1].record()
+        store.append(slots, d_off[k], d_tok[k])
+        ev[j][2].record()
+        if k in sample_steps:
+            saved[k] = {n: t.clone() for n, t in out.items()}
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    wall_ms = (time.perf_counter() - wall0) * 1e3
+    clocks = sampler.stop() if rank == 0 else None
+    spec_ms = [ev[j][0].elapsed_time(ev[j][1]) for j in range(K)]
+    app_ms = [ev[j][1].elapsed_time(ev[j][2]) for j in range(K)]
+    tot_ms = [ev[j][0].elapsed_time(ev[j][2]) for j in range(K)]
+    timed_ms = float(sum(tot_ms))
+    if world > 1:
+        t = torch.tensor([timed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        timed_ms = float(t.item())
+    ms_per_step = timed_ms / K
+
+    # ---- end to end: host buffers in, host buffers out, every step
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda a: torch.as_tensor(a).pin_memory()   # noqa: E731
+        h_off = [pin(o) for o in steps.offsets[W + K:]]
+        h_tok = [pin(t) for t in steps.tokens[W + K:]]
+        h_slots = pin(np.arange(B, dtype=np.int32))
+        max_tok = max(int(t.numel()) for t in h_tok)
+        s_slots = torch.empty(B, dtype=torch.int32, device=dev)
+        s_off = torch.empty(B + 1, dtype=torch.int64, device=dev)
+        s_tok = torch.empty(max_tok, dtype=torch.int32, device=dev)
+        h_out = {n: torch.empty(t.shape, dtype=t.dtype).pin_memory() for n, t in out.items()}
+        h2d = d2h = 0
+
+        def e2e_step(k):
+            nonlocal h2d, d2h
+            nt = int(h_tok[k].numel())
+            s_slots.copy_(h_slots, non_blocking=True)
+            s_off.copy_(h_off[k], non_blocking=True)
+            s_tok[:nt].copy_(h_tok[k], non_blocking=True)
+            store.speculate(s_slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
+            for n in h_out:
+                h_out[n].copy_(out[n], non_blocking=True)
+            store.append(s_slots, s_off, s_tok[:nt])
+            torch.cuda.synchronize()
+            h2d += 4 * B + 8 * (B + 1) + 4 * nt
+            d2h += sum(t.numel() * t.element_size() for t in h_out.values())
+
+        for k in range(We):
+            e2e_step(k)
+        h2d = d2h = 0
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for k in range(We, We + Ke):
+            flush.zero_()
+            e2e_step(k)
+        e2e_s = time.perf_counter() - t0
+        # the flush is not part of the path: time it alone and take it out
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        for _ in range(Ke):
+            flush.zero_()
+        torch.cuda.synchronize()
+        e2e_s -= (time.perf_counter() - t1)
+        if world > 1:
+            t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        e2e = {"value": B * world * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d // Ke,
+               "d2h_bytes_per_step": d2h // Ke, "ms_per_step": e2e_s / Ke * 1e3}
+
+    # ---- CPU oracle beside it (rank 0, one GPU): lock-step replay, sampled steps timed and compared
+    cpu_baseline = None
+    roofline = None
+    extra = {}
+    if n_samp:
+        import oracle
+        thr = oracle_threads(B)
+        t0 = time.perf_counter()
+        ref = oracle.SuffixOracle(c.depth_cap, B)
+        ref.global_build(w.corpus(), w.corpus_offsets())
+        ref.slot_append_batch(list(range(B)), prompts, n_threads=thr)
+        setup_s = time.perf_counter() - t0
+        o_times, desc, adds, ok = [], [], [], True
+        for k in range(max(sample_steps) + 1):
+            t0 = time.perf_counter()
+            if k in sample_steps:
+                r = ref.speculate(list(range(B)), c.max_pattern, c.alpha, c.max_spec, n_threads=thr)
+            ref.slot_append_batch(list(range(B)), steps.lists[k], n_threads=thr)
+            if k in sample_steps:
+                o_times.append(time.perf_counter() - t0)
+                desc.append(int(r["visited"][:, 0].sum()))
+                adds.append(int(r["visited"][:, 1].sum()))
+                g = {n: t.cpu().numpy() for n, t in saved[k].items()}
+                for n in ("n_draft", "tokens", "parents", "positions", "chosen_tree", "chosen_p"):
+                    ok = ok and np.array_equal(g[n], r[n])
+                ok = ok and np.array_equal(g["mask"].view(np.uint32), r["mask"])
+                ok = ok and np.array_equal(g["score"].view(np.int64), r["score"].view(np.int64))
+        o_step = statistics.mean(o_times)
+        cpu_baseline = {"value": B / o_step, "unit": UNIT, "cores": thr, "kind": "oracle",
+                        "sample": f"{len(sample_steps)} of the {K} timed steps (all {B} requests each), "
+                                  f"{sum(o_times):.1f} s wall on {thr} threads; setup {setup_s:.0f} s untimed"}
+        visits = statistics.mean(d + a for d, a in zip(desc, adds))
+        alg_bytes = statistics.mean(32 * d + 64 * a for d, a in zip(desc, adds)) + B * OUT_BYTES_PER_REQ
+        peak, which = measured_peak()
+        spec_s = statistics.mean(spec_ms) / 1e3
+        achieved = alg_bytes / spec_s / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": None, "peak_source": which, "kernel": "sd_speculate (match_expand + select_emit)",
+                    "algorithmic_bytes_per_launch": alg_bytes}
+        extra = {"parity_vs_oracle": "bit-exact" if ok else "MISMATCH", "parity_steps": len(sample_steps),
+                 "nodes_visited_per_step": visits,
+                 "nodes_visited_per_s": visits * world / (ms_per_step / 1e3)}
+        ref.close()
+
+    if rank == 0:
+        st = store.stats()
+        line = {
+            "metric": METRIC, "value": B * world / (ms_per_step / 1e3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int32 trees, f64 scores", "data": "synthetic",
+            "config": {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": B,
+                       "global_tokens": int(c.n_seqs * c.seq_len), "prompt_len": c.prompt_len, "vocab": c.vocab,
+                       "D": c.depth_cap, "P": c.max_pattern, "alpha": c.alpha, "max_spec": c.max_spec,
+                       "l2": "flushed between steps (256 MiB write outside the timed events)",
+                       "parallelism": f"replica x{world}, requests sharded" if world > 1 else "single GPU"},
+            "speculate_us": {"mean": statistics.mean(spec_ms) * 1e3, "p50": statistics.median(spec_ms) * 1e3,
+                             "max": max(spec_ms) * 1e3},
+            "append_us": {"mean": statistics.mean(app_ms) * 1e3, "p50": statistics.median(app_ms) * 1e3},
+            "tokens_appended_per_step": float(np.mean([t.size for t in steps.tokens[W:W + K]])),
+            "build_ms": build_ms, "prompt_build_ms": prompt_ms, "global_nodes": st["global_nodes"],
+            "device_bytes": st["device_bytes"], "wall_ms_timed_region": wall_ms,
+            "gpu_launches": 3 * K, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "clocks": clocks,
+        }
+        line.update(extra)
+        print(json.dumps(line), flush=True)
+    store.free()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The CPU oracle as it stands, on the host cores, same metric and config.
+    Each step is a bounded sample of the workload's requests."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    w = make_workload(args)
+    c = w.cfg
+    B, K, W = c.batch, args.steps, args.warmup
+    thr = oracle_threads(B)
+    prompts = [w.prompt(i) for i in range(B)]
+    steps = StepInputs(w, 0, B, W + K, prompts)
+    ref = oracle.SuffixOracle(c.depth_cap, B)
+    ref.global_build(w.corpus(), w.corpus_offsets())
+    ref.slot_append_batch(list(range(B)), prompts, n_threads=thr)
+    sample = list(range(B))
+    budget_s = 150.0
+
+    def step(k):
+        ref.speculate(sample, c.max_pattern, c.alpha, c.max_spec, n_threads=thr)
+        ref.slot_append_batch(sample, [steps.lists[k][i] for i in sample], n_threads=thr)
+
+    t0 = time.perf_counter()
+    step(0) if W > 0 else None
+    t1 = time.perf_counter() - t0
+    if W > 0 and t1 * (K + W) > budget_s:
+        keep = max(8, int(B * budget_s / (t1 * (K + W))))
+        sample = list(range(min(B, keep)))
+    for k in range(1, W):
+        step(k)
+    t0 = time.perf_counter()
+    for k in range(W, W + K):
+        step(k)
+    dt = time.perf_counter() - t0
+    value = len(sample) * K / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+            "warmup": W, "ms_per_step": dt / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32 trees, f64 scores", "data": "synthetic",
+            "config": {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": B,
+                       "global_tokens": int(c.n_seqs * c.seq_len), "prompt_len": c.prompt_len, "vocab": c.vocab,
+                       "D": c.depth_cap, "P": c.max_pattern, "alpha": c.alpha, "max_spec": c.max_spec},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": thr, "kind": "oracle",
+                             "sample": f"{len(sample)} of {B} requests per step, {K} steps"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

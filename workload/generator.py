@@ -288,3 +288,14 @@ def get_workload(name: str, **overrides) -> Workload:
     if overrides:
         cfg = cfg.scaled(**overrides)
     return Workload(cfg)
+
+
+def accept_schedule(n_requests: int, n_steps: int, seed_index: int = 0, mean_extra: float = 3.0,
+                    cap: int = 16) -> np.ndarray:
+    """int32[n_steps][n_requests]: tokens appended per request per decode step in
+    the open-loop benchmark (1 bonus token + a geometric number of accepted
+    drafts, capped), from the counter-based generator."""
+    u = _unit(splitmix_block(stream_seed(99, PURPOSE_OUTLEN, seed_index), n_requests * n_steps))
+    p = 1.0 / (mean_extra + 1.0)
+    extra = np.floor(np.log1p(-u) / math.log(1.0 - p)).astype(np.int64)
+    return (1 + np.minimum(extra, cap - 1)).astype(np.int32).reshape(n_steps, n_requests)

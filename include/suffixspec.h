@@ -153,6 +153,39 @@ int sd_speculate(sd_store* store, int32_t n, const int32_t* d_slot, const sd_spe
                  double* d_score, int32_t* d_status, void* stream);
 
 /*
+ * sd_speculate_noalloc: sd_speculate for callers that must not allocate.
+ * (The paper has no counterpart; this is a deployment convenience.)
+ *
+ * Some hosts of this library run where device allocation is off limits: a
+ * serving loop that has handed all free device memory to its own pool, a
+ * plug-in that is only given buffers and a stream, or a real-time thread that
+ * may not take the allocator's locks.  sd_speculate itself does not allocate
+ * either, but its per-job scratch records come from memory that sd_build
+ * obtained with cudaMalloc; this variant keeps those records in a fixed array
+ * inside the library image instead, and calls no allocating routine at all.
+ *
+ * Same arguments, outputs and results as sd_speculate.  Differences:
+ *  - Size limit: n * 2 * depth_cap must not exceed SD_NOALLOC_MAX_JOBS (e.g. 64
+ *    requests at depth_cap 32); a larger batch returns SD_ERR_CAPACITY
+ *    ("capacity exceeded") and launches nothing.  Split the batch instead.
+ *  - The array (about 2.1 MB) is held on every GPU that loads the library,
+ *    until the process exits.
+ *  - The first call on each device looks up the array's device address (a
+ *    short, synchronous runtime query; that device must be current).  Make
+ *    that first call before starting any stream capture.
+ *  - All calls on a device share the one array.  Its contents carry over from
+ *    call to call but are never read before being rewritten, so no clearing is
+ *    needed; two calls whose kernels overlap on the GPU (different streams,
+ *    different stores) would overwrite each other's records, so keep calls on
+ *    one device ordered.
+ */
+#define SD_NOALLOC_MAX_JOBS 4096
+int sd_speculate_noalloc(sd_store* store, int32_t n, const int32_t* d_slot, const sd_spec_params* params,
+                         const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
+                         int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
+                         int32_t* d_chosen_p, double* d_score, int32_t* d_status, void* stream);
+
+/*
  * sd_query_counts: COUNT of arbitrary token paths (the quantity Eq. 1 divides),
  * for checking a store against an independent implementation.
  *   d_tree int32[n]: -1 global tree, else slot; path i is

@@ -6,4 +6,4 @@ not load the library; the first use does, and fails loudly if it is missing.
 """
 from .binding import (FLAG_GLOBAL_ONLY, FLAG_LINEAR, FLAG_REQUEST_ONLY, STATUS_BAD_SLOT, STATUS_BAD_TOKEN,  # noqa: F401
                       STATUS_GLOBAL_FULL, STATUS_POOL_FULL, SuffixSpecError, SuffixStore, library, sd_build,
-                      sd_append, sd_speculate, sd_free)
+                      sd_append, sd_speculate, sd_speculate_noalloc, sd_free)

@@ -18,7 +18,7 @@ from . import build as _build
 FLAG_GLOBAL_ONLY, FLAG_REQUEST_ONLY, FLAG_LINEAR = 1, 2, 4
 STATUS_BAD_SLOT, STATUS_POOL_FULL, STATUS_GLOBAL_FULL, STATUS_BAD_TOKEN = 1, 2, 4, 8
 
-EXPORTS = ["sd_build", "sd_append", "sd_speculate", "sd_query_counts", "sd_slot_info", "sd_stats", "sd_free",
+EXPORTS = ["sd_build", "sd_append", "sd_speculate", "sd_speculate_noalloc", "sd_query_counts", "sd_slot_info", "sd_stats", "sd_free",
            "sd_strerror"]
 
 
@@ -63,6 +63,8 @@ def library() -> C.CDLL:
         lib.sd_append.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
         lib.sd_speculate.restype = C.c_int
         lib.sd_speculate.argtypes = [vp, C.c_int32, vp, C.POINTER(_SpecParams)] + [vp] * 11
+        lib.sd_speculate_noalloc.restype = C.c_int
+        lib.sd_speculate_noalloc.argtypes = lib.sd_speculate.argtypes
         lib.sd_query_counts.restype = C.c_int
         lib.sd_query_counts.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
         lib.sd_slot_info.restype = C.c_int
@@ -126,6 +128,24 @@ def sd_speculate(store: int, slots: torch.Tensor, P: int, alpha: float, max_spec
         _ptr(out["score"], torch.float64, "score"), _ptr(out["status"], torch.int32, "status"), _stream())
     if rc != 0:
         raise SuffixSpecError(rc, "sd_speculate")
+
+
+def sd_speculate_noalloc(store: int, slots: torch.Tensor, P: int, alpha: float, max_spec: int, flags: int,
+                         budget_cap: Optional[torch.Tensor], out: Dict[str, torch.Tensor]) -> None:
+    """sd_speculate for callers that may not allocate device memory: the scratch
+    records live in a fixed array inside the library, so the batch is limited
+    (n * 2 * depth_cap <= 4096 jobs) and calls on one device must not overlap.
+    `out` must be preallocated by the caller; nothing is allocated here."""
+    prm = _SpecParams(P, alpha, max_spec, flags)
+    rc = library().sd_speculate_noalloc(
+        store, int(slots.numel()), _ptr(slots, torch.int32, "slots"), C.byref(prm),
+        _ptr(budget_cap, torch.int32, "budget_cap"), _ptr(out["n_draft"], torch.int32, "n_draft"),
+        _ptr(out["tokens"], torch.int32, "tokens"), _ptr(out["parents"], torch.int32, "parents"),
+        _ptr(out["positions"], torch.int32, "positions"), _ptr(out["mask"], torch.int32, "mask"),
+        _ptr(out["chosen_tree"], torch.int32, "chosen_tree"), _ptr(out["chosen_p"], torch.int32, "chosen_p"),
+        _ptr(out["score"], torch.float64, "score"), _ptr(out["status"], torch.int32, "status"), _stream())
+    if rc != 0:
+        raise SuffixSpecError(rc, "sd_speculate_noalloc")
 
 
 def sd_free(store: int) -> None:

@@ -8,6 +8,8 @@
 // fp64 rules: C = count / sibling-sum (Eq. 1), D = D(parent) * C (Eq. 2), SCORE
 // adds D in insertion order; __ddiv_rn / __dmul_rn / __dadd_rn keep every
 // operation a separately rounded IEEE binary64 operation (no FMA contraction).
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -277,6 +279,83 @@ extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const
     match_expand_kernel<<<(unsigned)((jobs + SPEC_WARPS - 1) / SPEC_WARPS), SPEC_WARPS * 32, 0, st>>>(
         *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap);
     select_emit_kernel<<<(unsigned)((n + 3) / 4), 128, 0, st>>>(*s, n, d_slot, Pe, d_n_draft, d_tokens, d_parents,
+                                                                d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score,
+                                                                d_status);
+    SD_CUDA_OK(cudaGetLastError());
+    return SD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// sd_speculate_noalloc: the same two kernels, with the per-job scratch records kept in a
+// fixed array that is part of the loaded library image instead of in memory obtained
+// from cudaMalloc.  Meant for callers that must not touch the CUDA allocator at all
+// (see the declaration in suffixspec.h).
+//
+// The array's name below is only meaningful to device code.  Host code holds a stand-in
+// symbol of the same name, so the launch code first asks the runtime for the array's
+// real device address (once per device, with that device current) and passes that on.
+namespace {
+
+constexpr long long NOALLOC_BYTES =
+    (long long)SD_NOALLOC_MAX_JOBS * (sizeof(double) + sizeof(int32_t) + 2ll * SD_MAX_SPEC * sizeof(int32_t));
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+unsigned char* g_noalloc_ptr[NOALLOC_MAX_DEVICES];      // device address of the array, per device
+bool g_noalloc_ready[NOALLOC_MAX_DEVICES];
+std::mutex g_noalloc_mutex;
+
+// Device address of the scratch array on the current device (looked up on first use).
+int noalloc_scratch_address(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return SD_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ready[dev]) {
+        unsigned char* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return SD_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = p;
+        g_noalloc_ready[dev] = true;
+    }
+    *out = g_noalloc_ptr[dev];
+    return SD_OK;
+}
+
+}  // namespace
+
+extern "C" int sd_speculate_noalloc(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
+                                    const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
+                                    int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
+                                    int32_t* d_chosen_p, double* d_score, int32_t* d_status, void* stream) {
+    if (!s || !prm || n < 0 || n > s->R) return SD_ERR_INVALID_ARG;
+    if (prm->P < 1 || prm->max_spec < 0 || prm->max_spec > s->M || !(prm->alpha >= 0.0)) return SD_ERR_INVALID_ARG;
+    if ((prm->flags & SD_FLAG_GLOBAL_ONLY) && (prm->flags & SD_FLAG_REQUEST_ONLY)) return SD_ERR_INVALID_ARG;
+    // one record per (request, tree, depth): the batch must fit the fixed array
+    if ((long long)n * 2 * s->D > SD_NOALLOC_MAX_JOBS) return SD_ERR_CAPACITY;
+    if (n == 0) return SD_OK;
+    if (!d_slot || !d_n_draft || !d_tokens || !d_parents || !d_positions || !d_mask || !d_chosen_tree || !d_chosen_p ||
+        !d_score)
+        return SD_ERR_INVALID_ARG;
+    unsigned char* base = nullptr;
+    const int rc = noalloc_scratch_address(&base);
+    if (rc != SD_OK) return rc;
+    // Same record layout as the store's own scratch, carved out of the fixed array.  Every
+    // record the second kernel reads is written by the first kernel of the same call, so
+    // nothing left over from an earlier call is ever consumed and nothing needs clearing.
+    sd_store view = *s;
+    view.j_score = reinterpret_cast<double*>(base);
+    view.j_n = reinterpret_cast<int32_t*>(base + (long long)SD_NOALLOC_MAX_JOBS * sizeof(double));
+    view.j_tok = view.j_n + SD_NOALLOC_MAX_JOBS;
+    view.j_par = view.j_tok + (long long)SD_NOALLOC_MAX_JOBS * SD_MAX_SPEC;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int Pe = prm->P < s->D ? prm->P : s->D;
+    const long long jobs = (long long)n * 2 * Pe;
+    match_expand_kernel<<<(unsigned)((jobs + SPEC_WARPS - 1) / SPEC_WARPS), SPEC_WARPS * 32, 0, st>>>(
+        view, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap);
+    select_emit_kernel<<<(unsigned)((n + 3) / 4), 128, 0, st>>>(view, n, d_slot, Pe, d_n_draft, d_tokens, d_parents,
                                                                 d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score,
                                                                 d_status);
     SD_CUDA_OK(cudaGetLastError());

@@ -231,3 +231,64 @@ def test_speculate_is_deterministic(U):
     for k in a:
         assert torch.equal(a[k], b[k])
     pr.close()
+
+
+# ---------------------------------------------------------------- BASELINE configs, scaled so the oracle takes seconds
+def _config_pair(U, name, n_seqs, batch, prompt_len=None, extra_tokens=64):
+    from workload.generator import get_workload
+    kw = dict(n_seqs=n_seqs, batch=batch)
+    if prompt_len:
+        kw["prompt_len"] = prompt_len
+    w = get_workload(name, **kw)
+    c = w.cfg
+    corpus = w.corpus()
+    seqs = [corpus[i * c.seq_len:(i + 1) * c.seq_len] for i in range(c.n_seqs)]
+    pr = U.Pair(seqs, vocab=c.vocab, D=c.depth_cap, n_slots=c.batch, max_req_tokens=c.prompt_len + extra_tokens,
+                M=c.max_spec)
+    return w, c, pr
+
+
+@pytest.mark.parametrize("name,n_seqs,batch", [("agentic", 300, 6), ("large_batch", 256, 24),
+                                               ("low_repetition", 256, 32)])
+def test_configs_scaled_prompts_then_decode_steps(U, name, n_seqs, batch):
+    """Corpus cut to a few hundred sequences, prompts at full length (8,192 / 4,096 tokens),
+    every other parameter as the benchmark spec gives it; three decode steps of appends."""
+    w, c, pr = _config_pair(U, name, n_seqs, batch)
+    prompts = w.prompts()
+    pr.append(list(range(batch)), prompts, reset=[1] * batch)
+    pr.check_tree(-1)
+    for s in (0, batch - 1):
+        pr.check_tree(s)
+    got, _ = pr.check_speculate(list(range(batch)), c.max_pattern, c.alpha, c.max_spec)
+    assert (got["n_draft"] > 0).any()
+    cont = [w.continuation(i, prompts[i], length=40) for i in range(batch)]
+    cur = 0
+    for step, k in enumerate((1, 7, 3)):
+        pr.append(list(range(batch)), [x[cur:cur + k] for x in cont])
+        cur += k
+        pr.check_speculate(list(range(batch)), c.max_pattern, c.alpha, c.max_spec)
+        pr.check_speculate(list(range(batch)), c.max_pattern, c.alpha, c.max_spec, flags=4)
+    pr.check_tree(1)
+    pr.close()
+
+
+def test_closed_loop_scaled(U):
+    """BASELINE config 4 in miniature: speculate, accept against the hidden continuation, append
+    accepted + bonus tokens, insert finished outputs into the global tree, refill the slot."""
+    from workload.closed_loop import ClosedLoop
+    w, c, pr = _config_pair(U, "closed_loop", 128, 12, prompt_len=300, extra_tokens=80)
+    loop = ClosedLoop(w, 12, prompt_len=300, out_lo=10, out_hi=60)
+    pr.append(*loop.start())
+    for step in range(40):
+        got, _ = pr.check_speculate(list(range(12)), c.max_pattern, c.alpha, c.max_spec)
+        slots, lists, reset = loop.advance(got)
+        pr.append(slots, lists, reset)
+        if step % 13 == 0:
+            pr.check_tree(-1)
+            pr.check_tree(step % 12)
+    s = loop.summary()
+    assert s["finished_requests"] >= 12 and s["mean_accepted_drafts"] > 0.5
+    pr.check_tree(-1)
+    for sl in range(12):
+        pr.check_tree(sl)
+    pr.close()

@@ -7,6 +7,11 @@
 // most D tokens long: lane L extends the ACTIVE node of depth L (the node of
 // the last L tokens; lane 0 extends the root) by child x, creating it or
 // raising its count.  The 32 lanes work on 32 different parents at once.
+//
+// Placement.  A suffix that has left the known text creates one new leaf per appended token,
+// each the only child of the previous one.  The first such leaf reserves room for the whole
+// chain down to depth D and every later leaf goes directly behind its parent, so chains of
+// only children are consecutive entries (what the wide window loads of sd_speculate exploit).
 #include "common.cuh"
 
 namespace {
@@ -44,9 +49,11 @@ __device__ int insert_child(int4* ent, int parent, int cb, int n, int pos, int x
 // on return it is the active node after x was appended.  `t` is the context length
 // before the append.  `used` / `live` are warp-uniform pool counters.
 // Returns false, changing nothing, if the pool cannot hold the new nodes.
-__device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, int& act, int& used, int& live) {
+__device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, int& act, int& room, int& used,
+                             int& live) {
     const unsigned FULL = 0xffffffffu;
     const int parent = __shfl_up_sync(FULL, act, 1);            // node of depth `lane`
+    const int parent_room = __shfl_up_sync(FULL, room, 1);      // free entries reserved behind it
     const bool valid = lane <= min(t, D - 1);
     int found = -1, pos = 0, cb = 0, n = 0;
     unsigned w = 0;
@@ -67,9 +74,16 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
     }
     const bool need = valid && found < 0;
     int asz = 0;                                                 // fresh entries this lane needs
+    bool behind_parent = false;                                  // the new leaf goes to parent + 1
+    int new_room = 0;
     if (need) {
-        if (lane == 0) asz = 1;
-        else if ((uint32_t)n == sd_run_capacity(w)) asz = (int)sd_pow2ceil((uint32_t)n + 1u);
+        if (lane == 0 || n == 0) {
+            // first child of a leaf (or a new depth-1 node): start or continue a chain block
+            if (lane > 0 && parent_room > 0) { behind_parent = true; new_room = parent_room - 1; }
+            else { asz = D - lane; new_room = asz - 1; }
+        } else if ((uint32_t)n == sd_run_capacity(w)) {
+            asz = (int)sd_pow2ceil((uint32_t)n + 1u);
+        }
     }
     int inc = asz;
 #pragma unroll
@@ -79,7 +93,8 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
     }
     const int total = __shfl_sync(FULL, inc, 31);
     if ((long long)used + total > (long long)tr.cap) return false;
-    const int fresh = used + inc - asz;
+    const int fresh = behind_parent ? parent + 1 : used + inc - asz;
+    const bool moves = behind_parent || asz > 0;
     used += total;
 
     // A lane that moves entries of its run must not do so while the next lane edits the
@@ -94,6 +109,7 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
         *word(&tr.ent[found], 1) += 1;
         act = found;
     }
+    room = new_room;
     if (!serial) {
         if (need) {
             if (lane == 0) {
@@ -101,7 +117,7 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
                 tr.root[x] = fresh;
                 act = fresh;
             } else {
-                act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, asz > 0);
+                act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, moves);
             }
         }
         __syncwarp();
@@ -113,13 +129,13 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
                     tr.root[x] = fresh;
                     act = fresh;
                 } else {
-                    act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, asz > 0);
+                    act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, moves);
                 }
             }
             __syncwarp();
         }
     }
-    if (!valid) act = -1;
+    if (!valid) { act = -1; room = 0; }
     live += __popc(__ballot_sync(FULL, need));
     return true;
 }
@@ -139,12 +155,12 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
         for (int i = 0; i < n; ++i) {
             if (d_slot[i] != -1) continue;
             any = true;
-            int act = -1;
+            int act = -1, room = 0;
             const long long b = d_offsets[i], e = d_offsets[i + 1];
             for (long long k = b; k < e && !(status & SD_STATUS_GLOBAL_FULL); ++k) {
                 const int x = d_tokens[k];
                 if (x < 0 || x >= sv.V) { status |= SD_STATUS_BAD_TOKEN; break; }
-                if (!append_token(tr, sv.D, x, (int)(k - b), lane, act, used, live)) {
+                if (!append_token(tr, sv.D, x, (int)(k - b), lane, act, room, used, live)) {
                     status |= SD_STATUS_GLOBAL_FULL;
                     break;
                 }
@@ -152,6 +168,7 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
             }
         }
         if (any && lane == 0) {
+            sv.g_state->epoch += 1;                  // cached match nodes of every slot are stale now
             sv.g_state->used = used; sv.g_state->live = live; sv.g_state->status = status;
             sv.g_state->tokens = tokens;
         }
@@ -164,18 +181,19 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
     int32_t* text = sv.s_text + (long long)slot * sv.T;
     TreeRef tr{sv.s_ent + (long long)slot * sv.spn, sv.s_root + (long long)slot * sv.V, (int)sv.spn};
     int len = ss->len, used = ss->used, live = ss->live, status = ss->status;
-    int act = lane < SD_MAX_DEPTH ? ss->active[lane] : -1;
+    int act = ss->active[lane], room = ss->room[lane];
     if (d_reset && d_reset[i]) {
         // forget the old tree: only root-table cells of tokens that occur can be set
         for (int k = lane; k < len; k += 32) tr.root[text[k]] = -1;
         __syncwarp();
-        len = 0; used = 0; live = 0; status = 0; act = -1;
+        len = 0; used = 0; live = 0; status = 0; act = -1; room = 0;
+        if (lane == 0) ss->gen += 1;
     }
     const long long b = d_offsets[i], e = d_offsets[i + 1];
     for (long long k = b; k < e && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)); ++k) {
         const int x = d_tokens[k];
         if (x < 0 || x >= sv.V) { status |= SD_STATUS_BAD_TOKEN; break; }
-        if (len >= sv.T || !append_token(tr, sv.D, x, len, lane, act, used, live)) {
+        if (len >= sv.T || !append_token(tr, sv.D, x, len, lane, act, room, used, live)) {
             status |= SD_STATUS_POOL_FULL;
             break;
         }
@@ -183,6 +201,7 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
         ++len;
     }
     ss->active[lane] = act;
+    ss->room[lane] = room;
     if (lane == 0) { ss->len = len; ss->used = used; ss->live = live; ss->status = status; }
 }
 

@@ -316,32 +316,62 @@ __global__ void seg_pos_kernel(const uint8_t* lcp, int d, const int* bscan, i64 
     if (lcp[j] < d) segpos[bscan[j]] = (int)j;
 }
 
-// Lay down the depth-d nodes.  Nodes of one depth are numbered in suffix order, so
-// the children of a node are consecutive at depth d + 1 and sorted by token.
+struct NewNodes {             // nodes opened by suffix j
+    const uint8_t* lcp;
+    const uint8_t* len;
+    __device__ int operator()(i64 j) const { return (int)len[j] - (int)lcp[j]; }
+};
+
+// Nodes are numbered in depth-first pre-order: the root is 0 and the node that suffix j opens
+// at depth d is 1 + nbase[j] + (d - lcp[j] - 1).  Pre-order is what makes paths contiguous:
+// child runs are laid down in node order, so the run of a node's first child directly follows
+// the node's own run, and a chain of only children is one run of consecutive entries.
+__global__ void count_children_kernel(const uint8_t* lcp, const uint8_t* len, i64 n, int d, int D, const int* r_d,
+                                      const int* r_next, const int* bscan, const int* segpos, const int* nbase,
+                                      int* nchild) {
+    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    if (j == 0 && d == 1) nchild[0] = r_d[n];             // the root's children: all depth-1 nodes
+    if (!(lcp[j] < d && d <= len[j])) return;
+    int nc = 0;
+    if (d < D) {
+        const int nb = segpos[bscan[j] + 1];              // first suffix past this node's range
+        nc = r_next[nb] - r_next[j];
+    }
+    nchild[1 + nbase[j] + (d - (int)lcp[j] - 1)] = nc;
+}
+
+// Write the depth-d nodes.  A node's entry sits in its parent's child run at its rank among
+// the siblings (suffix order = token order).
 __global__ void emit_level_kernel(const int32_t* tok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len,
-                                  i64 n, int d, int D, const int* r_d, const int* r_next, const int* bscan,
-                                  const int* segpos, i64 base_d, i64 base_next, int4* ent, int32_t* root) {
+                                  i64 n, int d, const int* r_d, const int* bscan, const int* segpos,
+                                  const int* bscan_prev, const int* segpos_prev, const int* nbase, const int* nchild,
+                                  const int* runstart, int4* ent, int32_t* root) {
     i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
     if (!(lcp[j] < d && d <= len[j])) return;
-    const int nb = segpos[bscan[j] + 1];              // first suffix past this node's range
+    const int nb = segpos[bscan[j] + 1];
+    int pnid = 0, rank = r_d[j];
+    if (d > 1) {
+        const int seg = bscan_prev[j] + (lcp[j] < d - 1 ? 1 : 0) - 1;   // depth d-1 range holding j
+        const int jx = segpos_prev[seg];                               // its first suffix opened the parent
+        pnid = 1 + nbase[jx] + (d - 1 - (int)lcp[jx] - 1);
+        rank = r_d[j] - r_d[jx];
+    }
+    const int nid = 1 + nbase[j] + (d - (int)lcp[j] - 1);
+    const int nc = nchild[nid];
     int4 e;
     e.x = tok[(i64)sa[j] + d - 1];
-    e.y = nb - (int)j;                                // every suffix in the range is an occurrence
-    int nc = 0, cb = 0;
-    if (d < D) {
-        nc = r_next[nb] - r_next[j];
-        if (nc > 0) cb = (int)(base_next + r_next[j]);
-    }
-    e.z = cb;
+    e.y = nb - (int)j;                                    // every suffix in the range is an occurrence
+    e.z = nc > 0 ? runstart[nid] : 0;
     e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC) : 0;
-    const i64 idx = base_d + r_d[j];
-    ent[idx] = e;
-    if (d == 1) root[e.x] = (int)idx;
+    const int pos = runstart[pnid] + rank;
+    ent[pos] = e;
+    if (d == 1) root[e.x] = pos;
 }
 
 __global__ void init_global_state_kernel(GlobalState* g, int used, long long tokens) {
-    g->used = used; g->live = used; g->status = 0; g->pad = 0; g->tokens = tokens;
+    g->used = used; g->live = used; g->status = 0; g->epoch = 1; g->tokens = tokens;
 }
 
 struct DeviceArena {          // temporaries of one build, released together
@@ -424,7 +454,6 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
     if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
 
     i64 n_nodes = 0;
-    i64 level_base[SD_MAX_DEPTH + 2] = {0};
     DeviceArena tmp;
     SortBuffers sb;
     int *end_pos = nullptr, *rank[8] = {nullptr}, *comb[2] = {nullptr, nullptr}, *ex = nullptr;
@@ -500,8 +529,7 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
             ce = cudaMemcpyAsync(h_level, level_nodes, sizeof(h_level), cudaMemcpyDeviceToHost, st);
         if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
         if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
-        for (int d = 1; d <= D; ++d) { level_base[d] = n_nodes; n_nodes += (i64)h_level[d]; }
-        level_base[D + 1] = n_nodes;
+        for (int d = 1; d <= D; ++d) n_nodes += (i64)h_level[d];
     }
 
     i64 extra = p->global_extra_nodes >= 0 ? p->global_extra_nodes : std::max<i64>(1ll << 22, n_nodes);
@@ -510,20 +538,37 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
     if (!store_alloc(s, &s->g_ent, s->g_cap)) { store_release(s); return SD_ERR_NOMEM; }
 
     if (N > 0) {
-        int *r_a = nullptr, *r_b = nullptr, *bscan = nullptr, *segpos = nullptr;
-        ok = tmp.get(&r_a, N + 1) && tmp.get(&r_b, N + 1) && tmp.get(&segpos, N + 2);
-        bscan = ex;
+        int *r_a = nullptr, *r_b = nullptr, *b_a = ex, *b_b = nullptr, *seg_a = nullptr, *seg_b = nullptr;
+        int *nbase = nullptr, *nchild = nullptr, *runstart = nullptr, *big_tmp = nullptr;
+        ok = tmp.get(&r_a, N + 1) && tmp.get(&r_b, N + 1) && tmp.get(&seg_a, N + 2) && tmp.get(&seg_b, N + 2) &&
+             tmp.get(&b_b, N + 1) && tmp.get(&nbase, N + 1) && tmp.get(&nchild, n_nodes + 1) &&
+             tmp.get(&runstart, n_nodes + 2) && tmp.get(&big_tmp, scan_tmp_ints(n_nodes + 1));
         if (!ok) { store_release(s); return SD_ERR_NOMEM; }
-        int* r_next = r_a;  // scan of depth d + 1 (unused at d == D)
+        exclusive_scan(NewNodes{lcp, len}, N, nbase, sb.scan_tmp, st);
+        // pass 1, deepest level first: children per node
+        int* r_next = r_a;
         int* r_cur = r_b;
         for (int d = D; d >= 1; --d) {
             exclusive_scan(OpensNode{lcp, len, d}, N, r_cur, sb.scan_tmp, st);
-            exclusive_scan(Boundary{lcp, d}, N, bscan, sb.scan_tmp, st);
-            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(lcp, d, bscan, N, segpos);
-            emit_level_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, sa, lcp, len, N, d, D, r_cur, r_next, bscan,
-                                                                 segpos, level_base[d], level_base[d + 1], s->g_ent,
-                                                                 s->g_root);
+            exclusive_scan(Boundary{lcp, d}, N, b_a, sb.scan_tmp, st);
+            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(lcp, d, b_a, N, seg_a);
+            count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, N, d, D, r_cur, r_next, b_a, seg_a,
+                                                                      nbase, nchild);
             std::swap(r_cur, r_next);
+        }
+        // child runs in node (pre-)order
+        exclusive_scan(LoadInt{nchild}, n_nodes + 1, runstart, big_tmp, st);
+        // pass 2, top level first: write the entries
+        int *b_cur = b_a, *b_prev = b_b, *seg_cur = seg_a, *seg_prev = seg_b;
+        for (int d = 1; d <= D; ++d) {
+            exclusive_scan(OpensNode{lcp, len, d}, N, r_cur, sb.scan_tmp, st);
+            exclusive_scan(Boundary{lcp, d}, N, b_cur, sb.scan_tmp, st);
+            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(lcp, d, b_cur, N, seg_cur);
+            emit_level_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, sa, lcp, len, N, d, r_cur, b_cur, seg_cur,
+                                                                 b_prev, seg_prev, nbase, nchild, runstart, s->g_ent,
+                                                                 s->g_root);
+            std::swap(b_cur, b_prev);
+            std::swap(seg_cur, seg_prev);
         }
     }
     init_global_state_kernel<<<1, 1, 0, st>>>(s->g_state, (int)n_nodes, N);

@@ -28,7 +28,7 @@ struct GlobalState {          // device-resident bookkeeping of the global tree
     int32_t used;             // entries handed out
     int32_t live;             // live nodes
     int32_t status;           // SD_STATUS_GLOBAL_FULL or 0
-    int32_t pad;
+    int32_t epoch;            // grows whenever an online insert changed the tree
     long long tokens;         // tokens inserted
 };
 
@@ -38,6 +38,15 @@ struct SlotState {            // device-resident bookkeeping of one request slot
     int32_t live;             // live nodes
     int32_t status;           // SD_STATUS_*
     int32_t active[SD_MAX_DEPTH];   // active[d-1]: entry of the node for the last d tokens
+    int32_t room[SD_MAX_DEPTH];     // free entries reserved right behind that node for its chain
+    // Match nodes of this request in the GLOBAL tree, kept from the last sd_speculate so that
+    // the next one only descends the tokens appended since (a cache: losing it costs a full walk).
+    int32_t gen;              // grows when the slot is reset
+    int32_t g_gen;            // value of gen the cache was taken at
+    int32_t g_epoch;          // global epoch the cache was taken at
+    int32_t g_len;            // context length the cache was taken at
+    int32_t g_depths;         // depths 1..g_depths are cached
+    int32_t g_node[SD_MAX_DEPTH];   // g_node[d-1]: global node of the last d tokens, -1 none
 };
 
 struct sd_store {

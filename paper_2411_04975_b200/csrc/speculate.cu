@@ -26,10 +26,10 @@ struct Frontier {                             // candidates of one job, best fir
 };
 
 // strict total order of candidates: larger D, then smaller token, then smaller parent index
+// (D values are non-negative, so their bit patterns order like the values: branch-free compare.)
 __device__ __forceinline__ bool better(double da, int ta, int pa, double db, int tb, int pb) {
-    if (da != db) return da > db;
-    if (ta != tb) return ta < tb;
-    return pa < pb;
+    const long long a = __double_as_longlong(da), b = __double_as_longlong(db);
+    return (a > b) | ((a == b) & ((ta < tb) | ((ta == tb) & (pa < pb))));
 }
 
 // Entry index of child `x` in the sorted run ent[cb .. cb+n), or -1.  Whole warp.
@@ -260,6 +260,654 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Fused path: one block of CTA_WARPS warps per request.
+//   1. match: the per-request match nodes are the slot's active nodes; the global match
+//      nodes are advanced from the nodes cached at the previous call by descending only the
+//      tokens appended since (full walks when the cache is stale).  Warp w serves pattern
+//      lengths w + 1 and w + 1 + CTA_WARPS.
+//   2. expand: the (tree, p) jobs that matched go into a queue, costliest first; warps pull
+//      jobs until it is empty.  A job is dropped, exactly, as soon as an upper bound of its
+//      SCORE (every D <= 1 and D never grows along a path) falls below a score already
+//      reached by another job of the request.
+//   3. select + emit from shared memory; no global scratch.
+constexpr int CTA_WARPS = 16;
+
+struct WarpWork {
+    Frontier F;
+    Frontier T;                               // scratch list for the children of one wide node
+    int one_tok[SD_MAX_SPEC];                 // its first children of count 1, in token order
+    int one_cb[SD_MAX_SPEC];
+    unsigned one_nc[SD_MAX_SPEC];
+    int tok[2][SD_MAX_SPEC];                  // draft tokens: working buffer and best-so-far buffer
+    unsigned char par[2][SD_MAX_SPEC];        // parent index + 1 (0: child of the match node)
+    double best_score;
+    int best_order, best_n, best_buf;
+};
+
+struct BlockShared {
+    WarpWork w[CTA_WARPS];
+    int node[2][SD_MAX_DEPTH];                // match node per tree and pattern length (-1: none)
+    int cb[2][SD_MAX_DEPTH];                  // its child run
+    unsigned nc[2][SD_MAX_DEPTH];
+    int cost[2 * SD_MAX_DEPTH];
+    int job[2 * SD_MAX_DEPTH];
+    int wide[2 * SD_MAX_DEPTH];               // jobs whose match node has a wide child run
+    int njobs, next, nwide, nwide_kept;
+    long long slice_sum[CTA_WARPS];
+    int slice_fs[CTA_WARPS];
+    unsigned long long best_bits;             // largest finished SCORE so far, as ordered bits
+    int win_warp;
+};
+
+// find_child that also hands back the matched entry (valid when the result is >= 0)
+__device__ int find_child_entry(const int4* __restrict__ ent, int cb, int n, int x, int lane, int4& out) {
+    int lo = 0, hi = n;
+    for (int it = 0; it < 6 && hi - lo > 32; ++it) {
+        const int q = lo + (int)(((long long)(hi - lo) * (lane + 1)) / 33);
+        const int tk = ent[cb + q].x;
+        const unsigned ge = __ballot_sync(FULL, tk >= x);
+        const int f = ge ? __ffs(ge) - 1 : 32;
+        const int q_prev = __shfl_sync(FULL, q, f > 0 ? f - 1 : 0);
+        const int q_at = __shfl_sync(FULL, q, f < 32 ? f : 31);
+        if (f > 0) lo = q_prev + 1;
+        if (f < 32) hi = q_at + 1;
+    }
+    int found = -1;
+    for (int base = lo; base < hi && found < 0; base += 32) {
+        const int idx = base + lane;
+        int4 e = make_int4(-1, 0, 0, 0);
+        if (idx < hi) e = ent[cb + idx];
+        const unsigned eq = __ballot_sync(FULL, idx < hi && e.x == x);
+        if (eq) {
+            const int src = __ffs(eq) - 1;
+            found = cb + base + src;
+            out.x = __shfl_sync(FULL, e.x, src); out.y = __shfl_sync(FULL, e.y, src);
+            out.z = __shfl_sync(FULL, e.z, src); out.w = __shfl_sync(FULL, e.w, src);
+        }
+    }
+    return found;
+}
+
+
+
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// Start fetching the `n` entries at ent[cb ...] into L2 (whole warp; at most `max_lines` 128-byte lines per lane).
+__device__ __forceinline__ void prefetch_run(const int4* __restrict__ ent, int cb, int n, int lane, int max_rounds) {
+    const int lines = (n + 7) >> 3;
+    for (int r = 0, l = lane; r < max_rounds && l < lines; ++r, l += 32) prefetch_l2(ent + cb + l * 8);
+}
+
+// Merge up to 32 candidates (one per lane with `pass`) into the sorted frontier of at most K
+// entries in one go: every survivor's final position is its number of betters, found by
+// broadcasting the candidates once; then all entries move together.
+__device__ void frontier_merge(Frontier& F, int fh, int& fs, int K, bool pass, double d, int tok, int par, int cb,
+                               unsigned nc, int lane) {
+    const unsigned m = __ballot_sync(FULL, pass);
+    if (!m) return;
+    const int i0 = lane, i1 = lane + 32;
+    const int s0 = (fh + i0) & (SD_MAX_SPEC - 1), s1 = (fh + i1) & (SD_MAX_SPEC - 1);
+    const bool v0 = i0 < fs, v1 = i1 < fs;
+    double e0d = 0.0, e1d = 0.0;
+    int e0t = 0, e1t = 0, e0p = 0, e1p = 0;
+    if (v0) { e0d = F.d[s0]; e0t = F.tok[s0]; e0p = F.par[s0]; }
+    if (v1) { e1d = F.d[s1]; e1t = F.tok[s1]; e1p = F.par[s1]; }
+    int up0 = 0, up1 = 0;                                       // candidates that go before E[i0], E[i1]
+    int my_rank = 0;
+    unsigned mm = m;
+    while (mm) {
+        const int src = __ffs(mm) - 1;
+        mm &= mm - 1;
+        const double bd = __shfl_sync(FULL, d, src);
+        const int bt = __shfl_sync(FULL, tok, src), bp = __shfl_sync(FULL, par, src);
+        const bool b0 = v0 && better(bd, bt, bp, e0d, e0t, e0p);
+        const bool b1 = v1 && better(bd, bt, bp, e1d, e1t, e1p);
+        up0 += b0 ? 1 : 0;
+        up1 += b1 ? 1 : 0;
+        const int worse_old = __popc(__ballot_sync(FULL, b0)) + __popc(__ballot_sync(FULL, b1));
+        const int better_new = __popc(__ballot_sync(FULL, pass && lane != src && better(d, tok, par, bd, bt, bp)));
+        if (lane == src) my_rank = (fs - worse_old) + better_new;
+    }
+    const int n0 = i0 + up0, n1 = i1 + up1;
+    int c0 = 0, c1 = 0;
+    unsigned w0 = 0, w1 = 0;
+    const bool k0 = v0 && n0 < K && up0 > 0, k1 = v1 && n1 < K && up1 > 0;   // entries that move
+    if (k0) { c0 = F.cb[s0]; w0 = F.nc[s0]; }
+    if (k1) { c1 = F.cb[s1]; w1 = F.nc[s1]; }
+    __syncwarp();
+    if (k0) { const int q = (fh + n0) & (SD_MAX_SPEC - 1); F.d[q] = e0d; F.tok[q] = e0t; F.par[q] = e0p; F.cb[q] = c0; F.nc[q] = w0; }
+    if (k1) { const int q = (fh + n1) & (SD_MAX_SPEC - 1); F.d[q] = e1d; F.tok[q] = e1t; F.par[q] = e1p; F.cb[q] = c1; F.nc[q] = w1; }
+    if (pass && my_rank < K) {
+        const int q = (fh + my_rank) & (SD_MAX_SPEC - 1);
+        F.d[q] = d; F.tok[q] = tok; F.par[q] = par; F.cb[q] = cb; F.nc[q] = nc;
+    }
+    __syncwarp();
+    fs = min(fs + __popc(m), K);
+}
+
+// Offer the first `cnt` entries of list O (ordered, ring head 0) to F.
+__device__ void frontier_merge_list(Frontier& F, int fh, int& fs, int K, const Frontier& O, int cnt, int par, int lane) {
+    for (int base = 0; base < cnt; base += 32) {
+        const int q = base + lane;
+        bool pass = q < cnt;
+        double d = 0.0; int tok = 0, cb = 0; unsigned nc = 0;
+        if (pass) { d = O.d[q]; tok = O.tok[q]; cb = O.cb[q]; nc = O.nc[q]; }
+        if (pass && fs == K) {
+            const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+            pass = better(d, tok, par, F.d[last], F.tok[last], F.par[last]);
+        }
+        if (!__any_sync(FULL, pass)) break;                     // O is ordered: nothing further can enter
+        frontier_merge(F, fh, fs, K, pass, d, tok, par, cb, nc, lane);
+    }
+}
+
+// A WINDOW is 32 consecutive entries, one per lane, starting at `base`.  Trees are laid out so
+// that the child run of a node's first (often only) child tends to follow the node's own
+// child run, so one window usually holds several levels of a path at once.
+__device__ __forceinline__ int4 load_window(const int4* __restrict__ ent, int base, int limit, int lane) {
+    const int idx = base + lane;
+    // the entries behind the window hold the rest of the node's sub-tree (pre-order layout):
+    // bring the next 1.5 KB into L2 so that the following windows of this job hit there
+    if (lane < 12 && base + 32 + lane * 8 < limit)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(ent + base + 32 + lane * 8));
+    return idx < limit ? ent[idx] : make_int4(-1, 0, 0, 0);
+}
+
+// Offer the children of a node to the frontier; `w` already holds the first 32 entries of the run.
+__device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int4 w, double d_parent, int par_index,
+                                Frontier& F, int fh, int& fs, int K, int lane) {
+    if (n <= 0 || K <= 0) return;
+    // sibling sum: the denominator of Eq. 1 (a parent's occurrences fit 31 bits)
+    unsigned part = lane < n ? (unsigned)w.y : 0u;
+    for (int base = 32; base < n; base += 128) {                // wide runs: four loads in flight
+        int y[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { const int idx = base + u * 32 + lane; y[u] = idx < n ? ent[cb + idx].y : 0; }
+        part += (unsigned)(y[0] + y[1] + y[2] + y[3]);
+    }
+    const unsigned sum = __reduce_add_sync(FULL, part);
+    const double dsum = (double)sum;
+    // With a full frontier only a child that beats its worst entry matters:
+    // D = d_parent * count / sum, so counts below `cmin` lose without any fp64 work.
+    int cmin = 1;
+    double ld = 0.0; int lt = 0, lp = 0;
+    const bool full = fs == K;
+    if (full) {
+        const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+        ld = F.d[last]; lt = F.tok[last]; lp = F.par[last];
+        const double need = ld / d_parent * dsum * 0.999999;
+        cmin = need >= 2.0e9 ? 2000000000 : max(1, (int)need);
+    }
+    for (int base = 0; base < n; base += 32) {
+        const int idx = base + lane;
+        int4 e = w;
+        if (base != 0) { e = make_int4(0, 0, 0, 0); if (idx < n) e = ent[cb + idx]; }
+        bool pass = idx < n && e.y >= cmin;
+        if (!__any_sync(FULL, pass)) continue;
+        double dc = 0.0;
+        if (pass) {
+            dc = __dmul_rn(d_parent, __ddiv_rn((double)e.y, dsum));      // Eq. 2 with Eq. 1
+            if (full) pass = better(dc, e.x, par_index, ld, lt, lp);
+            if (pass && ((unsigned)e.w & RUN_COUNT_MASK)) prefetch_l2(ent + e.z);   // likely looked at soon
+        }
+        frontier_merge(F, fh, fs, K, pass, dc, e.x, par_index, e.z, (unsigned)e.w, lane);
+        if (!full && fs == K) {                                 // it filled up while merging
+            const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+            const double d2 = F.d[last];
+            const int t2 = F.tok[last], p2 = F.par[last];
+            // from here on compare exactly against the new worst entry (no count shortcut)
+            for (int b2 = base + 32; b2 < n; b2 += 32) {
+                const int i2 = b2 + lane;
+                int4 e2 = make_int4(0, 0, 0, 0);
+                if (i2 < n) e2 = ent[cb + i2];
+                double dc2 = 0.0;
+                bool pass2 = i2 < n;
+                if (pass2) {
+                    dc2 = __dmul_rn(d_parent, __ddiv_rn((double)e2.y, dsum));
+                    const int l3 = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+                    pass2 = better(dc2, e2.x, par_index, F.d[l3], F.tok[l3], F.par[l3]);
+                }
+                frontier_merge(F, fh, fs, K, pass2, dc2, e2.x, par_index, e2.z, (unsigned)e2.w, lane);
+            }
+            (void)d2; (void)t2; (void)p2;
+            return;
+        }
+    }
+}
+
+// MatchPattern from a known node: descend text[from .. to).  Levels whose child run lies inside
+// the window already in registers cost no memory access.  Returns the node reached (-1: no
+// match) and its child run in (cb, n).
+__device__ int walk_from(const int4* __restrict__ ent, int limit, int node, const int32_t* __restrict__ text, int from,
+                         int to, int lane, int& cb, int& n) {
+    if (node < 0) return -1;
+    int wb = node;
+    int4 w = load_window(ent, wb, limit, lane);
+    cb = __shfl_sync(FULL, w.z, 0);
+    n = (int)((unsigned)__shfl_sync(FULL, w.w, 0) & RUN_COUNT_MASK);
+    for (int pos = from; pos < to; ++pos) {
+        const int x = text[pos];
+        if (n == 0) return -1;
+        if (n > 32) {                                           // wide run: 32-way search
+            int4 e;
+            node = find_child_entry(ent, cb, n, x, lane, e);
+            if (node < 0) return -1;
+            cb = e.z; n = (int)((unsigned)e.w & RUN_COUNT_MASK);
+            wb = -64;                                           // no usable window
+            continue;
+        }
+        if (!(cb >= wb && cb + n <= wb + 32)) { wb = cb; w = load_window(ent, wb, limit, lane); }
+        const int rel = wb + lane - cb;
+        const unsigned hit = __ballot_sync(FULL, rel >= 0 && rel < n && w.x == x);
+        if (!hit) return -1;
+        const int src = __ffs(hit) - 1;
+        node = wb + src;
+        cb = __shfl_sync(FULL, w.z, src);
+        n = (int)((unsigned)__shfl_sync(FULL, w.w, src) & RUN_COUNT_MASK);
+    }
+    return node;
+}
+
+
+constexpr int WIDE_RUN = 256;                 // child runs longer than this are scanned by several warps
+
+// One pass over chunks first, first + stride, ... of a child run: adds up the counts and keeps
+// the K children with the largest counts (then smallest tokens) in F, ordered, with the COUNT
+// in the d field.  Among the children of one parent that is the order of D (Eq. 2), so no
+// division is needed while scanning.  F starts empty at ring head fh.
+// Most children of a wide node occur once.  Those tie on the count and rank by token, i.e. in
+// run order: the first K of them are simply copied (ones list) and appended behind the
+// children that occur more often, which alone go through the ordered merge.
+// Children with a count below `cmin` are known not to matter and are skipped.
+__device__ void scan_run_by_count(const int4* __restrict__ ent, int cb, int n, int first, int stride, int par_index,
+                                  int cmin, WarpWork& W, Frontier& F, int fh, int& fs, int K, long long& sum_out,
+                                  int lane) {
+    long long sum = 0;
+    fs = 0;
+    int ones = 0;                                               // count-1 children copied so far (warp-uniform)
+    if (stride == 1) prefetch_run(ent, cb, n, lane, 64);        // the whole run, all lines in flight at once
+    for (int c = first; c * 32 < n; c += 4 * stride) {
+        int4 e[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {                           // four loads in flight
+            const int idx = (c + u * stride) * 32 + lane;
+            e[u] = make_int4(-1, 0, 0, 0);
+            if (idx < n) e[u] = ent[cb + idx];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            sum += e[u].y;
+            const unsigned m1 = __ballot_sync(FULL, e[u].y == 1 && cmin <= 1);
+            if (m1 && ones < K) {
+                const int at = ones + __popc(m1 & ((1u << lane) - 1u));
+                if (e[u].y == 1 && at < K) { W.one_tok[at] = e[u].x; W.one_cb[at] = e[u].z; W.one_nc[at] = (unsigned)e[u].w; }
+                ones = min(K, ones + __popc(m1));
+            }
+            bool pass = e[u].y >= 2 && e[u].y >= cmin;
+            if (pass && fs == K) {
+                const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+                pass = better((double)e[u].y, e[u].x, par_index, F.d[last], F.tok[last], F.par[last]);
+            }
+            if (pass && ((unsigned)e[u].w & RUN_COUNT_MASK)) prefetch_l2(ent + e[u].z);
+            frontier_merge(F, fh, fs, K, pass, (double)e[u].y, e[u].x, par_index, e[u].z, (unsigned)e[u].w, lane);
+        }
+    }
+    __syncwarp();
+    // the count-1 children go behind the others, in token order, as far as there is room
+    const int take = min(ones, K - fs);
+    for (int i = lane; i < take; i += 32) {
+        const int q = (fh + fs + i) & (SD_MAX_SPEC - 1);
+        F.d[q] = 1.0; F.tok[q] = W.one_tok[i]; F.par[q] = par_index; F.cb[q] = W.one_cb[i]; F.nc[q] = W.one_nc[i];
+    }
+    fs += take;
+    __syncwarp();
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+    sum_out = sum;
+}
+
+// counts in F.d -> D = d_parent * count / sum (Eq. 1, Eq. 2)
+__device__ void counts_to_d(Frontier& F, int fh, int fs, double d_parent, long long sum, int lane) {
+    const double dsum = (double)sum;
+    for (int i = lane; i < fs; i += 32) {
+        const int q = (fh + i) & (SD_MAX_SPEC - 1);
+        F.d[q] = __dmul_rn(d_parent, __ddiv_rn(F.d[q], dsum));
+    }
+    __syncwarp();
+}
+
+__device__ __forceinline__ double best_so_far(BlockShared& sh) {
+    return __shfl_sync(FULL, __longlong_as_double((long long)*(volatile unsigned long long*)&sh.best_bits), 0);
+}
+
+// ExpandSpeculationTree + SCORE for one (tree, p) job by one warp.  With `seeded` the frontier
+// already holds the match node's children (fs entries from ring head 0).
+__device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict__ ent, int limit, int tree, int p,
+                           int budget, unsigned flags, bool seeded, int fs, int lane) {
+    const int order = tree * SD_MAX_DEPTH + p;                  // loop order of Algorithm 1
+    const int buf = W.best_buf ^ 1;
+    int fh = 0, cnt = 0;
+    double score = 0.0;
+    bool dropped = false;
+    // the node whose children are to be offered next: the match node first, D(N_p) = 1
+    double cur_d = 1.0;
+    int cur_cb = sh.cb[tree][p - 1], cur_n = (int)sh.nc[tree][p - 1], cur_idx = -1;
+    bool have_cur = !seeded;
+    if (!seeded) fs = 0;
+    int4 w = make_int4(-1, 0, 0, 0);                            // window in registers: entries wb .. wb + wvalid
+    int wb = -1, wvalid = 0;
+    while (true) {
+        if (!have_cur) {
+            if (cnt >= budget || fs == 0) break;
+            cur_d = W.F.d[fh];
+            const int tok = W.F.tok[fh], par = W.F.par[fh];
+            cur_cb = W.F.cb[fh];
+            cur_n = (int)(W.F.nc[fh] & RUN_COUNT_MASK);
+            // everything still to come is at most cur_d each
+            if ((score + (double)(budget - cnt) * cur_d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
+            __syncwarp();
+            fh = (fh + 1) & (SD_MAX_SPEC - 1);
+            --fs;
+            if (lane == 0) { W.tok[buf][cnt] = tok; W.par[buf][cnt] = (unsigned char)(par + 1); }
+            score = __dadd_rn(score, cur_d);                    // Eq. 4, insertion order
+            cur_idx = cnt++;
+            const int K = budget - cnt;
+            if (fs > K) fs = K;
+            if (flags & SD_FLAG_LINEAR) fs = 0;
+        }
+        have_cur = false;
+        if (cnt >= budget) break;
+        if (cur_n == 0) continue;
+        if (cur_n > 32) {
+            // wide run: one pass that keeps the best children by count, then D for those only
+            const int K = budget - cnt;
+            long long sum;
+            if (fs == 0) {
+                scan_run_by_count(ent, cur_cb, cur_n, 0, 1, cur_idx, 1, W, W.F, fh, fs, K, sum, lane);
+                counts_to_d(W.F, fh, fs, cur_d, sum, lane);
+            } else if (fs == K) {
+                // full frontier: sum pass, then a pass that only looks at counts large enough
+                prefetch_run(ent, cur_cb, cur_n, lane, 64);
+                push_children_w(ent, cur_cb, cur_n, load_window(ent, cur_cb, limit, lane), cur_d, cur_idx, W.F, fh, fs, K,
+                                lane);
+            } else {
+                // With a full frontier a child only matters if it beats the worst entry.  Counts are
+                // at least 1, so the sibling sum is at least cur_n and D <= cur_d * count / cur_n:
+                // children below the count that needs are skipped without any arithmetic.
+                int cmin = 1;
+                if (fs == K) {
+                    const double need = W.F.d[(fh + fs - 1) & (SD_MAX_SPEC - 1)] / cur_d * (double)cur_n * 0.999999;
+                    cmin = need >= 2.0e9 ? 2000000000 : max(1, (int)need);
+                }
+                int ts;
+                scan_run_by_count(ent, cur_cb, cur_n, 0, 1, cur_idx, cmin, W, W.T, 0, ts, K, sum, lane);
+                counts_to_d(W.T, 0, ts, cur_d, sum, lane);
+                frontier_merge_list(W.F, fh, fs, K, W.T, ts, cur_idx, lane);
+            }
+            continue;
+        }
+        {
+            const int off = cur_cb - wb;
+            if (wb >= 0 && off >= 0 && off + cur_n <= wvalid) {  // the run is already in registers
+                if (off > 0) {
+                    w.x = __shfl_down_sync(FULL, w.x, off); w.y = __shfl_down_sync(FULL, w.y, off);
+                    w.z = __shfl_down_sync(FULL, w.z, off); w.w = __shfl_down_sync(FULL, w.w, off);
+                    wvalid -= off;
+                    wb = cur_cb;
+                }
+            } else {
+                w = load_window(ent, cur_cb, limit, lane);
+                wb = cur_cb;
+                wvalid = min(32, limit - cur_cb);
+            }
+        }
+        if (cur_n == 1 && (fs == 0 || W.F.d[fh] < cur_d)) {
+            // An only child has C = 1, so D stays cur_d: while the best waiting candidate is
+            // strictly worse, the whole chain of only children is added in one go.
+            const bool link = lane < wvalid && ((unsigned)w.w & RUN_COUNT_MASK) == 1u && w.z == cur_cb + lane + 1;
+            const unsigned links = __ballot_sync(FULL, link);
+            const int len = min(wvalid, 1 + (links == 0xffffffffu ? 32 : __ffs(~links) - 1));
+            const int m = min(len, budget - cnt);
+            if (lane < m) {
+                W.tok[buf][cnt + lane] = w.x;
+                W.par[buf][cnt + lane] = (unsigned char)((lane == 0 ? cur_idx : cnt + lane - 1) + 1);
+            }
+            for (int q = 0; q < m; ++q) score = __dadd_rn(score, cur_d);
+            cnt += m;
+            if (fs > budget - cnt) fs = budget - cnt;
+            cur_idx = cnt - 1;
+            cur_cb = __shfl_sync(FULL, w.z, m - 1);
+            cur_n = (int)((unsigned)__shfl_sync(FULL, w.w, m - 1) & RUN_COUNT_MASK);
+            have_cur = true;
+            if ((score + (double)(budget - cnt) * cur_d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
+            continue;
+        }
+        push_children_w(ent, cur_cb, cur_n, w, cur_d, cur_idx, W.F, fh, fs, budget - cnt, lane);
+    }
+    __syncwarp();
+    if (!dropped && (score > W.best_score || (score == W.best_score && score > 0.0 && order < W.best_order))) {
+        if (lane == 0) {
+            W.best_score = score; W.best_order = order; W.best_n = cnt; W.best_buf = buf;
+            atomicMax(&sh.best_bits, (unsigned long long)__double_as_longlong(score));
+        }
+    }
+    __syncwarp();
+}
+
+__global__ void __launch_bounds__(CTA_WARPS * 32, 2)
+speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
+                       unsigned flags, const int32_t* __restrict__ d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
+                       int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
+                       int32_t* d_chosen_p, double* d_score, int32_t* d_status) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    BlockShared& sh = *reinterpret_cast<BlockShared*>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, wib = tid >> 5;
+    const int i = blockIdx.x;
+    const int M = sv.M, words = (M + 31) / 32;
+    const int slot = d_slot[i];
+    const bool ok = slot >= 0 && slot < sv.R;
+    int t = 0, status = SD_STATUS_BAD_SLOT;
+    SlotState* ss = nullptr;
+    if (ok) { ss = sv.s_state + slot; t = ss->len; status = ss->status; }
+    const bool usable = ok && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && t > 0;
+    int cap = max_spec;
+    if (d_budget_cap && d_budget_cap[i] >= 0) cap = min(cap, d_budget_cap[i]);
+    if (tid < 2 * SD_MAX_DEPTH) { (&sh.node[0][0])[tid] = -1; (&sh.nc[0][0])[tid] = 0; }
+    if (tid == 0) { sh.njobs = 0; sh.next = 0; sh.nwide = 0; sh.nwide_kept = 0; sh.best_bits = 0ull; sh.win_warp = -1; }
+    WarpWork& W = sh.w[wib];
+    if (lane == 0) { W.best_score = 0.0; W.best_order = 1 << 30; W.best_n = 0; W.best_buf = 0; }
+
+    // ---------------- 1. match
+    const bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
+    const bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
+    int src_node[2] = {-1, -1}, src_from[2] = {0, 0};           // per target: start node and first text index
+    const int32_t* text = ok ? sv.s_text + (long long)slot * sv.T : nullptr;
+    if (want_g) {
+        const bool cache_ok = ss->g_gen == ss->gen && ss->g_epoch == sv.g_state->epoch && ss->g_len <= t;
+        const int k = t - ss->g_len;                            // tokens appended since the cache was taken
+        const int depths = ss->g_depths;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int d = wib + 1 + h * CTA_WARPS;              // target pattern length
+            if (d > Pe || d > t) continue;
+            if (cache_ok && d > k && d - k <= depths) {
+                src_node[h] = ss->g_node[d - k - 1];            // node of the tokens before the new ones
+                src_from[h] = t - k;
+            } else {
+                src_node[h] = sv.g_root[text[t - d]];
+                src_from[h] = t - d + 1;
+            }
+        }
+    }
+    __syncthreads();                                            // all cached nodes read before any is replaced
+    if (want_g) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int d = wib + 1 + h * CTA_WARPS;
+            if (d > Pe) continue;
+            int cb = 0, nn = 0;
+            const int node = (d > t) ? -1 : walk_from(sv.g_ent, (int)sv.g_cap, src_node[h], text, src_from[h], t, lane, cb, nn);
+            if (lane == 0) {
+                ss->g_node[d - 1] = node;
+                sh.node[0][d - 1] = node;
+                if (node >= 0) { sh.cb[0][d - 1] = cb; sh.nc[0][d - 1] = (unsigned)nn; }
+            }
+        }
+        if (tid == 0) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = Pe; }
+    }
+    if (want_r && wib == CTA_WARPS - 1) {
+        const int d = lane + 1;
+        if (d <= Pe && d <= t) {
+            const int node = ss->active[d - 1];
+            const int4 e = (sv.s_ent + (long long)slot * sv.spn)[node];
+            sh.node[1][d - 1] = node; sh.cb[1][d - 1] = e.z; sh.nc[1][d - 1] = (unsigned)e.w & RUN_COUNT_MASK;
+        }
+    }
+    __syncthreads();
+
+    // ---------------- 2. job queue, costliest first; jobs that start at a wide node wait
+    if (tid < 2 * SD_MAX_DEPTH) {
+        const int tree = tid / SD_MAX_DEPTH, p = tid % SD_MAX_DEPTH + 1;
+        int c = 0;
+        if (p <= Pe && sh.node[tree][p - 1] >= 0 && sh.nc[tree][p - 1] > 0) {
+            // all first runs start their way to L2 now, long before a warp gets to them
+            const int4* base = (tree == 0 ? sv.g_ent : sv.s_ent + (long long)slot * sv.spn) + sh.cb[tree][p - 1];
+            const int lines = min(4, ((int)sh.nc[tree][p - 1] + 7) >> 3);
+            for (int l = 0; l < lines; ++l) prefetch_l2(base + l * 8);
+            c = min(budget_for(alpha, p, cap), 2 * (sv.D - p));
+            if (c > 0 && sh.nc[tree][p - 1] > WIDE_RUN) { sh.wide[atomicAdd(&sh.nwide, 1)] = tid; c = 0; }
+        }
+        sh.cost[tid] = c;
+    }
+    __syncthreads();
+    if (tid < 2 * SD_MAX_DEPTH) {
+        const int c = sh.cost[tid];
+        if (c > 0) {
+            int rank = 0;
+            for (int q = 0; q < 2 * SD_MAX_DEPTH; ++q) {
+                const int cq = sh.cost[q];
+                rank += (cq > c || (cq == c && q < tid)) ? 1 : 0;
+            }
+            sh.job[rank] = tid;
+            atomicAdd(&sh.njobs, 1);
+        }
+    }
+    __syncthreads();
+    const int njobs = sh.njobs;
+    const int4* s_ent = ok ? sv.s_ent + (long long)slot * sv.spn : nullptr;
+    while (true) {
+        int j = 0;
+        if (lane == 0) j = atomicAdd(&sh.next, 1);
+        j = __shfl_sync(FULL, j, 0);
+        if (j >= njobs) break;
+        const int code = sh.job[j];
+        const int tree = code / SD_MAX_DEPTH, p = code % SD_MAX_DEPTH + 1;
+        const int budget = budget_for(alpha, p, cap);
+        if ((double)budget < best_so_far(sh)) continue;         // SCORE <= number of draft nodes
+        expand_job(sh, W, tree == 0 ? sv.g_ent : s_ent, tree == 0 ? (int)sv.g_cap : (int)sv.spn, tree, p, budget, flags,
+                   false, 0, lane);
+    }
+    __syncthreads();
+    // Jobs that start at a wide node (short patterns, hence small budgets): most cannot reach
+    // the best score any more and are dropped here.  For the rest the warps of the block share
+    // the scan of the run, then one warp merges the partial lists and finishes the job.
+    if (tid == 0) {
+        const double best = __longlong_as_double((long long)sh.best_bits);
+        int kept = 0;
+        for (int q = 0; q < sh.nwide; ++q) {
+            const int p = sh.wide[q] % SD_MAX_DEPTH + 1;
+            if (!((double)budget_for(alpha, p, cap) < best)) sh.wide[kept++] = sh.wide[q];
+        }
+        sh.nwide_kept = kept;
+    }
+    __syncthreads();
+    const int nwide = sh.nwide_kept;
+    for (int base = 0; base < nwide; base += CTA_WARPS) {
+        const int nj = min(CTA_WARPS, nwide - base);
+        const int G = CTA_WARPS / nj;                           // warps per job
+        const int my_job = wib / G, my_slice = wib % G;
+        const bool active = my_job < nj;
+        int tree = 0, p = 1, budget = 0, fs = 0;
+        const int4* ent = sv.g_ent;
+        if (active) {
+            const int code = sh.wide[base + my_job];
+            tree = code / SD_MAX_DEPTH; p = code % SD_MAX_DEPTH + 1;
+            budget = budget_for(alpha, p, cap);
+            ent = tree == 0 ? sv.g_ent : s_ent;
+            long long sum;
+            scan_run_by_count(ent, sh.cb[tree][p - 1], (int)sh.nc[tree][p - 1], my_slice, G, -1, 1, W, W.F, 0, fs,
+                              budget, sum, lane);
+            if (lane == 0) { sh.slice_sum[wib] = sum; sh.slice_fs[wib] = fs; }
+        }
+        __syncthreads();
+        if (active && my_slice == 0) {
+            long long sum = sh.slice_sum[wib];
+            for (int g = 1; g < G; ++g) {
+                const Frontier& O = sh.w[wib + g].F;
+                const int ofs = sh.slice_fs[wib + g];
+                sum += sh.slice_sum[wib + g];
+                frontier_merge_list(W.F, 0, fs, budget, O, ofs, -1, lane);
+            }
+            counts_to_d(W.F, 0, fs, 1.0, sum, lane);
+            expand_job(sh, W, ent, tree == 0 ? (int)sv.g_cap : (int)sv.spn, tree, p, budget, flags, true, fs, lane);
+        }
+        __syncthreads();
+    }
+
+    // ---------------- 3. select (first in loop order among the largest scores) and emit
+    if (wib == 0) {
+        double sc = lane < CTA_WARPS ? sh.w[lane].best_score : 0.0;
+        int od = lane < CTA_WARPS ? sh.w[lane].best_order : 1 << 30;
+        int ww = lane;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const double osc = __shfl_xor_sync(FULL, sc, off);
+            const int ood = __shfl_xor_sync(FULL, od, off);
+            const int oww = __shfl_xor_sync(FULL, ww, off);
+            if (osc > sc || (osc == sc && ood < od)) { sc = osc; od = ood; ww = oww; }
+        }
+        if (lane == 0) sh.win_warp = sc > 0.0 ? ww : -1;
+    }
+    __syncthreads();
+    const int win = sh.win_warp;
+    int nd = 0, ctree = -1, cp = 0;
+    double best = 0.0;
+    const int* wtok = nullptr;
+    const unsigned char* wpar = nullptr;
+    if (win >= 0) {
+        const WarpWork& B = sh.w[win];
+        nd = B.best_n; best = B.best_score;
+        ctree = B.best_order / SD_MAX_DEPTH; cp = B.best_order % SD_MAX_DEPTH;
+        if (cp == 0) { cp = SD_MAX_DEPTH; ctree -= 1; }          // order = tree * 32 + p with p in 1..32
+        wtok = B.tok[B.best_buf]; wpar = B.par[B.best_buf];
+    }
+    if (tid < M) {
+        const int j = tid;
+        int tok = -1, par = -1, pos = -1;
+        unsigned long long bits = 0;
+        if (j < nd) {
+            tok = wtok[j];
+            par = (int)wpar[j] - 1;
+            int depth = 0;
+            for (int a = j, hops = 0; a >= 0 && hops < SD_MAX_SPEC; a = (int)wpar[a] - 1, ++hops) {
+                bits |= 1ull << a;
+                ++depth;
+            }
+            pos = t + depth - 1;
+        }
+        const long long o = (long long)i * M + j;
+        d_tokens[o] = tok; d_parents[o] = par; d_positions[o] = pos;
+        d_mask[o * words] = (uint32_t)bits;
+        if (words > 1) d_mask[o * words + 1] = (uint32_t)(bits >> 32);
+    }
+    if (tid == 0) {
+        d_n_draft[i] = nd; d_chosen_tree[i] = ctree; d_chosen_p[i] = cp; d_score[i] = best;
+        if (d_status) d_status[i] = status;
+    }
+}
+
 }  // namespace
 
 extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
@@ -275,12 +923,21 @@ extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const
         return SD_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int Pe = prm->P < s->D ? prm->P : s->D;               // longer patterns never match
-    const long long jobs = (long long)n * 2 * Pe;
-    match_expand_kernel<<<(unsigned)((jobs + SPEC_WARPS - 1) / SPEC_WARPS), SPEC_WARPS * 32, 0, st>>>(
-        *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap);
-    select_emit_kernel<<<(unsigned)((n + 3) / 4), 128, 0, st>>>(*s, n, d_slot, Pe, d_n_draft, d_tokens, d_parents,
-                                                                d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score,
-                                                                d_status);
+    {
+        // the block's shared memory exceeds the default limit: raise it once per device
+        static bool raised[64] = {false};
+        int dev = 0;
+        SD_CUDA_OK(cudaGetDevice(&dev));
+        if (dev >= 0 && dev < 64 && !raised[dev]) {
+            SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)sizeof(BlockShared)));
+            raised[dev] = true;
+        }
+    }
+    speculate_fused_kernel<<<(unsigned)n, CTA_WARPS * 32, sizeof(BlockShared), st>>>(*s, n, d_slot, Pe, prm->alpha, prm->max_spec,
+                                                                  prm->flags, d_budget_cap, d_n_draft, d_tokens,
+                                                                  d_parents, d_positions, d_mask, d_chosen_tree,
+                                                                  d_chosen_p, d_score, d_status);
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }

@@ -45,31 +45,91 @@ __device__ int insert_child(int4* ent, int parent, int cb, int n, int pos, int x
     return idx;
 }
 
+// The same insert done by the whole warp for a long run (all arguments warp-uniform):
+// entries move 32 at a time instead of one by one.
+__device__ int insert_child_warp(int4* ent, int parent, int cb, int n, int pos, int x, int fresh, bool moves, int lane) {
+    const int4 ne = make_int4(x, 1, 0, 0);
+    int idx;
+    if (moves) {
+        for (int i = lane; i < n; i += 32) ent[fresh + i + (i >= pos ? 1 : 0)] = ent[cb + i];
+        idx = fresh + pos;
+        if (lane == 0) { ent[idx] = ne; *word(&ent[parent], 2) = fresh; }
+    } else {
+        for (int hi = n; hi > pos; hi -= 32) {                   // from the top down, a chunk at a time
+            const int lo = max(pos, hi - 32);
+            const int i = lo + lane;
+            int4 e = make_int4(0, 0, 0, 0);
+            if (i < hi) e = ent[cb + i];
+            __syncwarp();
+            if (i < hi) ent[cb + i + 1] = e;
+            __syncwarp();
+        }
+        idx = cb + pos;
+        if (lane == 0) ent[idx] = ne;
+    }
+    if (lane == 0) *word(&ent[parent], 3) = n + 1;
+    __syncwarp();
+    return idx;
+}
+
+// lower_bound of token x in the sorted run ent[cb .. cb+n): eight-way, so that the seven
+// probes of a round are in flight together (a long run costs log8 n dependent rounds).
+__device__ int lower_bound_run(const int4* ent, int cb, int n, int x) {
+    int lo = 0, hi = n;
+    while (hi - lo > 8) {                                        // at most 8 rounds: n < 2^24
+        const int step = (hi - lo) >> 3;
+        int t[7];
+#pragma unroll
+        for (int k = 0; k < 7; ++k) t[k] = ent[cb + lo + (k + 1) * step].x;
+        int sel = 0;
+#pragma unroll
+        for (int k = 0; k < 7; ++k) sel += t[k] < x ? 1 : 0;     // pivots below x
+        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
+        const int nhi = sel == 7 ? hi : lo + (sel + 1) * step;
+        lo = nlo; hi = nhi;
+    }
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (ent[cb + mid].x < x) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
 // All 32 lanes call.  `act` is this lane's active node of depth lane + 1 (-1: none);
 // on return it is the active node after x was appended.  `t` is the context length
 // before the append.  `used` / `live` are warp-uniform pool counters.
 // Returns false, changing nothing, if the pool cannot hold the new nodes.
-__device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, int& act, int& room, int& used,
-                             int& live) {
+// (run_cb, run_w) travel with `act`: the active node's child run as of now, so that the
+// next token's look-up starts at the run itself instead of first reading the node.
+__device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, int& act, int& room, int& run_cb,
+                             unsigned& run_w, int& used, int& live) {
     const unsigned FULL = 0xffffffffu;
     const int parent = __shfl_up_sync(FULL, act, 1);            // node of depth `lane`
     const int parent_room = __shfl_up_sync(FULL, room, 1);      // free entries reserved behind it
+    const int parent_cb = __shfl_up_sync(FULL, run_cb, 1);
+    const unsigned parent_w = __shfl_up_sync(FULL, run_w, 1);
     const bool valid = lane <= min(t, D - 1);
     int found = -1, pos = 0, cb = 0, n = 0;
     unsigned w = 0;
+    int4 fe = make_int4(0, 0, 0, 0);                             // the child's entry when found
     if (valid) {
         if (lane == 0) {
             found = tr.root[x];
+            if (found >= 0) fe = tr.ent[found];
         } else {
-            const int4 pe = tr.ent[parent];
-            cb = pe.z; w = (unsigned)pe.w; n = (int)(w & RUN_COUNT_MASK);
-            int lo = 0, hi = n;
-            while (lo < hi) {                                    // at most 24 rounds: n < 2^24
-                const int mid = (lo + hi) >> 1;
-                if (tr.ent[cb + mid].x < x) lo = mid + 1; else hi = mid;
+            cb = parent_cb; w = parent_w;
+            if (w == RUN_UNKNOWN) { const int4 pe = tr.ent[parent]; cb = pe.z; w = (unsigned)pe.w; }
+            n = (int)(w & RUN_COUNT_MASK);
+            if (n <= 2) {                                        // the usual case: both loads at once
+                int4 e0 = make_int4(0x7fffffff, 0, 0, 0), e1 = e0;
+                if (n > 0) e0 = tr.ent[cb];
+                if (n > 1) e1 = tr.ent[cb + 1];
+                pos = (n > 0 && e0.x < x) ? ((n > 1 && e1.x < x) ? 2 : 1) : 0;
+                if (pos < n) { fe = pos == 0 ? e0 : e1; if (fe.x == x) found = cb + pos; }
+            } else {
+                pos = lower_bound_run(tr.ent, cb, n, x);
+                if (pos < n) { fe = tr.ent[cb + pos]; if (fe.x == x) found = cb + pos; }
             }
-            pos = lo;
-            if (pos < n && tr.ent[cb + pos].x == x) found = cb + pos;
         }
     }
     const bool need = valid && found < 0;
@@ -106,12 +166,22 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
     const bool serial = __any_sync(FULL, clash);
 
     if (valid && found >= 0) {
-        *word(&tr.ent[found], 1) += 1;
+        *word(&tr.ent[found], 1) = fe.y + 1;
         act = found;
+        run_cb = fe.z;
+        run_w = (unsigned)fe.w;
+        // the next lane is about to give this very node a child: what was read is stale then
+        if (lane < 31 && next_need && next_parent == found) run_w = RUN_UNKNOWN;
+        else if (run_w & RUN_COUNT_MASK) asm volatile("prefetch.global.L2 [%0];" ::"l"(tr.ent + run_cb));
+    } else {
+        run_cb = 0;
+        run_w = 0;                                               // a new leaf (or no node at all)
     }
     room = new_room;
     if (!serial) {
-        if (need) {
+        // inserts that move many entries are done by the whole warp, one after the other
+        const bool big = need && lane > 0 && (moves ? n : n - pos) > 8;
+        if (need && !big) {
             if (lane == 0) {
                 tr.ent[fresh] = make_int4(x, 1, 0, 0);
                 tr.root[x] = fresh;
@@ -121,6 +191,16 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
             }
         }
         __syncwarp();
+        unsigned bm = __ballot_sync(FULL, big);
+        while (bm) {
+            const int src = __ffs(bm) - 1;
+            bm &= bm - 1;
+            const int idx = insert_child_warp(tr.ent, __shfl_sync(FULL, parent, src), __shfl_sync(FULL, cb, src),
+                                              __shfl_sync(FULL, n, src), __shfl_sync(FULL, pos, src), x,
+                                              __shfl_sync(FULL, fresh, src), __shfl_sync(FULL, moves ? 1 : 0, src) != 0,
+                                              lane);
+            if (lane == src) act = idx;
+        }
     } else {
         for (int l = 31; l >= 0; --l) {
             if (lane == l && need) {
@@ -135,7 +215,7 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
             __syncwarp();
         }
     }
-    if (!valid) { act = -1; room = 0; }
+    if (!valid) { act = -1; room = 0; run_cb = 0; run_w = 0; }
     live += __popc(__ballot_sync(FULL, need));
     return true;
 }
@@ -155,12 +235,13 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
         for (int i = 0; i < n; ++i) {
             if (d_slot[i] != -1) continue;
             any = true;
-            int act = -1, room = 0;
+            int act = -1, room = 0, run_cb = 0;
+            unsigned run_w = 0;
             const long long b = d_offsets[i], e = d_offsets[i + 1];
             for (long long k = b; k < e && !(status & SD_STATUS_GLOBAL_FULL); ++k) {
                 const int x = d_tokens[k];
                 if (x < 0 || x >= sv.V) { status |= SD_STATUS_BAD_TOKEN; break; }
-                if (!append_token(tr, sv.D, x, (int)(k - b), lane, act, room, used, live)) {
+                if (!append_token(tr, sv.D, x, (int)(k - b), lane, act, room, run_cb, run_w, used, live)) {
                     status |= SD_STATUS_GLOBAL_FULL;
                     break;
                 }
@@ -181,19 +262,20 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
     int32_t* text = sv.s_text + (long long)slot * sv.T;
     TreeRef tr{sv.s_ent + (long long)slot * sv.spn, sv.s_root + (long long)slot * sv.V, (int)sv.spn};
     int len = ss->len, used = ss->used, live = ss->live, status = ss->status;
-    int act = ss->active[lane], room = ss->room[lane];
+    int act = ss->active[lane], room = ss->room[lane], run_cb = ss->run_cb[lane];
+    unsigned run_w = ss->run_w[lane];
     if (d_reset && d_reset[i]) {
         // forget the old tree: only root-table cells of tokens that occur can be set
         for (int k = lane; k < len; k += 32) tr.root[text[k]] = -1;
         __syncwarp();
-        len = 0; used = 0; live = 0; status = 0; act = -1; room = 0;
+        len = 0; used = 0; live = 0; status = 0; act = -1; room = 0; run_cb = 0; run_w = 0;
         if (lane == 0) ss->gen += 1;
     }
     const long long b = d_offsets[i], e = d_offsets[i + 1];
     for (long long k = b; k < e && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)); ++k) {
         const int x = d_tokens[k];
         if (x < 0 || x >= sv.V) { status |= SD_STATUS_BAD_TOKEN; break; }
-        if (len >= sv.T || !append_token(tr, sv.D, x, len, lane, act, room, used, live)) {
+        if (len >= sv.T || !append_token(tr, sv.D, x, len, lane, act, room, run_cb, run_w, used, live)) {
             status |= SD_STATUS_POOL_FULL;
             break;
         }
@@ -202,6 +284,8 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
     }
     ss->active[lane] = act;
     ss->room[lane] = room;
+    ss->run_cb[lane] = run_cb;
+    ss->run_w[lane] = run_w;
     if (lane == 0) { ss->len = len; ss->used = used; ss->live = live; ss->status = status; }
 }
 

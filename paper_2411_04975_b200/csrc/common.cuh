@@ -23,6 +23,7 @@
 #define SD_MAX_SPEC 64
 #define RUN_STATIC 0x80000000u
 #define RUN_COUNT_MASK 0x00FFFFFFu
+#define RUN_UNKNOWN 0xFFFFFFFFu
 
 struct GlobalState {          // device-resident bookkeeping of the global tree
     int32_t used;             // entries handed out
@@ -39,6 +40,8 @@ struct SlotState {            // device-resident bookkeeping of one request slot
     int32_t status;           // SD_STATUS_*
     int32_t active[SD_MAX_DEPTH];   // active[d-1]: entry of the node for the last d tokens
     int32_t room[SD_MAX_DEPTH];     // free entries reserved right behind that node for its chain
+    int32_t run_cb[SD_MAX_DEPTH];   // that node's child run: first entry ...
+    uint32_t run_w[SD_MAX_DEPTH];   // ... and its w field (count | flags); RUN_UNKNOWN: read the entry
     // Match nodes of this request in the GLOBAL tree, kept from the last sd_speculate so that
     // the next one only descends the tokens appended since (a cache: losing it costs a full walk).
     int32_t gen;              // grows when the slot is reset

@@ -761,8 +761,13 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
         const int d = lane + 1;
         if (d <= Pe && d <= t) {
             const int node = ss->active[d - 1];
-            const int4 e = (sv.s_ent + (long long)slot * sv.spn)[node];
-            sh.node[1][d - 1] = node; sh.cb[1][d - 1] = e.z; sh.nc[1][d - 1] = (unsigned)e.w & RUN_COUNT_MASK;
+            int rcb = ss->run_cb[d - 1];
+            unsigned rw = ss->run_w[d - 1];                      // kept current by sd_append
+            if (rw == RUN_UNKNOWN) {
+                const int4 e = (sv.s_ent + (long long)slot * sv.spn)[node];
+                rcb = e.z; rw = (unsigned)e.w;
+            }
+            sh.node[1][d - 1] = node; sh.cb[1][d - 1] = rcb; sh.nc[1][d - 1] = rw & RUN_COUNT_MASK;
         }
     }
     __syncthreads();

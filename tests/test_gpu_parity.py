@@ -292,3 +292,81 @@ def test_closed_loop_scaled(U):
     for sl in range(12):
         pr.check_tree(sl)
     pr.close()
+
+
+def test_large_batch_full_size_sampled_against_oracle(U):
+    """BASELINE config 2 at full size (4,194,304-token global tree, 256 requests x 4,096-token
+    prompts) in the launch configuration bench.py times.  The oracle holds the full global tree
+    but only a sample of the requests; their rows must be bit-exact, and every row must satisfy
+    the properties that hold for any draft."""
+    from workload.generator import accept_schedule, get_workload
+    import oracle as oracle_pkg
+    import paper_2411_04975_b200 as sfx
+    w = get_workload("large_batch")
+    c = w.cfg
+    B = c.batch
+    sample = [0, 1, 37, 100, 101, 180, 254, 255]
+    dev = U.DEV
+    store = sfx.SuffixStore(torch.as_tensor(w.corpus(), device=dev), torch.as_tensor(w.corpus_offsets(), device=dev),
+                            vocab=c.vocab, depth_cap=c.depth_cap, max_requests=B, max_req_tokens=c.prompt_len + 64,
+                            max_spec_cap=c.max_spec)
+    prompts = [w.prompt(i) for i in range(B)]
+    off, flat = U.ragged(prompts)
+    slots = torch.arange(B, dtype=torch.int32, device=dev)
+    store.append(slots, torch.as_tensor(off, device=dev), U.dev_i32(flat), torch.ones(B, dtype=torch.uint8, device=dev))
+    ref = oracle_pkg.SuffixOracle(c.depth_cap, len(sample))
+    ref.global_build(w.corpus(), w.corpus_offsets())
+    ref.slot_append_batch(list(range(len(sample))), [prompts[i] for i in sample], n_threads=8)
+    assert store.stats()["global_nodes"] == ref.node_count(-1)
+    sched = accept_schedule(B, 3)
+    cont = [w.continuation(i, prompts[i], length=int(sched[:, i].sum()) + 1) for i in range(B)]
+    cur = np.zeros(B, dtype=np.int64)
+    for step in range(3):
+        out = store.speculate(slots, c.max_pattern, c.alpha, c.max_spec)
+        torch.cuda.synchronize()
+        got = {k: v.cpu().numpy() for k, v in out.items()}
+        got["mask"] = got["mask"].view(np.uint32)
+        want = ref.speculate(list(range(len(sample))), c.max_pattern, c.alpha, c.max_spec, n_threads=8)
+        U.assert_same_drafts({k: v[sample] for k, v in got.items()}, want)
+        # properties of every row
+        n = got["n_draft"]
+        assert (got["status"] == 0).all() and (n >= 0).all() and (n <= c.max_spec).all()
+        assert ((got["score"] > 0) == (n > 0)).all() and (got["score"] <= n).all()
+        for i in range(B):
+            k = int(n[i])
+            par = got["parents"][i, :k]
+            assert (par < np.arange(k)).all() and (par >= -1).all()
+            depth = np.zeros(k, dtype=np.int64)
+            for j in range(k):
+                depth[j] = 1 if par[j] < 0 else depth[par[j]] + 1
+                row = int(got["mask"][i, j, 0]) | (int(got["mask"][i, j, 1]) << 32)
+                prow = 0 if par[j] < 0 else int(got["mask"][i, par[j], 0]) | (int(got["mask"][i, par[j], 1]) << 32)
+                assert row == prow | (1 << j)
+            t = c.prompt_len + int(cur[i])
+            assert (got["positions"][i, :k] == t + depth - 1).all()
+            assert (got["tokens"][i, k:] == -1).all() and (got["mask"][i, k:] == 0).all()
+            assert k <= max(1, int(c.alpha * got["chosen_p"][i])) and depth.max(initial=0) <= c.depth_cap - got["chosen_p"][i]
+        # next decode step
+        a = sched[step]
+        lists = [cont[i][cur[i]:cur[i] + a[i]] for i in range(B)]
+        cur += a
+        o2, f2 = U.ragged(lists)
+        store.append(slots, torch.as_tensor(o2, device=dev), U.dev_i32(f2))
+        ref.slot_append_batch(list(range(len(sample))), [lists[i] for i in sample], n_threads=8)
+    # the sampled per-request trees, node by node
+    for k, i in enumerate(sample[:3]):
+        depth, parent, tok, cnt = ref.dump(k)
+        nn = len(tok)
+        offp = np.zeros(nn + 1, dtype=np.int64); offp[1:] = np.cumsum(depth)
+        flatp = np.empty(int(offp[-1]), dtype=np.int32)
+        for q in range(nn):
+            b = offp[q]
+            if parent[q] >= 0:
+                pb = offp[parent[q]]
+                flatp[b:b + depth[q] - 1] = flatp[pb:pb + depth[q] - 1]
+            flatp[b + depth[q] - 1] = tok[q]
+        gotc = store.query_counts(U.dev_i32(np.full(nn, i)), torch.as_tensor(offp, device=dev), U.dev_i32(flatp))
+        assert np.array_equal(gotc.cpu().numpy(), cnt)
+        assert int(store.slot_info(U.dev_i32([i]))["nodes"][0]) == nn
+    store.free()
+    ref.close()

@@ -166,12 +166,14 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
     const bool serial = __any_sync(FULL, clash);
 
     if (valid && found >= 0) {
+        // a count changes: the copies in the run's top block (if any) are stale from now on
+        if (lane > 0 && (w & RUN_HAS_TOP)) *word(&tr.ent[parent], 3) = (int)(w & ~RUN_HAS_TOP);
         *word(&tr.ent[found], 1) = fe.y + 1;
         act = found;
         run_cb = fe.z;
         run_w = (unsigned)fe.w;
-        // the next lane is about to give this very node a child: what was read is stale then
-        if (lane < 31 && next_need && next_parent == found) run_w = RUN_UNKNOWN;
+        // the next lane works on this very node's run (new child, or flag dropped): what was read may be stale
+        if (lane < 31 && next_parent == found) run_w = RUN_UNKNOWN;
         else if (run_w & RUN_COUNT_MASK) asm volatile("prefetch.global.L2 [%0];" ::"l"(tr.ent + run_cb));
     } else {
         run_cb = 0;

@@ -341,6 +341,67 @@ __global__ void count_children_kernel(const uint8_t* lcp, const uint8_t* len, i6
     nchild[1 + nbase[j] + (d - (int)lcp[j] - 1)] = nc;
 }
 
+__device__ __forceinline__ int top_block_of(int nid, int nc) { return (nid > 0 && nc > SD_TOP_MIN) ? SD_TOP_BLOCK : 0; }
+
+struct RunAlloc {             // entries a node's child run takes, top block included
+    const int* nchild;
+    __device__ int operator()(i64 nid) const { return nchild[nid] + top_block_of((int)nid, nchild[nid]); }
+};
+
+__global__ void collect_wide_kernel(const int* nchild, i64 n_nodes_plus1, int* list, int* counter) {
+    i64 nid = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (nid >= n_nodes_plus1) return;
+    if (top_block_of((int)nid, nchild[nid])) list[atomicAdd(counter, 1)] = (int)nid;
+}
+
+// One block per long run: header (sum of counts) and the 64 best children by (count desc,
+// token asc), found by 64 rounds of "largest key below the previous one".
+__global__ void fill_top_kernel(const int* list, const int* nchild, const int* runstart, int4* ent) {
+    __shared__ u64 skey[256];
+    __shared__ int sidx[256];
+    __shared__ u64 ssum[256];
+    const int nid = list[blockIdx.x];
+    const int n = nchild[nid];
+    const int top = runstart[nid];                 // header; the run itself starts SD_TOP_BLOCK later
+    const int4* run = ent + top + SD_TOP_BLOCK;
+    u64 sum = 0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) sum += (u64)(unsigned)run[i].y;
+    ssum[threadIdx.x] = sum;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) ssum[threadIdx.x] += ssum[threadIdx.x + o];
+        __syncthreads();
+    }
+    const int ntop = n < 64 ? n : 64;
+    if (threadIdx.x == 0) ent[top] = make_int4((int)(unsigned)(ssum[0] & 0xffffffffu), (int)(unsigned)(ssum[0] >> 32), ntop, 0);
+    u64 prev = ~0ull;
+    for (int r = 0; r < ntop; ++r) {
+        u64 best = 0;
+        int bi = -1;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int4 e = run[i];
+            const u64 key = ((u64)(unsigned)e.y << 32) | (u64)(0xffffffffu - (unsigned)e.x);
+            if (key < prev && (bi < 0 || key > best)) { best = key; bi = i; }
+        }
+        skey[threadIdx.x] = bi >= 0 ? best : 0;
+        sidx[threadIdx.x] = bi;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if (threadIdx.x < o) {
+                const int oi = sidx[threadIdx.x + o];
+                if (oi >= 0 && (sidx[threadIdx.x] < 0 || skey[threadIdx.x + o] > skey[threadIdx.x])) {
+                    skey[threadIdx.x] = skey[threadIdx.x + o];
+                    sidx[threadIdx.x] = oi;
+                }
+            }
+            __syncthreads();
+        }
+        prev = skey[0];
+        if (threadIdx.x == 0) ent[top + 1 + r] = run[sidx[0]];
+        __syncthreads();
+    }
+}
+
 // Write the depth-d nodes.  A node's entry sits in its parent's child run at its rank among
 // the siblings (suffix order = token order).
 __global__ void emit_level_kernel(const int32_t* tok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len,
@@ -363,15 +424,16 @@ __global__ void emit_level_kernel(const int32_t* tok, const uint32_t* sa, const 
     int4 e;
     e.x = tok[(i64)sa[j] + d - 1];
     e.y = nb - (int)j;                                    // every suffix in the range is an occurrence
-    e.z = nc > 0 ? runstart[nid] : 0;
-    e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC) : 0;
-    const int pos = runstart[pnid] + rank;
+    const int tb = top_block_of(nid, nc);
+    e.z = nc > 0 ? runstart[nid] + tb : 0;
+    e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC | (tb ? RUN_HAS_TOP : 0u)) : 0;
+    const int pos = runstart[pnid] + top_block_of(pnid, nchild[pnid]) + rank;
     ent[pos] = e;
     if (d == 1) root[e.x] = pos;
 }
 
-__global__ void init_global_state_kernel(GlobalState* g, int used, long long tokens) {
-    g->used = used; g->live = used; g->status = 0; g->epoch = 1; g->tokens = tokens;
+__global__ void init_global_state_kernel(GlobalState* g, int used, int live, long long tokens) {
+    g->used = used; g->live = live; g->status = 0; g->epoch = 1; g->tokens = tokens;
 }
 
 struct DeviceArena {          // temporaries of one build, released together
@@ -532,22 +594,21 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
         for (int d = 1; d <= D; ++d) n_nodes += (i64)h_level[d];
     }
 
-    i64 extra = p->global_extra_nodes >= 0 ? p->global_extra_nodes : std::max<i64>(1ll << 22, n_nodes);
-    s->g_cap = n_nodes + extra;
-    if (s->g_cap >= (1ll << 31) - 2) { store_release(s); return SD_ERR_INVALID_ARG; }
-    if (!store_alloc(s, &s->g_ent, s->g_cap)) { store_release(s); return SD_ERR_NOMEM; }
-
+    i64 used_entries = 0;
+    int *r_a = nullptr, *r_b = nullptr, *b_a = ex, *b_b = nullptr, *seg_a = nullptr, *seg_b = nullptr;
+    int *nbase = nullptr, *nchild = nullptr, *runstart = nullptr, *big_tmp = nullptr, *wide_list = nullptr;
+    int* r_cur = nullptr;
+    int n_wide = 0;
     if (N > 0) {
-        int *r_a = nullptr, *r_b = nullptr, *b_a = ex, *b_b = nullptr, *seg_a = nullptr, *seg_b = nullptr;
-        int *nbase = nullptr, *nchild = nullptr, *runstart = nullptr, *big_tmp = nullptr;
         ok = tmp.get(&r_a, N + 1) && tmp.get(&r_b, N + 1) && tmp.get(&seg_a, N + 2) && tmp.get(&seg_b, N + 2) &&
              tmp.get(&b_b, N + 1) && tmp.get(&nbase, N + 1) && tmp.get(&nchild, n_nodes + 1) &&
-             tmp.get(&runstart, n_nodes + 2) && tmp.get(&big_tmp, scan_tmp_ints(n_nodes + 1));
+             tmp.get(&runstart, n_nodes + 2) && tmp.get(&big_tmp, scan_tmp_ints(n_nodes + 1)) &&
+             tmp.get(&wide_list, n_nodes / SD_TOP_MIN + 2);
         if (!ok) { store_release(s); return SD_ERR_NOMEM; }
         exclusive_scan(NewNodes{lcp, len}, N, nbase, sb.scan_tmp, st);
         // pass 1, deepest level first: children per node
         int* r_next = r_a;
-        int* r_cur = r_b;
+        r_cur = r_b;
         for (int d = D; d >= 1; --d) {
             exclusive_scan(OpensNode{lcp, len, d}, N, r_cur, sb.scan_tmp, st);
             exclusive_scan(Boundary{lcp, d}, N, b_a, sb.scan_tmp, st);
@@ -556,8 +617,25 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
                                                                       nbase, nchild);
             std::swap(r_cur, r_next);
         }
-        // child runs in node (pre-)order
-        exclusive_scan(LoadInt{nchild}, n_nodes + 1, runstart, big_tmp, st);
+        // child runs (with their top blocks) in node (pre-)order
+        exclusive_scan(RunAlloc{nchild}, n_nodes + 1, runstart, big_tmp, st);
+        int* wide_counter = (int*)level_nodes;
+        ce = cudaMemsetAsync(wide_counter, 0, sizeof(int), st);
+        collect_wide_kernel<<<grid_for(n_nodes + 1, T256), T256, 0, st>>>(nchild, n_nodes + 1, wide_list, wide_counter);
+        int h_total = 0;
+        if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_total, runstart + n_nodes + 1, sizeof(int), cudaMemcpyDeviceToHost, st);
+        if (ce == cudaSuccess) ce = cudaMemcpyAsync(&n_wide, wide_counter, sizeof(int), cudaMemcpyDeviceToHost, st);
+        if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+        if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
+        used_entries = h_total;
+    }
+
+    i64 extra = p->global_extra_nodes >= 0 ? p->global_extra_nodes : std::max<i64>(1ll << 22, n_nodes);
+    s->g_cap = used_entries + extra;
+    if (s->g_cap >= (1ll << 31) - 2) { store_release(s); return SD_ERR_INVALID_ARG; }
+    if (!store_alloc(s, &s->g_ent, s->g_cap)) { store_release(s); return SD_ERR_NOMEM; }
+
+    if (N > 0) {
         // pass 2, top level first: write the entries
         int *b_cur = b_a, *b_prev = b_b, *seg_cur = seg_a, *seg_prev = seg_b;
         for (int d = 1; d <= D; ++d) {
@@ -570,8 +648,9 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
             std::swap(b_cur, b_prev);
             std::swap(seg_cur, seg_prev);
         }
+        if (n_wide > 0) fill_top_kernel<<<n_wide, 256, 0, st>>>(wide_list, nchild, runstart, s->g_ent);
     }
-    init_global_state_kernel<<<1, 1, 0, st>>>(s->g_state, (int)n_nodes, N);
+    init_global_state_kernel<<<1, 1, 0, st>>>(s->g_state, (int)used_entries, (int)n_nodes, N);
     ce = cudaStreamSynchronize(st);
     if (ce == cudaSuccess) ce = cudaGetLastError();
     if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }

@@ -4,7 +4,7 @@
 // child run:
 //     x = token id          y = count (occurrences of the root-to-node path)
 //     z = index of the first entry of this node's own child run
-//     w = number of children (low 24 bits) | RUN_STATIC (bit 31)
+//     w = number of children (low 24 bits) | RUN_STATIC (bit 31) | RUN_HAS_TOP (bit 30)
 // A child run is a contiguous array of entries sorted by token id, so one
 // 16-byte load per child yields everything Eq. 1 needs (token, count) plus the
 // way down.  A run with n children built online has room for pow2ceil(n)
@@ -24,6 +24,14 @@
 #define RUN_STATIC 0x80000000u
 #define RUN_COUNT_MASK 0x00FFFFFFu
 #define RUN_UNKNOWN 0xFFFFFFFFu
+// A long child run laid down by the offline build is preceded by a TOP BLOCK: one header entry
+// {sum of the children's counts (lo, hi), number of top entries, 0} and copies of the 64
+// children with the largest counts (then smallest tokens), best first.  Only those can ever
+// enter a speculation tree of at most 64 nodes, so expanding such a node reads 1 KB instead
+// of the whole run.  The flag is dropped by the first online update that touches the run.
+#define RUN_HAS_TOP 0x40000000u
+#define SD_TOP_MIN 128            // runs longer than this get a top block
+#define SD_TOP_BLOCK 65           // entries of a top block
 
 struct GlobalState {          // device-resident bookkeeping of the global tree
     int32_t used;             // entries handed out

@@ -290,7 +290,7 @@ struct BlockShared {
     WarpWork w[CTA_WARPS];
     int node[2][SD_MAX_DEPTH];                // match node per tree and pattern length (-1: none)
     int cb[2][SD_MAX_DEPTH];                  // its child run
-    unsigned nc[2][SD_MAX_DEPTH];
+    unsigned nc[2][SD_MAX_DEPTH];             // ... as the node's w field (count | flags)
     int cost[2 * SD_MAX_DEPTH];
     int job[2 * SD_MAX_DEPTH];
     int wide[2 * SD_MAX_DEPTH];               // jobs whose match node has a wide child run
@@ -481,12 +481,13 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
 // the window already in registers cost no memory access.  Returns the node reached (-1: no
 // match) and its child run in (cb, n).
 __device__ int walk_from(const int4* __restrict__ ent, int limit, int node, const int32_t* __restrict__ text, int from,
-                         int to, int lane, int& cb, int& n) {
+                         int to, int lane, int& cb, unsigned& wfull) {
     if (node < 0) return -1;
     int wb = node;
     int4 w = load_window(ent, wb, limit, lane);
     cb = __shfl_sync(FULL, w.z, 0);
-    n = (int)((unsigned)__shfl_sync(FULL, w.w, 0) & RUN_COUNT_MASK);
+    wfull = (unsigned)__shfl_sync(FULL, w.w, 0);
+    int n = (int)(wfull & RUN_COUNT_MASK);
     for (int pos = from; pos < to; ++pos) {
         const int x = text[pos];
         if (n == 0) return -1;
@@ -494,7 +495,7 @@ __device__ int walk_from(const int4* __restrict__ ent, int limit, int node, cons
             int4 e;
             node = find_child_entry(ent, cb, n, x, lane, e);
             if (node < 0) return -1;
-            cb = e.z; n = (int)((unsigned)e.w & RUN_COUNT_MASK);
+            cb = e.z; wfull = (unsigned)e.w; n = (int)(wfull & RUN_COUNT_MASK);
             wb = -64;                                           // no usable window
             continue;
         }
@@ -505,11 +506,39 @@ __device__ int walk_from(const int4* __restrict__ ent, int limit, int node, cons
         const int src = __ffs(hit) - 1;
         node = wb + src;
         cb = __shfl_sync(FULL, w.z, src);
-        n = (int)((unsigned)__shfl_sync(FULL, w.w, src) & RUN_COUNT_MASK);
+        wfull = (unsigned)__shfl_sync(FULL, w.w, src);
+        n = (int)(wfull & RUN_COUNT_MASK);
     }
     return node;
 }
 
+
+// Children of a node whose run has a top block (see RUN_HAS_TOP): the 64 best by count are
+// listed, best first, right before the run, together with the sum of all counts.
+__device__ void push_top(const int4* __restrict__ ent, int cb, double d_parent, int par_index, Frontier& F, int fh,
+                         int& fs, int K, int lane) {
+    if (K <= 0) return;
+    const int4 hdr = ent[cb - SD_TOP_BLOCK];
+    const double dsum = (double)(((unsigned long long)(unsigned)hdr.y << 32) | (unsigned long long)(unsigned)hdr.x);
+    const int ntop = min(hdr.z, K);                             // only the K best can enter
+    for (int base = 0; base < ntop; base += 32) {
+        const int idx = base + lane;
+        bool pass = idx < ntop;
+        int4 e = make_int4(0, 0, 0, 0);
+        double dc = 0.0;
+        if (pass) {
+            e = ent[cb - SD_TOP_BLOCK + 1 + idx];
+            dc = __dmul_rn(d_parent, __ddiv_rn((double)e.y, dsum));      // Eq. 2 with Eq. 1
+            if (fs == K) {
+                const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+                pass = better(dc, e.x, par_index, F.d[last], F.tok[last], F.par[last]);
+            }
+            if (pass && ((unsigned)e.w & RUN_COUNT_MASK)) prefetch_l2(ent + e.z);
+        }
+        if (!__any_sync(FULL, pass)) break;                     // best first: nothing further can enter
+        frontier_merge(F, fh, fs, K, pass, dc, e.x, par_index, e.z, (unsigned)e.w, lane);
+    }
+}
 
 constexpr int WIDE_RUN = 256;                 // child runs longer than this are scanned by several warps
 
@@ -593,7 +622,9 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
     bool dropped = false;
     // the node whose children are to be offered next: the match node first, D(N_p) = 1
     double cur_d = 1.0;
-    int cur_cb = sh.cb[tree][p - 1], cur_n = (int)sh.nc[tree][p - 1], cur_idx = -1;
+    int cur_cb = sh.cb[tree][p - 1], cur_idx = -1;
+    unsigned cur_w = sh.nc[tree][p - 1];
+    int cur_n = (int)(cur_w & RUN_COUNT_MASK);
     bool have_cur = !seeded;
     if (!seeded) fs = 0;
     int4 w = make_int4(-1, 0, 0, 0);                            // window in registers: entries wb .. wb + wvalid
@@ -604,7 +635,8 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
             cur_d = W.F.d[fh];
             const int tok = W.F.tok[fh], par = W.F.par[fh];
             cur_cb = W.F.cb[fh];
-            cur_n = (int)(W.F.nc[fh] & RUN_COUNT_MASK);
+            cur_w = W.F.nc[fh];
+            cur_n = (int)(cur_w & RUN_COUNT_MASK);
             // everything still to come is at most cur_d each
             if ((score + (double)(budget - cnt) * cur_d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
             __syncwarp();
@@ -620,6 +652,10 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
         have_cur = false;
         if (cnt >= budget) break;
         if (cur_n == 0) continue;
+        if (cur_w & RUN_HAS_TOP) {                              // long run with a ready-made list of its best children
+            push_top(ent, cur_cb, cur_d, cur_idx, W.F, fh, fs, budget - cnt, lane);
+            continue;
+        }
         if (cur_n > 32) {
             // wide run: one pass that keeps the best children by count, then D for those only
             const int K = budget - cnt;
@@ -679,7 +715,8 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
             if (fs > budget - cnt) fs = budget - cnt;
             cur_idx = cnt - 1;
             cur_cb = __shfl_sync(FULL, w.z, m - 1);
-            cur_n = (int)((unsigned)__shfl_sync(FULL, w.w, m - 1) & RUN_COUNT_MASK);
+            cur_w = (unsigned)__shfl_sync(FULL, w.w, m - 1);
+            cur_n = (int)(cur_w & RUN_COUNT_MASK);
             have_cur = true;
             if ((score + (double)(budget - cnt) * cur_d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
             continue;
@@ -747,12 +784,13 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
         for (int h = 0; h < 2; ++h) {
             const int d = wib + 1 + h * CTA_WARPS;
             if (d > Pe) continue;
-            int cb = 0, nn = 0;
-            const int node = (d > t) ? -1 : walk_from(sv.g_ent, (int)sv.g_cap, src_node[h], text, src_from[h], t, lane, cb, nn);
+            int cb = 0;
+            unsigned wf = 0;
+            const int node = (d > t) ? -1 : walk_from(sv.g_ent, (int)sv.g_cap, src_node[h], text, src_from[h], t, lane, cb, wf);
             if (lane == 0) {
                 ss->g_node[d - 1] = node;
                 sh.node[0][d - 1] = node;
-                if (node >= 0) { sh.cb[0][d - 1] = cb; sh.nc[0][d - 1] = (unsigned)nn; }
+                if (node >= 0) { sh.cb[0][d - 1] = cb; sh.nc[0][d - 1] = wf; }
             }
         }
         if (tid == 0) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = Pe; }
@@ -767,7 +805,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
                 const int4 e = (sv.s_ent + (long long)slot * sv.spn)[node];
                 rcb = e.z; rw = (unsigned)e.w;
             }
-            sh.node[1][d - 1] = node; sh.cb[1][d - 1] = rcb; sh.nc[1][d - 1] = rw & RUN_COUNT_MASK;
+            sh.node[1][d - 1] = node; sh.cb[1][d - 1] = rcb; sh.nc[1][d - 1] = rw;
         }
     }
     __syncthreads();
@@ -776,13 +814,15 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     if (tid < 2 * SD_MAX_DEPTH) {
         const int tree = tid / SD_MAX_DEPTH, p = tid % SD_MAX_DEPTH + 1;
         int c = 0;
-        if (p <= Pe && sh.node[tree][p - 1] >= 0 && sh.nc[tree][p - 1] > 0) {
+        const unsigned wf = sh.nc[tree][p - 1];
+        const int nch = (int)(wf & RUN_COUNT_MASK);
+        if (p <= Pe && sh.node[tree][p - 1] >= 0 && nch > 0) {
             // all first runs start their way to L2 now, long before a warp gets to them
             const int4* base = (tree == 0 ? sv.g_ent : sv.s_ent + (long long)slot * sv.spn) + sh.cb[tree][p - 1];
-            const int lines = min(4, ((int)sh.nc[tree][p - 1] + 7) >> 3);
+            const int lines = min(4, (nch + 7) >> 3);
             for (int l = 0; l < lines; ++l) prefetch_l2(base + l * 8);
             c = min(budget_for(alpha, p, cap), 2 * (sv.D - p));
-            if (c > 0 && sh.nc[tree][p - 1] > WIDE_RUN) { sh.wide[atomicAdd(&sh.nwide, 1)] = tid; c = 0; }
+            if (c > 0 && nch > WIDE_RUN && !(wf & RUN_HAS_TOP)) { sh.wide[atomicAdd(&sh.nwide, 1)] = tid; c = 0; }
         }
         sh.cost[tid] = c;
     }
@@ -842,8 +882,8 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
             budget = budget_for(alpha, p, cap);
             ent = tree == 0 ? sv.g_ent : s_ent;
             long long sum;
-            scan_run_by_count(ent, sh.cb[tree][p - 1], (int)sh.nc[tree][p - 1], my_slice, G, -1, 1, W, W.F, 0, fs,
-                              budget, sum, lane);
+            scan_run_by_count(ent, sh.cb[tree][p - 1], (int)(sh.nc[tree][p - 1] & RUN_COUNT_MASK), my_slice, G, -1, 1, W,
+                              W.F, 0, fs, budget, sum, lane);
             if (lane == 0) { sh.slice_sum[wib] = sum; sh.slice_fs[wib] = fs; }
         }
         __syncthreads();

@@ -431,20 +431,18 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
     const double dsum = (double)sum;
     // With a full frontier only a child that beats its worst entry matters:
     // D = d_parent * count / sum, so counts below `cmin` lose without any fp64 work.
-    int cmin = 1;
-    double ld = 0.0; int lt = 0, lp = 0;
+    double ld = 0.0, need = 0.0; int lt = 0, lp = 0;
     const bool full = fs == K;
     if (full) {
         const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
         ld = F.d[last]; lt = F.tok[last]; lp = F.par[last];
-        const double need = ld / d_parent * dsum * 0.999999;
-        cmin = need >= 2.0e9 ? 2000000000 : max(1, (int)need);
+        need = ld * dsum * 0.999999;                            // count * d_parent must reach this
     }
     for (int base = 0; base < n; base += 32) {
         const int idx = base + lane;
         int4 e = w;
         if (base != 0) { e = make_int4(0, 0, 0, 0); if (idx < n) e = ent[cb + idx]; }
-        bool pass = idx < n && e.y >= cmin;
+        bool pass = idx < n && (double)e.y * d_parent >= need;
         if (!__any_sync(FULL, pass)) continue;
         double dc = 0.0;
         if (pass) {
@@ -644,6 +642,8 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
             --fs;
             if (lane == 0) { W.tok[buf][cnt] = tok; W.par[buf][cnt] = (unsigned char)(par + 1); }
             score = __dadd_rn(score, cur_d);                    // Eq. 4, insertion order
+            // the final SCORE of this job is at least its running value: let the others prune on it
+            if (lane == 0) atomicMax(&sh.best_bits, (unsigned long long)__double_as_longlong(score));
             cur_idx = cnt++;
             const int K = budget - cnt;
             if (fs > K) fs = K;
@@ -711,6 +711,7 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
                 W.par[buf][cnt + lane] = (unsigned char)((lane == 0 ? cur_idx : cnt + lane - 1) + 1);
             }
             for (int q = 0; q < m; ++q) score = __dadd_rn(score, cur_d);
+            if (lane == 0) atomicMax(&sh.best_bits, (unsigned long long)__double_as_longlong(score));
             cnt += m;
             if (fs > budget - cnt) fs = budget - cnt;
             cur_idx = cnt - 1;

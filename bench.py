@@ -33,6 +33,9 @@ METRIC = "speculation trees/s at batch 256 (one sd_speculate + sd_append per ste
 UNIT = "trees/s"
 OUT_BYTES_PER_REQ = 4 * 64 * 3 + 64 * 8 + 4 * 3 + 8          # tokens, parents, positions, mask, scalars
 FLUSH_BYTES = 256 << 20
+# dram__bytes_read + dram__bytes_write of one speculate_fused_kernel launch on the full-size
+# large_batch workload, from the ncu capture summarised in profiles/ (set to None when the kernel changes)
+SPECULATE_DRAM_TRAFFIC = 25.9e6
 
 
 def parse():
@@ -313,7 +316,8 @@ def run_ours(args):
         spec_s = statistics.mean(spec_ms) / 1e3
         achieved = alg_bytes / spec_s / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": None, "peak_source": which, "kernel": "speculate_fused_kernel (all of sd_speculate)",
+                    "traffic": SPECULATE_DRAM_TRAFFIC if c.name == "large_batch" and not args.small else None,
+                    "peak_source": which, "kernel": "speculate_fused_kernel (all of sd_speculate)",
                     "algorithmic_bytes_per_launch": alg_bytes}
         extra = {"parity_vs_oracle": "bit-exact" if ok else "MISMATCH", "parity_steps": len(sample_steps),
                  "nodes_visited_per_step": visits,

@@ -159,11 +159,10 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
 
     // A lane that moves entries of its run must not do so while the next lane edits the
     // header of an entry inside that run (only possible when the last tokens repeat one
-    // token).  Then the inserts go one at a time, deepest first.
+    // token): it then waits for that lane, see the rounds below.
     const int next_parent = __shfl_down_sync(FULL, parent, 1);
     const int next_need = __shfl_down_sync(FULL, need ? 1 : 0, 1);
     const bool clash = need && lane >= 1 && lane < 31 && next_need && next_parent >= cb && next_parent < cb + n;
-    const bool serial = __any_sync(FULL, clash);
 
     if (valid && found >= 0) {
         // a count changes: the copies in the run's top block (if any) are stale from now on
@@ -180,10 +179,16 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
         run_w = 0;                                               // a new leaf (or no node at all)
     }
     room = new_room;
-    if (!serial) {
+    // Inserts run in rounds: a lane whose insert would move an entry that the next lane still has
+    // to edit waits for that lane (deepest first); everybody else goes at once.  Almost always
+    // there is one round; a tail of k equal tokens needs up to k.
+    unsigned pend = __ballot_sync(FULL, need);
+    for (int round = 0; round < 33 && pend; ++round) {
+        const bool next_pending = lane < 31 && ((pend >> (lane + 1)) & 1u);
+        const bool ready = need && ((pend >> lane) & 1u) && !(clash && next_pending);
         // inserts that move many entries are done by the whole warp, one after the other
-        const bool big = need && lane > 0 && (moves ? n : n - pos) > 8;
-        if (need && !big) {
+        const bool big = ready && lane > 0 && (moves ? n : n - pos) > 8;
+        if (ready && !big) {
             if (lane == 0) {
                 tr.ent[fresh] = make_int4(x, 1, 0, 0);
                 tr.root[x] = fresh;
@@ -203,19 +208,8 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
                                               lane);
             if (lane == src) act = idx;
         }
-    } else {
-        for (int l = 31; l >= 0; --l) {
-            if (lane == l && need) {
-                if (lane == 0) {
-                    tr.ent[fresh] = make_int4(x, 1, 0, 0);
-                    tr.root[x] = fresh;
-                    act = fresh;
-                } else {
-                    act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, moves);
-                }
-            }
-            __syncwarp();
-        }
+        pend &= ~__ballot_sync(FULL, ready);
+        __syncwarp();
     }
     if (!valid) { act = -1; room = 0; run_cb = 0; run_w = 0; }
     live += __popc(__ballot_sync(FULL, need));

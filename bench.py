@@ -49,6 +49,8 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--oracle-samples", type=int, default=4)
     ap.add_argument("--small", action="store_true", help="1/16 corpus, batch 32: quick functional run")
+    ap.add_argument("--closed-loop-oracle", action="store_true",
+                    help="closed_loop config: run the CPU oracle in lock-step and compare every step (slow)")
     return ap.parse_args()
 
 
@@ -352,6 +354,99 @@ def run_ours(args):
 
 
 # --------------------------------------------------------------------------------------------
+def run_closed_loop(args):
+    """BASELINE config 4: speculate -> simulated verification against the hidden continuation ->
+    append accepted + bonus tokens; finished outputs go into the global tree, their slots are
+    refilled.  Reports mean accepted length and steps/s (one GPU)."""
+    import torch
+
+    import paper_2411_04975_b200 as sfx
+    from workload.closed_loop import ClosedLoop
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = make_workload(args)
+    c = w.cfg
+    B = c.batch
+    K = args.steps if args.steps != 100 else (c.steps or 1000)
+    store = sfx.SuffixStore(torch.as_tensor(w.corpus(), device=dev), torch.as_tensor(w.corpus_offsets(), device=dev),
+                            vocab=c.vocab, depth_cap=c.depth_cap, max_requests=B,
+                            max_req_tokens=c.prompt_len + c.out_len_hi + 8, max_spec_cap=c.max_spec)
+    ref = None
+    if args.closed_loop_oracle:
+        import oracle
+        ref = oracle.SuffixOracle(c.depth_cap, B)
+        ref.global_build(w.corpus(), w.corpus_offsets())
+    loop = ClosedLoop(w, B)
+    slots_all = torch.arange(B, dtype=torch.int32, device=dev)
+    out = store.alloc_outputs(B)
+
+    def append(items):
+        sl, lists, reset = items
+        off = np.zeros(len(sl) + 1, dtype=np.int64)
+        off[1:] = np.cumsum([len(x) for x in lists])
+        flat = np.concatenate(lists).astype(np.int32) if off[-1] else np.zeros(0, dtype=np.int32)
+        store.append(torch.as_tensor(np.asarray(sl, dtype=np.int32), device=dev), torch.as_tensor(off, device=dev),
+                     torch.as_tensor(flat, device=dev) if flat.size else torch.zeros(0, dtype=torch.int32, device=dev),
+                     torch.as_tensor(np.asarray(reset, dtype=np.uint8), device=dev))
+        if ref is not None:
+            for s_, l_, r_ in zip(sl, lists, reset):
+                if s_ < 0:
+                    ref.global_insert(l_)
+                elif r_:
+                    ref.slot_reset(s_)
+            idx = [i for i, s_ in enumerate(sl) if s_ >= 0]
+            ref.slot_append_batch([sl[i] for i in idx], [lists[i] for i in idx], n_threads=oracle_threads(B))
+
+    append(loop.start())
+    torch.cuda.synchronize()
+    spec_ms, app_ms, ok = [], [], True
+    t_wall = time.perf_counter()
+    for k in range(K):
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record()
+        store.speculate(slots_all, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
+        e1.record()
+        host = {n: out[n].cpu().numpy() for n in ("n_draft", "tokens", "parents")}
+        if ref is not None:
+            r = ref.speculate(list(range(B)), c.max_pattern, c.alpha, c.max_spec, n_threads=oracle_threads(B))
+            g = {n: t.cpu().numpy() for n, t in out.items()}
+            for n in ("n_draft", "tokens", "parents", "positions", "chosen_tree", "chosen_p"):
+                ok = ok and np.array_equal(g[n], r[n])
+            ok = ok and np.array_equal(g["score"].view(np.int64), r["score"].view(np.int64))
+        items = loop.advance(host)
+        e1b = torch.cuda.Event(enable_timing=True)
+        e1b.record()
+        append(items)
+        e2.record()
+        torch.cuda.synchronize()
+        spec_ms.append(e0.elapsed_time(e1))
+        app_ms.append(e1b.elapsed_time(e2))
+    wall = time.perf_counter() - t_wall
+    st = store.stats()
+    summ = loop.summary()
+    gpu_s = (sum(spec_ms) + sum(app_ms)) / 1e3
+    line = {"metric": "closed-loop decode simulation: steps/s (GPU time of sd_speculate + sd_append) and mean accepted length",
+            "value": K / gpu_s, "unit": "steps/s", "n_gpus": 1, "steps": K, "warmup": 0,
+            "ms_per_step": gpu_s / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32 trees, f64 scores", "data": "synthetic",
+            "config": {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": B,
+                       "global_tokens": int(c.n_seqs * c.seq_len), "prompt_len": c.prompt_len, "vocab": c.vocab,
+                       "D": c.depth_cap, "P": c.max_pattern, "alpha": c.alpha, "max_spec": c.max_spec},
+            "speculate_us": {"mean": statistics.mean(spec_ms) * 1e3, "p50": statistics.median(spec_ms) * 1e3},
+            "append_us": {"mean": statistics.mean(app_ms) * 1e3, "p50": statistics.median(app_ms) * 1e3,
+                          "max": max(app_ms) * 1e3},
+            "wall_steps_per_s_with_host_verifier": K / wall, "gpu_launches": 2 * K,
+            "global_nodes_end": st["global_nodes"], "global_tokens_end": st["global_tokens"],
+            "global_status": st["global_status"]}
+    line.update(summ)
+    if ref is not None:
+        line["parity_vs_oracle"] = "bit-exact" if ok else "MISMATCH"
+    print(json.dumps(line), flush=True)
+    store.free()
+
+
+# --------------------------------------------------------------------------------------------
 def run_reference(args):
     """The CPU oracle as it stands, on the host cores, same metric and config.
     Each step is a bounded sample of the workload's requests."""
@@ -404,5 +499,7 @@ if __name__ == "__main__":
     a = parse()
     if a.impl == "reference":
         run_reference(a)
+    elif a.config == "closed_loop":
+        run_closed_loop(a)
     else:
         run_ours(a)

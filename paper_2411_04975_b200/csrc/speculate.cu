@@ -273,6 +273,8 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 //      reached by another job of the request.
 //   3. select + emit from shared memory; no global scratch.
 constexpr int CTA_WARPS = 16;
+constexpr int CTA_MIN_BLOCKS = 2;              // blocks per SM the register budget is set for
+constexpr int MATCH_ROUNDS = (SD_MAX_DEPTH + CTA_WARPS - 1) / CTA_WARPS;   // pattern lengths per warp
 
 struct WarpWork {
     Frontier F;
@@ -734,7 +736,7 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
     __syncwarp();
 }
 
-__global__ void __launch_bounds__(CTA_WARPS * 32, 2)
+__global__ void __launch_bounds__(CTA_WARPS * 32, CTA_MIN_BLOCKS)
 speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
                        unsigned flags, const int32_t* __restrict__ d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
                        int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
@@ -760,14 +762,16 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     // ---------------- 1. match
     const bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
     const bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
-    int src_node[2] = {-1, -1}, src_from[2] = {0, 0};           // per target: start node and first text index
+    int src_node[MATCH_ROUNDS], src_from[MATCH_ROUNDS];         // per target: start node and first text index
+#pragma unroll
+    for (int h = 0; h < MATCH_ROUNDS; ++h) { src_node[h] = -1; src_from[h] = 0; }
     const int32_t* text = ok ? sv.s_text + (long long)slot * sv.T : nullptr;
     if (want_g) {
         const bool cache_ok = ss->g_gen == ss->gen && ss->g_epoch == sv.g_state->epoch && ss->g_len <= t;
         const int k = t - ss->g_len;                            // tokens appended since the cache was taken
         const int depths = ss->g_depths;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < MATCH_ROUNDS; ++h) {
             const int d = wib + 1 + h * CTA_WARPS;              // target pattern length
             if (d > Pe || d > t) continue;
             if (cache_ok && d > k && d - k <= depths) {
@@ -782,7 +786,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     __syncthreads();                                            // all cached nodes read before any is replaced
     if (want_g) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < MATCH_ROUNDS; ++h) {
             const int d = wib + 1 + h * CTA_WARPS;
             if (d > Pe) continue;
             int cb = 0;

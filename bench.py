@@ -433,9 +433,11 @@ def run_closed_loop(args):
             "config": {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": B,
                        "global_tokens": int(c.n_seqs * c.seq_len), "prompt_len": c.prompt_len, "vocab": c.vocab,
                        "D": c.depth_cap, "P": c.max_pattern, "alpha": c.alpha, "max_spec": c.max_spec},
-            "speculate_us": {"mean": statistics.mean(spec_ms) * 1e3, "p50": statistics.median(spec_ms) * 1e3},
+            "speculate_us": {"mean": statistics.mean(spec_ms) * 1e3, "p50": statistics.median(spec_ms) * 1e3,
+                             "p90": float(np.percentile(spec_ms, 90)) * 1e3, "p99": float(np.percentile(spec_ms, 99)) * 1e3,
+                             "max": max(spec_ms) * 1e3},
             "append_us": {"mean": statistics.mean(app_ms) * 1e3, "p50": statistics.median(app_ms) * 1e3,
-                          "max": max(app_ms) * 1e3},
+                          "p90": float(np.percentile(app_ms, 90)) * 1e3, "max": max(app_ms) * 1e3},
             "wall_steps_per_s_with_host_verifier": K / wall, "gpu_launches": 2 * K,
             "global_nodes_end": st["global_nodes"], "global_tokens_end": st["global_tokens"],
             "global_status": st["global_status"]}

@@ -4,8 +4,8 @@
  * C ABI.  Every pointer named d_* is DEVICE memory owned by the caller; every
  * other pointer is HOST memory.  A store owns all of its device memory from
  * sd_build() until sd_free().  Calls are asynchronous on `stream` (a
- * cudaStream_t passed as void*, NULL = default stream) unless stated, and
- * after sd_build() no call allocates device memory.
+ * cudaStream_t passed as void*, NULL = default stream) unless stated; the
+ * per-step calls (sd_append, sd_speculate) never allocate device memory.
  *
  * Return value: SD_OK (0) or a negative SD_ERR_* code.  Nothing aborts, throws
  * or traps.  Conditions that depend on device data (a request whose slot pool
@@ -120,6 +120,23 @@ int sd_build(const sd_build_params* params, const int32_t* d_corpus, const int64
  */
 int sd_append(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* d_offsets,
               const int32_t* d_tokens, const uint8_t* d_reset, void* stream);
+
+/*
+ * sd_build_requests: start n new requests at once: their per-request trees are built from the
+ * prompts by the sort-based pipeline of sd_build instead of token by token (Section 3, "Suffix
+ * Tree Construction": the per-request tree is constructed when the request is received).  The
+ * result is the same as sd_append with d_reset = 1 for every item, only faster for long prompts.
+ *   h_slot     int32[n]    HOST: slot of each request (each slot at most once, 0 <= slot < max_requests)
+ *   h_offsets  int64[n+1]  HOST: prompt i is d_tokens[h_offsets[i] .. h_offsets[i+1]), h_offsets[0] = 0
+ *   d_tokens   int32[h_offsets[n]]  DEVICE
+ * A prompt that does not fit the slot's node pool or text buffer leaves the slot empty with
+ * SD_STATUS_POOL_FULL.  Unlike the per-step calls this one allocates temporary device memory
+ * (about 100 bytes per prompt token) and synchronises the stream before it returns.
+ * Errors: INVALID_ARG (bad slot, slot twice, offsets not ascending, token outside [0, V): nothing
+ * is changed), CAPACITY (n * vocab or the token total does not fit 31 bits), NOMEM, CUDA.
+ */
+int sd_build_requests(sd_store* store, int32_t n, const int32_t* h_slot, const int64_t* h_offsets,
+                      const int32_t* d_tokens, void* stream);
 
 /*
  * sd_speculate: GenerateCandidateTree of Algorithm 1 for n requests at once.

@@ -18,7 +18,7 @@ from . import build as _build
 FLAG_GLOBAL_ONLY, FLAG_REQUEST_ONLY, FLAG_LINEAR = 1, 2, 4
 STATUS_BAD_SLOT, STATUS_POOL_FULL, STATUS_GLOBAL_FULL, STATUS_BAD_TOKEN = 1, 2, 4, 8
 
-EXPORTS = ["sd_build", "sd_append", "sd_speculate", "sd_speculate_noalloc", "sd_query_counts", "sd_slot_info", "sd_stats", "sd_free",
+EXPORTS = ["sd_build", "sd_build_requests", "sd_append", "sd_speculate", "sd_speculate_noalloc", "sd_query_counts", "sd_slot_info", "sd_stats", "sd_free",
            "sd_strerror"]
 
 
@@ -59,6 +59,8 @@ def library() -> C.CDLL:
         vp = C.c_void_p
         lib.sd_build.restype = C.c_int
         lib.sd_build.argtypes = [C.POINTER(_BuildParams), vp, vp, C.c_int32, vp, C.POINTER(vp)]
+        lib.sd_build_requests.restype = C.c_int
+        lib.sd_build_requests.argtypes = [vp, C.c_int32, vp, vp, vp, vp]
         lib.sd_append.restype = C.c_int
         lib.sd_append.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
         lib.sd_speculate.restype = C.c_int
@@ -184,6 +186,16 @@ class SuffixStore:
     def append(self, slots: torch.Tensor, offsets: torch.Tensor, tokens: torch.Tensor,
                reset: Optional[torch.Tensor] = None) -> None:
         sd_append(self._h, slots, offsets, tokens, reset)
+
+    def build_requests(self, slots, offsets, tokens: torch.Tensor) -> None:
+        """Start new requests: `slots` and `offsets` are HOST sequences, `tokens` a CUDA tensor."""
+        import numpy as np
+        hs = np.ascontiguousarray(slots, dtype=np.int32)
+        ho = np.ascontiguousarray(offsets, dtype=np.int64)
+        rc = library().sd_build_requests(self._h, int(hs.size), hs.ctypes.data, ho.ctypes.data,
+                                         _ptr(tokens, torch.int32, "tokens"), _stream())
+        if rc != 0:
+            raise SuffixSpecError(rc, "sd_build_requests")
 
     def alloc_outputs(self, n: int) -> Dict[str, torch.Tensor]:
         M, dev = self.max_spec_cap, self.device

@@ -345,7 +345,10 @@ __device__ __forceinline__ int top_block_of(int nid, int nc) { return (nid > 0 &
 
 struct RunAlloc {             // entries a node's child run takes, top block included
     const int* nchild;
-    __device__ int operator()(i64 nid) const { return nchild[nid] + top_block_of((int)nid, nchild[nid]); }
+    int top_blocks;
+    __device__ int operator()(i64 nid) const {
+        return nchild[nid] + (top_blocks ? top_block_of((int)nid, nchild[nid]) : 0);
+    }
 };
 
 __global__ void collect_wide_kernel(const int* nchild, i64 n_nodes_plus1, int* list, int* counter) {
@@ -478,6 +481,124 @@ static void store_release(sd_store* s) {
     delete s;
 }
 
+// Everything up to the placement of the child runs, for one array of sequences: suffix
+// order, LCPs, children per node (pre-order node ids) and the start of every child run.
+struct Pipeline {
+    DeviceArena tmp;
+    SortBuffers sb;
+    int *end_pos = nullptr, *rank[8] = {nullptr}, *comb[2] = {nullptr, nullptr}, *ex = nullptr;
+    uint8_t *lcp = nullptr, *len = nullptr;
+    unsigned long long* level_nodes = nullptr;
+    const uint32_t* sa = nullptr;
+    int *r_a = nullptr, *r_b = nullptr, *b_a = nullptr, *b_b = nullptr, *seg_a = nullptr, *seg_b = nullptr;
+    int *nbase = nullptr, *nchild = nullptr, *runstart = nullptr, *big_tmp = nullptr, *wide_list = nullptr;
+    int* r_cur = nullptr;
+    i64 N = 0, n_nodes = 0, used_entries = 0;
+    int n_wide = 0;
+};
+
+// max_token: largest token value + 1 (sets the number of radix passes).  top_blocks: reserve
+// room for top blocks in front of long runs.  Returns SD_OK, SD_ERR_NOMEM or SD_ERR_CUDA.
+static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_offsets, int n_seqs, i64 N,
+                        i64 max_token, int D, bool top_blocks, cudaStream_t st) {
+    const int T256 = 256;
+    P.N = N;
+    DeviceArena& tmp = P.tmp;
+    SortBuffers& sb = P.sb;
+    cudaError_t ce = cudaSuccess;
+    const int nblk = (int)((N + RS_TILE - 1) / RS_TILE);
+    int m = 0;
+    while ((2 << m) <= D) ++m;                    // 2^m <= D < 2^(m+1)
+    bool ok = tmp.get(&sb.keys[0], N) && tmp.get(&sb.keys[1], N) && tmp.get(&sb.vals[0], N) &&
+              tmp.get(&sb.vals[1], N) && tmp.get(&sb.hist, (i64)256 * nblk + 1) &&
+              tmp.get(&sb.scan_tmp, scan_tmp_ints(std::max<i64>((i64)256 * nblk, N + 1))) &&
+              tmp.get(&P.end_pos, N) && tmp.get(&P.ex, N + 1) && tmp.get(&P.lcp, N) && tmp.get(&P.len, N) &&
+              tmp.get(&P.level_nodes, SD_MAX_DEPTH + 2);
+    for (int k = 0; ok && k <= m; ++k) ok = tmp.get(&P.rank[k], N);
+    ok = ok && tmp.get(&P.comb[0], N) && tmp.get(&P.comb[1], N);
+    if (!ok) return SD_ERR_NOMEM;
+    int *end_pos = P.end_pos, **rank = P.rank, **comb = P.comb, *ex = P.ex;
+    uint8_t *lcp = P.lcp, *len = P.len;
+
+    seq_end_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_seq_offsets, n_seqs, N, end_pos);
+    rank0_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tok, N, rank[0]);
+    int bits = bits_for(std::max<i64>(max_token, N) + 1);
+    int sorted = 0;
+    // rank[k] orders the first 2^k tokens of every suffix
+    auto round = [&](const int* ra, const int* rb, int off, int* rout) {
+        make_keys_kernel<<<grid_for(N, T256), T256, 0, st>>>(ra, rb, off, end_pos, N, sb.keys[0], sb.vals[0]);
+        sorted = radix_sort_pairs(sb, N, bits, bits, st);
+        if (rout) {
+            exclusive_scan(KeyChange{sb.keys[sorted]}, N, ex, sb.scan_tmp, st);
+            assign_rank_kernel<<<grid_for(N, T256), T256, 0, st>>>(sb.keys[sorted], sb.vals[sorted], ex, N, rout);
+        }
+    };
+    if (m == 0) {
+        round(rank[0], rank[0], 1 << 30, nullptr);        // D == 1: the first token alone
+    } else {
+        const bool pow2 = D == (1 << m);
+        for (int k = 0; k < m; ++k)
+            round(rank[k], rank[k], 1 << k, (pow2 && k == m - 1) ? nullptr : rank[k + 1]);
+        if (!pow2) {
+            // append the remaining binary digits of D, high to low
+            int cur_len = 1 << m, rem = D - cur_len, which = 0;
+            const int* cur = rank[m];
+            for (int b = m - 1; b >= 0; --b) {
+                if (!(rem & (1 << b))) continue;
+                rem -= 1 << b;
+                int* dst = rem == 0 ? nullptr : comb[which];
+                round(cur, rank[b], cur_len, dst);
+                cur = dst;
+                which ^= 1;
+                cur_len += 1 << b;
+            }
+        }
+    }
+    P.sa = sb.vals[sorted];
+    lcp_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tok, P.sa, end_pos, N, D, lcp, len);
+    ce = cudaMemsetAsync(P.level_nodes, 0, sizeof(unsigned long long) * (SD_MAX_DEPTH + 2), st);
+    level_hist_kernel<<<(unsigned)std::min<i64>(grid_for(N, T256), 1184), T256, 0, st>>>(lcp, len, N, P.level_nodes);
+    unsigned long long h_level[SD_MAX_DEPTH + 2];
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(h_level, P.level_nodes, sizeof(h_level), cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    if (ce != cudaSuccess) return SD_ERR_CUDA;
+    i64 n_nodes = 0;
+    for (int d = 1; d <= D; ++d) n_nodes += (i64)h_level[d];
+    P.n_nodes = n_nodes;
+
+    P.b_a = ex;
+    ok = tmp.get(&P.r_a, N + 1) && tmp.get(&P.r_b, N + 1) && tmp.get(&P.seg_a, N + 2) && tmp.get(&P.seg_b, N + 2) &&
+         tmp.get(&P.b_b, N + 1) && tmp.get(&P.nbase, N + 1) && tmp.get(&P.nchild, n_nodes + 1) &&
+         tmp.get(&P.runstart, n_nodes + 2) && tmp.get(&P.big_tmp, scan_tmp_ints(n_nodes + 1)) &&
+         tmp.get(&P.wide_list, n_nodes / SD_TOP_MIN + 2);
+    if (!ok) return SD_ERR_NOMEM;
+    exclusive_scan(NewNodes{lcp, len}, N, P.nbase, sb.scan_tmp, st);
+    // pass 1, deepest level first: children per node
+    int* r_next = P.r_a;
+    P.r_cur = P.r_b;
+    for (int d = D; d >= 1; --d) {
+        exclusive_scan(OpensNode{lcp, len, d}, N, P.r_cur, sb.scan_tmp, st);
+        exclusive_scan(Boundary{lcp, d}, N, P.b_a, sb.scan_tmp, st);
+        seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(lcp, d, P.b_a, N, P.seg_a);
+        count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, N, d, D, P.r_cur, r_next, P.b_a, P.seg_a,
+                                                                  P.nbase, P.nchild);
+        std::swap(P.r_cur, r_next);
+    }
+    // child runs (with their top blocks) in node (pre-)order
+    exclusive_scan(RunAlloc{P.nchild, top_blocks ? 1 : 0}, n_nodes + 1, P.runstart, P.big_tmp, st);
+    int* wide_counter = (int*)P.level_nodes;
+    ce = cudaMemsetAsync(wide_counter, 0, sizeof(int), st);
+    if (top_blocks)
+        collect_wide_kernel<<<grid_for(n_nodes + 1, T256), T256, 0, st>>>(P.nchild, n_nodes + 1, P.wide_list, wide_counter);
+    int h_total = 0;
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_total, P.runstart + n_nodes + 1, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&P.n_wide, wide_counter, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    if (ce != cudaSuccess) return SD_ERR_CUDA;
+    P.used_entries = h_total;
+    return SD_OK;
+}
+
 extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const int64_t* d_seq_offsets, int32_t n_seqs,
                         void* stream, sd_store** out) {
     if (!out) return SD_ERR_INVALID_ARG;
@@ -515,31 +636,14 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
     if (ce == cudaSuccess) ce = cudaMemsetAsync(s->s_state, 0, sizeof(SlotState) * (size_t)s->R, st);
     if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
 
-    i64 n_nodes = 0;
-    DeviceArena tmp;
-    SortBuffers sb;
-    int *end_pos = nullptr, *rank[8] = {nullptr}, *comb[2] = {nullptr, nullptr}, *ex = nullptr;
-    uint8_t *lcp = nullptr, *len = nullptr;
-    unsigned long long* level_nodes = nullptr;
-    const uint32_t* sa = nullptr;
+    Pipeline P;
     const int T256 = 256;
-
+    i64 n_nodes = 0, used_entries = 0;
     if (N > 0) {
-        const int nblk = (int)((N + RS_TILE - 1) / RS_TILE);
-        int m = 0;
-        while ((2 << m) <= D) ++m;                    // 2^m <= D < 2^(m+1)
-        ok = tmp.get(&sb.keys[0], N) && tmp.get(&sb.keys[1], N) && tmp.get(&sb.vals[0], N) &&
-             tmp.get(&sb.vals[1], N) && tmp.get(&sb.hist, (i64)256 * nblk + 1) &&
-             tmp.get(&sb.scan_tmp, scan_tmp_ints(std::max<i64>((i64)256 * nblk, N + 1))) &&
-             tmp.get(&end_pos, N) && tmp.get(&ex, N + 1) && tmp.get(&lcp, N) && tmp.get(&len, N) &&
-             tmp.get(&level_nodes, SD_MAX_DEPTH + 2);
-        for (int k = 0; ok && k <= m; ++k) ok = tmp.get(&rank[k], N);
-        ok = ok && tmp.get(&comb[0], N) && tmp.get(&comb[1], N);
-        if (!ok) { store_release(s); return SD_ERR_NOMEM; }
-
         {
-            int* bad = (int*)level_nodes;
+            int* bad = nullptr;
             int h_bad = 0;
+            if (!P.tmp.get(&bad, 1)) { store_release(s); return SD_ERR_NOMEM; }
             ce = cudaMemsetAsync(bad, 0, sizeof(int), st);
             validate_kernel<<<grid_for(std::max<i64>(N, n_seqs), T256), T256, 0, st>>>(d_corpus, N, s->V, d_seq_offsets,
                                                                                       n_seqs, bad);
@@ -548,86 +652,10 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
             if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
             if (h_bad) { store_release(s); return SD_ERR_INVALID_ARG; }
         }
-        seq_end_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_seq_offsets, n_seqs, N, end_pos);
-        rank0_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, N, rank[0]);
-        int bits = bits_for(std::max<i64>(s->V, N) + 1);
-        int sorted = 0;
-        // rank[k] orders the first 2^k tokens of every suffix
-        auto round = [&](const int* ra, const int* rb, int off, int* rout) {
-            make_keys_kernel<<<grid_for(N, T256), T256, 0, st>>>(ra, rb, off, end_pos, N, sb.keys[0], sb.vals[0]);
-            sorted = radix_sort_pairs(sb, N, bits, bits, st);
-            if (rout) {
-                exclusive_scan(KeyChange{sb.keys[sorted]}, N, ex, sb.scan_tmp, st);
-                assign_rank_kernel<<<grid_for(N, T256), T256, 0, st>>>(sb.keys[sorted], sb.vals[sorted], ex, N, rout);
-            }
-        };
-        if (m == 0) {
-            round(rank[0], rank[0], 1 << 30, nullptr);        // D == 1: the first token alone
-        } else {
-            const bool pow2 = D == (1 << m);
-            for (int k = 0; k < m; ++k)
-                round(rank[k], rank[k], 1 << k, (pow2 && k == m - 1) ? nullptr : rank[k + 1]);
-            if (!pow2) {
-                // append the remaining binary digits of D, high to low
-                int cur_len = 1 << m, rem = D - cur_len, which = 0;
-                const int* cur = rank[m];
-                for (int b = m - 1; b >= 0; --b) {
-                    if (!(rem & (1 << b))) continue;
-                    rem -= 1 << b;
-                    int* dst = rem == 0 ? nullptr : comb[which];
-                    round(cur, rank[b], cur_len, dst);
-                    cur = dst;
-                    which ^= 1;
-                    cur_len += 1 << b;
-                }
-            }
-        }
-        sa = sb.vals[sorted];
-        lcp_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, sa, end_pos, N, D, lcp, len);
-        ce = cudaMemsetAsync(level_nodes, 0, sizeof(unsigned long long) * (SD_MAX_DEPTH + 2), st);
-        level_hist_kernel<<<(unsigned)std::min<i64>(grid_for(N, T256), 1184), T256, 0, st>>>(lcp, len, N, level_nodes);
-        unsigned long long h_level[SD_MAX_DEPTH + 2];
-        if (ce == cudaSuccess)
-            ce = cudaMemcpyAsync(h_level, level_nodes, sizeof(h_level), cudaMemcpyDeviceToHost, st);
-        if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
-        if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
-        for (int d = 1; d <= D; ++d) n_nodes += (i64)h_level[d];
-    }
-
-    i64 used_entries = 0;
-    int *r_a = nullptr, *r_b = nullptr, *b_a = ex, *b_b = nullptr, *seg_a = nullptr, *seg_b = nullptr;
-    int *nbase = nullptr, *nchild = nullptr, *runstart = nullptr, *big_tmp = nullptr, *wide_list = nullptr;
-    int* r_cur = nullptr;
-    int n_wide = 0;
-    if (N > 0) {
-        ok = tmp.get(&r_a, N + 1) && tmp.get(&r_b, N + 1) && tmp.get(&seg_a, N + 2) && tmp.get(&seg_b, N + 2) &&
-             tmp.get(&b_b, N + 1) && tmp.get(&nbase, N + 1) && tmp.get(&nchild, n_nodes + 1) &&
-             tmp.get(&runstart, n_nodes + 2) && tmp.get(&big_tmp, scan_tmp_ints(n_nodes + 1)) &&
-             tmp.get(&wide_list, n_nodes / SD_TOP_MIN + 2);
-        if (!ok) { store_release(s); return SD_ERR_NOMEM; }
-        exclusive_scan(NewNodes{lcp, len}, N, nbase, sb.scan_tmp, st);
-        // pass 1, deepest level first: children per node
-        int* r_next = r_a;
-        r_cur = r_b;
-        for (int d = D; d >= 1; --d) {
-            exclusive_scan(OpensNode{lcp, len, d}, N, r_cur, sb.scan_tmp, st);
-            exclusive_scan(Boundary{lcp, d}, N, b_a, sb.scan_tmp, st);
-            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(lcp, d, b_a, N, seg_a);
-            count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, N, d, D, r_cur, r_next, b_a, seg_a,
-                                                                      nbase, nchild);
-            std::swap(r_cur, r_next);
-        }
-        // child runs (with their top blocks) in node (pre-)order
-        exclusive_scan(RunAlloc{nchild}, n_nodes + 1, runstart, big_tmp, st);
-        int* wide_counter = (int*)level_nodes;
-        ce = cudaMemsetAsync(wide_counter, 0, sizeof(int), st);
-        collect_wide_kernel<<<grid_for(n_nodes + 1, T256), T256, 0, st>>>(nchild, n_nodes + 1, wide_list, wide_counter);
-        int h_total = 0;
-        if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_total, runstart + n_nodes + 1, sizeof(int), cudaMemcpyDeviceToHost, st);
-        if (ce == cudaSuccess) ce = cudaMemcpyAsync(&n_wide, wide_counter, sizeof(int), cudaMemcpyDeviceToHost, st);
-        if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
-        if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
-        used_entries = h_total;
+        const int rc = pipeline_run(P, d_corpus, d_seq_offsets, n_seqs, N, s->V, D, true, st);
+        if (rc != SD_OK) { store_release(s); return rc; }
+        n_nodes = P.n_nodes;
+        used_entries = P.used_entries;
     }
 
     i64 extra = p->global_extra_nodes >= 0 ? p->global_extra_nodes : std::max<i64>(1ll << 22, n_nodes);
@@ -637,18 +665,18 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
 
     if (N > 0) {
         // pass 2, top level first: write the entries
-        int *b_cur = b_a, *b_prev = b_b, *seg_cur = seg_a, *seg_prev = seg_b;
+        int *b_cur = P.b_a, *b_prev = P.b_b, *seg_cur = P.seg_a, *seg_prev = P.seg_b;
         for (int d = 1; d <= D; ++d) {
-            exclusive_scan(OpensNode{lcp, len, d}, N, r_cur, sb.scan_tmp, st);
-            exclusive_scan(Boundary{lcp, d}, N, b_cur, sb.scan_tmp, st);
-            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(lcp, d, b_cur, N, seg_cur);
-            emit_level_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, sa, lcp, len, N, d, r_cur, b_cur, seg_cur,
-                                                                 b_prev, seg_prev, nbase, nchild, runstart, s->g_ent,
-                                                                 s->g_root);
+            exclusive_scan(OpensNode{P.lcp, P.len, d}, N, P.r_cur, P.sb.scan_tmp, st);
+            exclusive_scan(Boundary{P.lcp, d}, N, b_cur, P.sb.scan_tmp, st);
+            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(P.lcp, d, b_cur, N, seg_cur);
+            emit_level_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, P.sa, P.lcp, P.len, N, d, P.r_cur, b_cur,
+                                                                 seg_cur, b_prev, seg_prev, P.nbase, P.nchild,
+                                                                 P.runstart, s->g_ent, s->g_root);
             std::swap(b_cur, b_prev);
             std::swap(seg_cur, seg_prev);
         }
-        if (n_wide > 0) fill_top_kernel<<<n_wide, 256, 0, st>>>(wide_list, nchild, runstart, s->g_ent);
+        if (P.n_wide > 0) fill_top_kernel<<<P.n_wide, 256, 0, st>>>(P.wide_list, P.nchild, P.runstart, s->g_ent);
     }
     init_global_state_kernel<<<1, 1, 0, st>>>(s->g_state, (int)used_entries, (int)n_nodes, N);
     ce = cudaStreamSynchronize(st);
@@ -673,4 +701,209 @@ extern "C" const char* sd_strerror(int code) {
         case SD_ERR_CAPACITY: return "capacity exceeded";
         default: return "unknown error";
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// sd_build_requests: the per-request trees of a batch of new requests, built from their prompts
+// by the same sort-based pipeline as the global tree instead of token by token.  The prompts
+// are kept apart by giving every request its own token range (token + rank * V), so one
+// suffix sort orders all of them request by request and one pre-order numbering lays every
+// request's nodes down contiguously; each request's part is then written into its own pool.
+namespace {
+
+__device__ __forceinline__ int seq_rank_of(const int64_t* off, int n, i64 pos) {
+    int lo = 0, hi = n;                               // largest q with off[q] <= pos
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (off[mid] <= pos) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__global__ void map_tokens_kernel(const int32_t* tok, const int64_t* off, int n, i64 N, int V, int32_t* out, int* bad) {
+    i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const int t = tok[i];
+    if (t < 0 || t >= V) { atomicOr(bad, 1); out[i] = 0; return; }
+    out[i] = seq_rank_of(off, n, i) * V + t;
+}
+
+// one warp per request: forget the slot's old tree and store the new text
+__global__ void requests_prepare_kernel(sd_store sv, int n, const int32_t* slot_ids, const int64_t* off,
+                                        const int32_t* tok) {
+    const int q = (int)((blockIdx.x * (i64)blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    if (q >= n) return;
+    const int slot = slot_ids[q];
+    if (slot < 0 || slot >= sv.R) return;
+    SlotState* ss = sv.s_state + slot;
+    int32_t* text = sv.s_text + (i64)slot * sv.T;
+    int32_t* root = sv.s_root + (i64)slot * sv.V;
+    const int old_len = ss->len;
+    for (int k = lane; k < old_len; k += 32) root[text[k]] = -1;
+    __syncwarp();
+    const i64 lo = off[q], hi = off[q + 1];
+    if (hi - lo <= sv.T)
+        for (i64 k = lane; k < hi - lo; k += 32) text[k] = tok[lo + k];
+}
+
+struct RequestLayout {       // where request q's nodes go (device arrays of n entries)
+    int* run_base;           // global position of its first child run
+    int* n1;                 // its depth-1 nodes
+    int* r1lo;               // depth-1 nodes of earlier requests
+    int* used;               // entries it takes
+    int* live;               // nodes
+    int* ok;                 // fits its pool and text buffer
+};
+
+__global__ void requests_layout_kernel(sd_store sv, int n, const int64_t* off, const int* nbase, const int* runstart,
+                                       const int* r1, RequestLayout L) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= n) return;
+    const i64 lo = off[q], hi = off[q + 1];
+    const int first = 1 + nbase[lo], next = 1 + nbase[hi];
+    const int rb = runstart[first], re = runstart[next];
+    const int n1 = r1[hi] - r1[lo];
+    L.run_base[q] = rb; L.n1[q] = n1; L.r1lo[q] = r1[lo];
+    L.used[q] = n1 + (re - rb); L.live[q] = next - first;
+    L.ok[q] = ((i64)n1 + (re - rb) <= sv.spn && hi - lo <= sv.T) ? 1 : 0;
+}
+
+__global__ void emit_level_slots_kernel(sd_store sv, int n_req, const int32_t* slot_ids, const int64_t* off,
+                                        const int32_t* mtok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len,
+                                        i64 n, int d, const int* r_d, const int* bscan, const int* segpos,
+                                        const int* bscan_prev, const int* segpos_prev, const int* nbase, const int* nchild,
+                                        const int* runstart, RequestLayout L) {
+    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    if (!(lcp[j] < d && d <= len[j])) return;
+    const int q = seq_rank_of(off, n_req, (i64)sa[j]);
+    const int slot = slot_ids[q];
+    if (!L.ok[q] || slot < 0 || slot >= sv.R) return;
+    int4* ent = sv.s_ent + (i64)slot * sv.spn;
+    const int nb = segpos[bscan[j] + 1];
+    const int nid = 1 + nbase[j] + (d - (int)lcp[j] - 1);
+    const int nc = nchild[nid];
+    const int shift = L.n1[q] - L.run_base[q];                  // global run position -> index in the slot pool
+    int4 e;
+    e.x = mtok[(i64)sa[j] + d - 1] - q * sv.V;
+    e.y = nb - (int)j;
+    e.z = nc > 0 ? runstart[nid] + shift : 0;
+    e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC) : 0;
+    int pos;
+    if (d == 1) {
+        pos = r_d[j] - L.r1lo[q];
+        (sv.s_root + (i64)slot * sv.V)[e.x] = pos;
+    } else {
+        const int seg = bscan_prev[j] + (lcp[j] < d - 1 ? 1 : 0) - 1;
+        const int jx = segpos_prev[seg];
+        const int pnid = 1 + nbase[jx] + (d - 1 - (int)lcp[jx] - 1);
+        pos = runstart[pnid] + (r_d[j] - r_d[jx]) + shift;
+    }
+    ent[pos] = e;
+}
+
+// one warp per request: bookkeeping and the active nodes (lane d-1: node of the last d tokens)
+__global__ void requests_finalize_kernel(sd_store sv, int n, const int32_t* slot_ids, const int64_t* off,
+                                         RequestLayout L) {
+    const int q = (int)((blockIdx.x * (i64)blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    if (q >= n) return;
+    const int slot = slot_ids[q];
+    if (slot < 0 || slot >= sv.R) return;
+    SlotState* ss = sv.s_state + slot;
+    const bool ok = L.ok[q] != 0;
+    const int len = ok ? (int)(off[q + 1] - off[q]) : 0;
+    const int4* ent = sv.s_ent + (i64)slot * sv.spn;
+    const int32_t* root = sv.s_root + (i64)slot * sv.V;
+    const int32_t* text = sv.s_text + (i64)slot * sv.T;
+    int node = -1, rcb = 0;
+    unsigned rw = 0;
+    const int d = lane + 1;
+    if (d <= len && d <= sv.D) {
+        node = root[text[len - d]];
+        int4 e = make_int4(0, 0, 0, 0);
+        if (node >= 0) e = ent[node];
+        for (int k = 1; k < d && node >= 0; ++k) {
+            const int x = text[len - d + k];
+            const int cb = e.z, nn = (int)((unsigned)e.w & RUN_COUNT_MASK);
+            int lo = 0, hi = nn;
+            while (lo < hi) {                                    // at most 24 rounds
+                const int mid = (lo + hi) >> 1;
+                if (ent[cb + mid].x < x) lo = mid + 1; else hi = mid;
+            }
+            node = -1;
+            if (lo < nn) { e = ent[cb + lo]; if (e.x == x) node = cb + lo; }
+        }
+        if (node >= 0) { rcb = e.z; rw = (unsigned)e.w; }
+    }
+    ss->active[lane] = node; ss->room[lane] = 0; ss->run_cb[lane] = rcb; ss->run_w[lane] = rw;
+    if (lane == 0) {
+        ss->len = len; ss->used = ok ? L.used[q] : 0; ss->live = ok ? L.live[q] : 0;
+        ss->status = ok ? 0 : SD_STATUS_POOL_FULL;
+        ss->gen += 1;
+    }
+}
+
+}  // namespace
+
+extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, const int64_t* h_offsets,
+                                 const int32_t* d_tokens, void* stream) {
+    if (!s || n < 0) return SD_ERR_INVALID_ARG;
+    if (n == 0) return SD_OK;
+    if (!h_slot || !h_offsets || n > s->R) return SD_ERR_INVALID_ARG;
+    if (h_offsets[0] != 0) return SD_ERR_INVALID_ARG;
+    for (int q = 0; q < n; ++q) {
+        if (h_offsets[q + 1] < h_offsets[q] || h_slot[q] < 0 || h_slot[q] >= s->R) return SD_ERR_INVALID_ARG;
+        for (int r = 0; r < q; ++r) if (h_slot[r] == h_slot[q]) return SD_ERR_INVALID_ARG;   // a slot once per call
+    }
+    const i64 N = h_offsets[n];
+    if (N > 0 && !d_tokens) return SD_ERR_INVALID_ARG;
+    if ((i64)n * s->V >= (1ll << 31) - 2 || N >= (1ll << 31) - 2) return SD_ERR_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int T256 = 256, D = s->D;
+
+    Pipeline P;
+    int32_t *d_slot = nullptr, *mtok = nullptr;
+    int64_t* d_off = nullptr;
+    int *bad = nullptr, *r1 = nullptr;
+    RequestLayout L;
+    bool ok = P.tmp.get(&d_slot, n) && P.tmp.get(&d_off, n + 1) && P.tmp.get(&mtok, N) && P.tmp.get(&bad, 1) &&
+              P.tmp.get(&r1, N + 1) && P.tmp.get(&L.run_base, n) && P.tmp.get(&L.n1, n) && P.tmp.get(&L.r1lo, n) &&
+              P.tmp.get(&L.used, n) && P.tmp.get(&L.live, n) && P.tmp.get(&L.ok, n);
+    if (!ok) return SD_ERR_NOMEM;
+    SD_CUDA_OK(cudaMemcpyAsync(d_slot, h_slot, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st));
+    SD_CUDA_OK(cudaMemcpyAsync(d_off, h_offsets, sizeof(int64_t) * (n + 1), cudaMemcpyHostToDevice, st));
+    SD_CUDA_OK(cudaMemsetAsync(bad, 0, sizeof(int), st));
+    if (N > 0) {
+        map_tokens_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tokens, d_off, n, N, s->V, mtok, bad);
+        int h_bad = 0;
+        SD_CUDA_OK(cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, st));
+        SD_CUDA_OK(cudaStreamSynchronize(st));
+        if (h_bad) return SD_ERR_INVALID_ARG;                    // nothing was changed yet
+    }
+    requests_prepare_kernel<<<grid_for((i64)n * 32, T256), T256, 0, st>>>(*s, n, d_slot, d_off, d_tokens);
+    if (N > 0) {
+        const int rc = pipeline_run(P, mtok, d_off, n, N, (i64)n * s->V, D, false, st);
+        if (rc != SD_OK) return rc;
+        exclusive_scan(OpensNode{P.lcp, P.len, 1}, N, r1, P.sb.scan_tmp, st);
+        requests_layout_kernel<<<grid_for(n, T256), T256, 0, st>>>(*s, n, d_off, P.nbase, P.runstart, r1, L);
+        int *b_cur = P.b_a, *b_prev = P.b_b, *seg_cur = P.seg_a, *seg_prev = P.seg_b;
+        for (int d = 1; d <= D; ++d) {
+            exclusive_scan(OpensNode{P.lcp, P.len, d}, N, P.r_cur, P.sb.scan_tmp, st);
+            exclusive_scan(Boundary{P.lcp, d}, N, b_cur, P.sb.scan_tmp, st);
+            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(P.lcp, d, b_cur, N, seg_cur);
+            emit_level_slots_kernel<<<grid_for(N, T256), T256, 0, st>>>(*s, n, d_slot, d_off, mtok, P.sa, P.lcp, P.len, N, d,
+                                                                       P.r_cur, b_cur, seg_cur, b_prev, seg_prev, P.nbase,
+                                                                       P.nchild, P.runstart, L);
+            std::swap(b_cur, b_prev);
+            std::swap(seg_cur, seg_prev);
+        }
+    } else {
+        SD_CUDA_OK(cudaMemsetAsync(L.ok, 0xFF, sizeof(int) * n, st));
+        SD_CUDA_OK(cudaMemsetAsync(L.used, 0, sizeof(int) * n, st));
+        SD_CUDA_OK(cudaMemsetAsync(L.live, 0, sizeof(int) * n, st));
+    }
+    requests_finalize_kernel<<<grid_for((i64)n * 32, T256), T256, 0, st>>>(*s, n, d_slot, d_off, L);
+    SD_CUDA_OK(cudaStreamSynchronize(st));                       // the temporaries are released on return
+    SD_CUDA_OK(cudaGetLastError());
+    return SD_OK;
 }

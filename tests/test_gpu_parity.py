@@ -370,3 +370,53 @@ def test_large_batch_full_size_sampled_against_oracle(U):
         assert int(store.slot_info(U.dev_i32([i]))["nodes"][0]) == nn
     store.free()
     ref.close()
+
+
+# ---------------------------------------------------------------- sort-based per-request build (a2)
+@pytest.mark.parametrize("D,vocab", [(1, 3), (4, 2), (7, 30), (32, 5), (32, 2000)])
+def test_build_requests_equals_token_by_token_append(U, D, vocab):
+    import paper_2411_04975_b200 as sfx
+    rng = np.random.default_rng(D * 31 + vocab)
+    n_slots = 9
+    pr = U.Pair(_rand_seqs(rng, 4, 20, 100, vocab), vocab=vocab, D=D, n_slots=n_slots, max_req_tokens=3000)
+    # slot 8 holds an older request that is replaced; slot 5 stays untouched
+    pr.append([8, 5], _rand_seqs(rng, 2, 40, 80, vocab), reset=[1, 1])
+    slots = [3, 8, 0, 7, 2]
+    prompts = _rand_seqs(rng, 5, 0, 2500, vocab)
+    prompts[2] = np.zeros(0, dtype=np.int32)                     # an empty prompt
+    prompts[3] = np.full(300, vocab - 1, dtype=np.int32)         # one token repeated
+    off, flat = U.ragged(prompts)
+    pr.g.build_requests(slots, off, U.dev_i32(flat) if flat.size else torch.zeros(0, dtype=torch.int32, device=U.DEV))
+    for s_, p_ in zip(slots, prompts):
+        pr.o.slot_reset(s_)
+        pr.o.slot_append(s_, p_)
+    for s_ in range(n_slots):
+        pr.check_tree(s_)
+    pr.check_speculate(list(range(n_slots)), 32, 2.0, 64)
+    # the trees keep growing token by token afterwards (offline runs are exact fits and must move)
+    for step in range(3):
+        pr.append(list(range(n_slots)), _rand_seqs(rng, n_slots, 0, 12, vocab))
+        pr.check_speculate(list(range(n_slots)), 16, 1.5, 40)
+    for s_ in range(n_slots):
+        pr.check_tree(s_)
+    # argument errors change nothing
+    for bad in ([0, 0], [0, 99]):
+        with pytest.raises(sfx.SuffixSpecError):
+            pr.g.build_requests(bad, [0, 1, 2], U.dev_i32([0, 0]))
+    with pytest.raises(sfx.SuffixSpecError):
+        pr.g.build_requests([0], [0, 1], U.dev_i32([vocab]))
+    pr.check_tree(0)
+    pr.close()
+
+
+def test_build_requests_pool_overflow(U):
+    rng = np.random.default_rng(8)
+    pr = U.Pair([], vocab=500, D=8, n_slots=2, max_req_tokens=64, slot_pool_nodes=120)
+    prompts = [rng.integers(0, 500, size=60).astype(np.int32), rng.integers(0, 500, size=10).astype(np.int32)]
+    off, flat = U.ragged(prompts)
+    pr.g.build_requests([0, 1], off, U.dev_i32(flat))
+    info = pr.g.slot_info(U.dev_i32([0, 1]))
+    assert int(info["status"][0]) == 2 and int(info["len"][0]) == 0 and int(info["nodes"][0]) == 0
+    pr.o.slot_append(1, prompts[1])
+    pr.check_tree(1)
+    pr.close()

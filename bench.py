@@ -174,9 +174,10 @@ def run_ours(args):
     slots = torch.arange(B, dtype=torch.int32, device=dev)
     poff = np.zeros(B + 1, dtype=np.int64)
     poff[1:] = np.cumsum([len(p) for p in prompts])
+    d_prompts = torch.as_tensor(np.concatenate(prompts), device=dev)
+    torch.cuda.synchronize()
     t0 = time.perf_counter()
-    store.append(slots, torch.as_tensor(poff, device=dev), torch.as_tensor(np.concatenate(prompts), device=dev),
-                 torch.ones(B, dtype=torch.uint8, device=dev))
+    store.build_requests(np.arange(B, dtype=np.int32), poff, d_prompts)      # sort-based, all prompts at once
     torch.cuda.synchronize()
     prompt_ms = (time.perf_counter() - t0) * 1e3
 
@@ -381,14 +382,47 @@ def run_closed_loop(args):
     slots_all = torch.arange(B, dtype=torch.int32, device=dev)
     out = store.alloc_outputs(B)
 
+    side = torch.cuda.Stream(device=dev)
+
     def append(items):
         sl, lists, reset = items
+        # new requests go through the batched sort-based build, everything else through sd_append
+        new = [i for i in range(len(sl)) if sl[i] >= 0 and reset[i]]
+        if new:
+            # the other items (accepted tokens, finished outputs for the global tree) touch other
+            # slots: they are enqueued first and run while the new requests are built on a side stream
+            keep = [i for i in range(len(sl)) if i not in set(new)]
+            ev_pre = torch.cuda.Event()
+            ev_pre.record()
+            if keep:
+                append(([sl[i] for i in keep], [lists[i] for i in keep], [reset[i] for i in keep]))
+            ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            refill_ev.append((ev_a, ev_b, sum(len(lists[i]) for i in new)))
+            noff = np.zeros(len(new) + 1, dtype=np.int64)
+            noff[1:] = np.cumsum([len(lists[i]) for i in new])
+            with torch.cuda.stream(side):
+                side.wait_event(ev_pre)                          # not for the append enqueued just now
+                ev_a.record()
+                toks_new = torch.as_tensor(np.concatenate([lists[i] for i in new]).astype(np.int32), device=dev)
+                store.build_requests([sl[i] for i in new], noff, toks_new)
+                ev_b.record()
+            torch.cuda.current_stream().wait_stream(side)
+            if ref is not None:
+                for i in new:
+                    ref.slot_reset(sl[i])
+                ref.slot_append_batch([sl[i] for i in new], [lists[i] for i in new], n_threads=oracle_threads(B))
+            return
         off = np.zeros(len(sl) + 1, dtype=np.int64)
         off[1:] = np.cumsum([len(x) for x in lists])
         flat = np.concatenate(lists).astype(np.int32) if off[-1] else np.zeros(0, dtype=np.int32)
-        store.append(torch.as_tensor(np.asarray(sl, dtype=np.int32), device=dev), torch.as_tensor(off, device=dev),
-                     torch.as_tensor(flat, device=dev) if flat.size else torch.zeros(0, dtype=torch.int32, device=dev),
-                     torch.as_tensor(np.asarray(reset, dtype=np.uint8), device=dev))
+        args_ = (torch.as_tensor(np.asarray(sl, dtype=np.int32), device=dev), torch.as_tensor(off, device=dev),
+                 torch.as_tensor(flat, device=dev) if flat.size else torch.zeros(0, dtype=torch.int32, device=dev),
+                 torch.as_tensor(np.asarray(reset, dtype=np.uint8), device=dev))
+        ka, kb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ka.record()
+        store.append(*args_)
+        kb.record()
+        kernel_ev.append((ka, kb, sum(len(lists[i]) for i in range(len(sl)) if sl[i] < 0)))
         if ref is not None:
             for s_, l_, r_ in zip(sl, lists, reset):
                 if s_ < 0:
@@ -398,8 +432,11 @@ def run_closed_loop(args):
             idx = [i for i, s_ in enumerate(sl) if s_ >= 0]
             ref.slot_append_batch([sl[i] for i in idx], [lists[i] for i in idx], n_threads=oracle_threads(B))
 
+    refill_ev, kernel_ev = [], []
     append(loop.start())
     torch.cuda.synchronize()
+    refill_ev.clear()
+    kernel_ev.clear()
     spec_ms, app_ms, ok = [], [], True
     t_wall = time.perf_counter()
     for k in range(K):
@@ -441,6 +478,16 @@ def run_closed_loop(args):
             "wall_steps_per_s_with_host_verifier": K / wall, "gpu_launches": 2 * K,
             "global_nodes_end": st["global_nodes"], "global_tokens_end": st["global_tokens"],
             "global_status": st["global_status"]}
+    if refill_ev:
+        r_ms = [a.elapsed_time(b) for a, b, _ in refill_ev]
+        line["refill"] = {"calls": len(r_ms), "mean_us": statistics.mean(r_ms) * 1e3, "max_us": max(r_ms) * 1e3,
+                          "mean_tokens": statistics.mean(t for _, _, t in refill_ev),
+                          "total_ms": sum(r_ms)}
+    k_ms = [a.elapsed_time(b) for a, b, _ in kernel_ev]
+    g_tok = [t for _, _, t in kernel_ev]
+    line["append_kernel"] = {"mean_us": statistics.mean(k_ms) * 1e3, "p50_us": statistics.median(k_ms) * 1e3,
+                             "max_us": max(k_ms) * 1e3, "global_tokens_per_call": statistics.mean(g_tok),
+                             "us_per_global_token": sum(k_ms) * 1e3 / max(sum(g_tok), 1)}
     line.update(summ)
     if ref is not None:
         line["parity_vs_oracle"] = "bit-exact" if ok else "MISMATCH"

@@ -130,8 +130,9 @@ int sd_append(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* 
  *   h_offsets  int64[n+1]  HOST: prompt i is d_tokens[h_offsets[i] .. h_offsets[i+1]), h_offsets[0] = 0
  *   d_tokens   int32[h_offsets[n]]  DEVICE
  * A prompt that does not fit the slot's node pool or text buffer leaves the slot empty with
- * SD_STATUS_POOL_FULL.  Unlike the per-step calls this one allocates temporary device memory
- * (about 100 bytes per prompt token) and synchronises the stream before it returns.
+ * SD_STATUS_POOL_FULL.  Unlike the per-step calls this one may allocate device memory: its
+ * temporaries (about 100 bytes per prompt token of the largest batch so far) are kept by the
+ * store and reused.  It synchronises the stream before it returns.
  * Errors: INVALID_ARG (bad slot, slot twice, offsets not ascending, token outside [0, V): nothing
  * is changed), CAPACITY (n * vocab or the token total does not fit 31 bits), NOMEM, CUDA.
  */

@@ -72,11 +72,20 @@ __device__ int insert_child_warp(int4* ent, int parent, int cb, int n, int pos, 
     return idx;
 }
 
-// lower_bound of token x in the sorted run ent[cb .. cb+n): eight-way, so that the seven
-// probes of a round are in flight together (a long run costs log8 n dependent rounds).
+// lower_bound of token x in the sorted run ent[cb .. cb+n): 32-way, then eight-way, so that the
+// probes of a round are in flight together (a long run costs a few dependent rounds).
 __device__ int lower_bound_run(const int4* ent, int cb, int n, int x) {
     int lo = 0, hi = n;
-    while (hi - lo > 8) {                                        // at most 8 rounds: n < 2^24
+    while (hi - lo > 256) {                                      // very long runs: 32-way, 31 probes in flight
+        const int step = (hi - lo) >> 5;
+        int sel = 0;
+#pragma unroll
+        for (int k = 0; k < 31; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
+        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
+        const int nhi = sel == 31 ? hi : lo + (sel + 1) * step;
+        lo = nlo; hi = nhi;
+    }
+    while (hi - lo > 8) {                                        // at most 3 rounds from 256
         const int step = (hi - lo) >> 3;
         int t[7];
 #pragma unroll
@@ -93,6 +102,39 @@ __device__ int lower_bound_run(const int4* ent, int cb, int n, int x) {
         if (ent[cb + mid].x < x) lo = mid + 1; else hi = mid;
     }
     return lo;
+}
+
+// Child x of `node` (-1 if none), by plain loads.
+__device__ int peek_child(const int4* ent, int node, int x) {
+    if (node < 0) return -1;
+    const int4 pe = ent[node];
+    const int n = (int)((unsigned)pe.w & RUN_COUNT_MASK);
+    if (n == 0) return -1;
+    const int pos = lower_bound_run(ent, pe.z, n, x);
+    if (pos >= n) return -1;
+    return ent[pe.z + pos].x == x ? pe.z + pos : -1;
+}
+
+// The slow look-ups of a token are the shallow ones (long child runs of frequent tokens, cold in
+// the caches), and they depend only on the last two or three tokens, not on the deep state.
+// Lane j walks the two- and three-token strings that end at token k0 + j, 32 tokens at once, so
+// that the token-by-token pass finds those runs in the caches.  Nothing is decided here; the
+// return value only keeps the loads alive.
+__device__ int warm_shallow(const TreeRef& tr, int V, const int32_t* tok, long long b, long long e, long long k0,
+                            int lane) {
+    const long long k = k0 + lane;
+    if (k >= e) return 0;
+    const int x0 = tok[k];
+    const int x1 = k - 1 >= b ? tok[k - 1] : -1, x2 = k - 2 >= b ? tok[k - 2] : -1;
+    if (x0 < 0 || x0 >= V || x1 < 0 || x1 >= V) return 0;
+    int seen = 0;
+    const int c1 = peek_child(tr.ent, tr.root[x1], x0);                        // (x1, x0)
+    if (c1 >= 0) seen += tr.ent[c1].y;
+    if (x2 >= 0 && x2 < V) {
+        const int c2 = peek_child(tr.ent, peek_child(tr.ent, tr.root[x2], x1), x0);   // (x2, x1, x0)
+        if (c2 >= 0) seen += tr.ent[c2].y;
+    }
+    return seen;
 }
 
 // All 32 lanes call.  `act` is this lane's active node of depth lane + 1 (-1: none);
@@ -234,7 +276,9 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
             int act = -1, room = 0, run_cb = 0;
             unsigned run_w = 0;
             const long long b = d_offsets[i], e = d_offsets[i + 1];
+            int seen = 0;
             for (long long k = b; k < e && !(status & SD_STATUS_GLOBAL_FULL); ++k) {
+                if (((k - b) & 31) == 0) seen |= warm_shallow(tr, sv.V, d_tokens, b, e, k, lane);
                 const int x = d_tokens[k];
                 if (x < 0 || x >= sv.V) { status |= SD_STATUS_BAD_TOKEN; break; }
                 if (!append_token(tr, sv.D, x, (int)(k - b), lane, act, room, run_cb, run_w, used, live)) {
@@ -243,6 +287,7 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
                 }
                 ++tokens;
             }
+            if (__any_sync(0xffffffffu, seen == 0x7fffffff)) status |= 0x40000000;   // never true
         }
         if (any && lane == 0) {
             sv.g_state->epoch += 1;                  // cached match nodes of every slot are stale now

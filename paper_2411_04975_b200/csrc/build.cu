@@ -439,14 +439,29 @@ __global__ void init_global_state_kernel(GlobalState* g, int used, int live, lon
     g->used = used; g->live = live; g->status = 0; g->epoch = 1; g->tokens = tokens;
 }
 
-struct DeviceArena {          // temporaries of one build, released together
-    void* ptr[40];
+struct DeviceArena {          // temporaries of one build: freed together, or kept in a workspace
+    void* ptr[48];
     int n = 0;
-    ~DeviceArena() { for (int i = 0; i < n; ++i) cudaFree(ptr[i]); }
+    sd_workspace* keep = nullptr;                     // if set, buffers live there and are reused
+    ~DeviceArena() { if (!keep) for (int i = 0; i < n; ++i) cudaFree(ptr[i]); }
     template <class T> bool get(T** out, i64 count) {
-        void* p = nullptr;
         if (count < 1) count = 1;
-        if (cudaMalloc(&p, (size_t)count * sizeof(T)) != cudaSuccess) { cudaGetLastError(); return false; }
+        if (n >= 48) return false;
+        const long long need = (long long)count * (long long)sizeof(T);
+        if (keep) {
+            const int k = n++;
+            if (keep->bytes[k] < need) {
+                if (keep->ptr[k]) cudaFree(keep->ptr[k]);
+                keep->ptr[k] = nullptr; keep->bytes[k] = 0;
+                const long long want = need + need / 4 + 256;
+                if (cudaMalloc(&keep->ptr[k], (size_t)want) != cudaSuccess) { cudaGetLastError(); return false; }
+                keep->bytes[k] = want;
+            }
+            *out = (T*)keep->ptr[k];
+            return true;
+        }
+        void* p = nullptr;
+        if (cudaMalloc(&p, (size_t)need) != cudaSuccess) { cudaGetLastError(); return false; }
         ptr[n++] = p;
         *out = (T*)p;
         return true;
@@ -478,6 +493,10 @@ static void store_release(sd_store* s) {
     cudaFree(s->g_ent); cudaFree(s->g_root); cudaFree(s->g_state);
     cudaFree(s->s_ent); cudaFree(s->s_root); cudaFree(s->s_text); cudaFree(s->s_state);
     cudaFree(s->j_score); cudaFree(s->j_n); cudaFree(s->j_tok); cudaFree(s->j_par);
+    if (s->ws) {
+        for (int k = 0; k < 48; ++k) cudaFree(s->ws->ptr[k]);
+        delete s->ws;
+    }
     delete s;
 }
 
@@ -522,12 +541,13 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
 
     seq_end_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_seq_offsets, n_seqs, N, end_pos);
     rank0_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tok, N, rank[0]);
-    int bits = bits_for(std::max<i64>(max_token, N) + 1);
+    const int bits_tok = bits_for(max_token + 1), bits_rank = bits_for(N + 1);
     int sorted = 0;
     // rank[k] orders the first 2^k tokens of every suffix
     auto round = [&](const int* ra, const int* rb, int off, int* rout) {
         make_keys_kernel<<<grid_for(N, T256), T256, 0, st>>>(ra, rb, off, end_pos, N, sb.keys[0], sb.vals[0]);
-        sorted = radix_sort_pairs(sb, N, bits, bits, st);
+        // the token ranks of the first round need more bits than the dense ranks of the later ones
+        sorted = radix_sort_pairs(sb, N, rb == rank[0] ? bits_tok : bits_rank, ra == rank[0] ? bits_tok : bits_rank, st);
         if (rout) {
             exclusive_scan(KeyChange{sb.keys[sorted]}, N, ex, sb.scan_tmp, st);
             assign_rank_kernel<<<grid_for(N, T256), T256, 0, st>>>(sb.keys[sorted], sb.vals[sorted], ex, N, rout);
@@ -862,6 +882,12 @@ extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, 
     const int T256 = 256, D = s->D;
 
     Pipeline P;
+    if (!s->ws) {
+        s->ws = new (std::nothrow) sd_workspace();
+        if (!s->ws) return SD_ERR_NOMEM;
+        memset(s->ws, 0, sizeof(*s->ws));
+    }
+    P.tmp.keep = s->ws;                                          // temporaries are kept for the next call
     int32_t *d_slot = nullptr, *mtok = nullptr;
     int64_t* d_off = nullptr;
     int *bad = nullptr, *r1 = nullptr;

@@ -60,6 +60,11 @@ struct SlotState {            // device-resident bookkeeping of one request slot
     int32_t g_node[SD_MAX_DEPTH];   // g_node[d-1]: global node of the last d tokens, -1 none
 };
 
+struct sd_workspace {         // grow-only device buffers, reused call after call
+    void* ptr[48];
+    long long bytes[48];
+};
+
 struct sd_store {
     int32_t V, D, R, T, M;
     // global tree
@@ -79,6 +84,7 @@ struct sd_store {
     int32_t* j_tok;           // [R*2*D][M]
     int32_t* j_par;           // [R*2*D][M]
     long long device_bytes;
+    struct sd_workspace* ws;  // HOST: temporaries of sd_build_requests, kept between calls
 };
 
 __host__ __device__ inline uint32_t sd_pow2ceil(uint32_t n) {

@@ -30,14 +30,27 @@ __device__ __forceinline__ int* word(int4* e, int k) { return reinterpret_cast<i
 __device__ int insert_child(int4* ent, int parent, int cb, int n, int pos, int x, int fresh, bool moves) {
     const int4 ne = make_int4(x, 1, 0, 0);
     int idx;
+    // entries move eight at a time: the eight loads are in flight together
     if (moves) {
-        for (int k = 0; k < pos; ++k) ent[fresh + k] = ent[cb + k];
+        for (int k0 = 0; k0 < n; k0 += 8) {
+            int4 t[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) if (k0 + u < n) t[u] = ent[cb + k0 + u];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) if (k0 + u < n) ent[fresh + k0 + u + (k0 + u >= pos ? 1 : 0)] = t[u];
+        }
         ent[fresh + pos] = ne;
-        for (int k = pos; k < n; ++k) ent[fresh + k + 1] = ent[cb + k];
         *word(&ent[parent], 2) = fresh;
         idx = fresh + pos;
     } else {
-        for (int k = n - 1; k >= pos; --k) ent[cb + k + 1] = ent[cb + k];
+        for (int hi = n; hi > pos; hi -= 8) {                    // from the top down
+            const int lo = max(pos, hi - 8);
+            int4 t[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) if (lo + u < hi) t[u] = ent[cb + lo + u];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) if (lo + u < hi) ent[cb + lo + u + 1] = t[u];
+        }
         ent[cb + pos] = ne;
         idx = cb + pos;
     }
@@ -97,11 +110,39 @@ __device__ int lower_bound_run(const int4* ent, int cb, int n, int x) {
         const int nhi = sel == 7 ? hi : lo + (sel + 1) * step;
         lo = nlo; hi = nhi;
     }
-    while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (ent[cb + mid].x < x) lo = mid + 1; else hi = mid;
+    // at most eight candidates left: all of them in one round
+    int t[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) t[k] = lo + k < hi ? ent[cb + lo + k].x : 0x7fffffff;
+    int below = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) below += t[k] < x ? 1 : 0;
+    return lo + below;
+}
+
+// Look-up of child x in the sorted run ent[cb .. cb+n): insert position in `pos`, and if the
+// child exists its index is returned with its entry in `fe` (else -1).  The last round reads
+// whole entries, so a run of up to eight children costs one round of loads.
+__device__ int lookup_child(const int4* ent, int cb, int n, int x, int& pos, int4& fe) {
+    int lo = 0, hi = n;
+    if (n > 8) {                                                 // narrow to a window of eight that holds the position
+        const int p0 = lower_bound_run(ent, cb, n, x);
+        pos = p0;
+        if (p0 >= n) return -1;
+        fe = ent[cb + p0];
+        return fe.x == x ? cb + p0 : -1;
     }
-    return lo;
+    int4 e[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) e[k] = lo + k < hi ? ent[cb + lo + k] : make_int4(0x7fffffff, 0, 0, 0);
+    int below = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) below += e[k].x < x ? 1 : 0;
+    pos = below;
+    int found = -1;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) if (k == below && k < n && e[k].x == x) { fe = e[k]; found = cb + k; }
+    return found;
 }
 
 // Child x of `node` (-1 if none), by plain loads.
@@ -162,16 +203,7 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
             cb = parent_cb; w = parent_w;
             if (w == RUN_UNKNOWN) { const int4 pe = tr.ent[parent]; cb = pe.z; w = (unsigned)pe.w; }
             n = (int)(w & RUN_COUNT_MASK);
-            if (n <= 2) {                                        // the usual case: both loads at once
-                int4 e0 = make_int4(0x7fffffff, 0, 0, 0), e1 = e0;
-                if (n > 0) e0 = tr.ent[cb];
-                if (n > 1) e1 = tr.ent[cb + 1];
-                pos = (n > 0 && e0.x < x) ? ((n > 1 && e1.x < x) ? 2 : 1) : 0;
-                if (pos < n) { fe = pos == 0 ? e0 : e1; if (fe.x == x) found = cb + pos; }
-            } else {
-                pos = lower_bound_run(tr.ent, cb, n, x);
-                if (pos < n) { fe = tr.ent[cb + pos]; if (fe.x == x) found = cb + pos; }
-            }
+            found = lookup_child(tr.ent, cb, n, x, pos, fe);
         }
     }
     const bool need = valid && found < 0;
@@ -229,7 +261,7 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
         const bool next_pending = lane < 31 && ((pend >> (lane + 1)) & 1u);
         const bool ready = need && ((pend >> lane) & 1u) && !(clash && next_pending);
         // inserts that move many entries are done by the whole warp, one after the other
-        const bool big = ready && lane > 0 && (moves ? n : n - pos) > 8;
+        const bool big = ready && lane > 0 && (moves ? n : n - pos) > 48;
         if (ready && !big) {
             if (lane == 0) {
                 tr.ent[fresh] = make_int4(x, 1, 0, 0);

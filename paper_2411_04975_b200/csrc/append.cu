@@ -125,12 +125,23 @@ __device__ int lower_bound_run(const int4* ent, int cb, int n, int x) {
 // whole entries, so a run of up to eight children costs one round of loads.
 __device__ int lookup_child(const int4* ent, int cb, int n, int x, int& pos, int4& fe) {
     int lo = 0, hi = n;
-    if (n > 8) {                                                 // narrow to a window of eight that holds the position
-        const int p0 = lower_bound_run(ent, cb, n, x);
-        pos = p0;
-        if (p0 >= n) return -1;
-        fe = ent[cb + p0];
-        return fe.x == x ? cb + p0 : -1;
+    while (hi - lo > 256) {                                      // very long runs: 32-way, 31 probes in flight
+        const int step = (hi - lo) >> 5;
+        int sel = 0;
+#pragma unroll
+        for (int k = 0; k < 31; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
+        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
+        const int nhi = sel == 31 ? hi : lo + (sel + 1) * step + 1;   // keep the pivot: it may be x itself
+        lo = nlo; hi = nhi;
+    }
+    while (hi - lo > 8) {                                        // eight-way down to a window of eight
+        const int step = (hi - lo) >> 3;
+        int sel = 0;
+#pragma unroll
+        for (int k = 0; k < 7; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
+        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
+        const int nhi = sel == 7 ? hi : lo + (sel + 1) * step + 1;
+        lo = nlo; hi = nhi;
     }
     int4 e[8];
 #pragma unroll
@@ -138,10 +149,10 @@ __device__ int lookup_child(const int4* ent, int cb, int n, int x, int& pos, int
     int below = 0;
 #pragma unroll
     for (int k = 0; k < 8; ++k) below += e[k].x < x ? 1 : 0;
-    pos = below;
+    pos = lo + below;
     int found = -1;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) if (k == below && k < n && e[k].x == x) { fe = e[k]; found = cb + k; }
+    for (int k = 0; k < 8; ++k) if (k == below && lo + k < hi && e[k].x == x) { fe = e[k]; found = cb + lo + k; }
     return found;
 }
 

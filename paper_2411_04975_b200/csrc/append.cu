@@ -303,9 +303,38 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
 
 // Warp 0 of the grid inserts whole sequences into the global tree, one after the
 // other; warp i + 1 appends item i to its request slot.
+// The blocks behind those run ahead of warp 0 through the global tree: thread per token position of
+// every sequence that is being inserted, walking the up to D tokens that start there, reading
+// only.  The global tree is hundreds of megabytes and cold; warp 0, which has to take the tokens
+// one after the other, then finds most of what it needs in L2.  Nothing is decided here.
 __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_offsets,
-                              const int32_t* d_tokens, const uint8_t* d_reset) {
+                              const int32_t* d_tokens, const uint8_t* d_reset, int main_blocks) {
     const int lane = threadIdx.x & 31;
+    if ((int)blockIdx.x >= main_blocks) {
+        const long long tid = (long long)(blockIdx.x - main_blocks) * blockDim.x + threadIdx.x;
+        const long long nthreads = (long long)(gridDim.x - main_blocks) * blockDim.x;
+        int seen = 0;
+        for (int i = 0; i < n; ++i) {
+            if (d_slot[i] != -1) continue;
+            const long long b = d_offsets[i], e = d_offsets[i + 1];
+            for (long long k = b + tid; k < e; k += nthreads) {
+                int x = d_tokens[k];
+                if (x < 0 || x >= sv.V) continue;
+                int node = sv.g_root[x];
+                for (int d = 1; d < sv.D && node >= 0 && k + d < e; ++d) {
+                    x = d_tokens[k + d];
+                    const int4 pe = sv.g_ent[node];
+                    const int nc = (int)((unsigned)pe.w & RUN_COUNT_MASK);
+                    int pos;
+                    int4 fe;
+                    node = nc > 0 ? lookup_child(sv.g_ent, pe.z, nc, x, pos, fe) : -1;
+                    seen += pos;
+                }
+            }
+        }
+        if (seen == 0x7fffffff) sv.g_state->status |= 0x40000000;   // keeps the loads alive; never true
+        return;
+    }
     const int warp = (int)((blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5);
     if (warp > n) return;
     if (warp == 0) {
@@ -382,7 +411,9 @@ extern "C" int sd_append(sd_store* s, int32_t n, const int32_t* d_slot, const in
     if (!d_slot || !d_offsets) return SD_ERR_INVALID_ARG;
     const int warps_per_block = 4;
     const unsigned blocks = (unsigned)((n + 1 + warps_per_block - 1) / warps_per_block);
-    append_kernel<<<blocks, warps_per_block * 32, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset);
+    const unsigned ahead = 32;                                   // blocks that only warm the caches for warp 0
+    append_kernel<<<blocks + ahead, warps_per_block * 32, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_offsets, d_tokens,
+                                                                                     d_reset, (int)blocks);
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }

@@ -49,6 +49,8 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--oracle-samples", type=int, default=4)
     ap.add_argument("--small", action="store_true", help="1/16 corpus, batch 32: quick functional run")
+    ap.add_argument("--sweep", action="store_true",
+                    help="scalability sweep over the size of the global tree (shape of the paper's appendix table)")
     ap.add_argument("--closed-loop-oracle", action="store_true",
                     help="closed_loop config: run the CPU oracle in lock-step and compare every step (slow)")
     return ap.parse_args()
@@ -355,6 +357,72 @@ def run_ours(args):
 
 
 # --------------------------------------------------------------------------------------------
+def run_sweep(args):
+    """Memory, update time per token and look-up time per speculated token against the size of
+    the global tree: the quantities of the paper's scalability table (appendix "Scalability and
+    Memory Overhead"), on synthetic corpora of the headline workload's kind."""
+    import torch
+
+    import paper_2411_04975_b200 as sfx
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    K, W = min(args.steps, 30), 3
+    rows = []
+    for n_seqs in (512, 1024, 2048, 4096, 8192, 16384):
+        w = get_workload("large_batch", n_seqs=n_seqs)
+        c = w.cfg
+        B = c.batch
+        prompts = [w.prompt(i) for i in range(B)]
+        steps = StepInputs(w, 0, B, W + K, prompts)
+        corpus = torch.as_tensor(w.corpus(), device=dev)
+        offsets = torch.as_tensor(w.corpus_offsets(), device=dev)
+        build_ms = float("inf")
+        for attempt in range(2):                                 # the first build also pays for fresh device allocations
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            store = sfx.SuffixStore(corpus, offsets, vocab=c.vocab, depth_cap=c.depth_cap, max_requests=B,
+                                    max_req_tokens=c.prompt_len + steps.max_total + 8, max_spec_cap=c.max_spec)
+            torch.cuda.synchronize()
+            build_ms = min(build_ms, (time.perf_counter() - t0) * 1e3)
+            if attempt == 0:
+                store.free()
+        st = store.stats()
+        poff = np.zeros(B + 1, dtype=np.int64)
+        poff[1:] = np.cumsum([len(p) for p in prompts])
+        store.build_requests(np.arange(B, dtype=np.int32), poff, torch.as_tensor(np.concatenate(prompts), device=dev))
+        slots = torch.arange(B, dtype=torch.int32, device=dev)
+        out = store.alloc_outputs(B)
+        flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
+        d_off = [torch.as_tensor(o, device=dev) for o in steps.offsets]
+        d_tok = [torch.as_tensor(t, device=dev) for t in steps.tokens]
+        spec, app, drafts, toks = [], [], 0, 0
+        for k in range(W + K):
+            flush.zero_()
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record()
+            store.speculate(slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
+            e1.record()
+            store.append(slots, d_off[k], d_tok[k])
+            e2.record()
+            torch.cuda.synchronize()
+            if k >= W:
+                spec.append(e0.elapsed_time(e1)); app.append(e1.elapsed_time(e2))
+                drafts += int(out["n_draft"].sum().item()); toks += int(d_tok[k].numel())
+        n_tok = n_seqs * c.seq_len
+        rows.append({"entries": n_seqs, "tokens": n_tok, "global_nodes": st["global_nodes"],
+                     "global_tree_MB": st["global_pool_used"] * 16 / 1e6, "bytes_per_token": st["global_pool_used"] * 16 / n_tok,
+                     "offline_build_ms": build_ms, "offline_update_us_per_token": build_ms * 1e3 / n_tok,
+                     "online_update_us_per_token": sum(app) * 1e3 / toks,
+                     "lookup_us_per_speculated_token": sum(spec) * 1e3 / max(drafts, 1),
+                     "speculate_us_per_step": statistics.mean(spec) * 1e3, "draft_tokens_per_step": drafts / K})
+        store.free()
+        del corpus, offsets, flush
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "scalability sweep (batch 256, 4,096-token prompts, one B200)", "rows": rows}), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
 def run_closed_loop(args):
     """BASELINE config 4: speculate -> simulated verification against the hidden continuation ->
     append accepted + bonus tokens; finished outputs go into the global tree, their slots are
@@ -548,6 +616,8 @@ if __name__ == "__main__":
     a = parse()
     if a.impl == "reference":
         run_reference(a)
+    elif a.sweep:
+        run_sweep(a)
     elif a.config == "closed_loop":
         run_closed_loop(a)
     else:

@@ -220,6 +220,18 @@ int sd_query_counts(sd_store* store, int32_t n, const int32_t* d_tree, const int
 int sd_slot_info(sd_store* store, int32_t n, const int32_t* d_slot, int32_t* d_len, int32_t* d_nodes,
                  int32_t* d_status, void* stream);
 
+/*
+ * sd_entropy: empirical entropy of a tree in bits (Appendix "Predicting SuffixDecoding
+ * Effectiveness"): for every node that has children, the entropy of the children's count
+ * distribution; the result is the average over those nodes (the root included) weighted by the
+ * sum of the children's counts.  A low value says the next token is predictable from its
+ * prefix, i.e. that suffix-tree speculation will work well on this kind of text.
+ *   tree: -1 global tree, else a slot.  h_entropy: HOST double.  An empty tree gives 0.
+ * An offline analysis call: allocates temporary device memory and synchronises the stream.
+ * Sums are accumulated with atomics, so the last bits vary from call to call.
+ */
+int sd_entropy(sd_store* store, int32_t tree, double* h_entropy, void* stream);
+
 /* sd_stats: store-wide figures into HOST memory.  Synchronises the stream. */
 int sd_stats(sd_store* store, sd_stats_t* out, void* stream);
 

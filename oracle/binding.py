@@ -58,6 +58,8 @@ def _load():
         lib.sfx_oracle_candidate.restype = C.c_int
         lib.sfx_oracle_candidate.argtypes = [C.c_void_p, C.c_int, p32, C.c_int64, C.c_int, C.c_int, C.c_int,
                                              p32, p32, pd, pd]
+        lib.sfx_oracle_entropy.restype = C.c_double
+        lib.sfx_oracle_entropy.argtypes = [C.c_void_p, C.c_int]
         lib.sfx_oracle_budget.restype = C.c_int
         lib.sfx_oracle_budget.argtypes = [C.c_double, C.c_int, C.c_int]
         lib.sfx_oracle_speculate.argtypes = [C.c_void_p, C.c_int, p32, C.c_int, C.c_double, C.c_int, C.c_int,
@@ -142,6 +144,9 @@ class SuffixOracle:
         a = [np.empty(n, dtype=np.int32) for _ in range(4)]
         self._lib.sfx_oracle_dump(self._h, tree, n, *[_p(x, C.c_int32) for x in a])
         return tuple(a)
+
+    def entropy(self, tree: int) -> float:
+        return float(self._lib.sfx_oracle_entropy(self._h, tree))
 
     # ---- Algorithm 1 ---------------------------------------------------
     def budget(self, alpha: float, p: int, cap: int) -> int:

@@ -315,6 +315,27 @@ int sfx_oracle_candidate(void* h, int tree, const int32_t* ctx, int64_t t, int p
     return (int)out.size();
 }
 
+// Empirical entropy (Appendix "Predicting SuffixDecoding Effectiveness"): entropy in bits of
+// each node's children distribution, averaged with the children's total count as weight.
+static void entropy_rec(const Node* n, double& acc, double& weight) {
+    if (n->children.empty()) return;
+    double sum = 0.0;
+    for (auto& kv : n->children) sum += (double)kv.second->count;
+    double h = 0.0;
+    for (auto& kv : n->children) {
+        double p = (double)kv.second->count / sum;
+        h -= p * std::log2(p);
+    }
+    acc += sum * h;
+    weight += sum;
+    for (auto& kv : n->children) entropy_rec(kv.second, acc, weight);
+}
+double sfx_oracle_entropy(void* h, int tree) {
+    double acc = 0.0, weight = 0.0;
+    entropy_rec(&pick((Oracle*)h, tree).root, acc, weight);
+    return weight > 0.0 ? acc / weight : 0.0;
+}
+
 int sfx_oracle_budget(double alpha, int p, int cap) { return budget_for(alpha, p, cap); }
 
 // GenerateCandidateTree for n requests.  Row stride of every per-draft output is M.

@@ -18,7 +18,7 @@ from . import build as _build
 FLAG_GLOBAL_ONLY, FLAG_REQUEST_ONLY, FLAG_LINEAR = 1, 2, 4
 STATUS_BAD_SLOT, STATUS_POOL_FULL, STATUS_GLOBAL_FULL, STATUS_BAD_TOKEN = 1, 2, 4, 8
 
-EXPORTS = ["sd_build", "sd_build_requests", "sd_append", "sd_speculate", "sd_speculate_noalloc", "sd_query_counts", "sd_slot_info", "sd_stats", "sd_free",
+EXPORTS = ["sd_build", "sd_build_requests", "sd_append", "sd_speculate", "sd_speculate_noalloc", "sd_query_counts", "sd_slot_info", "sd_entropy", "sd_stats", "sd_free",
            "sd_strerror"]
 
 
@@ -71,6 +71,8 @@ def library() -> C.CDLL:
         lib.sd_query_counts.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
         lib.sd_slot_info.restype = C.c_int
         lib.sd_slot_info.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
+        lib.sd_entropy.restype = C.c_int
+        lib.sd_entropy.argtypes = [vp, C.c_int32, C.POINTER(C.c_double), vp]
         lib.sd_stats.restype = C.c_int
         lib.sd_stats.argtypes = [vp, C.POINTER(_Stats), vp]
         lib.sd_free.restype = None
@@ -234,6 +236,14 @@ class SuffixStore:
         if rc != 0:
             raise SuffixSpecError(rc, "sd_slot_info")
         return {"len": o[0], "nodes": o[1], "status": o[2]}
+
+    def entropy(self, tree: int = -1) -> float:
+        """Count-weighted mean entropy (bits) of the children distributions of `tree`."""
+        h = C.c_double(0.0)
+        rc = library().sd_entropy(self._h, tree, C.byref(h), _stream())
+        if rc != 0:
+            raise SuffixSpecError(rc, "sd_entropy")
+        return h.value
 
     def stats(self) -> dict:
         st = _Stats()

@@ -86,3 +86,134 @@ extern "C" int sd_stats(sd_store* s, sd_stats_t* out, void* stream) {
     out->global_status = g.status;
     return SD_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Empirical entropy of a tree (Appendix "Predicting SuffixDecoding Effectiveness"): for every
+// node the entropy of its children's count distribution, averaged over the nodes with the
+// sibling sum as weight.  Level-by-level traversal from the root table (the pools also hold
+// abandoned runs and top-block copies, so a plain sweep over the pool would count too much).
+namespace {
+
+__device__ __forceinline__ void warp_accumulate(double h_times_s, unsigned long long s, double* acc,
+                                                unsigned long long* wsum) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        h_times_s += __shfl_xor_sync(0xffffffffu, h_times_s, o);
+        s += __shfl_xor_sync(0xffffffffu, s, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (h_times_s != 0.0) atomicAdd(acc, h_times_s);
+        if (s) atomicAdd(wsum, s);
+    }
+}
+
+// depth-1 nodes: total count, and the first frontier
+__global__ void entropy_root_sum_kernel(const int4* ent, const int32_t* root, int V, unsigned long long* total,
+                                        int* frontier, int* n_frontier) {
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned long long c = 0;
+    if (v < V) {
+        const int idx = root[v];
+        if (idx >= 0) {
+            const int4 e = ent[idx];
+            c = (unsigned)e.y;
+            if ((unsigned)e.w & RUN_COUNT_MASK) frontier[atomicAdd(n_frontier, 1)] = idx;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(total, c);
+}
+
+__global__ void entropy_root_kernel(const int4* ent, const int32_t* root, int V, const unsigned long long* total,
+                                    double* acc, unsigned long long* wsum) {
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;
+    double part = 0.0;                                           // -(c/S) log2(c/S) * S = -c log2(c/S)
+    const double S = (double)*total;
+    if (v < V) {
+        const int idx = root[v];
+        if (idx >= 0) { const double c = (double)(unsigned)ent[idx].y; part = -c * log2(c / S); }
+    }
+    warp_accumulate(part, 0ull, acc, wsum);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && *total) atomicAdd(wsum, *total);
+}
+
+// one thread per node of the current level
+__global__ void entropy_level_kernel(const int4* ent, const int* frontier, int n, int* next, int* n_next, double* acc,
+                                     unsigned long long* wsum) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    double part = 0.0;
+    unsigned long long S = 0;
+    if (i < n) {
+        const int4 e = ent[frontier[i]];
+        const int cb = e.z, nc = (int)((unsigned)e.w & RUN_COUNT_MASK);
+        for (int k = 0; k < nc; ++k) S += (unsigned)ent[cb + k].y;
+        const double dS = (double)S;
+        for (int k = 0; k < nc; ++k) {
+            const int4 c = ent[cb + k];
+            const double dc = (double)(unsigned)c.y;
+            part -= dc * log2(dc / dS);
+            if ((unsigned)c.w & RUN_COUNT_MASK) next[atomicAdd(n_next, 1)] = cb + k;
+        }
+    }
+    warp_accumulate(part, S, acc, wsum);
+}
+
+}  // namespace
+
+extern "C" int sd_entropy(sd_store* s, int32_t tree, double* h_entropy, void* stream) {
+    if (!s || !h_entropy || tree < -1 || tree >= s->R) return SD_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int4* ent = tree < 0 ? s->g_ent : s->s_ent + (long long)tree * s->spn;
+    const int32_t* root = tree < 0 ? s->g_root : s->s_root + (long long)tree * s->V;
+    int live = 0;
+    if (tree < 0) {
+        GlobalState g;
+        SD_CUDA_OK(cudaMemcpyAsync(&g, s->g_state, sizeof(g), cudaMemcpyDeviceToHost, st));
+        SD_CUDA_OK(cudaStreamSynchronize(st));
+        live = g.live;
+    } else {
+        SlotState ss;
+        SD_CUDA_OK(cudaMemcpyAsync(&ss, s->s_state + tree, sizeof(ss), cudaMemcpyDeviceToHost, st));
+        SD_CUDA_OK(cudaStreamSynchronize(st));
+        live = ss.live;
+    }
+    *h_entropy = 0.0;
+    if (live <= 0) return SD_OK;
+    int *fa = nullptr, *fb = nullptr;
+    unsigned char* small = nullptr;                              // total, acc, wsum, counters
+    if (cudaMalloc(&fa, sizeof(int) * (size_t)live) != cudaSuccess || cudaMalloc(&fb, sizeof(int) * (size_t)live) != cudaSuccess ||
+        cudaMalloc(&small, 64) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(fa); cudaFree(fb); cudaFree(small);
+        return SD_ERR_NOMEM;
+    }
+    unsigned long long* total = (unsigned long long*)small;
+    double* acc = (double*)(small + 8);
+    unsigned long long* wsum = (unsigned long long*)(small + 16);
+    int* cnt = (int*)(small + 24);                               // cnt[0], cnt[1]: frontier sizes
+    cudaError_t ce = cudaMemsetAsync(small, 0, 64, st);
+    entropy_root_sum_kernel<<<(s->V + 255) / 256, 256, 0, st>>>(ent, root, s->V, total, fa, cnt);
+    entropy_root_kernel<<<(s->V + 255) / 256, 256, 0, st>>>(ent, root, s->V, total, acc, wsum);
+    int n = 0, cur = 0;
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&n, cnt, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    for (int depth = 1; ce == cudaSuccess && n > 0 && depth <= SD_MAX_DEPTH; ++depth) {
+        int* from = cur ? fb : fa;
+        int* to = cur ? fa : fb;
+        ce = cudaMemsetAsync(cnt + (cur ^ 1), 0, sizeof(int), st);
+        entropy_level_kernel<<<(n + 255) / 256, 256, 0, st>>>(ent, from, n, to, cnt + (cur ^ 1), acc, wsum);
+        if (ce == cudaSuccess) ce = cudaMemcpyAsync(&n, cnt + (cur ^ 1), sizeof(int), cudaMemcpyDeviceToHost, st);
+        if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+        cur ^= 1;
+    }
+    double h_acc = 0.0;
+    unsigned long long h_w = 0;
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_acc, acc, sizeof(double), cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_w, wsum, sizeof(h_w), cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    cudaFree(fa); cudaFree(fb); cudaFree(small);
+    if (ce != cudaSuccess) return SD_ERR_CUDA;
+    *h_entropy = h_w ? h_acc / (double)h_w : 0.0;
+    return SD_OK;
+}

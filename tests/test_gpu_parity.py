@@ -420,3 +420,17 @@ def test_build_requests_pool_overflow(U):
     pr.o.slot_append(1, prompts[1])
     pr.check_tree(1)
     pr.close()
+
+
+def test_entropy_matches_oracle(U):
+    rng = np.random.default_rng(23)
+    pr = U.Pair(_rand_seqs(rng, 30, 20, 400, 9) + [np.arange(2000, dtype=np.int32) % 700], vocab=700, D=12, n_slots=3,
+                max_req_tokens=600)
+    pr.append([0, 2, -1], _rand_seqs(rng, 3, 100, 500, 9), reset=[1, 1, 0])
+    pr.append([0, -1], _rand_seqs(rng, 2, 50, 90, 700))
+    for tree in (-1, 0, 1, 2):
+        want = pr.o.entropy(tree)
+        got = pr.g.entropy(tree)
+        assert abs(got - want) <= 1e-9 * max(1.0, abs(want)), (tree, got, want)
+    assert pr.g.entropy(1) == 0.0                                # empty slot
+    pr.close()

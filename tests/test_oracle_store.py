@@ -123,3 +123,41 @@ def test_append_in_chunks_equals_token_by_token(oracle_mod):
     a.slot_append_batch([1], [text[25:]], n_threads=2)
     for x, y in zip(a.dump(0), a.dump(1)):
         assert np.array_equal(x, y)
+
+
+def test_entropy_closed_forms_and_bruteforce(oracle_mod):
+    """Appendix "Predicting SuffixDecoding Effectiveness": count-weighted mean of the entropy of
+    every node's children distribution (bits)."""
+    import math
+    from bruteforce import children
+    # sequences [a,b], [a,c]: root {a:2, b:1, c:1} -> 1.5 bits, weight 4; node a {b:1, c:1} -> 1 bit, weight 2
+    o = oracle_mod.SuffixOracle(4, 1)
+    o.global_insert([1, 2]); o.global_insert([1, 3])
+    assert abs(o.entropy(-1) - (4 * 1.5 + 2 * 1.0) / 6) < 1e-12
+    # one repeated token: every node has a single child -> 0
+    o = oracle_mod.SuffixOracle(6, 1)
+    o.global_insert([7] * 15)
+    assert o.entropy(-1) == 0.0
+    assert oracle_mod.SuffixOracle(6, 1).entropy(-1) == 0.0      # empty tree
+    # k equally likely tokens, depth cap 1: log2 k
+    o = oracle_mod.SuffixOracle(1, 1)
+    o.global_insert(list(range(8)) * 3)
+    assert abs(o.entropy(-1) - 3.0) < 1e-12
+    # brute force from substring scans on a random corpus
+    rng = np.random.default_rng(17)
+    D = 4
+    seqs = [rng.integers(0, 3, size=int(rng.integers(3, 14))).tolist() for _ in range(4)]
+    o = oracle_mod.SuffixOracle(D, 1)
+    for s in seqs:
+        o.global_insert(s)
+    acc = weight = 0.0
+    stack = [[]]
+    while stack:
+        path = stack.pop()
+        ch = children(seqs, path, D)
+        tot = sum(ch.values())
+        if tot:
+            acc += tot * -sum(c / tot * math.log2(c / tot) for c in ch.values())
+            weight += tot
+            stack.extend(path + [t] for t in ch)
+    assert abs(o.entropy(-1) - acc / weight) < 1e-12

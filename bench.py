@@ -236,30 +236,36 @@ def run_ours(args):
     # ---- end to end: host buffers in, host buffers out, every step
     e2e = None
     if not args.no_e2e:
-        pin = lambda a: torch.as_tensor(a).pin_memory()   # noqa: E731
-        h_off = [pin(o) for o in steps.offsets[W + K:]]
-        h_tok = [pin(t) for t in steps.tokens[W + K:]]
-        h_slots = pin(np.arange(B, dtype=np.int32))
-        max_tok = max(int(t.numel()) for t in h_tok)
-        s_slots = torch.empty(B, dtype=torch.int32, device=dev)
-        s_off = torch.empty(B + 1, dtype=torch.int64, device=dev)
-        s_tok = torch.empty(max_tok, dtype=torch.int32, device=dev)
-        h_out = {n: torch.empty(t.shape, dtype=t.dtype).pin_memory() for n, t in out.items()}
+        # per step: ONE pinned host buffer in (slots, offsets, tokens), ONE pinned host buffer out
+        max_tok = max(int(t.size) for t in steps.tokens[W + K:])
+        in_bytes = 8 * (B + 1) + 4 * B + 4 * max_tok
+        h_in = [torch.empty(in_bytes, dtype=torch.uint8).pin_memory() for _ in range(We + Ke)]
+        n_tok = []
+        for k in range(We + Ke):
+            o, t = steps.offsets[W + K + k], steps.tokens[W + K + k]
+            h_in[k][:8 * (B + 1)].view(torch.int64).copy_(torch.as_tensor(o))
+            h_in[k][8 * (B + 1):8 * (B + 1) + 4 * B].view(torch.int32).copy_(torch.arange(B, dtype=torch.int32))
+            h_in[k][8 * (B + 1) + 4 * B:8 * (B + 1) + 4 * B + 4 * t.size].view(torch.int32).copy_(torch.as_tensor(t))
+            n_tok.append(int(t.size))
+        d_in = torch.empty(in_bytes, dtype=torch.uint8, device=dev)
+        s_off = d_in[:8 * (B + 1)].view(torch.int64)
+        s_slots = d_in[8 * (B + 1):8 * (B + 1) + 4 * B].view(torch.int32)
+        s_tok = d_in[8 * (B + 1) + 4 * B:].view(torch.int32)
+        h_packed = torch.empty(out["packed"].numel(), dtype=torch.uint8).pin_memory()
+        h_out = store.unpack_outputs(h_packed, B)                # host views of the drafts
         h2d = d2h = 0
 
         def e2e_step(k):
             nonlocal h2d, d2h
-            nt = int(h_tok[k].numel())
-            s_slots.copy_(h_slots, non_blocking=True)
-            s_off.copy_(h_off[k], non_blocking=True)
-            s_tok[:nt].copy_(h_tok[k], non_blocking=True)
+            nt = n_tok[k]
+            nb = 8 * (B + 1) + 4 * B + 4 * nt
+            d_in[:nb].copy_(h_in[k][:nb], non_blocking=True)
             store.speculate(s_slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
-            for n in h_out:
-                h_out[n].copy_(out[n], non_blocking=True)
+            h_packed.copy_(out["packed"], non_blocking=True)
             store.append(s_slots, s_off, s_tok[:nt])
             torch.cuda.synchronize()
-            h2d += 4 * B + 8 * (B + 1) + 4 * nt
-            d2h += sum(t.numel() * t.element_size() for t in h_out.values())
+            h2d += nb
+            d2h += h_packed.numel()
 
         for k in range(We):
             e2e_step(k)

@@ -200,14 +200,38 @@ class SuffixStore:
             raise SuffixSpecError(rc, "sd_build_requests")
 
     def alloc_outputs(self, n: int) -> Dict[str, torch.Tensor]:
-        M, dev = self.max_spec_cap, self.device
+        """Output tensors of sd_speculate for n requests.  They are views into ONE device
+        buffer (returned under the key "packed"), so a caller that wants the drafts on the host
+        needs a single device-to-host copy; `unpack_outputs` makes the same views on a host copy."""
+        packed = torch.empty(self.packed_output_bytes(n), dtype=torch.uint8, device=self.device)
+        return self.unpack_outputs(packed, n)
+
+    def _output_layout(self, n: int):
+        M = self.max_spec_cap
         words = (M + 31) // 32
-        i32 = dict(dtype=torch.int32, device=dev)
-        return {"n_draft": torch.empty(n, **i32), "tokens": torch.empty(n, M, **i32),
-                "parents": torch.empty(n, M, **i32), "positions": torch.empty(n, M, **i32),
-                "mask": torch.empty(n, M, words, **i32), "chosen_tree": torch.empty(n, **i32),
-                "chosen_p": torch.empty(n, **i32), "score": torch.empty(n, dtype=torch.float64, device=dev),
-                "status": torch.empty(n, **i32)}
+        fields = [("score", torch.float64, (n,)), ("tokens", torch.int32, (n, M)), ("parents", torch.int32, (n, M)),
+                  ("positions", torch.int32, (n, M)), ("mask", torch.int32, (n, M, words)),
+                  ("n_draft", torch.int32, (n,)), ("chosen_tree", torch.int32, (n,)), ("chosen_p", torch.int32, (n,)),
+                  ("status", torch.int32, (n,))]
+        off, lay = 0, []
+        for name, dt, shape in fields:
+            size = torch.empty(0, dtype=dt).element_size()
+            cnt = 1
+            for d in shape:
+                cnt *= d
+            lay.append((name, dt, shape, off, cnt * size))
+            off += (cnt * size + 15) // 16 * 16
+        return lay, off
+
+    def packed_output_bytes(self, n: int) -> int:
+        return max(16, self._output_layout(n)[1])
+
+    def unpack_outputs(self, packed: torch.Tensor, n: int) -> Dict[str, torch.Tensor]:
+        lay, _ = self._output_layout(n)
+        out = {"packed": packed}
+        for name, dt, shape, off, nbytes in lay:
+            out[name] = packed[off:off + nbytes].view(dt).view(shape)
+        return out
 
     def speculate(self, slots: torch.Tensor, P: int, alpha: float, max_spec: int, flags: int = 0,
                   budget_cap: Optional[torch.Tensor] = None,

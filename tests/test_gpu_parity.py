@@ -229,7 +229,8 @@ def test_speculate_is_deterministic(U):
     a = {k: v.clone() for k, v in a.items()}
     b = pr.g.speculate(U.dev_i32(list(range(16))), 16, 2.0, 64)
     for k in a:
-        assert torch.equal(a[k], b[k])
+        if k != "packed":                                        # the one buffer behind the views: has padding
+            assert torch.equal(a[k], b[k])
     pr.close()
 
 

@@ -16,7 +16,8 @@ pytestmark = pytest.mark.gpu
 
 def _same(a, b):
     for k in a:
-        assert torch.equal(a[k], b[k]), k          # integers and fp64 score bits alike: exact
+        if k != "packed":                          # the buffer behind the views (has padding bytes)
+            assert torch.equal(a[k], b[k]), k      # integers and fp64 score bits alike: exact
 
 
 def test_noalloc_matches_sd_speculate_twice_in_a_row():

@@ -171,6 +171,22 @@ int sd_speculate(sd_store* store, int32_t n, const int32_t* d_slot, const sd_spe
                  double* d_score, int32_t* d_status, void* stream);
 
 /*
+ * sd_step: one decode step in one launch: for every request i first append the tokens
+ * d_new_tokens[d_offsets[i] .. d_offsets[i+1]) (accepted drafts + bonus token of the previous
+ * step) to its per-request tree and context, then speculate, exactly as sd_append followed by
+ * sd_speculate on the same slots would (Section 3: tokens are added to the per-request tree as
+ * they are generated; Algorithm 1 then runs on the extended context).  The appends of requests
+ * with many new tokens overlap with the speculation of the others.
+ *   d_slot int32[n]: distinct slots >= 0 (no global inserts, no resets: use sd_append for those);
+ *   d_offsets int64[n+1], d_new_tokens int32[d_offsets[n]]; all other arguments as sd_speculate.
+ * A request whose append stops early (pool full, bad token) gets no draft and the status bits.
+ */
+int sd_step(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_new_tokens,
+            const sd_spec_params* params, const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
+            int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
+            double* d_score, int32_t* d_status, void* stream);
+
+/*
  * sd_speculate_noalloc: sd_speculate for callers that must not allocate.
  * (The paper has no counterpart; this is a deployment convenience.)
  *

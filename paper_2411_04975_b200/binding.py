@@ -18,7 +18,7 @@ from . import build as _build
 FLAG_GLOBAL_ONLY, FLAG_REQUEST_ONLY, FLAG_LINEAR = 1, 2, 4
 STATUS_BAD_SLOT, STATUS_POOL_FULL, STATUS_GLOBAL_FULL, STATUS_BAD_TOKEN = 1, 2, 4, 8
 
-EXPORTS = ["sd_build", "sd_build_requests", "sd_append", "sd_speculate", "sd_speculate_noalloc", "sd_query_counts", "sd_slot_info", "sd_entropy", "sd_stats", "sd_free",
+EXPORTS = ["sd_build", "sd_build_requests", "sd_append", "sd_speculate", "sd_step", "sd_speculate_noalloc", "sd_query_counts", "sd_slot_info", "sd_entropy", "sd_stats", "sd_free",
            "sd_strerror"]
 
 
@@ -65,6 +65,8 @@ def library() -> C.CDLL:
         lib.sd_append.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
         lib.sd_speculate.restype = C.c_int
         lib.sd_speculate.argtypes = [vp, C.c_int32, vp, C.POINTER(_SpecParams)] + [vp] * 11
+        lib.sd_step.restype = C.c_int
+        lib.sd_step.argtypes = [vp, C.c_int32, vp, vp, vp, C.POINTER(_SpecParams)] + [vp] * 11
         lib.sd_speculate_noalloc.restype = C.c_int
         lib.sd_speculate_noalloc.argtypes = lib.sd_speculate.argtypes
         lib.sd_query_counts.restype = C.c_int
@@ -240,6 +242,26 @@ class SuffixStore:
         if out is None:
             out = self.alloc_outputs(int(slots.numel()))
         sd_speculate(self._h, slots, P, alpha, max_spec, flags, budget_cap, out)
+        return out
+
+    def step(self, slots: torch.Tensor, offsets: torch.Tensor, new_tokens: torch.Tensor, P: int, alpha: float,
+             max_spec: int, flags: int = 0, budget_cap: Optional[torch.Tensor] = None,
+             out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        """One decode step in one launch: append `new_tokens` (ragged by `offsets`) to the slots,
+        then speculate.  Same result as append() followed by speculate()."""
+        if out is None:
+            out = self.alloc_outputs(int(slots.numel()))
+        prm = _SpecParams(P, alpha, max_spec, flags)
+        rc = library().sd_step(
+            self._h, int(slots.numel()), _ptr(slots, torch.int32, "slots"), _ptr(offsets, torch.int64, "offsets"),
+            _ptr(new_tokens, torch.int32, "new_tokens"), C.byref(prm), _ptr(budget_cap, torch.int32, "budget_cap"),
+            _ptr(out["n_draft"], torch.int32, "n_draft"), _ptr(out["tokens"], torch.int32, "tokens"),
+            _ptr(out["parents"], torch.int32, "parents"), _ptr(out["positions"], torch.int32, "positions"),
+            _ptr(out["mask"], torch.int32, "mask"), _ptr(out["chosen_tree"], torch.int32, "chosen_tree"),
+            _ptr(out["chosen_p"], torch.int32, "chosen_p"), _ptr(out["score"], torch.float64, "score"),
+            _ptr(out["status"], torch.int32, "status"), _stream())
+        if rc != 0:
+            raise SuffixSpecError(rc, "sd_step")
         return out
 
     def query_counts(self, tree: torch.Tensor, offsets: torch.Tensor, paths: torch.Tensor) -> torch.Tensor:

@@ -1,305 +1,7 @@
-// Online update of the suffix trees (Section 3, "Suffix Tree Construction": the
-// tokens of the ongoing request are added as they are generated, a finished
-// request's output is added to the global tree).
-//
-// One warp owns one tree for the duration of the kernel.  Appending token x at
-// context length t adds one occurrence to every string that ends at x and is at
-// most D tokens long: lane L extends the ACTIVE node of depth L (the node of
-// the last L tokens; lane 0 extends the root) by child x, creating it or
-// raising its count.  The 32 lanes work on 32 different parents at once.
-//
-// Placement.  A suffix that has left the known text creates one new leaf per appended token,
-// each the only child of the previous one.  The first such leaf reserves room for the whole
-// chain down to depth D and every later leaf goes directly behind its parent, so chains of
-// only children are consecutive entries (what the wide window loads of sd_speculate exploit).
-#include "common.cuh"
+// Batched append kernel (sd_append): see append_core.cuh for how one token is appended.
+#include "append_core.cuh"
 
 namespace {
-
-struct TreeRef {
-    int4* ent;
-    int32_t* root;
-    int cap;                 // entries in the pool
-};
-
-__device__ __forceinline__ int* word(int4* e, int k) { return reinterpret_cast<int*>(e) + k; }
-
-// Inserts child x at sorted position `pos` into the child run of `parent`
-// (cb, n children, flags in w).  `fresh` > 0: the run is full and moves to
-// ent[fresh ...).  Returns the new child's entry index.
-__device__ int insert_child(int4* ent, int parent, int cb, int n, int pos, int x, int fresh, bool moves) {
-    const int4 ne = make_int4(x, 1, 0, 0);
-    int idx;
-    // entries move eight at a time: the eight loads are in flight together
-    if (moves) {
-        for (int k0 = 0; k0 < n; k0 += 8) {
-            int4 t[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) if (k0 + u < n) t[u] = ent[cb + k0 + u];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) if (k0 + u < n) ent[fresh + k0 + u + (k0 + u >= pos ? 1 : 0)] = t[u];
-        }
-        ent[fresh + pos] = ne;
-        *word(&ent[parent], 2) = fresh;
-        idx = fresh + pos;
-    } else {
-        for (int hi = n; hi > pos; hi -= 8) {                    // from the top down
-            const int lo = max(pos, hi - 8);
-            int4 t[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) if (lo + u < hi) t[u] = ent[cb + lo + u];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) if (lo + u < hi) ent[cb + lo + u + 1] = t[u];
-        }
-        ent[cb + pos] = ne;
-        idx = cb + pos;
-    }
-    *word(&ent[parent], 3) = n + 1;               // dynamic run from now on (no RUN_STATIC)
-    return idx;
-}
-
-// The same insert done by the whole warp for a long run (all arguments warp-uniform):
-// entries move 32 at a time instead of one by one.
-__device__ int insert_child_warp(int4* ent, int parent, int cb, int n, int pos, int x, int fresh, bool moves, int lane) {
-    const int4 ne = make_int4(x, 1, 0, 0);
-    int idx;
-    if (moves) {
-        for (int i = lane; i < n; i += 32) ent[fresh + i + (i >= pos ? 1 : 0)] = ent[cb + i];
-        idx = fresh + pos;
-        if (lane == 0) { ent[idx] = ne; *word(&ent[parent], 2) = fresh; }
-    } else {
-        for (int hi = n; hi > pos; hi -= 32) {                   // from the top down, a chunk at a time
-            const int lo = max(pos, hi - 32);
-            const int i = lo + lane;
-            int4 e = make_int4(0, 0, 0, 0);
-            if (i < hi) e = ent[cb + i];
-            __syncwarp();
-            if (i < hi) ent[cb + i + 1] = e;
-            __syncwarp();
-        }
-        idx = cb + pos;
-        if (lane == 0) ent[idx] = ne;
-    }
-    if (lane == 0) *word(&ent[parent], 3) = n + 1;
-    __syncwarp();
-    return idx;
-}
-
-// lower_bound of token x in the sorted run ent[cb .. cb+n): 32-way, then eight-way, so that the
-// probes of a round are in flight together (a long run costs a few dependent rounds).
-__device__ int lower_bound_run(const int4* ent, int cb, int n, int x) {
-    int lo = 0, hi = n;
-    while (hi - lo > 256) {                                      // very long runs: 32-way, 31 probes in flight
-        const int step = (hi - lo) >> 5;
-        int sel = 0;
-#pragma unroll
-        for (int k = 0; k < 31; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
-        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
-        const int nhi = sel == 31 ? hi : lo + (sel + 1) * step;
-        lo = nlo; hi = nhi;
-    }
-    while (hi - lo > 8) {                                        // at most 3 rounds from 256
-        const int step = (hi - lo) >> 3;
-        int t[7];
-#pragma unroll
-        for (int k = 0; k < 7; ++k) t[k] = ent[cb + lo + (k + 1) * step].x;
-        int sel = 0;
-#pragma unroll
-        for (int k = 0; k < 7; ++k) sel += t[k] < x ? 1 : 0;     // pivots below x
-        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
-        const int nhi = sel == 7 ? hi : lo + (sel + 1) * step;
-        lo = nlo; hi = nhi;
-    }
-    // at most eight candidates left: all of them in one round
-    int t[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) t[k] = lo + k < hi ? ent[cb + lo + k].x : 0x7fffffff;
-    int below = 0;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) below += t[k] < x ? 1 : 0;
-    return lo + below;
-}
-
-// Look-up of child x in the sorted run ent[cb .. cb+n): insert position in `pos`, and if the
-// child exists its index is returned with its entry in `fe` (else -1).  The last round reads
-// whole entries, so a run of up to eight children costs one round of loads.
-__device__ int lookup_child(const int4* ent, int cb, int n, int x, int& pos, int4& fe) {
-    int lo = 0, hi = n;
-    while (hi - lo > 256) {                                      // very long runs: 32-way, 31 probes in flight
-        const int step = (hi - lo) >> 5;
-        int sel = 0;
-#pragma unroll
-        for (int k = 0; k < 31; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
-        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
-        const int nhi = sel == 31 ? hi : lo + (sel + 1) * step + 1;   // keep the pivot: it may be x itself
-        lo = nlo; hi = nhi;
-    }
-    while (hi - lo > 8) {                                        // eight-way down to a window of eight
-        const int step = (hi - lo) >> 3;
-        int sel = 0;
-#pragma unroll
-        for (int k = 0; k < 7; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
-        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
-        const int nhi = sel == 7 ? hi : lo + (sel + 1) * step + 1;
-        lo = nlo; hi = nhi;
-    }
-    int4 e[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) e[k] = lo + k < hi ? ent[cb + lo + k] : make_int4(0x7fffffff, 0, 0, 0);
-    int below = 0;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) below += e[k].x < x ? 1 : 0;
-    pos = lo + below;
-    int found = -1;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) if (k == below && lo + k < hi && e[k].x == x) { fe = e[k]; found = cb + lo + k; }
-    return found;
-}
-
-// Child x of `node` (-1 if none), by plain loads.
-__device__ int peek_child(const int4* ent, int node, int x) {
-    if (node < 0) return -1;
-    const int4 pe = ent[node];
-    const int n = (int)((unsigned)pe.w & RUN_COUNT_MASK);
-    if (n == 0) return -1;
-    const int pos = lower_bound_run(ent, pe.z, n, x);
-    if (pos >= n) return -1;
-    return ent[pe.z + pos].x == x ? pe.z + pos : -1;
-}
-
-// The slow look-ups of a token are the shallow ones (long child runs of frequent tokens, cold in
-// the caches), and they depend only on the last two or three tokens, not on the deep state.
-// Lane j walks the two- and three-token strings that end at token k0 + j, 32 tokens at once, so
-// that the token-by-token pass finds those runs in the caches.  Nothing is decided here; the
-// return value only keeps the loads alive.
-__device__ int warm_shallow(const TreeRef& tr, int V, const int32_t* tok, long long b, long long e, long long k0,
-                            int lane) {
-    const long long k = k0 + lane;
-    if (k >= e) return 0;
-    const int x0 = tok[k];
-    const int x1 = k - 1 >= b ? tok[k - 1] : -1, x2 = k - 2 >= b ? tok[k - 2] : -1;
-    if (x0 < 0 || x0 >= V || x1 < 0 || x1 >= V) return 0;
-    int seen = 0;
-    const int c1 = peek_child(tr.ent, tr.root[x1], x0);                        // (x1, x0)
-    if (c1 >= 0) seen += tr.ent[c1].y;
-    if (x2 >= 0 && x2 < V) {
-        const int c2 = peek_child(tr.ent, peek_child(tr.ent, tr.root[x2], x1), x0);   // (x2, x1, x0)
-        if (c2 >= 0) seen += tr.ent[c2].y;
-    }
-    return seen;
-}
-
-// All 32 lanes call.  `act` is this lane's active node of depth lane + 1 (-1: none);
-// on return it is the active node after x was appended.  `t` is the context length
-// before the append.  `used` / `live` are warp-uniform pool counters.
-// Returns false, changing nothing, if the pool cannot hold the new nodes.
-// (run_cb, run_w) travel with `act`: the active node's child run as of now, so that the
-// next token's look-up starts at the run itself instead of first reading the node.
-__device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, int& act, int& room, int& run_cb,
-                             unsigned& run_w, int& used, int& live) {
-    const unsigned FULL = 0xffffffffu;
-    const int parent = __shfl_up_sync(FULL, act, 1);            // node of depth `lane`
-    const int parent_room = __shfl_up_sync(FULL, room, 1);      // free entries reserved behind it
-    const int parent_cb = __shfl_up_sync(FULL, run_cb, 1);
-    const unsigned parent_w = __shfl_up_sync(FULL, run_w, 1);
-    const bool valid = lane <= min(t, D - 1);
-    int found = -1, pos = 0, cb = 0, n = 0;
-    unsigned w = 0;
-    int4 fe = make_int4(0, 0, 0, 0);                             // the child's entry when found
-    if (valid) {
-        if (lane == 0) {
-            found = tr.root[x];
-            if (found >= 0) fe = tr.ent[found];
-        } else {
-            cb = parent_cb; w = parent_w;
-            if (w == RUN_UNKNOWN) { const int4 pe = tr.ent[parent]; cb = pe.z; w = (unsigned)pe.w; }
-            n = (int)(w & RUN_COUNT_MASK);
-            found = lookup_child(tr.ent, cb, n, x, pos, fe);
-        }
-    }
-    const bool need = valid && found < 0;
-    int asz = 0;                                                 // fresh entries this lane needs
-    bool behind_parent = false;                                  // the new leaf goes to parent + 1
-    int new_room = 0;
-    if (need) {
-        if (lane == 0 || n == 0) {
-            // first child of a leaf (or a new depth-1 node): start or continue a chain block
-            if (lane > 0 && parent_room > 0) { behind_parent = true; new_room = parent_room - 1; }
-            else { asz = D - lane; new_room = asz - 1; }
-        } else if ((uint32_t)n == sd_run_capacity(w)) {
-            asz = (int)sd_pow2ceil((uint32_t)n + 1u);
-        }
-    }
-    int inc = asz;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(FULL, inc, o);
-        if (lane >= o) inc += y;
-    }
-    const int total = __shfl_sync(FULL, inc, 31);
-    if ((long long)used + total > (long long)tr.cap) return false;
-    const int fresh = behind_parent ? parent + 1 : used + inc - asz;
-    const bool moves = behind_parent || asz > 0;
-    used += total;
-
-    // A lane that moves entries of its run must not do so while the next lane edits the
-    // header of an entry inside that run (only possible when the last tokens repeat one
-    // token): it then waits for that lane, see the rounds below.
-    const int next_parent = __shfl_down_sync(FULL, parent, 1);
-    const int next_need = __shfl_down_sync(FULL, need ? 1 : 0, 1);
-    const bool clash = need && lane >= 1 && lane < 31 && next_need && next_parent >= cb && next_parent < cb + n;
-
-    if (valid && found >= 0) {
-        // a count changes: the copies in the run's top block (if any) are stale from now on
-        if (lane > 0 && (w & RUN_HAS_TOP)) *word(&tr.ent[parent], 3) = (int)(w & ~RUN_HAS_TOP);
-        *word(&tr.ent[found], 1) = fe.y + 1;
-        act = found;
-        run_cb = fe.z;
-        run_w = (unsigned)fe.w;
-        // the next lane works on this very node's run (new child, or flag dropped): what was read may be stale
-        if (lane < 31 && next_parent == found) run_w = RUN_UNKNOWN;
-        else if (run_w & RUN_COUNT_MASK) asm volatile("prefetch.global.L2 [%0];" ::"l"(tr.ent + run_cb));
-    } else {
-        run_cb = 0;
-        run_w = 0;                                               // a new leaf (or no node at all)
-    }
-    room = new_room;
-    // Inserts run in rounds: a lane whose insert would move an entry that the next lane still has
-    // to edit waits for that lane (deepest first); everybody else goes at once.  Almost always
-    // there is one round; a tail of k equal tokens needs up to k.
-    unsigned pend = __ballot_sync(FULL, need);
-    for (int round = 0; round < 33 && pend; ++round) {
-        const bool next_pending = lane < 31 && ((pend >> (lane + 1)) & 1u);
-        const bool ready = need && ((pend >> lane) & 1u) && !(clash && next_pending);
-        // inserts that move many entries are done by the whole warp, one after the other
-        const bool big = ready && lane > 0 && (moves ? n : n - pos) > 48;
-        if (ready && !big) {
-            if (lane == 0) {
-                tr.ent[fresh] = make_int4(x, 1, 0, 0);
-                tr.root[x] = fresh;
-                act = fresh;
-            } else {
-                act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, moves);
-            }
-        }
-        __syncwarp();
-        unsigned bm = __ballot_sync(FULL, big);
-        while (bm) {
-            const int src = __ffs(bm) - 1;
-            bm &= bm - 1;
-            const int idx = insert_child_warp(tr.ent, __shfl_sync(FULL, parent, src), __shfl_sync(FULL, cb, src),
-                                              __shfl_sync(FULL, n, src), __shfl_sync(FULL, pos, src), x,
-                                              __shfl_sync(FULL, fresh, src), __shfl_sync(FULL, moves ? 1 : 0, src) != 0,
-                                              lane);
-            if (lane == src) act = idx;
-        }
-        pend &= ~__ballot_sync(FULL, ready);
-        __syncwarp();
-    }
-    if (!valid) { act = -1; room = 0; run_cb = 0; run_w = 0; }
-    live += __popc(__ballot_sync(FULL, need));
-    return true;
-}
 
 // Warp 0 of the grid inserts whole sequences into the global tree, one after the
 // other; warp i + 1 appends item i to its request slot.

@@ -10,7 +10,7 @@
 // operation a separately rounded IEEE binary64 operation (no FMA contraction).
 #include <mutex>
 
-#include "common.cuh"
+#include "append_core.cuh"
 
 namespace {
 
@@ -480,8 +480,10 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
 // MatchPattern from a known node: descend text[from .. to).  Levels whose child run lies inside
 // the window already in registers cost no memory access.  Returns the node reached (-1: no
 // match) and its child run in (cb, n).
-__device__ int walk_from(const int4* __restrict__ ent, int limit, int node, const int32_t* __restrict__ text, int from,
-                         int to, int lane, int& cb, unsigned& wfull) {
+// The context is `text` up to position t_old and `newtok` from there on (tokens that are
+// being appended in the same launch).
+__device__ int walk_from(const int4* __restrict__ ent, int limit, int node, const int32_t* __restrict__ text, int t_old,
+                         const int32_t* __restrict__ newtok, int from, int to, int lane, int& cb, unsigned& wfull) {
     if (node < 0) return -1;
     int wb = node;
     int4 w = load_window(ent, wb, limit, lane);
@@ -489,7 +491,7 @@ __device__ int walk_from(const int4* __restrict__ ent, int limit, int node, cons
     wfull = (unsigned)__shfl_sync(FULL, w.w, 0);
     int n = (int)(wfull & RUN_COUNT_MASK);
     for (int pos = from; pos < to; ++pos) {
-        const int x = text[pos];
+        const int x = pos < t_old ? text[pos] : newtok[pos - t_old];
         if (n == 0) return -1;
         if (n > 32) {                                           // wide run: 32-way search
             int4 e;
@@ -736,11 +738,17 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
     __syncwarp();
 }
 
+// STEP: the block first appends the request's newly accepted tokens (warp 0, exactly what
+// sd_append does for the slot) while its other warps already advance the global match nodes
+// over those tokens, then speculates: one launch per decode step, and the appends of long
+// token lists overlap with the speculation of the other requests.
+template <bool STEP>
 __global__ void __launch_bounds__(CTA_WARPS * 32, CTA_MIN_BLOCKS)
 speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
                        unsigned flags, const int32_t* __restrict__ d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
                        int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
-                       int32_t* d_chosen_p, double* d_score, int32_t* d_status) {
+                       int32_t* d_chosen_p, double* d_score, int32_t* d_status, const int64_t* __restrict__ d_app_off,
+                       const int32_t* __restrict__ d_app_tok) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     BlockShared& sh = *reinterpret_cast<BlockShared*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, wib = tid >> 5;
@@ -751,7 +759,17 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     int t = 0, status = SD_STATUS_BAD_SLOT;
     SlotState* ss = nullptr;
     if (ok) { ss = sv.s_state + slot; t = ss->len; status = ss->status; }
-    const bool usable = ok && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && t > 0;
+    // STEP: t_old tokens are in the slot's text, the next n_new come from the append list; the
+    // match below already runs on the context of t = t_old + n_new tokens
+    const int t_old = t;
+    const int32_t* newtok = nullptr;
+    int n_new = 0;
+    if (STEP && ok) {
+        newtok = d_app_tok + d_app_off[i];
+        n_new = (int)(d_app_off[i + 1] - d_app_off[i]);
+        t = t_old + n_new;
+    }
+    bool usable = ok && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && t > 0;
     int cap = max_spec;
     if (d_budget_cap && d_budget_cap[i] >= 0) cap = min(cap, d_budget_cap[i]);
     if (tid < 2 * SD_MAX_DEPTH) { (&sh.node[0][0])[tid] = -1; (&sh.nc[0][0])[tid] = 0; }
@@ -760,45 +778,85 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     if (lane == 0) { W.best_score = 0.0; W.best_order = 1 << 30; W.best_n = 0; W.best_buf = 0; }
 
     // ---------------- 1. match
-    const bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
-    const bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
-    int src_node[MATCH_ROUNDS], src_from[MATCH_ROUNDS];         // per target: start node and first text index
+    bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
+    bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
+    // warps that advance the global match nodes, and this warp's rank among them
+    const int mwarps = STEP ? CTA_WARPS - 1 : CTA_WARPS;
+    const int mrank = STEP ? wib - 1 : wib;
+    constexpr int MROUNDS = STEP ? (SD_MAX_DEPTH + CTA_WARPS - 2) / (CTA_WARPS - 1) : MATCH_ROUNDS;
+    int src_node[MROUNDS], src_from[MROUNDS];                   // per target: start node and first text index
 #pragma unroll
-    for (int h = 0; h < MATCH_ROUNDS; ++h) { src_node[h] = -1; src_from[h] = 0; }
+    for (int h = 0; h < MROUNDS; ++h) { src_node[h] = -1; src_from[h] = 0; }
     const int32_t* text = ok ? sv.s_text + (long long)slot * sv.T : nullptr;
-    if (want_g) {
+    if (want_g && mrank >= 0) {
         const bool cache_ok = ss->g_gen == ss->gen && ss->g_epoch == sv.g_state->epoch && ss->g_len <= t;
         const int k = t - ss->g_len;                            // tokens appended since the cache was taken
         const int depths = ss->g_depths;
 #pragma unroll
-        for (int h = 0; h < MATCH_ROUNDS; ++h) {
-            const int d = wib + 1 + h * CTA_WARPS;              // target pattern length
+        for (int h = 0; h < MROUNDS; ++h) {
+            const int d = mrank + 1 + h * mwarps;               // target pattern length
             if (d > Pe || d > t) continue;
             if (cache_ok && d > k && d - k <= depths) {
                 src_node[h] = ss->g_node[d - k - 1];            // node of the tokens before the new ones
                 src_from[h] = t - k;
             } else {
-                src_node[h] = sv.g_root[text[t - d]];
+                const int x0 = t - d < t_old ? text[t - d] : newtok[t - d - t_old];
+                src_node[h] = (x0 >= 0 && x0 < sv.V) ? sv.g_root[x0] : -1;
                 src_from[h] = t - d + 1;
             }
         }
     }
     __syncthreads();                                            // all cached nodes read before any is replaced
-    if (want_g) {
+    if (STEP && wib == 0 && ok && n_new > 0) {
+        // ---- the request's accepted tokens go into its tree and text (as sd_append does)
+        int32_t* wtext = sv.s_text + (long long)slot * sv.T;
+        TreeRef tr{sv.s_ent + (long long)slot * sv.spn, sv.s_root + (long long)slot * sv.V, (int)sv.spn};
+        int len = ss->len, used = ss->used, live = ss->live, st = ss->status;
+        int act = ss->active[lane], room = ss->room[lane], run_cb = ss->run_cb[lane];
+        unsigned run_w = ss->run_w[lane];
+        for (int k = 0; k < n_new && !(st & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)); ++k) {
+            const int x = newtok[k];
+            if (x < 0 || x >= sv.V) { st |= SD_STATUS_BAD_TOKEN; break; }
+            if (len >= sv.T || !append_token(tr, sv.D, x, len, lane, act, room, run_cb, run_w, used, live)) {
+                st |= SD_STATUS_POOL_FULL;
+                break;
+            }
+            if (lane == 0) wtext[len] = x;
+            ++len;
+        }
+        ss->active[lane] = act; ss->room[lane] = room; ss->run_cb[lane] = run_cb; ss->run_w[lane] = run_w;
+        if (lane == 0) { ss->len = len; ss->used = used; ss->live = live; ss->status = st; }
+    }
+    if (want_g && mrank >= 0) {
 #pragma unroll
-        for (int h = 0; h < MATCH_ROUNDS; ++h) {
-            const int d = wib + 1 + h * CTA_WARPS;
+        for (int h = 0; h < MROUNDS; ++h) {
+            const int d = mrank + 1 + h * mwarps;
             if (d > Pe) continue;
             int cb = 0;
             unsigned wf = 0;
-            const int node = (d > t) ? -1 : walk_from(sv.g_ent, (int)sv.g_cap, src_node[h], text, src_from[h], t, lane, cb, wf);
+            const int node = (d > t) ? -1 : walk_from(sv.g_ent, (int)sv.g_cap, src_node[h], text, t_old, newtok, src_from[h], t,
+                                                      lane, cb, wf);
             if (lane == 0) {
                 ss->g_node[d - 1] = node;
                 sh.node[0][d - 1] = node;
                 if (node >= 0) { sh.cb[0][d - 1] = cb; sh.nc[0][d - 1] = wf; }
             }
         }
-        if (tid == 0) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = Pe; }
+        if (tid == (STEP ? 32 : 0)) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = Pe; }
+    }
+    if (STEP) {
+        __syncthreads();                                        // the append is done and visible
+        if (ok) {
+            status = ss->status;
+            if (ss->len != t || (status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN))) {
+                // the append stopped early: no speculation for this request, and the match nodes
+                // taken above describe a context that does not exist
+                usable = false; want_g = false; want_r = false;
+                t = ss->len;
+                if (tid == 0) ss->g_gen = ss->gen - 1;
+                if (tid < 2 * SD_MAX_DEPTH) { (&sh.node[0][0])[tid] = -1; (&sh.nc[0][0])[tid] = 0; }
+            }
+        }
     }
     if (want_r && wib == CTA_WARPS - 1) {
         const int d = lane + 1;
@@ -960,10 +1018,11 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
 
 }  // namespace
 
-extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
-                            const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents,
-                            int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
-                            double* d_score, int32_t* d_status, void* stream) {
+static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
+                        const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents,
+                        int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
+                        double* d_score, int32_t* d_status, const int64_t* d_app_off, const int32_t* d_app_tok,
+                        bool step, void* stream) {
     if (!s || !prm || n < 0 || n > s->R) return SD_ERR_INVALID_ARG;
     if (prm->P < 1 || prm->max_spec < 0 || prm->max_spec > s->M || !(prm->alpha >= 0.0)) return SD_ERR_INVALID_ARG;
     if ((prm->flags & SD_FLAG_GLOBAL_ONLY) && (prm->flags & SD_FLAG_REQUEST_ONLY)) return SD_ERR_INVALID_ARG;
@@ -971,6 +1030,7 @@ extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const
     if (!d_slot || !d_n_draft || !d_tokens || !d_parents || !d_positions || !d_mask || !d_chosen_tree || !d_chosen_p ||
         !d_score)
         return SD_ERR_INVALID_ARG;
+    if (step && !d_app_off) return SD_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int Pe = prm->P < s->D ? prm->P : s->D;               // longer patterns never match
     {
@@ -979,17 +1039,39 @@ extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const
         int dev = 0;
         SD_CUDA_OK(cudaGetDevice(&dev));
         if (dev >= 0 && dev < 64 && !raised[dev]) {
-            SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)sizeof(BlockShared)));
+            SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)sizeof(BlockShared)));
             raised[dev] = true;
         }
     }
-    speculate_fused_kernel<<<(unsigned)n, CTA_WARPS * 32, sizeof(BlockShared), st>>>(*s, n, d_slot, Pe, prm->alpha, prm->max_spec,
-                                                                  prm->flags, d_budget_cap, d_n_draft, d_tokens,
-                                                                  d_parents, d_positions, d_mask, d_chosen_tree,
-                                                                  d_chosen_p, d_score, d_status);
+    if (step)
+        speculate_fused_kernel<true><<<(unsigned)n, CTA_WARPS * 32, sizeof(BlockShared), st>>>(
+            *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,
+            d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, d_app_off, d_app_tok);
+    else
+        speculate_fused_kernel<false><<<(unsigned)n, CTA_WARPS * 32, sizeof(BlockShared), st>>>(
+            *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,
+            d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, nullptr, nullptr);
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
+}
+
+extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
+                            const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents,
+                            int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
+                            double* d_score, int32_t* d_status, void* stream) {
+    return launch_fused(s, n, d_slot, prm, d_budget_cap, d_n_draft, d_tokens, d_parents, d_positions, d_mask, d_chosen_tree,
+                        d_chosen_p, d_score, d_status, nullptr, nullptr, false, stream);
+}
+
+extern "C" int sd_step(sd_store* s, int32_t n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_new_tokens,
+                       const sd_spec_params* prm, const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
+                       int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
+                       int32_t* d_chosen_p, double* d_score, int32_t* d_status, void* stream) {
+    return launch_fused(s, n, d_slot, prm, d_budget_cap, d_n_draft, d_tokens, d_parents, d_positions, d_mask, d_chosen_tree,
+                        d_chosen_p, d_score, d_status, d_offsets, d_new_tokens, true, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

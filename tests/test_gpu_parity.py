@@ -435,3 +435,52 @@ def test_entropy_matches_oracle(U):
         assert abs(got - want) <= 1e-9 * max(1.0, abs(want)), (tree, got, want)
     assert pr.g.entropy(1) == 0.0                                # empty slot
     pr.close()
+
+
+# ---------------------------------------------------------------- fused decode step
+@pytest.mark.parametrize("vocab,D", [(2, 32), (6, 8), (40, 16)])
+def test_step_equals_append_then_speculate(U, vocab, D):
+    rng = np.random.default_rng(vocab * 7 + D)
+    n_slots = 20
+    pr = U.Pair(_rand_seqs(rng, 15, 50, 300, vocab), vocab=vocab, D=D, n_slots=n_slots, max_req_tokens=400)
+    pr.append(list(range(n_slots)), _rand_seqs(rng, n_slots, 0, 150, vocab), reset=[1] * n_slots)
+    slots = list(range(n_slots))
+    for step in range(6):
+        lists = _rand_seqs(rng, n_slots, 0, 17, vocab)
+        if step == 2:
+            lists[3] = np.full(30, vocab - 1, dtype=np.int32)       # a repeated token
+        off, flat = U.ragged(lists)
+        out = pr.g.step(U.dev_i32(slots), torch.as_tensor(off, device=U.DEV),
+                        U.dev_i32(flat) if flat.size else torch.zeros(0, dtype=torch.int32, device=U.DEV), 32, 2.0, 64,
+                        flags=4 if step == 4 else 0)
+        torch.cuda.synchronize()
+        pr.o.slot_append_batch(slots, lists, n_threads=4)
+        want = pr.o.speculate(slots, 32, 2.0, 64, M=64, flags=4 if step == 4 else 0, n_threads=4)
+        got = {k: v.cpu().numpy() for k, v in out.items()}
+        got["mask"] = got["mask"].view(np.uint32)
+        U.assert_same_drafts(got, want)
+        # plain speculate on the stepped store agrees too (the cached match nodes are consistent)
+        pr.check_speculate(slots, 32, 2.0, 64)
+    for s_ in range(n_slots):
+        pr.check_tree(s_)
+    pr.close()
+
+
+def test_step_reports_a_stopped_append(U):
+    rng = np.random.default_rng(4)
+    pr = U.Pair(_rand_seqs(rng, 3, 30, 60, 50), vocab=50, D=8, n_slots=3, max_req_tokens=40)
+    pr.append([0, 1, 2], _rand_seqs(rng, 3, 10, 20, 50), reset=[1, 1, 1])
+    lists = [rng.integers(0, 50, size=60).astype(np.int32),        # overflows the text buffer of slot 0
+             np.array([3, 99], dtype=np.int32),                      # token outside the vocabulary
+             rng.integers(0, 50, size=4).astype(np.int32)]
+    off, flat = U.ragged(lists)
+    out = pr.g.step(U.dev_i32([0, 1, 2]), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat), 8, 2.0, 16)
+    torch.cuda.synchronize()
+    st = out["status"].cpu().numpy()
+    assert st[0] & 2 and st[1] & 8 and st[2] == 0
+    assert int(out["n_draft"][0]) == 0 and int(out["n_draft"][1]) == 0
+    pr.o.slot_append(2, lists[2])
+    want = pr.o.speculate([2], 8, 2.0, 16, M=64)
+    assert int(out["n_draft"][2]) == int(want["n_draft"][0])
+    assert out["tokens"][2].cpu().numpy().tolist() == want["tokens"][0].tolist()
+    pr.close()

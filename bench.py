@@ -3,9 +3,11 @@
 
 A step is one decode step of the whole batch on the headline workload
 (config "large_batch": 4M-token global corpus, 256 requests with 4,096-token
-prompts): sd_speculate for every request, then sd_append of the tokens each
-request accepted in that step (a seeded schedule, mean 4 tokens, taken from the
-request's hidden continuation).  The global tree and the prompts are built
+prompts): the tokens each request accepted in the previous step (a seeded
+schedule, mean 4 tokens, taken from the request's hidden continuation) are
+appended to its tree, then a draft tree is speculated for every request.  That is
+one sd_step launch; the same work as two calls (sd_append, sd_speculate) is timed
+beside it.  The global tree and the prompts are built
 before the timed region.  One JSON line is printed by rank 0.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
@@ -29,7 +31,7 @@ if ROOT not in sys.path:
 
 from workload.generator import accept_schedule, get_workload  # noqa: E402
 
-METRIC = "speculation trees/s at batch 256 (one sd_speculate + sd_append per step)"
+METRIC = "speculation trees/s at batch 256 (per step: append the accepted tokens, speculate)"
 UNIT = "trees/s"
 OUT_BYTES_PER_REQ = 4 * 64 * 3 + 64 * 8 + 4 * 3 + 8          # tokens, parents, positions, mask, scalars
 FLUSH_BYTES = 256 << 20
@@ -160,7 +162,8 @@ def run_ours(args):
     B, K, W = c.batch, args.steps, args.warmup
     Ke = 0 if args.no_e2e else K
     We = 0 if args.no_e2e else min(W, 3)
-    n_steps = W + K + We + Ke
+    K2 = min(K, 30)                                   # steps timed as two calls, for the breakdown
+    n_steps = W + K + We + Ke + K2
     first = sharding.request_range(rank, world, B)[0]   # weak scaling: every rank has its own requests
     prompts = [w.prompt(first + i) for i in range(B)]
     steps = StepInputs(w, first, B, n_steps, prompts)
@@ -185,12 +188,13 @@ def run_ours(args):
 
     d_off = [torch.as_tensor(o, device=dev) for o in steps.offsets[:W + K]]
     d_tok = [torch.as_tensor(t, device=dev) for t in steps.tokens[:W + K]]
+    d_off2 = [torch.as_tensor(o, device=dev) for o in steps.offsets[W + K + We + Ke:]]
+    d_tok2 = [torch.as_tensor(t, device=dev) for t in steps.tokens[W + K + We + Ke:]]
     out = store.alloc_outputs(B)
     flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
 
     def step(k):
-        store.speculate(slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
-        store.append(slots, d_off[k], d_tok[k])
+        store.step(slots, d_off[k], d_tok[k], c.max_pattern, c.alpha, c.max_spec, 0, None, out)
 
     n_samp = 0 if (args.no_oracle or world > 1) else max(1, min(args.oracle_samples, K))
     sample_steps = sorted({W + (j * K) // n_samp for j in range(n_samp)}) if n_samp else []
@@ -210,16 +214,14 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
     wall0 = time.perf_counter()
     for j in range(K):
         k = W + j
         flush.zero_()                                  # L2 flush, outside the per-step events
         ev[j][0].record()
-        store.speculate(slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
+        step(k)
         ev[j][1].record()
-        store.append(slots, d_off[k], d_tok[k])
-        ev[j][2].record()
         if k in sample_steps:
             saved[k] = {n: t.clone() for n, t in out.items()}
     torch.cuda.synchronize()
@@ -227,9 +229,7 @@ def run_ours(args):
         dist.barrier()
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - wall0) * 1e3
-    spec_ms = [ev[j][0].elapsed_time(ev[j][1]) for j in range(K)]
-    app_ms = [ev[j][1].elapsed_time(ev[j][2]) for j in range(K)]
-    tot_ms = [ev[j][0].elapsed_time(ev[j][2]) for j in range(K)]
+    tot_ms = [ev[j][0].elapsed_time(ev[j][1]) for j in range(K)]
     timed_ms = sharding.max_over_ranks(float(sum(tot_ms)), dev)
     ms_per_step = timed_ms / K
 
@@ -260,9 +260,8 @@ def run_ours(args):
             nt = n_tok[k]
             nb = 8 * (B + 1) + 4 * B + 4 * nt
             d_in[:nb].copy_(h_in[k][:nb], non_blocking=True)
-            store.speculate(s_slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
+            store.step(s_slots, s_off, s_tok[:nt], c.max_pattern, c.alpha, c.max_spec, 0, None, out)
             h_packed.copy_(out["packed"], non_blocking=True)
-            store.append(s_slots, s_off, s_tok[:nt])
             torch.cuda.synchronize()
             h2d += nb
             d2h += h_packed.numel()
@@ -288,6 +287,18 @@ def run_ours(args):
         e2e = {"value": B * world * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d // Ke,
                "d2h_bytes_per_step": d2h // Ke, "ms_per_step": e2e_s / Ke * 1e3}
 
+    # ---- the same work as two calls (sd_append, then sd_speculate), for the breakdown
+    app_ms, spec_ms = [], []
+    for k in range(K2):
+        flush.zero_()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record()
+        store.append(slots, d_off2[k], d_tok2[k])
+        e1.record()
+        store.speculate(slots, c.max_pattern, c.alpha, c.max_spec, 0, None, out)
+        e2.record()
+        torch.cuda.synchronize()
+        app_ms.append(e0.elapsed_time(e1)); spec_ms.append(e1.elapsed_time(e2))
     clocks = sampler.stop() if rank == 0 else None      # sampled from warm-up to the end of the e2e loop
 
     # ---- CPU oracle beside it (rank 0, one GPU): lock-step replay, sampled steps timed and compared
@@ -305,9 +316,9 @@ def run_ours(args):
         o_times, desc, adds, ok = [], [], [], True
         for k in range(max(sample_steps) + 1):
             t0 = time.perf_counter()
+            ref.slot_append_batch(list(range(B)), steps.lists[k], n_threads=thr)
             if k in sample_steps:
                 r = ref.speculate(list(range(B)), c.max_pattern, c.alpha, c.max_spec, n_threads=thr)
-            ref.slot_append_batch(list(range(B)), steps.lists[k], n_threads=thr)
             if k in sample_steps:
                 o_times.append(time.perf_counter() - t0)
                 desc.append(int(r["visited"][:, 0].sum()))
@@ -324,11 +335,11 @@ def run_ours(args):
         visits = statistics.mean(d + a for d, a in zip(desc, adds))
         alg_bytes = statistics.mean(32 * d + 64 * a for d, a in zip(desc, adds)) + B * OUT_BYTES_PER_REQ
         peak, which = measured_peak()
-        spec_s = statistics.mean(spec_ms) / 1e3
+        spec_s = statistics.mean(tot_ms) / 1e3               # the whole launch: append + speculate
         achieved = alg_bytes / spec_s / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": SPECULATE_DRAM_TRAFFIC if c.name == "large_batch" and not args.small else None,
-                    "peak_source": which, "kernel": "speculate_fused_kernel (all of sd_speculate)",
+                    "peak_source": which, "kernel": "speculate_fused_kernel<STEP> (all of sd_step)",
                     "algorithmic_bytes_per_launch": alg_bytes}
         extra = {"parity_vs_oracle": "bit-exact" if ok else "MISMATCH", "parity_steps": len(sample_steps),
                  "nodes_visited_per_step": visits,
@@ -346,13 +357,14 @@ def run_ours(args):
                        "D": c.depth_cap, "P": c.max_pattern, "alpha": c.alpha, "max_spec": c.max_spec,
                        "l2": "flushed between steps (256 MiB write outside the timed events)",
                        "parallelism": f"replica x{world}, requests sharded" if world > 1 else "single GPU"},
-            "speculate_us": {"mean": statistics.mean(spec_ms) * 1e3, "p50": statistics.median(spec_ms) * 1e3,
-                             "max": max(spec_ms) * 1e3},
-            "append_us": {"mean": statistics.mean(app_ms) * 1e3, "p50": statistics.median(app_ms) * 1e3},
+            "step_us": {"mean": statistics.mean(tot_ms) * 1e3, "p50": statistics.median(tot_ms) * 1e3,
+                        "max": max(tot_ms) * 1e3},
+            "two_calls": {"steps": K2, "append_us": statistics.mean(app_ms) * 1e3 if app_ms else None,
+                          "speculate_us": statistics.mean(spec_ms) * 1e3 if spec_ms else None},
             "tokens_appended_per_step": float(np.mean([t.size for t in steps.tokens[W:W + K]])),
             "build_ms": build_ms, "prompt_build_ms": prompt_ms, "global_nodes": st["global_nodes"],
             "device_bytes": st["device_bytes"], "wall_ms_timed_region": wall_ms,
-            "gpu_launches": 2 * K, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "gpu_launches": K, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "clocks": clocks,
         }
         line.update(extra)

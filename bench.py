@@ -35,9 +35,9 @@ METRIC = "speculation trees/s at batch 256 (per step: append the accepted tokens
 UNIT = "trees/s"
 OUT_BYTES_PER_REQ = 4 * 64 * 3 + 64 * 8 + 4 * 3 + 8          # tokens, parents, positions, mask, scalars
 FLUSH_BYTES = 256 << 20
-# dram__bytes_read + dram__bytes_write of one speculate_fused_kernel launch on the full-size
+# dram__bytes_read + dram__bytes_write of one speculate_fused_kernel<STEP> launch (sd_step) on the full-size
 # large_batch workload, from the ncu capture summarised in profiles/ (set to None when the kernel changes)
-SPECULATE_DRAM_TRAFFIC = 25.9e6
+SPECULATE_DRAM_TRAFFIC = 28.4e6
 
 
 def parse():

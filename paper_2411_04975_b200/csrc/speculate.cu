@@ -299,7 +299,9 @@ struct BlockShared {
     int njobs, next, nwide, nwide_kept;
     long long slice_sum[CTA_WARPS];
     int slice_fs[CTA_WARPS];
-    unsigned long long best_bits;             // largest finished SCORE so far, as ordered bits
+    unsigned best_hi;                         // high word of the largest SCORE reached so far: a lower
+                                              // bound of it (scores are non-negative doubles), which is
+                                              // all the pruning needs; 32 bits keep the atomic native
     int win_warp;
 };
 
@@ -610,7 +612,7 @@ __device__ void counts_to_d(Frontier& F, int fh, int fs, double d_parent, long l
 }
 
 __device__ __forceinline__ double best_so_far(BlockShared& sh) {
-    return __shfl_sync(FULL, __longlong_as_double((long long)*(volatile unsigned long long*)&sh.best_bits), 0);
+    return __hiloint2double((int)__shfl_sync(FULL, *(volatile unsigned*)&sh.best_hi, 0), 0);
 }
 
 // ExpandSpeculationTree + SCORE for one (tree, p) job by one warp.  With `seeded` the frontier
@@ -647,7 +649,7 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
             if (lane == 0) { W.tok[buf][cnt] = tok; W.par[buf][cnt] = (unsigned char)(par + 1); }
             score = __dadd_rn(score, cur_d);                    // Eq. 4, insertion order
             // the final SCORE of this job is at least its running value: let the others prune on it
-            if (lane == 0) atomicMax(&sh.best_bits, (unsigned long long)__double_as_longlong(score));
+            if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
             cur_idx = cnt++;
             const int K = budget - cnt;
             if (fs > K) fs = K;
@@ -715,7 +717,7 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
                 W.par[buf][cnt + lane] = (unsigned char)((lane == 0 ? cur_idx : cnt + lane - 1) + 1);
             }
             for (int q = 0; q < m; ++q) score = __dadd_rn(score, cur_d);
-            if (lane == 0) atomicMax(&sh.best_bits, (unsigned long long)__double_as_longlong(score));
+            if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
             cnt += m;
             if (fs > budget - cnt) fs = budget - cnt;
             cur_idx = cnt - 1;
@@ -732,7 +734,7 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
     if (!dropped && (score > W.best_score || (score == W.best_score && score > 0.0 && order < W.best_order))) {
         if (lane == 0) {
             W.best_score = score; W.best_order = order; W.best_n = cnt; W.best_buf = buf;
-            atomicMax(&sh.best_bits, (unsigned long long)__double_as_longlong(score));
+            atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
         }
     }
     __syncwarp();
@@ -773,7 +775,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     int cap = max_spec;
     if (d_budget_cap && d_budget_cap[i] >= 0) cap = min(cap, d_budget_cap[i]);
     if (tid < 2 * SD_MAX_DEPTH) { (&sh.node[0][0])[tid] = -1; (&sh.nc[0][0])[tid] = 0; }
-    if (tid == 0) { sh.njobs = 0; sh.next = 0; sh.nwide = 0; sh.nwide_kept = 0; sh.best_bits = 0ull; sh.win_warp = -1; }
+    if (tid == 0) { sh.njobs = 0; sh.next = 0; sh.nwide = 0; sh.nwide_kept = 0; sh.best_hi = 0u; sh.win_warp = -1; }
     WarpWork& W = sh.w[wib];
     if (lane == 0) { W.best_score = 0.0; W.best_order = 1 << 30; W.best_n = 0; W.best_buf = 0; }
 
@@ -922,7 +924,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     // the best score any more and are dropped here.  For the rest the warps of the block share
     // the scan of the run, then one warp merges the partial lists and finishes the job.
     if (tid == 0) {
-        const double best = __longlong_as_double((long long)sh.best_bits);
+        const double best = __hiloint2double((int)sh.best_hi, 0);
         int kept = 0;
         for (int q = 0; q < sh.nwide; ++q) {
             const int p = sh.wide[q] % SD_MAX_DEPTH + 1;

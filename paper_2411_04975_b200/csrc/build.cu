@@ -76,7 +76,48 @@ __global__ void scan_add_kernel(int* out, i64 n, const int* tile_offsets) {
     }
 }
 
-__global__ void copy_one_kernel(int* dst, const int* src) { *dst = *src; }
+// Second half of a two-launch scan for up to 1024 tiles: every block adds up the totals of the
+// tiles before it by itself (a block-wide reduction over at most 1024 numbers), so the tile
+// totals need no scan of their own.  The last block also writes the grand total.
+__global__ void scan_add_direct_kernel(int* out, i64 n, const int* sums, int nb, int* total_out) {
+    __shared__ int wpart[SCAN_THREADS / 32];
+    __shared__ int offset_sh, total_sh;
+    int before = 0, all = 0;
+    for (int k = threadIdx.x; k < nb; k += SCAN_THREADS) {
+        const int v = sums[k];
+        all += v;
+        if (k < (int)blockIdx.x) before += v;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, o);
+        all += __shfl_xor_sync(0xffffffffu, all, o);
+    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) wpart[w] = before;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int k = 0; k < SCAN_THREADS / 32; ++k) t += wpart[k];
+        offset_sh = t;
+    }
+    __syncthreads();
+    if (lane == 0) wpart[w] = all;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int k = 0; k < SCAN_THREADS / 32; ++k) t += wpart[k];
+        total_sh = t;
+    }
+    __syncthreads();
+    const int add = offset_sh;
+    const i64 base = (i64)blockIdx.x * SCAN_TILE;
+    for (int k = threadIdx.x; k < SCAN_TILE; k += SCAN_THREADS) {
+        const i64 idx = base + k;
+        if (idx < n) out[idx] += add;
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) *total_out = total_sh;
+}
 
 inline i64 scan_tmp_ints(i64 n) {       // ints of scratch exclusive_scan() needs
     i64 total = 0;
@@ -95,8 +136,8 @@ void scan_in_place(int* data, i64 n, int* tmp, int* total_out, cudaStream_t st) 
     i64 nb = (n + SCAN_TILE - 1) / SCAN_TILE;
     if (nb < 1) nb = 1;
     scan_tiles_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(LoadInt{data}, n, data, tmp);
-    if (nb == 1) {
-        copy_one_kernel<<<1, 1, 0, st>>>(total_out, tmp);
+    if (nb <= 1024) {
+        scan_add_direct_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(data, n, tmp, (int)nb, total_out);
     } else {
         scan_in_place(tmp, nb, tmp + (nb + 31) / 32 * 32, total_out, st);
         scan_add_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(data, n, tmp);
@@ -109,8 +150,8 @@ void exclusive_scan(F f, i64 n, int* out, int* tmp, cudaStream_t st) {
     i64 nb = (n + SCAN_TILE - 1) / SCAN_TILE;
     if (nb < 1) nb = 1;
     scan_tiles_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(f, n, out, tmp);
-    if (nb == 1) {
-        copy_one_kernel<<<1, 1, 0, st>>>(out + n, tmp);
+    if (nb <= 1024) {
+        scan_add_direct_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(out, n, tmp, (int)nb, out + n);
     } else {
         scan_in_place(tmp, nb, tmp + (nb + 31) / 32 * 32, out + n, st);
         scan_add_kernel<<<(unsigned)nb, SCAN_THREADS, 0, st>>>(out, n, tmp);

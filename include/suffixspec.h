@@ -2,7 +2,11 @@
  * suffixspec: batched SuffixDecoding draft generation on one NVIDIA B200.
  *
  * C ABI.  Every pointer named d_* is DEVICE memory owned by the caller; every
- * other pointer is HOST memory.  A store owns all of its device memory from
+ * other pointer is HOST memory.  For the per-step inputs and outputs "device
+ * memory" means any address the GPU can use: page-locked host memory
+ * (cudaHostAlloc / cudaHostRegister, unified addressing) is accepted as it is,
+ * and the kernels then read the few KB of inputs and write the drafts across
+ * the bus themselves, which saves the copies before and after a step.  A store owns all of its device memory from
  * sd_build() until sd_free().  Calls are asynchronous on `stream` (a
  * cudaStream_t passed as void*, NULL = default stream) unless stated; the
  * per-step calls (sd_append, sd_speculate) never allocate device memory.

@@ -88,8 +88,11 @@ def library() -> C.CDLL:
 def _ptr(t: Optional[torch.Tensor], dtype: torch.dtype, name: str) -> Optional[int]:
     if t is None:
         return None
-    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
-        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+    # pinned host memory has a device address of its own (unified addressing): the kernels then
+    # read or write it across the bus, with no copy before or after the call
+    if not (t.is_cuda or t.is_pinned()) or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name}: expected a contiguous CUDA (or pinned host) tensor of {dtype}, "
+                        f"got {t.dtype} on {t.device}")
     return t.data_ptr()
 
 

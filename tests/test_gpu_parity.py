@@ -466,6 +466,32 @@ def test_step_equals_append_then_speculate(U, vocab, D):
     pr.close()
 
 
+def test_step_with_pinned_host_buffers(U):
+    """Inputs and outputs in page-locked host memory: the kernel reads and writes them itself."""
+    rng = np.random.default_rng(77)
+    vocab, n_slots = 200, 12
+    pr = U.Pair(_rand_seqs(rng, 10, 50, 200, vocab), vocab=vocab, D=16, n_slots=n_slots, max_req_tokens=300)
+    pr.append(list(range(n_slots)), _rand_seqs(rng, n_slots, 20, 100, vocab), reset=[1] * n_slots)
+    slots = list(range(n_slots))
+    h_packed = torch.empty(pr.g.alloc_outputs(n_slots)["packed"].numel(), dtype=torch.uint8).pin_memory()
+    h_out = pr.g.unpack_outputs(h_packed, n_slots)
+    for step in range(3):
+        lists = _rand_seqs(rng, n_slots, 0, 9, vocab)
+        off, flat = U.ragged(lists)
+        h_slots = torch.as_tensor(np.asarray(slots, dtype=np.int32)).pin_memory()
+        h_off = torch.as_tensor(off).pin_memory()
+        h_tok = torch.as_tensor(flat if flat.size else np.zeros(1, dtype=np.int32)).pin_memory()
+        h_packed.fill_(0x5A)
+        pr.g.step(h_slots, h_off, h_tok[:flat.size], 16, 2.0, 32, 0, None, h_out)
+        torch.cuda.synchronize()
+        pr.o.slot_append_batch(slots, lists, n_threads=2)
+        want = pr.o.speculate(slots, 16, 2.0, 32, M=64, n_threads=2)
+        got = {k: v.numpy().copy() for k, v in h_out.items()}
+        got["mask"] = got["mask"].view(np.uint32)
+        U.assert_same_drafts(got, want)
+    pr.close()
+
+
 def test_step_reports_a_stopped_append(U):
     rng = np.random.default_rng(4)
     pr = U.Pair(_rand_seqs(rng, 3, 30, 60, 50), vocab=50, D=8, n_slots=3, max_req_tokens=40)

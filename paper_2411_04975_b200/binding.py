@@ -162,6 +162,31 @@ def sd_free(store: int) -> None:
 
 
 # ---- convenience wrapper ---------------------------------------------------------------------
+class BoundStep:
+    """One sd_step call with all of its arguments already converted (see SuffixStore.bind_step).
+    Calling the object launches the step; `out` holds the output tensors it writes."""
+
+    def __init__(self, store, slots, offsets, new_tokens, P, alpha, max_spec, flags, budget_cap, out, stream):
+        self.out = out
+        self._keep = (store, slots, offsets, new_tokens, budget_cap)       # the buffers must outlive the calls
+        self._prm = _SpecParams(P, alpha, max_spec, flags)
+        self._fn = library().sd_step
+        self._args = (
+            store._h, int(slots.numel()), _ptr(slots, torch.int32, "slots"), _ptr(offsets, torch.int64, "offsets"),
+            _ptr(new_tokens, torch.int32, "new_tokens"), C.byref(self._prm), _ptr(budget_cap, torch.int32, "budget_cap"),
+            _ptr(out["n_draft"], torch.int32, "n_draft"), _ptr(out["tokens"], torch.int32, "tokens"),
+            _ptr(out["parents"], torch.int32, "parents"), _ptr(out["positions"], torch.int32, "positions"),
+            _ptr(out["mask"], torch.int32, "mask"), _ptr(out["chosen_tree"], torch.int32, "chosen_tree"),
+            _ptr(out["chosen_p"], torch.int32, "chosen_p"), _ptr(out["score"], torch.float64, "score"),
+            _ptr(out["status"], torch.int32, "status"), stream)
+
+    def __call__(self) -> Dict[str, torch.Tensor]:
+        rc = self._fn(*self._args)
+        if rc != 0:
+            raise SuffixSpecError(rc, "sd_step")
+        return self.out
+
+
 class SuffixStore:
     """Global suffix tree + per-request trees on one GPU."""
 
@@ -266,6 +291,19 @@ class SuffixStore:
         if rc != 0:
             raise SuffixSpecError(rc, "sd_step")
         return out
+
+    def bind_step(self, slots: torch.Tensor, offsets: torch.Tensor, new_tokens: torch.Tensor, P: int, alpha: float,
+                  max_spec: int, flags: int = 0, budget_cap: Optional[torch.Tensor] = None,
+                  out: Optional[Dict[str, torch.Tensor]] = None, stream: Optional[int] = None) -> "BoundStep":
+        """step() with the argument marshalling done once.  A serving loop calls sd_step with the
+        same buffers every step (it refills them in place: `new_tokens` is the whole token buffer,
+        `offsets` says how much of it a step uses), so the returned object keeps the converted
+        pointers and each call of it is just the C call.  `stream`: a cudaStream_t as an integer;
+        default: the stream that is current now."""
+        if out is None:
+            out = self.alloc_outputs(int(slots.numel()))
+        return BoundStep(self, slots, offsets, new_tokens, P, alpha, max_spec, flags, budget_cap, out,
+                         _stream() if stream is None else stream)
 
     def query_counts(self, tree: torch.Tensor, offsets: torch.Tensor, paths: torch.Tensor) -> torch.Tensor:
         n = int(tree.numel())

@@ -482,7 +482,10 @@ def test_step_with_pinned_host_buffers(U):
         h_off = torch.as_tensor(off).pin_memory()
         h_tok = torch.as_tensor(flat if flat.size else np.zeros(1, dtype=np.int32)).pin_memory()
         h_packed.fill_(0x5A)
-        pr.g.step(h_slots, h_off, h_tok[:flat.size], 16, 2.0, 32, 0, None, h_out)
+        if step == 1:                                               # the pre-marshalled form of the same call
+            pr.g.bind_step(h_slots, h_off, h_tok, 16, 2.0, 32, 0, None, h_out)()
+        else:
+            pr.g.step(h_slots, h_off, h_tok[:flat.size], 16, 2.0, 32, 0, None, h_out)
         torch.cuda.synchronize()
         pr.o.slot_append_batch(slots, lists, n_threads=2)
         want = pr.o.speculate(slots, 16, 2.0, 32, M=64, n_threads=2)

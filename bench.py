@@ -473,7 +473,7 @@ def run_sweep(args):
 
 # --------------------------------------------------------------------------------------------
 def run_closed_loop(args):
-    """BASELINE config 4: speculate -> simulated verification against the hidden continuation ->
+    """The closed-loop workload: speculate -> simulated verification against the hidden continuation ->
     append accepted + bonus tokens; finished outputs go into the global tree, their slots are
     refilled.  Reports mean accepted length and steps/s (one GPU)."""
     import torch

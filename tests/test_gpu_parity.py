@@ -155,7 +155,7 @@ def test_speculate_small_vocab_stress(U, seed):
 
 
 def test_speculate_tiny_config(U):
-    """BASELINE config 0 at full size."""
+    """The tiny workload at full size."""
     from workload.generator import get_workload
     w = get_workload("tiny")
     c = w.cfg
@@ -234,7 +234,7 @@ def test_speculate_is_deterministic(U):
     pr.close()
 
 
-# ---------------------------------------------------------------- BASELINE configs, scaled so the oracle takes seconds
+# ---------------------------------------------------------------- the named workloads, scaled so the oracle takes seconds
 def _config_pair(U, name, n_seqs, batch, prompt_len=None, extra_tokens=64):
     from workload.generator import get_workload
     kw = dict(n_seqs=n_seqs, batch=batch)
@@ -253,7 +253,7 @@ def _config_pair(U, name, n_seqs, batch, prompt_len=None, extra_tokens=64):
                                                ("low_repetition", 256, 32)])
 def test_configs_scaled_prompts_then_decode_steps(U, name, n_seqs, batch):
     """Corpus cut to a few hundred sequences, prompts at full length (8,192 / 4,096 tokens),
-    every other parameter as the benchmark spec gives it; three decode steps of appends."""
+    every other parameter as the workload defines it; three decode steps of appends."""
     w, c, pr = _config_pair(U, name, n_seqs, batch)
     prompts = w.prompts()
     pr.append(list(range(batch)), prompts, reset=[1] * batch)
@@ -274,7 +274,7 @@ def test_configs_scaled_prompts_then_decode_steps(U, name, n_seqs, batch):
 
 
 def test_closed_loop_scaled(U):
-    """BASELINE config 4 in miniature: speculate, accept against the hidden continuation, append
+    """The closed-loop workload in miniature: speculate, accept against the hidden continuation, append
     accepted + bonus tokens, insert finished outputs into the global tree, refill the slot."""
     from workload.closed_loop import ClosedLoop
     w, c, pr = _config_pair(U, "closed_loop", 128, 12, prompt_len=300, extra_tokens=80)
@@ -296,7 +296,7 @@ def test_closed_loop_scaled(U):
 
 
 def test_large_batch_full_size_sampled_against_oracle(U):
-    """BASELINE config 2 at full size (4,194,304-token global tree, 256 requests x 4,096-token
+    """The headline workload (large_batch) at full size (4,194,304-token global tree, 256 requests x 4,096-token
     prompts) in the launch configuration bench.py times.  The oracle holds the full global tree
     but only a sample of the requests; their rows must be bit-exact, and every row must satisfy
     the properties that hold for any draft."""

@@ -316,70 +316,163 @@ __global__ void lcp_kernel(const int32_t* tok, const uint32_t* sa, const int* en
     lcp[j] = (uint8_t)l;
 }
 
-// nodes per depth: suffix j opens one node at every depth in (lcp[j], len[j]]
-__global__ void level_hist_kernel(const uint8_t* lcp, const uint8_t* len, i64 n, unsigned long long* level_nodes) {
-    __shared__ int diff[SD_MAX_DEPTH + 2];
-    if (threadIdx.x < SD_MAX_DEPTH + 2) diff[threadIdx.x] = 0;
-    __syncthreads();
-    for (i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (i64)gridDim.x * blockDim.x) {
-        int a = lcp[j], b = len[j];
-        if (b > a) {
-            atomicAdd(&diff[a + 1], 1);
-            atomicAdd(&diff[b + 1], -1);
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int run = 0;
-        for (int d = 1; d <= SD_MAX_DEPTH; ++d) {
-            run += diff[d];
-            if (run) atomicAdd(&level_nodes[d], (unsigned long long)run);
-        }
-    }
-}
-
-struct OpensNode {            // suffix j opens a node at depth d
-    const uint8_t* lcp;
-    const uint8_t* len;
-    int d;
-    __device__ int operator()(i64 j) const { return (lcp[j] < d && d <= len[j]) ? 1 : 0; }
-};
-struct Boundary {             // suffix j differs from its predecessor within the first d tokens
-    const uint8_t* lcp;
-    int d;
-    __device__ int operator()(i64 j) const { return lcp[j] < d ? 1 : 0; }
-};
-
-__global__ void seg_pos_kernel(const uint8_t* lcp, int d, const int* bscan, i64 n, int* segpos) {
-    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
-    if (j > n) return;
-    if (j == n) { segpos[bscan[n]] = (int)n; return; }
-    if (lcp[j] < d) segpos[bscan[j]] = (int)j;
-}
-
-struct NewNodes {             // nodes opened by suffix j
+struct NewNodes {             // nodes opened by suffix j: one at every depth in (lcp[j], len[j]]
     const uint8_t* lcp;
     const uint8_t* len;
     __device__ int operator()(i64 j) const { return (int)len[j] - (int)lcp[j]; }
 };
 
+// ------------------------------------------------------------------ all depths at once
+// Everything the tree needs beyond the suffix order follows from lcp[] and len[], for all
+// depths d = 1 .. D together.  "Channel" c stands for depth d = c + 1:
+//   opens_c(i)  = lcp[i] <= c < len[i]    suffix i opens a node at depth d
+//   bound_c(i)  = lcp[i] <= c             suffix i starts a new range of equal d-token prefixes
+//   E_c[j]      = #{ i < j : opens_c(i) }                  rank of a depth-d node among all of them
+//   end(j, d)   = min{ i > j : bound_c(i) } (else N)        one past the node's range: count = end - j
+//   before(j)   = max{ i < j : lcp[i] < lcp[j] }            first suffix of the parent's range when
+//                                                           the parent was opened by another suffix
+// One warp scans a tile of MS_TILE suffixes, 32 at a time: a ballot per channel turns the 32
+// suffixes' flags into one word, lane c keeps the running state of channel c.  Three launches:
+// tile totals, carries across tiles (one small block), then the tile again with its carries.
 // Nodes are numbered in depth-first pre-order: the root is 0 and the node that suffix j opens
 // at depth d is 1 + nbase[j] + (d - lcp[j] - 1).  Pre-order is what makes paths contiguous:
 // child runs are laid down in node order, so the run of a node's first child directly follows
 // the node's own run, and a chain of only children is one run of consecutive entries.
-__global__ void count_children_kernel(const uint8_t* lcp, const uint8_t* len, i64 n, int d, int D, const int* r_d,
-                                      const int* r_next, const int* bscan, const int* segpos, const int* nbase,
-                                      int* nchild) {
-    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= n) return;
-    if (j == 0 && d == 1) nchild[0] = r_d[n];             // the root's children: all depth-1 nodes
-    if (!(lcp[j] < d && d <= len[j])) return;
-    int nc = 0;
-    if (d < D) {
-        const int nb = segpos[bscan[j] + 1];              // first suffix past this node's range
-        nc = r_next[nb] - r_next[j];
+constexpr int MS_CHUNKS = 32;                     // chunks of 32 suffixes per tile
+constexpr int MS_TILE = 32 * MS_CHUNKS;
+constexpr int MS_WARPS = 4;                       // tiles (warps) per block
+
+struct LevelTables {
+    int* E;               // [D][N + 1]
+    int* node_end;        // [n_nodes + 1], by node id
+    int* before;          // [N]
+    int* agg;             // [tiles][3][32]: opens counts, last bound index, first bound index
+    i64 N;
+    int D, tiles;
+};
+
+__global__ void __launch_bounds__(MS_WARPS * 32)
+ms_tile_kernel(const uint8_t* __restrict__ lcp, const uint8_t* __restrict__ len, LevelTables T) {
+    const int lane = threadIdx.x & 31;
+    const int tile = blockIdx.x * MS_WARPS + (threadIdx.x >> 5);
+    if (tile >= T.tiles) return;
+    const i64 t0 = (i64)tile * MS_TILE;
+    int cnt = 0, last = -1, first = 0x7fffffff;                 // of channel `lane`
+    for (int ch = 0; ch < MS_CHUNKS; ++ch) {
+        const i64 base = t0 + (i64)ch * 32, i = base + lane;
+        const int l = i < T.N ? lcp[i] : 255, n = i < T.N ? len[i] : 0;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            const unsigned ob = __ballot_sync(0xffffffffu, l <= c && c < n);
+            const unsigned bb = __ballot_sync(0xffffffffu, l <= c);
+            if (lane == c) {
+                cnt += __popc(ob);
+                if (bb) {
+                    last = (int)base + 31 - __clz(bb);
+                    if (first == 0x7fffffff) first = (int)base + __ffs(bb) - 1;
+                }
+            }
+        }
     }
-    nchild[1 + nbase[j] + (d - (int)lcp[j] - 1)] = nc;
+    int* a = T.agg + (i64)tile * 96;
+    a[lane] = cnt; a[32 + lane] = last; a[64 + lane] = first;
+}
+
+// In place: counts -> sum over the tiles before; last -> nearest bound index before the tile
+// (-1: none); first -> nearest bound index behind the tile (N: none).  Also E_c[N].
+__global__ void ms_carry_kernel(LevelTables T) {
+    const int q = threadIdx.x >> 5, c = threadIdx.x & 31;
+    if (q == 0) {
+        int run = 0;
+        for (int t = 0; t < T.tiles; ++t) { int* a = T.agg + (i64)t * 96 + c; const int v = *a; *a = run; run += v; }
+        if (c < T.D) T.E[(i64)c * (T.N + 1) + T.N] = run;
+    } else if (q == 1) {
+        int run = -1;
+        for (int t = 0; t < T.tiles; ++t) { int* a = T.agg + (i64)t * 96 + 32 + c; const int v = *a; *a = run; run = max(run, v); }
+    } else {
+        int run = (int)T.N;
+        for (int t = T.tiles - 1; t >= 0; --t) { int* a = T.agg + (i64)t * 96 + 64 + c; const int v = *a; *a = run; run = min(run, v); }
+    }
+}
+
+__global__ void __launch_bounds__(MS_WARPS * 32)
+ms_apply_kernel(const uint8_t* __restrict__ lcp, const uint8_t* __restrict__ len, const int* __restrict__ nbase,
+                LevelTables T) {
+    __shared__ unsigned bmask[MS_WARPS][MS_CHUNKS][32];         // bound words of the tile, by chunk and channel
+    __shared__ int sfirst[MS_WARPS][32];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int tile = blockIdx.x * MS_WARPS + wib;
+    if (tile >= T.tiles) return;
+    const i64 t0 = (i64)tile * MS_TILE;
+    const unsigned lt = (1u << lane) - 1u;
+    const int* a = T.agg + (i64)tile * 96;
+    int run_cnt = a[lane], run_last = a[32 + lane], run_first = a[64 + lane];
+    // forward: E and `before`
+    for (int ch = 0; ch < MS_CHUNKS; ++ch) {
+        const i64 base = t0 + (i64)ch * 32, i = base + lane;
+        const int l = i < T.N ? lcp[i] : 255, n = i < T.N ? len[i] : 0;
+        const int prev_last = run_last;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            const unsigned ob = __ballot_sync(0xffffffffu, l <= c && c < n);
+            const unsigned bb = __ballot_sync(0xffffffffu, l <= c);
+            const int carry = __shfl_sync(0xffffffffu, run_cnt, c);
+            if (c < T.D && i < T.N) T.E[(i64)c * (T.N + 1) + i] = carry + __popc(ob & lt);
+            if (lane == c) {
+                run_cnt += __popc(ob);
+                if (bb) run_last = (int)base + 31 - __clz(bb);
+                bmask[wib][ch][c] = bb;
+            }
+        }
+        __syncwarp();
+        // nearest earlier suffix with a smaller lcp: bound channel lcp - 1
+        const int src = (l >= 1 && l <= 32) ? l - 1 : 0;
+        const int far = __shfl_sync(0xffffffffu, prev_last, src);
+        if (i < T.N) {
+            int b = -1;
+            if (l >= 1) {
+                const unsigned m = bmask[wib][ch][src] & lt;
+                b = m ? (int)base + 31 - __clz(m) : far;
+            }
+            T.before[i] = b;
+        }
+    }
+    // backward: the end of every node's range
+    for (int ch = MS_CHUNKS - 1; ch >= 0; --ch) {
+        const i64 base = t0 + (i64)ch * 32, i = base + lane;
+        sfirst[wib][lane] = run_first;
+        __syncwarp();
+        if (i < T.N) {
+            const int l = lcp[i], n = len[i];
+            const unsigned gt = ~lt & ~(1u << lane);
+            int nid = 1 + nbase[i];
+            for (int d = l + 1; d <= n; ++d, ++nid) {
+                const unsigned m = bmask[wib][ch][d - 1] & gt;
+                T.node_end[nid] = m ? (int)base + __ffs(m) - 1 : sfirst[wib][d - 1];
+            }
+        }
+        __syncwarp();
+        const unsigned bb = bmask[wib][ch][lane];
+        if (bb) run_first = (int)base + __ffs(bb) - 1;
+    }
+}
+
+// children per node: the depth d + 1 nodes opened inside the node's range
+__global__ void count_children_kernel(const uint8_t* __restrict__ lcp, const uint8_t* __restrict__ len,
+                                      const int* __restrict__ nbase, LevelTables T, int* nchild) {
+    const i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) nchild[0] = T.E[T.N];                            // the root's children: all depth-1 nodes
+    if (i >= T.N) return;
+    const int l = lcp[i], n = len[i];
+    int nid = 1 + nbase[i];
+    for (int d = l + 1; d <= n; ++d, ++nid) {
+        int nc = 0;
+        if (d < T.D) {
+            const int* row = T.E + (i64)d * (T.N + 1);          // channel of depth d + 1
+            nc = row[T.node_end[nid]] - row[i];
+        }
+        nchild[nid] = nc;
+    }
 }
 
 __device__ __forceinline__ int top_block_of(int nid, int nc) { return (nid > 0 && nc > SD_TOP_MIN) ? SD_TOP_BLOCK : 0; }
@@ -446,34 +539,39 @@ __global__ void fill_top_kernel(const int* list, const int* nchild, const int* r
     }
 }
 
-// Write the depth-d nodes.  A node's entry sits in its parent's child run at its rank among
-// the siblings (suffix order = token order).
-__global__ void emit_level_kernel(const int32_t* tok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len,
-                                  i64 n, int d, const int* r_d, const int* bscan, const int* segpos,
-                                  const int* bscan_prev, const int* segpos_prev, const int* nbase, const int* nchild,
-                                  const int* runstart, int4* ent, int32_t* root) {
-    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+// Write the nodes that suffix j opens.  A node's entry sits in its parent's child run at its
+// rank among the siblings (suffix order = token order).  The first node a suffix opens hangs
+// below a node of an earlier suffix (or the root); every further one is the only-so-far child
+// of the one before it.
+__global__ void emit_nodes_kernel(const int32_t* tok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len, i64 n,
+                                  LevelTables T, const int* nbase, const int* nchild, const int* runstart, int4* ent,
+                                  int32_t* root) {
+    const i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
-    if (!(lcp[j] < d && d <= len[j])) return;
-    const int nb = segpos[bscan[j] + 1];
-    int pnid = 0, rank = r_d[j];
-    if (d > 1) {
-        const int seg = bscan_prev[j] + (lcp[j] < d - 1 ? 1 : 0) - 1;   // depth d-1 range holding j
-        const int jx = segpos_prev[seg];                               // its first suffix opened the parent
-        pnid = 1 + nbase[jx] + (d - 1 - (int)lcp[jx] - 1);
-        rank = r_d[j] - r_d[jx];
+    const int l = lcp[j], m = len[j];
+    if (m <= l) return;
+    int nid = 1 + nbase[j];
+    int pnid = 0, rank = T.E[j];                                  // depth 1: below the root
+    if (l >= 1) {
+        const int jx = T.before[j];                               // its first suffix opened the parent
+        pnid = 1 + nbase[jx] + (l - (int)lcp[jx] - 1);
+        const int* row = T.E + (i64)l * (T.N + 1);                // channel of depth l + 1
+        rank = row[j] - row[jx];
     }
-    const int nid = 1 + nbase[j] + (d - (int)lcp[j] - 1);
-    const int nc = nchild[nid];
-    int4 e;
-    e.x = tok[(i64)sa[j] + d - 1];
-    e.y = nb - (int)j;                                    // every suffix in the range is an occurrence
-    const int tb = top_block_of(nid, nc);
-    e.z = nc > 0 ? runstart[nid] + tb : 0;
-    e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC | (tb ? RUN_HAS_TOP : 0u)) : 0;
-    const int pos = runstart[pnid] + top_block_of(pnid, nchild[pnid]) + rank;
-    ent[pos] = e;
-    if (d == 1) root[e.x] = pos;
+    const i64 text = (i64)sa[j];
+    for (int d = l + 1; d <= m; ++d, ++nid) {
+        const int nc = nchild[nid];
+        int4 e;
+        e.x = tok[text + d - 1];
+        e.y = T.node_end[nid] - (int)j;                           // every suffix in the range is an occurrence
+        const int tb = top_block_of(nid, nc);
+        e.z = nc > 0 ? runstart[nid] + tb : 0;
+        e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC | (tb ? RUN_HAS_TOP : 0u)) : 0;
+        const int pos = runstart[pnid] + top_block_of(pnid, nchild[pnid]) + rank;
+        ent[pos] = e;
+        if (d == 1) root[e.x] = pos;
+        pnid = nid; rank = 0;
+    }
 }
 
 __global__ void init_global_state_kernel(GlobalState* g, int used, int live, long long tokens) {
@@ -548,11 +646,10 @@ struct Pipeline {
     SortBuffers sb;
     int *end_pos = nullptr, *rank[8] = {nullptr}, *comb[2] = {nullptr, nullptr}, *ex = nullptr;
     uint8_t *lcp = nullptr, *len = nullptr;
-    unsigned long long* level_nodes = nullptr;
+    int* wide_counter = nullptr;
     const uint32_t* sa = nullptr;
-    int *r_a = nullptr, *r_b = nullptr, *b_a = nullptr, *b_b = nullptr, *seg_a = nullptr, *seg_b = nullptr;
+    LevelTables lv;
     int *nbase = nullptr, *nchild = nullptr, *runstart = nullptr, *big_tmp = nullptr, *wide_list = nullptr;
-    int* r_cur = nullptr;
     i64 N = 0, n_nodes = 0, used_entries = 0;
     int n_wide = 0;
 };
@@ -573,7 +670,7 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
               tmp.get(&sb.vals[1], N) && tmp.get(&sb.hist, (i64)256 * nblk + 1) &&
               tmp.get(&sb.scan_tmp, scan_tmp_ints(std::max<i64>((i64)256 * nblk, N + 1))) &&
               tmp.get(&P.end_pos, N) && tmp.get(&P.ex, N + 1) && tmp.get(&P.lcp, N) && tmp.get(&P.len, N) &&
-              tmp.get(&P.level_nodes, SD_MAX_DEPTH + 2);
+              tmp.get(&P.wide_counter, 1);
     for (int k = 0; ok && k <= m; ++k) ok = tmp.get(&P.rank[k], N);
     ok = ok && tmp.get(&P.comb[0], N) && tmp.get(&P.comb[1], N);
     if (!ok) return SD_ERR_NOMEM;
@@ -617,37 +714,32 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     }
     P.sa = sb.vals[sorted];
     lcp_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tok, P.sa, end_pos, N, D, lcp, len);
-    ce = cudaMemsetAsync(P.level_nodes, 0, sizeof(unsigned long long) * (SD_MAX_DEPTH + 2), st);
-    level_hist_kernel<<<(unsigned)std::min<i64>(grid_for(N, T256), 1184), T256, 0, st>>>(lcp, len, N, P.level_nodes);
-    unsigned long long h_level[SD_MAX_DEPTH + 2];
-    if (ce == cudaSuccess) ce = cudaMemcpyAsync(h_level, P.level_nodes, sizeof(h_level), cudaMemcpyDeviceToHost, st);
+    ok = tmp.get(&P.nbase, N + 1);
+    if (!ok) return SD_ERR_NOMEM;
+    exclusive_scan(NewNodes{lcp, len}, N, P.nbase, sb.scan_tmp, st);
+    int h_nodes = 0;
+    ce = cudaMemcpyAsync(&h_nodes, P.nbase + N, sizeof(int), cudaMemcpyDeviceToHost, st);
     if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
     if (ce != cudaSuccess) return SD_ERR_CUDA;
-    i64 n_nodes = 0;
-    for (int d = 1; d <= D; ++d) n_nodes += (i64)h_level[d];
+    const i64 n_nodes = h_nodes;
     P.n_nodes = n_nodes;
 
-    P.b_a = ex;
-    ok = tmp.get(&P.r_a, N + 1) && tmp.get(&P.r_b, N + 1) && tmp.get(&P.seg_a, N + 2) && tmp.get(&P.seg_b, N + 2) &&
-         tmp.get(&P.b_b, N + 1) && tmp.get(&P.nbase, N + 1) && tmp.get(&P.nchild, n_nodes + 1) &&
+    LevelTables& lv = P.lv;
+    lv.N = N; lv.D = D;
+    lv.tiles = (int)((N + MS_TILE - 1) / MS_TILE);
+    ok = tmp.get(&lv.E, (i64)D * (N + 1)) && tmp.get(&lv.node_end, n_nodes + 1) && tmp.get(&lv.before, N) &&
+         tmp.get(&lv.agg, (i64)lv.tiles * 96) && tmp.get(&P.nchild, n_nodes + 1) &&
          tmp.get(&P.runstart, n_nodes + 2) && tmp.get(&P.big_tmp, scan_tmp_ints(n_nodes + 1)) &&
          tmp.get(&P.wide_list, n_nodes / SD_TOP_MIN + 2);
     if (!ok) return SD_ERR_NOMEM;
-    exclusive_scan(NewNodes{lcp, len}, N, P.nbase, sb.scan_tmp, st);
-    // pass 1, deepest level first: children per node
-    int* r_next = P.r_a;
-    P.r_cur = P.r_b;
-    for (int d = D; d >= 1; --d) {
-        exclusive_scan(OpensNode{lcp, len, d}, N, P.r_cur, sb.scan_tmp, st);
-        exclusive_scan(Boundary{lcp, d}, N, P.b_a, sb.scan_tmp, st);
-        seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(lcp, d, P.b_a, N, P.seg_a);
-        count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, N, d, D, P.r_cur, r_next, P.b_a, P.seg_a,
-                                                                  P.nbase, P.nchild);
-        std::swap(P.r_cur, r_next);
-    }
+    const unsigned ms_grid = (unsigned)((lv.tiles + MS_WARPS - 1) / MS_WARPS);
+    ms_tile_kernel<<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, lv);
+    ms_carry_kernel<<<1, 96, 0, st>>>(lv);
+    ms_apply_kernel<<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, P.nbase, lv);
+    count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, P.nbase, lv, P.nchild);
     // child runs (with their top blocks) in node (pre-)order
     exclusive_scan(RunAlloc{P.nchild, top_blocks ? 1 : 0}, n_nodes + 1, P.runstart, P.big_tmp, st);
-    int* wide_counter = (int*)P.level_nodes;
+    int* wide_counter = P.wide_counter;
     ce = cudaMemsetAsync(wide_counter, 0, sizeof(int), st);
     if (top_blocks)
         collect_wide_kernel<<<grid_for(n_nodes + 1, T256), T256, 0, st>>>(P.nchild, n_nodes + 1, P.wide_list, wide_counter);
@@ -725,18 +817,9 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
     if (!store_alloc(s, &s->g_ent, s->g_cap)) { store_release(s); return SD_ERR_NOMEM; }
 
     if (N > 0) {
-        // pass 2, top level first: write the entries
-        int *b_cur = P.b_a, *b_prev = P.b_b, *seg_cur = P.seg_a, *seg_prev = P.seg_b;
-        for (int d = 1; d <= D; ++d) {
-            exclusive_scan(OpensNode{P.lcp, P.len, d}, N, P.r_cur, P.sb.scan_tmp, st);
-            exclusive_scan(Boundary{P.lcp, d}, N, b_cur, P.sb.scan_tmp, st);
-            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(P.lcp, d, b_cur, N, seg_cur);
-            emit_level_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, P.sa, P.lcp, P.len, N, d, P.r_cur, b_cur,
-                                                                 seg_cur, b_prev, seg_prev, P.nbase, P.nchild,
-                                                                 P.runstart, s->g_ent, s->g_root);
-            std::swap(b_cur, b_prev);
-            std::swap(seg_cur, seg_prev);
-        }
+        // write the entries
+        emit_nodes_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, P.sa, P.lcp, P.len, N, P.lv, P.nbase, P.nchild,
+                                                             P.runstart, s->g_ent, s->g_root);
         if (P.n_wide > 0) fill_top_kernel<<<P.n_wide, 256, 0, st>>>(P.wide_list, P.nchild, P.runstart, s->g_ent);
     }
     init_global_state_kernel<<<1, 1, 0, st>>>(s->g_state, (int)used_entries, (int)n_nodes, N);
@@ -829,38 +912,39 @@ __global__ void requests_layout_kernel(sd_store sv, int n, const int64_t* off, c
     L.ok[q] = ((i64)n1 + (re - rb) <= sv.spn && hi - lo <= sv.T) ? 1 : 0;
 }
 
-__global__ void emit_level_slots_kernel(sd_store sv, int n_req, const int32_t* slot_ids, const int64_t* off,
+__global__ void emit_nodes_slots_kernel(sd_store sv, int n_req, const int32_t* slot_ids, const int64_t* off,
                                         const int32_t* mtok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len,
-                                        i64 n, int d, const int* r_d, const int* bscan, const int* segpos,
-                                        const int* bscan_prev, const int* segpos_prev, const int* nbase, const int* nchild,
-                                        const int* runstart, RequestLayout L) {
-    i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+                                        i64 n, LevelTables T, const int* nbase, const int* nchild, const int* runstart,
+                                        RequestLayout L) {
+    const i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
-    if (!(lcp[j] < d && d <= len[j])) return;
-    const int q = seq_rank_of(off, n_req, (i64)sa[j]);
+    const int l = lcp[j], m = len[j];
+    if (m <= l) return;
+    const i64 text = (i64)sa[j];
+    const int q = seq_rank_of(off, n_req, text);
     const int slot = slot_ids[q];
     if (!L.ok[q] || slot < 0 || slot >= sv.R) return;
     int4* ent = sv.s_ent + (i64)slot * sv.spn;
-    const int nb = segpos[bscan[j] + 1];
-    const int nid = 1 + nbase[j] + (d - (int)lcp[j] - 1);
-    const int nc = nchild[nid];
     const int shift = L.n1[q] - L.run_base[q];                  // global run position -> index in the slot pool
-    int4 e;
-    e.x = mtok[(i64)sa[j] + d - 1] - q * sv.V;
-    e.y = nb - (int)j;
-    e.z = nc > 0 ? runstart[nid] + shift : 0;
-    e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC) : 0;
-    int pos;
-    if (d == 1) {
-        pos = r_d[j] - L.r1lo[q];
-        (sv.s_root + (i64)slot * sv.V)[e.x] = pos;
-    } else {
-        const int seg = bscan_prev[j] + (lcp[j] < d - 1 ? 1 : 0) - 1;
-        const int jx = segpos_prev[seg];
-        const int pnid = 1 + nbase[jx] + (d - 1 - (int)lcp[jx] - 1);
-        pos = runstart[pnid] + (r_d[j] - r_d[jx]) + shift;
+    int nid = 1 + nbase[j];
+    int pos = T.E[j] - L.r1lo[q];                               // depth 1: the request's own root table
+    if (l >= 1) {
+        const int jx = T.before[j];
+        const int pnid = 1 + nbase[jx] + (l - (int)lcp[jx] - 1);
+        const int* row = T.E + (i64)l * (T.N + 1);
+        pos = runstart[pnid] + (row[j] - row[jx]) + shift;
     }
-    ent[pos] = e;
+    for (int d = l + 1; d <= m; ++d, ++nid) {
+        const int nc = nchild[nid];
+        int4 e;
+        e.x = mtok[text + d - 1] - q * sv.V;
+        e.y = T.node_end[nid] - (int)j;
+        e.z = nc > 0 ? runstart[nid] + shift : 0;
+        e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC) : 0;
+        ent[pos] = e;
+        if (d == 1) (sv.s_root + (i64)slot * sv.V)[e.x] = pos;
+        pos = runstart[nid] + shift;                             // the next one is this node's first child
+    }
 }
 
 // one warp per request: bookkeeping and the active nodes (lane d-1: node of the last d tokens)
@@ -931,10 +1015,10 @@ extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, 
     P.tmp.keep = s->ws;                                          // temporaries are kept for the next call
     int32_t *d_slot = nullptr, *mtok = nullptr;
     int64_t* d_off = nullptr;
-    int *bad = nullptr, *r1 = nullptr;
+    int* bad = nullptr;
     RequestLayout L;
     bool ok = P.tmp.get(&d_slot, n) && P.tmp.get(&d_off, n + 1) && P.tmp.get(&mtok, N) && P.tmp.get(&bad, 1) &&
-              P.tmp.get(&r1, N + 1) && P.tmp.get(&L.run_base, n) && P.tmp.get(&L.n1, n) && P.tmp.get(&L.r1lo, n) &&
+              P.tmp.get(&L.run_base, n) && P.tmp.get(&L.n1, n) && P.tmp.get(&L.r1lo, n) &&
               P.tmp.get(&L.used, n) && P.tmp.get(&L.live, n) && P.tmp.get(&L.ok, n);
     if (!ok) return SD_ERR_NOMEM;
     SD_CUDA_OK(cudaMemcpyAsync(d_slot, h_slot, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st));
@@ -951,19 +1035,9 @@ extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, 
     if (N > 0) {
         const int rc = pipeline_run(P, mtok, d_off, n, N, (i64)n * s->V, D, false, st);
         if (rc != SD_OK) return rc;
-        exclusive_scan(OpensNode{P.lcp, P.len, 1}, N, r1, P.sb.scan_tmp, st);
-        requests_layout_kernel<<<grid_for(n, T256), T256, 0, st>>>(*s, n, d_off, P.nbase, P.runstart, r1, L);
-        int *b_cur = P.b_a, *b_prev = P.b_b, *seg_cur = P.seg_a, *seg_prev = P.seg_b;
-        for (int d = 1; d <= D; ++d) {
-            exclusive_scan(OpensNode{P.lcp, P.len, d}, N, P.r_cur, P.sb.scan_tmp, st);
-            exclusive_scan(Boundary{P.lcp, d}, N, b_cur, P.sb.scan_tmp, st);
-            seg_pos_kernel<<<grid_for(N + 1, T256), T256, 0, st>>>(P.lcp, d, b_cur, N, seg_cur);
-            emit_level_slots_kernel<<<grid_for(N, T256), T256, 0, st>>>(*s, n, d_slot, d_off, mtok, P.sa, P.lcp, P.len, N, d,
-                                                                       P.r_cur, b_cur, seg_cur, b_prev, seg_prev, P.nbase,
-                                                                       P.nchild, P.runstart, L);
-            std::swap(b_cur, b_prev);
-            std::swap(seg_cur, seg_prev);
-        }
+        requests_layout_kernel<<<grid_for(n, T256), T256, 0, st>>>(*s, n, d_off, P.nbase, P.runstart, P.lv.E, L);
+        emit_nodes_slots_kernel<<<grid_for(N, T256), T256, 0, st>>>(*s, n, d_slot, d_off, mtok, P.sa, P.lcp, P.len, N, P.lv,
+                                                                   P.nbase, P.nchild, P.runstart, L);
     } else {
         SD_CUDA_OK(cudaMemsetAsync(L.ok, 0xFF, sizeof(int) * n, st));
         SD_CUDA_OK(cudaMemsetAsync(L.used, 0, sizeof(int) * n, st));

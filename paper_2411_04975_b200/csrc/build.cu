@@ -346,7 +346,7 @@ struct LevelTables {
     int* E;               // [D][N + 1]
     int* node_end;        // [n_nodes + 1], by node id
     int* before;          // [N]
-    int* agg;             // [tiles][3][32]: opens counts, last bound index, first bound index
+    int* agg;             // [3][32][tiles]: opens counts, last bound index, first bound index, per channel
     i64 N;
     int D, tiles;
 };
@@ -374,25 +374,38 @@ ms_tile_kernel(const uint8_t* __restrict__ lcp, const uint8_t* __restrict__ len,
             }
         }
     }
-    int* a = T.agg + (i64)tile * 96;
-    a[lane] = cnt; a[32 + lane] = last; a[64 + lane] = first;
+    T.agg[(i64)lane * T.tiles + tile] = cnt;
+    T.agg[(i64)(32 + lane) * T.tiles + tile] = last;
+    T.agg[(i64)(64 + lane) * T.tiles + tile] = first;
 }
 
 // In place: counts -> sum over the tiles before; last -> nearest bound index before the tile
 // (-1: none); first -> nearest bound index behind the tile (N: none).  Also E_c[N].
-__global__ void ms_carry_kernel(LevelTables T) {
-    const int q = threadIdx.x >> 5, c = threadIdx.x & 31;
-    if (q == 0) {
-        int run = 0;
-        for (int t = 0; t < T.tiles; ++t) { int* a = T.agg + (i64)t * 96 + c; const int v = *a; *a = run; run += v; }
-        if (c < T.D) T.E[(i64)c * (T.N + 1) + T.N] = run;
-    } else if (q == 1) {
-        int run = -1;
-        for (int t = 0; t < T.tiles; ++t) { int* a = T.agg + (i64)t * 96 + 32 + c; const int v = *a; *a = run; run = max(run, v); }
-    } else {
-        int run = (int)T.N;
-        for (int t = T.tiles - 1; t >= 0; --t) { int* a = T.agg + (i64)t * 96 + 64 + c; const int v = *a; *a = run; run = min(run, v); }
+// One block per column (kind, channel) of agg[96][tiles]; every thread takes a contiguous
+// stretch of tiles, the stretches' totals are combined in shared memory.
+constexpr int MC_THREADS = 256;
+__global__ void __launch_bounds__(MC_THREADS) ms_carry_kernel(LevelTables T) {
+    __shared__ int part[MC_THREADS];
+    const int kind = blockIdx.x >> 5, c = blockIdx.x & 31;
+    int* col = T.agg + (i64)blockIdx.x * T.tiles;
+    const int per = (T.tiles + MC_THREADS - 1) / MC_THREADS;
+    // kind 2 runs over the tiles from the last to the first
+    const int ident = kind == 0 ? 0 : (kind == 1 ? -1 : (int)T.N);
+    auto at = [&](int k) { return kind == 2 ? T.tiles - 1 - k : k; };
+    auto op = [&](int x, int y) { return kind == 0 ? x + y : (kind == 1 ? max(x, y) : min(x, y)); };
+    const int k0 = threadIdx.x * per, k1 = min(T.tiles, k0 + per);
+    int acc = ident;
+    for (int k = k0; k < k1; ++k) acc = op(acc, col[at(k)]);
+    part[threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = ident;
+        for (int t = 0; t < MC_THREADS; ++t) { const int v = part[t]; part[t] = run; run = op(run, v); }
+        if (kind == 0 && c < T.D) T.E[(i64)c * (T.N + 1) + T.N] = run;
     }
+    __syncthreads();
+    int run = part[threadIdx.x];
+    for (int k = k0; k < k1; ++k) { const int v = col[at(k)]; col[at(k)] = run; run = op(run, v); }
 }
 
 __global__ void __launch_bounds__(MS_WARPS * 32)
@@ -405,8 +418,8 @@ ms_apply_kernel(const uint8_t* __restrict__ lcp, const uint8_t* __restrict__ len
     if (tile >= T.tiles) return;
     const i64 t0 = (i64)tile * MS_TILE;
     const unsigned lt = (1u << lane) - 1u;
-    const int* a = T.agg + (i64)tile * 96;
-    int run_cnt = a[lane], run_last = a[32 + lane], run_first = a[64 + lane];
+    int run_cnt = T.agg[(i64)lane * T.tiles + tile], run_last = T.agg[(i64)(32 + lane) * T.tiles + tile],
+        run_first = T.agg[(i64)(64 + lane) * T.tiles + tile];
     // forward: E and `before`
     for (int ch = 0; ch < MS_CHUNKS; ++ch) {
         const i64 base = t0 + (i64)ch * 32, i = base + lane;
@@ -582,11 +595,28 @@ struct DeviceArena {          // temporaries of one build: freed together, or ke
     void* ptr[48];
     int n = 0;
     sd_workspace* keep = nullptr;                     // if set, buffers live there and are reused
+    char* chunk = nullptr;                            // reserved block the next buffers are carved from
+    long long chunk_left = 0;
     ~DeviceArena() { if (!keep) for (int i = 0; i < n; ++i) cudaFree(ptr[i]); }
+    // One allocation for the buffers to come (an allocation of its own costs far more than the
+    // kernels that use a buffer).  If it fails the buffers are simply allocated one by one.
+    void reserve(long long bytes) {
+        if (keep || n >= 48 || bytes <= 0) return;
+        void* p = nullptr;
+        if (cudaMalloc(&p, (size_t)bytes) != cudaSuccess) { cudaGetLastError(); return; }
+        ptr[n++] = p;
+        chunk = (char*)p; chunk_left = bytes;
+    }
     template <class T> bool get(T** out, i64 count) {
         if (count < 1) count = 1;
-        if (n >= 48) return false;
         const long long need = (long long)count * (long long)sizeof(T);
+        const long long padded = (need + 255) / 256 * 256;
+        if (!keep && chunk_left >= padded) {
+            *out = (T*)chunk;
+            chunk += padded; chunk_left -= padded;
+            return true;
+        }
+        if (n >= 48) return false;
         if (keep) {
             const int k = n++;
             if (keep->bytes[k] < need) {
@@ -666,6 +696,11 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     const int nblk = (int)((N + RS_TILE - 1) / RS_TILE);
     int m = 0;
     while ((2 << m) <= D) ++m;                    // 2^m <= D < 2^(m+1)
+    {
+        const i64 scan_ints = scan_tmp_ints(std::max<i64>((i64)256 * nblk, N + 1));
+        tmp.reserve((long long)N * (16 + 8 + 4 + 4 + 2 + 4 * (m + 1) + 8 + 4) + 4ll * ((i64)256 * nblk + 1 + scan_ints) +
+                    64 * 256);
+    }
     bool ok = tmp.get(&sb.keys[0], N) && tmp.get(&sb.keys[1], N) && tmp.get(&sb.vals[0], N) &&
               tmp.get(&sb.vals[1], N) && tmp.get(&sb.hist, (i64)256 * nblk + 1) &&
               tmp.get(&sb.scan_tmp, scan_tmp_ints(std::max<i64>((i64)256 * nblk, N + 1))) &&
@@ -727,6 +762,8 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     LevelTables& lv = P.lv;
     lv.N = N; lv.D = D;
     lv.tiles = (int)((N + MS_TILE - 1) / MS_TILE);
+    tmp.reserve(4ll * ((i64)D * (N + 1) + 3 * (n_nodes + 2) + N + (i64)lv.tiles * 96 + scan_tmp_ints(n_nodes + 1) +
+                       n_nodes / SD_TOP_MIN + 2) + 64 * 256);
     ok = tmp.get(&lv.E, (i64)D * (N + 1)) && tmp.get(&lv.node_end, n_nodes + 1) && tmp.get(&lv.before, N) &&
          tmp.get(&lv.agg, (i64)lv.tiles * 96) && tmp.get(&P.nchild, n_nodes + 1) &&
          tmp.get(&P.runstart, n_nodes + 2) && tmp.get(&P.big_tmp, scan_tmp_ints(n_nodes + 1)) &&
@@ -734,7 +771,7 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     if (!ok) return SD_ERR_NOMEM;
     const unsigned ms_grid = (unsigned)((lv.tiles + MS_WARPS - 1) / MS_WARPS);
     ms_tile_kernel<<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, lv);
-    ms_carry_kernel<<<1, 96, 0, st>>>(lv);
+    ms_carry_kernel<<<96, MC_THREADS, 0, st>>>(lv);
     ms_apply_kernel<<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, P.nbase, lv);
     count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, P.nbase, lv, P.nchild);
     // child runs (with their top blocks) in node (pre-)order

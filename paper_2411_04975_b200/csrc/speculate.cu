@@ -262,19 +262,19 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 
 
 // ---------------------------------------------------------------------------------------------
-// Fused path: one block of CTA_WARPS warps per request.
+// Fused path: one block of W warps per request (W = 16, two blocks per SM; W = 32 when the batch
+// leaves SMs idle anyway and there are more jobs per request than 16 warps take at once).
 //   1. match: the per-request match nodes are the slot's active nodes; the global match
 //      nodes are advanced from the nodes cached at the previous call by descending only the
 //      tokens appended since (full walks when the cache is stale).  Warp w serves pattern
-//      lengths w + 1 and w + 1 + CTA_WARPS.
+//      lengths w + 1, w + 1 + W, ...
 //   2. expand: the (tree, p) jobs that matched go into a queue, costliest first; warps pull
 //      jobs until it is empty.  A job is dropped, exactly, as soon as an upper bound of its
 //      SCORE (every D <= 1 and D never grows along a path) falls below a score already
 //      reached by another job of the request.
 //   3. select + emit from shared memory; no global scratch.
-constexpr int CTA_WARPS = 16;
-constexpr int CTA_MIN_BLOCKS = 2;              // blocks per SM the register budget is set for
-constexpr int MATCH_ROUNDS = (SD_MAX_DEPTH + CTA_WARPS - 1) / CTA_WARPS;   // pattern lengths per warp
+constexpr int CTA_WARPS = 16;                  // the usual block
+constexpr int CTA_WARPS_WIDE = 32;             // small batches of requests with many jobs each
 
 struct WarpWork {
     Frontier F;
@@ -288,8 +288,9 @@ struct WarpWork {
     int best_order, best_n, best_buf;
 };
 
-struct BlockShared {
-    WarpWork w[CTA_WARPS];
+template <int WARPS>
+struct BlockSharedT {
+    WarpWork w[WARPS];
     int node[2][SD_MAX_DEPTH];                // match node per tree and pattern length (-1: none)
     int cb[2][SD_MAX_DEPTH];                  // its child run
     unsigned nc[2][SD_MAX_DEPTH];             // ... as the node's w field (count | flags)
@@ -297,8 +298,8 @@ struct BlockShared {
     int job[2 * SD_MAX_DEPTH];
     int wide[2 * SD_MAX_DEPTH];               // jobs whose match node has a wide child run
     int njobs, next, nwide, nwide_kept;
-    long long slice_sum[CTA_WARPS];
-    int slice_fs[CTA_WARPS];
+    long long slice_sum[WARPS];
+    int slice_fs[WARPS];
     unsigned best_hi;                         // high word of the largest SCORE reached so far: a lower
                                               // bound of it (scores are non-negative doubles), which is
                                               // all the pruning needs; 32 bits keep the atomic native
@@ -611,12 +612,14 @@ __device__ void counts_to_d(Frontier& F, int fh, int fs, double d_parent, long l
     __syncwarp();
 }
 
+template <class BlockShared>
 __device__ __forceinline__ double best_so_far(BlockShared& sh) {
     return __hiloint2double((int)__shfl_sync(FULL, *(volatile unsigned*)&sh.best_hi, 0), 0);
 }
 
 // ExpandSpeculationTree + SCORE for one (tree, p) job by one warp.  With `seeded` the frontier
 // already holds the match node's children (fs entries from ring head 0).
+template <class BlockShared>
 __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict__ ent, int limit, int tree, int p,
                            int budget, unsigned flags, bool seeded, int fs, int lane) {
     const int order = tree * SD_MAX_DEPTH + p;                  // loop order of Algorithm 1
@@ -744,14 +747,16 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
 // sd_append does for the slot) while its other warps already advance the global match nodes
 // over those tokens, then speculates: one launch per decode step, and the appends of long
 // token lists overlap with the speculation of the other requests.
-template <bool STEP>
-__global__ void __launch_bounds__(CTA_WARPS * 32, CTA_MIN_BLOCKS)
+template <bool STEP, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 1024 / (WARPS * 32))
 speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
                        unsigned flags, const int32_t* __restrict__ d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
                        int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
                        int32_t* d_chosen_p, double* d_score, int32_t* d_status, const int64_t* __restrict__ d_app_off,
                        const int32_t* __restrict__ d_app_tok) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    using BlockShared = BlockSharedT<WARPS>;
+    constexpr int CTA_WARPS = WARPS;
     BlockShared& sh = *reinterpret_cast<BlockShared*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, wib = tid >> 5;
     const int i = blockIdx.x;
@@ -785,7 +790,8 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     // warps that advance the global match nodes, and this warp's rank among them
     const int mwarps = STEP ? CTA_WARPS - 1 : CTA_WARPS;
     const int mrank = STEP ? wib - 1 : wib;
-    constexpr int MROUNDS = STEP ? (SD_MAX_DEPTH + CTA_WARPS - 2) / (CTA_WARPS - 1) : MATCH_ROUNDS;
+    constexpr int MROUNDS = STEP ? (SD_MAX_DEPTH + CTA_WARPS - 2) / (CTA_WARPS - 1)
+                                 : (SD_MAX_DEPTH + CTA_WARPS - 1) / CTA_WARPS;   // pattern lengths per warp
     int src_node[MROUNDS], src_from[MROUNDS];                   // per target: start node and first text index
 #pragma unroll
     for (int h = 0; h < MROUNDS; ++h) { src_node[h] = -1; src_from[h] = 0; }
@@ -1035,27 +1041,40 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
     if (step && !d_app_off) return SD_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int Pe = prm->P < s->D ? prm->P : s->D;               // longer patterns never match
-    {
+    static bool raised[64] = {false};
+    static int sm_count[64] = {0};
+    int dev = 0;
+    SD_CUDA_OK(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && !raised[dev]) {
         // the block's shared memory exceeds the default limit: raise it once per device
-        static bool raised[64] = {false};
-        int dev = 0;
-        SD_CUDA_OK(cudaGetDevice(&dev));
-        if (dev >= 0 && dev < 64 && !raised[dev]) {
-            SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)sizeof(BlockShared)));
-            SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)sizeof(BlockShared)));
-            raised[dev] = true;
-        }
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(BlockSharedT<CTA_WARPS>)));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(BlockSharedT<CTA_WARPS>)));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_WIDE>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(BlockSharedT<CTA_WARPS_WIDE>)));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_WIDE>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(BlockSharedT<CTA_WARPS_WIDE>)));
+        SD_CUDA_OK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+        raised[dev] = true;
     }
-    if (step)
-        speculate_fused_kernel<true><<<(unsigned)n, CTA_WARPS * 32, sizeof(BlockShared), st>>>(
-            *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,
-            d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, d_app_off, d_app_tok);
-    else
-        speculate_fused_kernel<false><<<(unsigned)n, CTA_WARPS * 32, sizeof(BlockShared), st>>>(
-            *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,
-            d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, nullptr, nullptr);
+    // one block per SM is all a small batch can use: give each block 32 warps if its request has
+    // more jobs (two trees, Pe pattern lengths each) than 16 warps start at once
+    const bool wide = dev >= 0 && dev < 64 && n <= sm_count[dev] && 2 * Pe > 2 * CTA_WARPS;
+#define SD_LAUNCH_FUSED(STEP, WARPS, OFF, TOK)                                                                          \
+    speculate_fused_kernel<STEP, WARPS><<<(unsigned)n, WARPS * 32, sizeof(BlockSharedT<WARPS>), st>>>(                    \
+        *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,          \
+        d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, OFF, TOK)
+    if (step) {
+        if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE, d_app_off, d_app_tok);
+        else SD_LAUNCH_FUSED(true, CTA_WARPS, d_app_off, d_app_tok);
+    } else {
+        if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, nullptr, nullptr);
+        else SD_LAUNCH_FUSED(false, CTA_WARPS, nullptr, nullptr);
+    }
+#undef SD_LAUNCH_FUSED
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }

@@ -262,8 +262,9 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 
 
 // ---------------------------------------------------------------------------------------------
-// Fused path: one block of W warps per request (W = 16, two blocks per SM; W = 32 when the batch
-// leaves SMs idle anyway and there are more jobs per request than 16 warps take at once).
+// Fused path: one block of W warps per request.  W = 16, two blocks per SM, is the usual shape;
+// W = 32 when the batch leaves SMs idle anyway and a request has more jobs than 16 warps take
+// at once; W = 8, four blocks per SM, when 16-warp blocks would need a second wave.
 //   1. match: the per-request match nodes are the slot's active nodes; the global match
 //      nodes are advanced from the nodes cached at the previous call by descending only the
 //      tokens appended since (full walks when the cache is stale).  Warp w serves pattern
@@ -275,6 +276,7 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 //   3. select + emit from shared memory; no global scratch.
 constexpr int CTA_WARPS = 16;                  // the usual block
 constexpr int CTA_WARPS_WIDE = 32;             // small batches of requests with many jobs each
+constexpr int CTA_WARPS_NARROW = 8;            // batches of more than two requests per SM
 
 struct WarpWork {
     Frontier F;
@@ -1057,21 +1059,32 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
         SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_WIDE>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_WIDE>)));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_NARROW>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(BlockSharedT<CTA_WARPS_NARROW>)));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_NARROW>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(BlockSharedT<CTA_WARPS_NARROW>)));
         SD_CUDA_OK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
         raised[dev] = true;
     }
     // one block per SM is all a small batch can use: give each block 32 warps if its request has
     // more jobs (two trees, Pe pattern lengths each) than 16 warps start at once
-    const bool wide = dev >= 0 && dev < 64 && n <= sm_count[dev] && 2 * Pe > 2 * CTA_WARPS;
+    const bool known = dev >= 0 && dev < 64;
+    const bool wide = known && n <= sm_count[dev] && 2 * Pe > 2 * CTA_WARPS;
+    // more requests than two 16-warp blocks per SM hold at once: smaller blocks, one wave
+    const bool narrow = known && n > 2 * sm_count[dev];
 #define SD_LAUNCH_FUSED(STEP, WARPS, OFF, TOK)                                                                          \
     speculate_fused_kernel<STEP, WARPS><<<(unsigned)n, WARPS * 32, sizeof(BlockSharedT<WARPS>), st>>>(                    \
         *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,          \
         d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, OFF, TOK)
     if (step) {
         if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE, d_app_off, d_app_tok);
+        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW, d_app_off, d_app_tok);
         else SD_LAUNCH_FUSED(true, CTA_WARPS, d_app_off, d_app_tok);
     } else {
         if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, nullptr, nullptr);
+        else if (narrow) SD_LAUNCH_FUSED(false, CTA_WARPS_NARROW, nullptr, nullptr);
         else SD_LAUNCH_FUSED(false, CTA_WARPS, nullptr, nullptr);
     }
 #undef SD_LAUNCH_FUSED

@@ -466,6 +466,26 @@ def test_step_equals_append_then_speculate(U, vocab, D):
     pr.close()
 
 
+def test_more_requests_than_block_slots(U):
+    """Over 296 requests (two 16-warp blocks per SM on 148 SMs) the kernel runs with smaller blocks."""
+    rng = np.random.default_rng(320)
+    vocab, n_slots = 60, 330
+    pr = U.Pair(_rand_seqs(rng, 12, 100, 400, vocab), vocab=vocab, D=32, n_slots=n_slots, max_req_tokens=200)
+    slots = list(range(n_slots))
+    pr.append(slots, _rand_seqs(rng, n_slots, 20, 90, vocab), reset=[1] * n_slots)
+    pr.check_speculate(slots, 32, 2.0, 64)
+    lists = _rand_seqs(rng, n_slots, 0, 9, vocab)
+    off, flat = U.ragged(lists)
+    out = pr.g.step(U.dev_i32(slots), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat), 32, 2.0, 64)
+    torch.cuda.synchronize()
+    pr.o.slot_append_batch(slots, lists, n_threads=4)
+    want = pr.o.speculate(slots, 32, 2.0, 64, M=64, n_threads=4)
+    got = {k: v.cpu().numpy() for k, v in out.items()}
+    got["mask"] = got["mask"].view(np.uint32)
+    U.assert_same_drafts(got, want)
+    pr.close()
+
+
 def test_step_with_pinned_host_buffers(U):
     """Inputs and outputs in page-locked host memory: the kernel reads and writes them itself."""
     rng = np.random.default_rng(77)

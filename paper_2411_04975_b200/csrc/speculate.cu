@@ -422,9 +422,22 @@ __device__ __forceinline__ int4 load_window(const int4* __restrict__ ent, int ba
     return idx < limit ? ent[idx] : make_int4(-1, 0, 0, 0);
 }
 
+// A child that was not put into the frontier because it would be taken out again at once.
+struct Taken {
+    bool any;
+    double d;
+    int tok, cb;
+    unsigned w;
+};
+
 // Offer the children of a node to the frontier; `w` already holds the first 32 entries of the run.
+// With `take` (runs of at most 32 children): if the best child (largest count, then smallest
+// token: among siblings that is the order of D) beats every waiting candidate, it is the next
+// node to be added whatever else is offered, so it is handed back instead of being merged in
+// and popped again; the frontier is then bounded by K - 1.
 __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int4 w, double d_parent, int par_index,
-                                Frontier& F, int fh, int& fs, int K, int lane) {
+                                Frontier& F, int fh, int& fs, int K, int lane, Taken* take = nullptr) {
+    if (take) take->any = false;
     if (n <= 0 || K <= 0) return;
     // sibling sum: the denominator of Eq. 1 (a parent's occurrences fit 31 bits)
     unsigned part = lane < n ? (unsigned)w.y : 0u;
@@ -436,6 +449,22 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
     }
     const unsigned sum = __reduce_add_sync(FULL, part);
     const double dsum = (double)sum;
+    int skip = -1;                                              // child handed back through `take`
+    if (take && n <= 32) {
+        const unsigned cmax = __reduce_max_sync(FULL, lane < n ? (unsigned)w.y : 0u);
+        const int b = __ffs(__ballot_sync(FULL, lane < n && (unsigned)w.y == cmax)) - 1;
+        const double db = __dmul_rn(d_parent, __ddiv_rn((double)cmax, dsum));    // Eq. 2 with Eq. 1
+        const int tb = __shfl_sync(FULL, w.x, b);
+        if (fs == 0 || better(db, tb, par_index, F.d[fh], F.tok[fh], F.par[fh])) {
+            take->any = true; take->d = db; take->tok = tb;
+            take->cb = __shfl_sync(FULL, w.z, b);
+            take->w = (unsigned)__shfl_sync(FULL, w.w, b);
+            skip = b;
+            --K;                                                // one node fewer is still to come
+            if (fs > K) fs = K;
+            if (K <= 0 || n == 1) return;
+        }
+    }
     // With a full frontier only a child that beats its worst entry matters:
     // D = d_parent * count / sum, so counts below `cmin` lose without any fp64 work.
     double ld = 0.0, need = 0.0; int lt = 0, lp = 0;
@@ -449,7 +478,7 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
         const int idx = base + lane;
         int4 e = w;
         if (base != 0) { e = make_int4(0, 0, 0, 0); if (idx < n) e = ent[cb + idx]; }
-        bool pass = idx < n && (double)e.y * d_parent >= need;
+        bool pass = idx < n && idx != skip && (double)e.y * d_parent >= need;
         if (!__any_sync(FULL, pass)) continue;
         double dc = 0.0;
         if (pass) {
@@ -733,7 +762,20 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
             if ((score + (double)(budget - cnt) * cur_d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
             continue;
         }
-        push_children_w(ent, cur_cb, cur_n, w, cur_d, cur_idx, W.F, fh, fs, budget - cnt, lane);
+        Taken tk;
+        push_children_w(ent, cur_cb, cur_n, w, cur_d, cur_idx, W.F, fh, fs, budget - cnt, lane, &tk);
+        if (tk.any) {
+            // the same steps as taking it from the frontier at the top of the loop
+            if ((score + (double)(budget - cnt) * tk.d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
+            if (lane == 0) { W.tok[buf][cnt] = tk.tok; W.par[buf][cnt] = (unsigned char)(cur_idx + 1); }
+            score = __dadd_rn(score, tk.d);
+            if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
+            cur_idx = cnt++;
+            cur_d = tk.d; cur_cb = tk.cb; cur_w = tk.w;
+            cur_n = (int)(cur_w & RUN_COUNT_MASK);
+            if (flags & SD_FLAG_LINEAR) fs = 0;
+            have_cur = true;
+        }
     }
     __syncwarp();
     if (!dropped && (score > W.best_score || (score == W.best_score && score > 0.0 && order < W.best_order))) {

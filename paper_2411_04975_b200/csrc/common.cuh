@@ -88,9 +88,13 @@ struct sd_store {
 };
 
 __host__ __device__ inline uint32_t sd_pow2ceil(uint32_t n) {
+#ifdef __CUDA_ARCH__
+    return n <= 1u ? 1u : 1u << (32 - __clz((int)(n - 1u)));
+#else
     uint32_t c = 1;
     while (c < n) c <<= 1;
     return c;
+#endif
 }
 
 // Room of a child run that currently holds n children.

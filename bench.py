@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 from workload.generator import accept_schedule, get_workload  # noqa: E402
 
-METRIC = "speculation trees/s at batch 256 (per step: append the accepted tokens, speculate)"
+METRIC = "speculation trees/s at batch {B} (per step: append the accepted tokens, speculate)"
 UNIT = "trees/s"
 OUT_BYTES_PER_REQ = 4 * 64 * 3 + 64 * 8 + 4 * 3 + 8          # tokens, parents, positions, mask, scalars
 FLUSH_BYTES = 256 << 20
@@ -380,7 +380,7 @@ def run_ours(args):
     if rank == 0:
         st = store.stats()
         line = {
-            "metric": METRIC, "value": B * world / (ms_per_step / 1e3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "metric": METRIC.format(B=B), "value": B * world / (ms_per_step / 1e3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32 trees, f64 scores", "data": "synthetic",
             "config": {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": B,
@@ -648,7 +648,7 @@ def run_reference(args):
         step(k)
     dt = time.perf_counter() - t0
     value = len(sample) * K / dt
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+    line = {"impl": "reference", "metric": METRIC.format(B=B), "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
             "warmup": W, "ms_per_step": dt / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int32 trees, f64 scores", "data": "synthetic",
             "config": {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": B,

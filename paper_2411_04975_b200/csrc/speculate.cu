@@ -486,6 +486,30 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
             if (full) pass = better(dc, e.x, par_index, ld, lt, lp);
             if (pass && ((unsigned)e.w & RUN_COUNT_MASK)) prefetch_l2(ent + e.z);   // likely looked at soon
         }
+        if (fs == 0 && n <= 32) {
+            // Nothing waits yet (the first children of a job): the candidates are siblings, and
+            // among siblings the order of D is the order of (count, then token).  Their places
+            // follow from one pass per distinct count, largest first, without any merging.
+            unsigned rem = __ballot_sync(FULL, pass);
+            const int np = __popc(rem);
+            const unsigned below = (1u << lane) - 1u;
+            int place = -1, taken = 0;
+            while (rem && taken < K) {
+                const bool in = (rem >> lane) & 1u;
+                const unsigned top = __reduce_max_sync(FULL, in ? (unsigned)e.y : 0u);
+                const unsigned grp = __ballot_sync(FULL, in && (unsigned)e.y == top);
+                if ((grp >> lane) & 1u) place = taken + __popc(grp & below);
+                taken += __popc(grp);
+                rem &= ~grp;
+            }
+            if (place >= 0 && place < K) {
+                const int q = (fh + place) & (SD_MAX_SPEC - 1);
+                F.d[q] = dc; F.tok[q] = e.x; F.par[q] = par_index; F.cb[q] = e.z; F.nc[q] = (unsigned)e.w;
+            }
+            __syncwarp();
+            fs = min(np, K);
+            return;
+        }
         frontier_merge(F, fh, fs, K, pass, dc, e.x, par_index, e.z, (unsigned)e.w, lane);
         if (!full && fs == K) {                                 // it filled up while merging
             const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);

@@ -262,7 +262,7 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 
 
 // ---------------------------------------------------------------------------------------------
-// Fused path: one block of W warps per request.  W = 16, two blocks per SM, is the usual shape;
+// Fused path: one block of W warps per request.  W = 16 (12 for sd_step), two blocks per SM, is the usual shape;
 // W = 32 when the batch leaves SMs idle anyway and a request has more jobs than 16 warps take
 // at once; W = 8, four blocks per SM, when 16-warp blocks would need a second wave.
 //   1. match: the per-request match nodes are the slot's active nodes; the global match
@@ -275,6 +275,9 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 //      reached by another job of the request.
 //   3. select + emit from shared memory; no global scratch.
 constexpr int CTA_WARPS = 16;                  // the usual block
+constexpr int CTA_WARPS_STEP = 12;             // the usual block of sd_step: fewer warps, 80 registers each, so
+                                               // that the append in front spills less (measured: 100 us per
+                                               // step against 104 us with 16 warps, 101 with 14, 113 with 10)
 constexpr int CTA_WARPS_WIDE = 32;             // small batches of requests with many jobs each
 constexpr int CTA_WARPS_NARROW = 8;            // batches of more than two requests per SM
 
@@ -1117,8 +1120,9 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
         // the block's shared memory exceeds the default limit: raise it once per device
         SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(BlockSharedT<CTA_WARPS>)));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_STEP>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(BlockSharedT<CTA_WARPS_STEP>)));
         SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_WIDE>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_WIDE>)));
@@ -1147,7 +1151,7 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
     if (step) {
         if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE, d_app_off, d_app_tok);
         else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW, d_app_off, d_app_tok);
-        else SD_LAUNCH_FUSED(true, CTA_WARPS, d_app_off, d_app_tok);
+        else SD_LAUNCH_FUSED(true, CTA_WARPS_STEP, d_app_off, d_app_tok);
     } else {
         if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, nullptr, nullptr);
         else if (narrow) SD_LAUNCH_FUSED(false, CTA_WARPS_NARROW, nullptr, nullptr);

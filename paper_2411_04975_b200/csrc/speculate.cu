@@ -262,9 +262,10 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 
 
 // ---------------------------------------------------------------------------------------------
-// Fused path: one block of W warps per request.  W = 16 (12 for sd_step), two blocks per SM, is the usual shape;
-// W = 32 when the batch leaves SMs idle anyway and a request has more jobs than 16 warps take
-// at once; W = 8, four blocks per SM, when 16-warp blocks would need a second wave.
+// Fused path: one block of W warps per request.  Two blocks per SM is the usual shape: W = 16
+// with 64 registers per thread for sd_speculate, W = 8 with 128 for sd_step, whose append is
+// register hungry.  A batch of at most one request per SM gets bigger blocks (W = 24 / 16), a
+// batch of more than two requests per SM smaller ones (W = 8, four per SM) to stay in one wave.
 //   1. match: the per-request match nodes are the slot's active nodes; the global match
 //      nodes are advanced from the nodes cached at the previous call by descending only the
 //      tokens appended since (full walks when the cache is stale).  Warp w serves pattern
@@ -275,10 +276,12 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 //      reached by another job of the request.
 //   3. select + emit from shared memory; no global scratch.
 constexpr int CTA_WARPS = 16;                  // the usual block
-constexpr int CTA_WARPS_STEP = 12;             // the usual block of sd_step: fewer warps, 80 registers each, so
-                                               // that the append in front spills less (measured: 100 us per
-                                               // step against 104 us with 16 warps, 101 with 14, 113 with 10)
-constexpr int CTA_WARPS_WIDE = 32;             // small batches of requests with many jobs each
+constexpr int CTA_WARPS_STEP = 8;              // the usual block of sd_step: 8 warps with 128 registers each, so
+                                               // that the append in front does not spill (measured per step:
+                                               // 95 us; 10 warps with 96 registers 100, 12 with 80 100, 16 with
+                                               // 64 104, 6 with 168 110)
+constexpr int CTA_WARPS_WIDE = 24;             // small batches (one block per SM at most): the block has the SM's
+constexpr int CTA_WARPS_WIDE_STEP = 16;        // registers to itself (80 per thread; sd_step: 128)
 constexpr int CTA_WARPS_NARROW = 8;            // batches of more than two requests per SM
 
 struct WarpWork {
@@ -818,8 +821,8 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
 // sd_append does for the slot) while its other warps already advance the global match nodes
 // over those tokens, then speculates: one launch per decode step, and the appends of long
 // token lists overlap with the speculation of the other requests.
-template <bool STEP, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32, 1024 / (WARPS * 32))
+template <bool STEP, int WARPS, int MINB = 1024 / (WARPS * 32)>
+__global__ void __launch_bounds__(WARPS * 32, MINB)
 speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
                        unsigned flags, const int32_t* __restrict__ d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
                        int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
@@ -1118,44 +1121,45 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
     SD_CUDA_OK(cudaGetDevice(&dev));
     if (dev >= 0 && dev < 64 && !raised[dev]) {
         // the block's shared memory exceeds the default limit: raise it once per device
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_STEP>,
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_STEP, 2>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_STEP>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_WIDE>,
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_WIDE, 1>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_WIDE>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_WIDE>,
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_WIDE_STEP, 1>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(BlockSharedT<CTA_WARPS_WIDE>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_NARROW>,
+                                        (int)sizeof(BlockSharedT<CTA_WARPS_WIDE_STEP>)));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_NARROW, 4>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_NARROW>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_NARROW>,
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_NARROW, 4>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_NARROW>)));
         SD_CUDA_OK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
         raised[dev] = true;
     }
-    // one block per SM is all a small batch can use: give each block 32 warps if its request has
-    // more jobs (two trees, Pe pattern lengths each) than 16 warps start at once
+    // one block per SM is all a small batch can use: sd_speculate then takes more warps if a
+    // request has more jobs (two trees, Pe pattern lengths each) than 16 warps start at once,
+    // sd_step takes more registers
     const bool known = dev >= 0 && dev < 64;
-    const bool wide = known && n <= sm_count[dev] && 2 * Pe > 2 * CTA_WARPS;
+    const bool wide = known && n <= sm_count[dev] && (step || 2 * Pe > 2 * CTA_WARPS);
     // more requests than two 16-warp blocks per SM hold at once: smaller blocks, one wave
     const bool narrow = known && n > 2 * sm_count[dev];
-#define SD_LAUNCH_FUSED(STEP, WARPS, OFF, TOK)                                                                          \
-    speculate_fused_kernel<STEP, WARPS><<<(unsigned)n, WARPS * 32, sizeof(BlockSharedT<WARPS>), st>>>(                    \
+#define SD_LAUNCH_FUSED(STEP, WARPS, MINB, OFF, TOK)                                                                    \
+    speculate_fused_kernel<STEP, WARPS, MINB><<<(unsigned)n, WARPS * 32, sizeof(BlockSharedT<WARPS>), st>>>(              \
         *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,          \
         d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, OFF, TOK)
     if (step) {
-        if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE, d_app_off, d_app_tok);
-        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW, d_app_off, d_app_tok);
-        else SD_LAUNCH_FUSED(true, CTA_WARPS_STEP, d_app_off, d_app_tok);
+        if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE_STEP, 1, d_app_off, d_app_tok);
+        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW, 4, d_app_off, d_app_tok);
+        else SD_LAUNCH_FUSED(true, CTA_WARPS_STEP, 2, d_app_off, d_app_tok);
     } else {
-        if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, nullptr, nullptr);
-        else if (narrow) SD_LAUNCH_FUSED(false, CTA_WARPS_NARROW, nullptr, nullptr);
-        else SD_LAUNCH_FUSED(false, CTA_WARPS, nullptr, nullptr);
+        if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, 1, nullptr, nullptr);
+        else if (narrow) SD_LAUNCH_FUSED(false, CTA_WARPS_NARROW, 4, nullptr, nullptr);
+        else SD_LAUNCH_FUSED(false, CTA_WARPS, 2, nullptr, nullptr);
     }
 #undef SD_LAUNCH_FUSED
     SD_CUDA_OK(cudaGetLastError());

@@ -29,7 +29,7 @@ __global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const i
                     const int nc = (int)((unsigned)pe.w & RUN_COUNT_MASK);
                     int pos;
                     int4 fe;
-                    node = nc > 0 ? lookup_child(sv.g_ent, pe.z, nc, x, pos, fe) : -1;
+                    node = nc > 0 ? lookup_child<8>(sv.g_ent, pe.z, nc, x, pos, fe) : -1;
                     seen += pos;
                 }
             }

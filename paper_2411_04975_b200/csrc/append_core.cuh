@@ -32,29 +32,32 @@ __device__ __forceinline__ int* word(int4* e, int k) { return reinterpret_cast<i
 // Inserts child x at sorted position `pos` into the child run of `parent`
 // (cb, n children, flags in w).  `fresh` > 0: the run is full and moves to
 // ent[fresh ...).  Returns the new child's entry index.
+// G: entries moved (or, in the look-up, read) per round.  Eight where registers are plentiful;
+// the decode-step kernel, which has to share its registers with the speculation code, uses four.
+template <int G>
 __device__ int insert_child(int4* ent, int parent, int cb, int n, int pos, int x, int fresh, bool moves) {
     const int4 ne = make_int4(x, 1, 0, 0);
     int idx;
-    // entries move eight at a time: the eight loads are in flight together
+    // entries move G at a time: the loads of a round are in flight together
     if (moves) {
-        for (int k0 = 0; k0 < n; k0 += 8) {
-            int4 t[8];
+        for (int k0 = 0; k0 < n; k0 += G) {
+            int4 t[G];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) if (k0 + u < n) t[u] = ent[cb + k0 + u];
+            for (int u = 0; u < G; ++u) if (k0 + u < n) t[u] = ent[cb + k0 + u];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) if (k0 + u < n) ent[fresh + k0 + u + (k0 + u >= pos ? 1 : 0)] = t[u];
+            for (int u = 0; u < G; ++u) if (k0 + u < n) ent[fresh + k0 + u + (k0 + u >= pos ? 1 : 0)] = t[u];
         }
         ent[fresh + pos] = ne;
         *word(&ent[parent], 2) = fresh;
         idx = fresh + pos;
     } else {
-        for (int hi = n; hi > pos; hi -= 8) {                    // from the top down
-            const int lo = max(pos, hi - 8);
-            int4 t[8];
+        for (int hi = n; hi > pos; hi -= G) {                    // from the top down
+            const int lo = max(pos, hi - G);
+            int4 t[G];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) if (lo + u < hi) t[u] = ent[cb + lo + u];
+            for (int u = 0; u < G; ++u) if (lo + u < hi) t[u] = ent[cb + lo + u];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) if (lo + u < hi) ent[cb + lo + u + 1] = t[u];
+            for (int u = 0; u < G; ++u) if (lo + u < hi) ent[cb + lo + u + 1] = t[u];
         }
         ent[cb + pos] = ne;
         idx = cb + pos;
@@ -127,7 +130,8 @@ __device__ int lower_bound_run(const int4* ent, int cb, int n, int x) {
 
 // Look-up of child x in the sorted run ent[cb .. cb+n): insert position in `pos`, and if the
 // child exists its index is returned with its entry in `fe` (else -1).  The last round reads
-// whole entries, so a run of up to eight children costs one round of loads.
+// whole entries, so a run of up to G children costs one round of loads.
+template <int G>
 __device__ int lookup_child(const int4* ent, int cb, int n, int x, int& pos, int4& fe) {
     int lo = 0, hi = n;
     while (hi - lo > 256) {                                      // very long runs: 32-way, 31 probes in flight
@@ -139,25 +143,41 @@ __device__ int lookup_child(const int4* ent, int cb, int n, int x, int& pos, int
         const int nhi = sel == 31 ? hi : lo + (sel + 1) * step + 1;   // keep the pivot: it may be x itself
         lo = nlo; hi = nhi;
     }
-    while (hi - lo > 8) {                                        // eight-way down to a window of eight
-        const int step = (hi - lo) >> 3;
-        int sel = 0;
+    if (G == 8) {
+        while (hi - lo > 8) {                                    // eight-way down to a window of eight
+            const int step = (hi - lo) >> 3;
+            int sel = 0;
 #pragma unroll
-        for (int k = 0; k < 7; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
-        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
-        const int nhi = sel == 7 ? hi : lo + (sel + 1) * step + 1;
-        lo = nlo; hi = nhi;
+            for (int k = 0; k < 7; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
+            const int nlo = sel == 0 ? lo : lo + sel * step + 1;
+            const int nhi = sel == 7 ? hi : lo + (sel + 1) * step + 1;
+            lo = nlo; hi = nhi;
+        }
+    } else {
+        // eight parts of `step` entries, probed at their last entries: the window becomes the
+        // first part that does not lie wholly below x (32 entries or fewer leave at most four)
+        while (hi - lo > G) {
+            const int step = (hi - lo + 7) >> 3;
+            int sel = 0;
+#pragma unroll
+            for (int k = 0; k < 7; ++k) {
+                const int q = lo + (k + 1) * step - 1;
+                sel += (q < hi && ent[cb + q].x < x) ? 1 : 0;
+            }
+            lo += sel * step;
+            hi = min(hi, lo + step);
+        }
     }
-    int4 e[8];
+    int4 e[G];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) e[k] = lo + k < hi ? ent[cb + lo + k] : make_int4(0x7fffffff, 0, 0, 0);
+    for (int k = 0; k < G; ++k) e[k] = lo + k < hi ? ent[cb + lo + k] : make_int4(0x7fffffff, 0, 0, 0);
     int below = 0;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) below += e[k].x < x ? 1 : 0;
+    for (int k = 0; k < G; ++k) below += e[k].x < x ? 1 : 0;
     pos = lo + below;
     int found = -1;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) if (k == below && lo + k < hi && e[k].x == x) { fe = e[k]; found = cb + lo + k; }
+    for (int k = 0; k < G; ++k) if (k == below && lo + k < hi && e[k].x == x) { fe = e[k]; found = cb + lo + k; }
     return found;
 }
 
@@ -200,6 +220,7 @@ __device__ int warm_shallow(const TreeRef& tr, int V, const int32_t* tok, long l
 // Returns false, changing nothing, if the pool cannot hold the new nodes.
 // (run_cb, run_w) travel with `act`: the active node's child run as of now, so that the
 // next token's look-up starts at the run itself instead of first reading the node.
+template <int G = 8>
 __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, int& act, int& room, int& run_cb,
                              unsigned& run_w, int& used, int& live) {
     const unsigned FULL = 0xffffffffu;
@@ -219,7 +240,7 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
             cb = parent_cb; w = parent_w;
             if (w == RUN_UNKNOWN) { const int4 pe = tr.ent[parent]; cb = pe.z; w = (unsigned)pe.w; }
             n = (int)(w & RUN_COUNT_MASK);
-            found = lookup_child(tr.ent, cb, n, x, pos, fe);
+            found = lookup_child<G>(tr.ent, cb, n, x, pos, fe);
         }
     }
     const bool need = valid && found < 0;
@@ -284,7 +305,7 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
                 tr.root[x] = fresh;
                 act = fresh;
             } else {
-                act = insert_child(tr.ent, parent, cb, n, pos, x, fresh, moves);
+                act = insert_child<G>(tr.ent, parent, cb, n, pos, x, fresh, moves);
             }
         }
         __syncwarp();

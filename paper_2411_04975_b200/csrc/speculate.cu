@@ -263,7 +263,7 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 
 // ---------------------------------------------------------------------------------------------
 // Fused path: one block of W warps per request.  Two blocks per SM is the usual shape: W = 16
-// with 64 registers per thread for sd_speculate, W = 8 with 128 for sd_step, whose append is
+// with 64 registers per thread for sd_speculate, W = 10 with 96 for sd_step, whose append is
 // register hungry.  A batch of at most one request per SM gets bigger blocks (W = 24 / 16), a
 // batch of more than two requests per SM smaller ones (W = 8 / 4, four per SM) to stay in one wave.
 //   1. match: the per-request match nodes are the slot's active nodes; the global match
@@ -276,10 +276,12 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 //      reached by another job of the request.
 //   3. select + emit from shared memory; no global scratch.
 constexpr int CTA_WARPS = 16;                  // the usual block
-constexpr int CTA_WARPS_STEP = 8;              // the usual block of sd_step: 8 warps with 128 registers each, so
-                                               // that the append in front does not spill (measured per step:
-                                               // 95 us; 10 warps with 96 registers 100, 12 with 80 100, 16 with
-                                               // 64 104, 6 with 168 110)
+constexpr int CTA_WARPS_STEP = 10;             // the usual block of sd_step: 10 warps with 96 registers each and
+constexpr int STEP_G = 4;                      // an append that moves four entries per round, so that the
+                                               // append in front does not spill.  Measured per step: 92.7 us;
+                                               // 9 warps 92.8, 11 (80 registers) 95, 8 (128) 96; with eight
+                                               // entries per round: 8 warps x 128 registers 95, 10 x 96 100,
+                                               // 12 x 80 100, 16 x 64 104, 6 x 168 110
 constexpr int CTA_WARPS_WIDE = 24;             // small batches (one block per SM at most): the block has the SM's
 constexpr int CTA_WARPS_WIDE_STEP = 16;        // registers to itself (80 per thread; sd_step: 128)
 constexpr int CTA_WARPS_NARROW = 8;            // batches of more than two requests per SM: four blocks per SM
@@ -822,7 +824,7 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
 // sd_append does for the slot) while its other warps already advance the global match nodes
 // over those tokens, then speculates: one launch per decode step, and the appends of long
 // token lists overlap with the speculation of the other requests.
-template <bool STEP, int WARPS, int MINB = 1024 / (WARPS * 32)>
+template <bool STEP, int WARPS, int MINB, int APPEND_G = 8>
 __global__ void __launch_bounds__(WARPS * 32, MINB)
 speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
                        unsigned flags, const int32_t* __restrict__ d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
@@ -900,7 +902,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
         for (int k = 0; k < n_new && !(st & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)); ++k) {
             const int x = newtok[k];
             if (x < 0 || x >= sv.V) { st |= SD_STATUS_BAD_TOKEN; break; }
-            if (len >= sv.T || !append_token(tr, sv.D, x, len, lane, act, room, run_cb, run_w, used, live)) {
+            if (len >= sv.T || !append_token<APPEND_G>(tr, sv.D, x, len, lane, act, room, run_cb, run_w, used, live)) {
                 st |= SD_STATUS_POOL_FULL;
                 break;
             }
@@ -1124,7 +1126,7 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
         // the block's shared memory exceeds the default limit: raise it once per device
         SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_STEP, 2>,
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_STEP, 2, STEP_G>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_STEP>)));
         SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_WIDE, 1>,
@@ -1149,18 +1151,18 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
     const bool wide = known && n <= sm_count[dev] && (step || 2 * Pe > 2 * CTA_WARPS);
     // more requests than two 16-warp blocks per SM hold at once: smaller blocks, one wave
     const bool narrow = known && n > 2 * sm_count[dev];
-#define SD_LAUNCH_FUSED(STEP, WARPS, MINB, OFF, TOK)                                                                    \
-    speculate_fused_kernel<STEP, WARPS, MINB><<<(unsigned)n, WARPS * 32, sizeof(BlockSharedT<WARPS>), st>>>(              \
+#define SD_LAUNCH_FUSED(STEP, WARPS, MINB, G, OFF, TOK)                                                                 \
+    speculate_fused_kernel<STEP, WARPS, MINB, G><<<(unsigned)n, WARPS * 32, sizeof(BlockSharedT<WARPS>), st>>>(           \
         *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,          \
         d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, OFF, TOK)
     if (step) {
-        if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE_STEP, 1, d_app_off, d_app_tok);
-        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW_STEP, 4, d_app_off, d_app_tok);
-        else SD_LAUNCH_FUSED(true, CTA_WARPS_STEP, 2, d_app_off, d_app_tok);
+        if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE_STEP, 1, 8, d_app_off, d_app_tok);
+        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW_STEP, 4, 8, d_app_off, d_app_tok);
+        else SD_LAUNCH_FUSED(true, CTA_WARPS_STEP, 2, STEP_G, d_app_off, d_app_tok);
     } else {
-        if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, 1, nullptr, nullptr);
-        else if (narrow) SD_LAUNCH_FUSED(false, CTA_WARPS_NARROW, 4, nullptr, nullptr);
-        else SD_LAUNCH_FUSED(false, CTA_WARPS, 2, nullptr, nullptr);
+        if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, 1, 8, nullptr, nullptr);
+        else if (narrow) SD_LAUNCH_FUSED(false, CTA_WARPS_NARROW, 4, 8, nullptr, nullptr);
+        else SD_LAUNCH_FUSED(false, CTA_WARPS, 2, 8, nullptr, nullptr);
     }
 #undef SD_LAUNCH_FUSED
     SD_CUDA_OK(cudaGetLastError());

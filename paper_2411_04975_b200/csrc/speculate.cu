@@ -265,7 +265,7 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 // Fused path: one block of W warps per request.  Two blocks per SM is the usual shape: W = 16
 // with 64 registers per thread for sd_speculate, W = 10 with 96 for sd_step, whose append is
 // register hungry.  A batch of at most one request per SM gets bigger blocks (W = 24 / 16), a
-// batch of more than two requests per SM smaller ones (W = 8 / 4, four per SM) to stay in one wave.
+// batch of more than two requests per SM smaller ones (W = 8 / 5, four per SM) to stay in one wave.
 //   1. match: the per-request match nodes are the slot's active nodes; the global match
 //      nodes are advanced from the nodes cached at the previous call by descending only the
 //      tokens appended since (full walks when the cache is stale).  Warp w serves pattern
@@ -285,7 +285,8 @@ constexpr int STEP_G = 4;                      // an append that moves four entr
 constexpr int CTA_WARPS_WIDE = 24;             // small batches (one block per SM at most): the block has the SM's
 constexpr int CTA_WARPS_WIDE_STEP = 16;        // registers to itself (80 per thread; sd_step: 128)
 constexpr int CTA_WARPS_NARROW = 8;            // batches of more than two requests per SM: four blocks per SM
-constexpr int CTA_WARPS_NARROW_STEP = 4;       // (sd_step: again 128 registers per thread)
+constexpr int CTA_WARPS_NARROW_STEP = 5;       // (sd_step: 96 registers and the four-entry append; 512 requests:
+                                               // 82 us per step, 88 with 4 warps x 128 registers, 100 with 8 x 64)
 
 struct WarpWork {
     Frontier F;
@@ -1138,7 +1139,7 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
         SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_NARROW, 4>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_NARROW>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_NARROW_STEP, 4>,
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_NARROW_STEP, 4, STEP_G>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(BlockSharedT<CTA_WARPS_NARROW_STEP>)));
         SD_CUDA_OK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
@@ -1157,7 +1158,7 @@ static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_
         d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, OFF, TOK)
     if (step) {
         if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE_STEP, 1, 8, d_app_off, d_app_tok);
-        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW_STEP, 4, 8, d_app_off, d_app_tok);
+        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW_STEP, 4, STEP_G, d_app_off, d_app_tok);
         else SD_LAUNCH_FUSED(true, CTA_WARPS_STEP, 2, STEP_G, d_app_off, d_app_tok);
     } else {
         if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, 1, 8, nullptr, nullptr);

@@ -35,9 +35,9 @@ METRIC = "speculation trees/s at batch {B} (per step: append the accepted tokens
 UNIT = "trees/s"
 OUT_BYTES_PER_REQ = 4 * 64 * 3 + 64 * 8 + 4 * 3 + 8          # tokens, parents, positions, mask, scalars
 FLUSH_BYTES = 256 << 20
-# dram__bytes_read + dram__bytes_write of one speculate_fused_kernel<1, 8, 2> launch (sd_step) on the full-size
+# dram__bytes_read + dram__bytes_write of one speculate_fused_kernel<1, 10, 2, 4> launch (sd_step) on the full-size
 # large_batch workload, from the ncu capture summarised in profiles/ (set to None when the kernel changes)
-SPECULATE_DRAM_TRAFFIC = 27.1e6
+SPECULATE_DRAM_TRAFFIC = 27.2e6
 
 
 def parse():
@@ -370,7 +370,7 @@ def run_ours(args):
         achieved = alg_bytes / spec_s / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": SPECULATE_DRAM_TRAFFIC if c.name == "large_batch" and not args.small else None,
-                    "peak_source": which, "kernel": "speculate_fused_kernel<1, 8, 2> (all of sd_step)",
+                    "peak_source": which, "kernel": "speculate_fused_kernel<1, 10, 2, 4> (all of sd_step)",
                     "algorithmic_bytes_per_launch": alg_bytes}
         extra = {"parity_vs_oracle": "bit-exact" if ok else "MISMATCH", "parity_steps": len(sample_steps),
                  "nodes_visited_per_step": visits,

@@ -295,11 +295,13 @@ def test_closed_loop_scaled(U):
     pr.close()
 
 
-def test_large_batch_full_size_sampled_against_oracle(U):
+@pytest.mark.parametrize("one_launch", [False, True])
+def test_large_batch_full_size_sampled_against_oracle(U, one_launch):
     """The headline workload (large_batch) at full size (4,194,304-token global tree, 256 requests x 4,096-token
-    prompts) in the launch configuration bench.py times.  The oracle holds the full global tree
-    but only a sample of the requests; their rows must be bit-exact, and every row must satisfy
-    the properties that hold for any draft."""
+    prompts) in the launch configurations bench.py times: sd_append + sd_speculate, and (one_launch)
+    prompts through sd_build_requests and every decode step as one sd_step.  The oracle holds the
+    full global tree but only a sample of the requests; their rows must be bit-exact, and every
+    row must satisfy the properties that hold for any draft."""
     from workload.generator import accept_schedule, get_workload
     import oracle as oracle_pkg
     import paper_2411_04975_b200 as sfx
@@ -314,7 +316,10 @@ def test_large_batch_full_size_sampled_against_oracle(U):
     prompts = [w.prompt(i) for i in range(B)]
     off, flat = U.ragged(prompts)
     slots = torch.arange(B, dtype=torch.int32, device=dev)
-    store.append(slots, torch.as_tensor(off, device=dev), U.dev_i32(flat), torch.ones(B, dtype=torch.uint8, device=dev))
+    if one_launch:
+        store.build_requests(np.arange(B, dtype=np.int32), off, U.dev_i32(flat))
+    else:
+        store.append(slots, torch.as_tensor(off, device=dev), U.dev_i32(flat), torch.ones(B, dtype=torch.uint8, device=dev))
     ref = oracle_pkg.SuffixOracle(c.depth_cap, len(sample))
     ref.global_build(w.corpus(), w.corpus_offsets())
     ref.slot_append_batch(list(range(len(sample))), [prompts[i] for i in sample], n_threads=8)
@@ -322,8 +327,13 @@ def test_large_batch_full_size_sampled_against_oracle(U):
     sched = accept_schedule(B, 3)
     cont = [w.continuation(i, prompts[i], length=int(sched[:, i].sum()) + 1) for i in range(B)]
     cur = np.zeros(B, dtype=np.int64)
+    pending = None                                             # (offsets, tokens) accepted in the last step
     for step in range(3):
-        out = store.speculate(slots, c.max_pattern, c.alpha, c.max_spec)
+        if one_launch and pending is not None:
+            out = store.step(slots, torch.as_tensor(pending[0], device=dev), U.dev_i32(pending[1]), c.max_pattern,
+                             c.alpha, c.max_spec)
+        else:
+            out = store.speculate(slots, c.max_pattern, c.alpha, c.max_spec)
         torch.cuda.synchronize()
         got = {k: v.cpu().numpy() for k, v in out.items()}
         got["mask"] = got["mask"].view(np.uint32)
@@ -352,7 +362,10 @@ def test_large_batch_full_size_sampled_against_oracle(U):
         lists = [cont[i][cur[i]:cur[i] + a[i]] for i in range(B)]
         cur += a
         o2, f2 = U.ragged(lists)
-        store.append(slots, torch.as_tensor(o2, device=dev), U.dev_i32(f2))
+        if one_launch and step < 2:
+            pending = (o2, f2)                                  # appended by the next step's launch
+        else:
+            store.append(slots, torch.as_tensor(o2, device=dev), U.dev_i32(f2))
         ref.slot_append_batch(list(range(len(sample))), [lists[i] for i in sample], n_threads=8)
     # the sampled per-request trees, node by node
     for k, i in enumerate(sample[:3]):

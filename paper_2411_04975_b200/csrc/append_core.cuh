@@ -284,7 +284,20 @@ __device__ bool append_token(const TreeRef& tr, int D, int x, int t, int lane, i
         run_w = (unsigned)fe.w;
         // the next lane works on this very node's run (new child, or flag dropped): what was read may be stale
         if (lane < 31 && next_parent == found) run_w = RUN_UNKNOWN;
-        else if (run_w & RUN_COUNT_MASK) asm volatile("prefetch.global.L2 [%0];" ::"l"(tr.ent + run_cb));
+        else if (run_w & RUN_COUNT_MASK) {
+            // The next token's look-up starts in this run: ask L2 for what its first round will
+            // read (the whole run if it is short, else the seven probes of an eight-way split).
+            const int nn = (int)(run_w & RUN_COUNT_MASK);
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(tr.ent + run_cb));
+            if (nn > G) {
+                const int step = G == 8 ? (nn >> 3) : ((nn + 7) >> 3);
+#pragma unroll
+                for (int k = 0; k < 7; ++k) {
+                    const int q = G == 8 ? (k + 1) * step : (k + 1) * step - 1;
+                    if (q < nn) asm volatile("prefetch.global.L2 [%0];" ::"l"(tr.ent + run_cb + q));
+                }
+            }
+        }
     } else {
         run_cb = 0;
         run_w = 0;                                               // a new leaf (or no node at all)

@@ -10,39 +10,116 @@ namespace {
 // of its positions: one root-to-depth-D PATH per start position.  Taking the tokens one after the
 // other makes a chain as long as the sequence.  Here one block takes up to 1,024 paths at once, a
 // thread per path, and all of them go down one level per round:
-//   A. every path looks its next token up in the child run of its current node; a child that
-//      exists gets its count raised by an atomic add, the others are PENDING;
-//   B. pending paths are served in rounds: per parent node one path is elected (a table of locks
-//      in shared memory, indexed by a hash of the parent), looks again (an earlier round may
-//      have added the very child) and inserts.  Runs of different parents are disjoint, so the
-//      elected paths do not disturb one another; paths of the same parent go one per round;
-//   C. an insert shifts or moves its run, so every path whose parent's run changed after it
-//      found its child looks the child's new place up.
+//   1. every path enters its current node (the parent of the node it is about to reach) into a
+//      hash set in shared memory, which counts the paths per parent;
+//   2. every path looks its next token up in the parent's child run.  A child that exists gets its
+//      count raised by an atomic add.  A missing child is inserted at once if the path is the
+//      only one at that parent: nobody else reads or writes that run during this level;
+//   3. the other missing children are PENDING and are served in rounds: per parent one path is
+//      elected per round (a turn counter in the parent's hash-set cell), looks again (an earlier
+//      round may have added the very child) and inserts.  Runs of different parents are
+//      disjoint, so the elected paths do not disturb one another;
+//   4. an insert shifts or moves its run, so every path that shares its parent and whose parent's
+//      run changed after it took its child looks the child's new place up.
 // Only runs of ONE depth change during a level, and the entries of their parents (one level up)
-// stay where they are, which is what makes the election by parent sufficient.  There is no
-// waiting on another thread anywhere, only block-wide barriers.  Placement follows the
+// stay where they are, which is what makes the election by parent sufficient.  A node's own
+// child run (first entry and size, as read with the node's entry) stays valid until the next
+// level, so it travels with the path and the next look-up starts at the run itself.  There is
+// no waiting on another thread anywhere, only block-wide barriers.  Placement follows the
 // token-by-token append: the first leaf of a path that leaves the known text reserves room down
 // to depth D and the later leaves go directly behind their parents.
 constexpr int GI_THREADS = 1024;
-constexpr int GI_LOCKS = 4096;
+constexpr int GI_SLOTS = 2048;                // cells of the parent set: at most half full
 constexpr int GI_ITEMS = 256;
 constexpr int GI_BIG = 48;                    // inserts that move more entries are done by a whole warp
 
 struct GiShared {
-    int lock[GI_LOCKS];
+    int key[GI_SLOTS];                        // parent + 1 (level 1: token + 1), 0 = free
+    int cnt[GI_SLOTS];                        // paths at that parent
+    int turn[GI_SLOTS];                       // rounds in which a path of that parent was elected
     int item[GI_ITEMS];
     long long begin[GI_ITEMS], end[GI_ITEMS], pref[GI_ITEMS + 1];
     unsigned long long used;
     int n_items, live, status;
 };
 
-__device__ __forceinline__ unsigned gi_hash(int key) { return ((unsigned)key * 2654435761u) >> 20; }   // 12 bits
+// Entries for new runs and chain blocks of a warp's lanes (`size` may be 0): one atomic per warp.
+// Returns the lane's first entry, -1 if it asked for none or the pool cannot hold the warp's
+// request (then the status bit is set as well).  All 32 lanes call.
+__device__ __forceinline__ int gi_alloc_warp(GiShared& sh, long long cap, int size, int lane) {
+    const unsigned FULL = 0xffffffffu;
+    int inc = size;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(FULL, inc, o);
+        if (lane >= o) inc += y;
+    }
+    const int total = __shfl_sync(FULL, inc, 31);
+    if (total == 0) return -1;
+    unsigned long long at = 0;
+    if (lane == 31) at = atomicAdd(&sh.used, (unsigned long long)total);
+    at = __shfl_sync(FULL, at, 31);
+    if (at + (unsigned long long)total > (unsigned long long)cap) {
+        if (lane == 31) atomicOr(&sh.status, SD_STATUS_GLOBAL_FULL);
+        return -1;
+    }
+    return size > 0 ? (int)at + inc - size : -1;
+}
 
-// Entries for a new run or chain block; -1 (and the status bit) when the pool cannot hold them.
-__device__ __forceinline__ int gi_alloc(GiShared& sh, long long cap, int size) {
-    const unsigned long long at = atomicAdd(&sh.used, (unsigned long long)size);
-    if (at + (unsigned long long)size > (unsigned long long)cap) { atomicOr(&sh.status, SD_STATUS_GLOBAL_FULL); return -1; }
-    return (int)at;
+// Child x of `cur` is missing and this path may add it (`ins`; lanes without an insert pass
+// false).  All 32 lanes call.  On return nxt is the new node and new_room the room reserved
+// behind it; (seen_cb, seen_n) describe the parent's run right after the insert.  A path whose
+// entries the pool cannot hold stops (rem = 0).
+__device__ __forceinline__ void gi_insert(GiShared& sh, const sd_store& sv, int d, int lane, bool ins, int x, int cur,
+                                          int room, int cb, int nc, unsigned w, int pos, int& nxt, int& new_room,
+                                          int& seen_cb, int& seen_n, int& rem, int& my_live) {
+    const unsigned FULL = 0xffffffffu;
+    int4* const ent = sv.g_ent;
+    const int D = sv.D;
+    bool moves = false, behind = false;
+    int asz = 0;
+    if (ins) {
+        if (d == 1) asz = D;                                     // a new depth-1 node starts a chain block
+        else if (nc == 0) {                                      // first child of a leaf: continue the chain block, or start one
+            moves = true;
+            if (room > 0) behind = true; else asz = D - d + 1;
+        } else if ((uint32_t)nc == sd_run_capacity(w)) {         // the run is full: it moves to twice the room
+            moves = true;
+            asz = (int)sd_pow2ceil((uint32_t)nc + 1u);
+        }
+    }
+    int fresh = gi_alloc_warp(sh, sv.g_cap, asz, lane);
+    bool big = false;
+    if (ins) {
+        if (asz > 0 && fresh < 0) rem = 0;
+        else {
+            ++my_live;
+            if (d == 1) {
+                ent[fresh] = make_int4(x, 1, 0, 0);
+                sv.g_root[x] = fresh;
+                nxt = fresh;
+                new_room = D - 1;
+            } else {
+                if (behind) { fresh = cur + 1; new_room = room - 1; }
+                else new_room = nc == 0 ? asz - 1 : 0;
+                seen_cb = moves ? fresh : cb;
+                seen_n = nc + 1;
+                big = (moves ? nc : nc - pos) > GI_BIG;
+                if (!big) nxt = insert_child<8>(ent, cur, cb, nc, pos, x, fresh, moves);
+            }
+        }
+    }
+    // inserts that move many entries: the warp does them one after the other
+    unsigned bm = __ballot_sync(FULL, big);
+    while (bm) {
+        const int src = __ffs(bm) - 1;
+        bm &= bm - 1;
+        const int idx = insert_child_warp(ent, __shfl_sync(FULL, cur, src), __shfl_sync(FULL, cb, src),
+                                          __shfl_sync(FULL, nc, src), __shfl_sync(FULL, pos, src),
+                                          __shfl_sync(FULL, x, src), __shfl_sync(FULL, fresh, src),
+                                          __shfl_sync(FULL, moves ? 1 : 0, src) != 0, lane);
+        if (lane == src) nxt = idx;
+    }
 }
 
 __global__ void __launch_bounds__(GI_THREADS, 1)
@@ -51,15 +128,16 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
     const unsigned FULL = 0xffffffffu;
     const int tid = threadIdx.x, lane = tid & 31;
     int4* const ent = sv.g_ent;
-    int32_t* const root = sv.g_root;
     const int D = sv.D;
 
     bool mine = false;
     for (int i = tid; i < n; i += GI_THREADS) mine |= d_slot[i] == -1;
     if (!__syncthreads_or(mine)) return;                         // the usual decode step: nothing for the global tree
     if (tid == 0) { sh.used = (unsigned long long)sv.g_state->used; sh.live = 0; sh.status = sv.g_state->status; }
+    for (int i = tid; i < GI_SLOTS; i += GI_THREADS) { sh.key[i] = 0; sh.cnt[i] = 0; sh.turn[i] = 0; }
     __syncthreads();
     long long tokens_done = 0;
+    int my_live = 0;
 
     for (int base = 0; base < n; base += GI_ITEMS) {
         if (__syncthreads_or(sh.status & SD_STATUS_GLOBAL_FULL)) break;
@@ -114,111 +192,91 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                 k = sh.begin[lo] + (p - sh.pref[lo]);
                 rem = (int)min((long long)D, sh.end[lo] - k);
             }
-            int cur = -1, room = 0;                              // node of the tokens taken so far; room reserved behind it
+            // the node of the tokens taken so far, the room reserved behind it, its child run
+            int cur = -1, room = 0, run_cb = 0;
+            unsigned run_w = 0;
             for (int d = 1; d <= D; ++d) {
-                if (!__syncthreads_or(rem >= d)) break;
+                if (!__syncthreads_or(rem >= d)) break;          // (the parent set is empty here)
                 const bool alive = rem >= d;
                 const int x = alive ? d_tokens[k + d - 1] : 0;
-                int found = -1, pos = 0, cb = 0, nc = 0;
-                unsigned w = 0;
-                int4 fe = make_int4(0, 0, 0, 0);
-                // A: look the token up
+                // 1. the parent set
+                int cell = 0;
                 if (alive) {
-                    if (d == 1) found = root[x];
-                    else {
-                        const int4 pe = ent[cur];
-                        cb = pe.z; w = (unsigned)pe.w; nc = (int)(w & RUN_COUNT_MASK);
-                        if (nc > 0) found = lookup_child<8>(ent, cb, nc, x, pos, fe);
+                    const int key = (d == 1 ? x : cur) + 1;
+                    cell = (int)(((unsigned)key * 2654435761u) >> 21);          // 11 bits
+                    for (int probe = 0; probe < GI_SLOTS; ++probe) {
+                        const int old = atomicCAS(&sh.key[cell], 0, key);
+                        if (old == 0 || old == key) break;
+                        cell = (cell + 1) & (GI_SLOTS - 1);
                     }
+                    atomicAdd(&sh.cnt[cell], 1);
+                }
+                __syncthreads();
+                const bool alone = alive && sh.cnt[cell] == 1;
+                // 2. look the token up
+                int found = -1, pos = 0;
+                int cb = run_cb, nc = (int)(run_w & RUN_COUNT_MASK);
+                unsigned w = run_w;
+                int4 fe = make_int4(0, 0, 0, 0);
+                if (alive) {
+                    if (d == 1) { found = sv.g_root[x]; if (found >= 0) fe = ent[found]; }
+                    else if (nc > 0) found = lookup_child<8>(ent, cb, nc, x, pos, fe);
                     if (found >= 0) {
                         atomicAdd(word(&ent[found], 1), 1);
                         // a count changes: the copies in the run's top block (if any) are stale from now on
                         if (d > 1 && (w & RUN_HAS_TOP)) atomicAnd(word(&ent[cur], 3), (int)~RUN_HAS_TOP);
                     }
                 }
-                bool pending = alive && found < 0;
                 int nxt = found, new_room = 0;
                 int seen_cb = cb, seen_n = nc;                    // the parent's run as it was when nxt was taken
-                // B: inserts, one path per parent and round
+                gi_insert(sh, sv, d, lane, alive && found < 0 && alone, x, cur, room, cb, nc, w, pos, nxt, new_room,
+                          seen_cb, seen_n, rem, my_live);
+                // 3. the other inserts: one path per parent and round
+                bool pending = alive && found < 0 && !alone;
                 for (int round = 0; round <= GI_THREADS; ++round) {
                     if (!__syncthreads_or(pending)) break;
-                    for (int i = tid; i < GI_LOCKS; i += GI_THREADS) sh.lock[i] = 0;
-                    __syncthreads();
-                    const bool win = pending && atomicCAS(&sh.lock[gi_hash(d == 1 ? x : cur)], 0, 1) == 0;
-                    bool big = false;
-                    int fresh = 0;
-                    bool moves = false;
+                    const bool win = pending && atomicCAS(&sh.turn[cell], round, round + 1) == round;
                     if (win) {
                         pending = false;
                         if (round > 0) {                         // an earlier round may have changed the run
                             found = -1; pos = 0;
-                            if (d == 1) found = root[x];
+                            if (d == 1) { found = sv.g_root[x]; if (found >= 0) fe = ent[found]; }
                             else {
                                 const int4 pe = ent[cur];
                                 cb = pe.z; w = (unsigned)pe.w; nc = (int)(w & RUN_COUNT_MASK);
                                 if (nc > 0) found = lookup_child<8>(ent, cb, nc, x, pos, fe);
                             }
-                        }
-                        if (found >= 0) {                        // added meanwhile by a path with the same string
-                            atomicAdd(word(&ent[found], 1), 1);
-                            nxt = found; seen_cb = cb; seen_n = nc;
-                        } else if (d == 1) {
-                            fresh = gi_alloc(sh, sv.g_cap, D);
-                            if (fresh >= 0) {
-                                ent[fresh] = make_int4(x, 1, 0, 0);
-                                root[x] = fresh;
-                                nxt = fresh; new_room = D - 1;
-                                atomicAdd(&sh.live, 1);
-                            } else rem = 0;
-                        } else {
-                            bool ok = true;
-                            if (nc == 0) {
-                                // first child of a leaf: continue the chain block, or start one
-                                moves = true;
-                                if (room > 0) { fresh = cur + 1; new_room = room - 1; }
-                                else { const int asz = D - d + 1; fresh = gi_alloc(sh, sv.g_cap, asz); new_room = asz - 1; ok = fresh >= 0; }
-                            } else if ((uint32_t)nc == sd_run_capacity(w)) {
-                                moves = true;
-                                fresh = gi_alloc(sh, sv.g_cap, (int)sd_pow2ceil((uint32_t)nc + 1u));
-                                ok = fresh >= 0;
-                            }
-                            if (!ok) { rem = 0; new_room = 0; }
-                            else {
-                                atomicAdd(&sh.live, 1);
-                                seen_cb = moves ? fresh : cb; seen_n = nc + 1;
-                                big = (moves ? nc : nc - pos) > GI_BIG;
-                                if (!big) nxt = insert_child<8>(ent, cur, cb, nc, pos, x, fresh, moves);
+                            if (found >= 0) {                    // added meanwhile by a path with the same string
+                                atomicAdd(word(&ent[found], 1), 1);
+                                nxt = found; seen_cb = cb; seen_n = nc;
                             }
                         }
                     }
-                    // inserts that move many entries: the warp does them one after the other
-                    unsigned bm = __ballot_sync(FULL, big);
-                    while (bm) {
-                        const int src = __ffs(bm) - 1;
-                        bm &= bm - 1;
-                        const int idx = insert_child_warp(ent, __shfl_sync(FULL, cur, src), __shfl_sync(FULL, cb, src),
-                                                          __shfl_sync(FULL, nc, src), __shfl_sync(FULL, pos, src),
-                                                          __shfl_sync(FULL, x, src), __shfl_sync(FULL, fresh, src),
-                                                          __shfl_sync(FULL, moves ? 1 : 0, src) != 0, lane);
-                        if (lane == src) nxt = idx;
-                    }
+                    gi_insert(sh, sv, d, lane, win && found < 0, x, cur, room, cb, nc, w, pos, nxt, new_room, seen_cb,
+                              seen_n, rem, my_live);
                 }
-                // C: the child's place after all inserts of this level
-                if (rem >= d && d > 1) {
+                // 4. the child's place after all inserts of this level
+                if (rem >= d && d > 1 && !alone) {
                     const int4 pe = ent[cur];
                     const int n2 = (int)((unsigned)pe.w & RUN_COUNT_MASK);
                     if (pe.z != seen_cb || n2 != seen_n) {
-                        nxt = n2 > 0 ? lookup_child<8>(ent, pe.z, n2, x, pos, fe) : -1;
+                        found = n2 > 0 ? lookup_child<8>(ent, pe.z, n2, x, pos, fe) : -1;
+                        nxt = found;
                         new_room = 0;                            // the node left its chain block
                     }
                 }
                 if (rem >= d && nxt < 0) rem = 0;                // cannot happen; the path stops rather than go astray
                 cur = nxt;
                 room = new_room;
+                run_cb = found >= 0 ? fe.z : 0;                  // a node made just now has no children
+                run_w = found >= 0 ? (unsigned)fe.w : 0u;
+                for (int i = tid; i < GI_SLOTS; i += GI_THREADS) { sh.key[i] = 0; sh.cnt[i] = 0; sh.turn[i] = 0; }
             }
             tokens_done += min((long long)GI_THREADS, total - c0);
         }
     }
+    __syncthreads();
+    if (my_live) atomicAdd(&sh.live, my_live);
     __syncthreads();
     if (tid == 0) {
         GlobalState* gs = sv.g_state;

@@ -37,7 +37,7 @@ OUT_BYTES_PER_REQ = 4 * 64 * 3 + 64 * 8 + 4 * 3 + 8          # tokens, parents, 
 FLUSH_BYTES = 256 << 20
 # dram__bytes_read + dram__bytes_write of one speculate_fused_kernel<1, 10, 2, 4> launch (sd_step) on the full-size
 # large_batch workload, from the ncu capture summarised in profiles/ (set to None when the kernel changes)
-SPECULATE_DRAM_TRAFFIC = 27.2e6
+SPECULATE_DRAM_TRAFFIC = 27.3e6
 
 
 def parse():

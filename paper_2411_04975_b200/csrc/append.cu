@@ -229,8 +229,20 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                 }
                 int nxt = found, new_room = 0;
                 int seen_cb = cb, seen_n = nc;                    // the parent's run as it was when nxt was taken
-                gi_insert(sh, sv, d, lane, alive && found < 0 && alone, x, cur, room, cb, nc, w, pos, nxt, new_room,
-                          seen_cb, seen_n, rem, my_live);
+                const bool own = alive && found < 0 && alone;
+                gi_insert(sh, sv, d, lane, own, x, cur, room, cb, nc, w, pos, nxt, new_room, seen_cb, seen_n, rem, my_live);
+                // A node made by a path that was alone at the parent can be reached by no other path
+                // of this pass, and neither can anything below it: the rest of the path is a chain
+                // of new leaves, written here in one go if the room behind the node holds it.
+                if (own && rem > d && new_room >= rem - d) {
+                    *word(&ent[nxt], 2) = nxt + 1;
+                    *word(&ent[nxt], 3) = 1;
+                    for (int j = d + 1; j <= rem; ++j)
+                        ent[nxt + j - d] = j < rem ? make_int4(d_tokens[k + j - 1], 1, nxt + j - d + 1, 1)
+                                                   : make_int4(d_tokens[k + j - 1], 1, 0, 0);
+                    my_live += rem - d;
+                    rem = 0;
+                }
                 // 3. the other inserts: one path per parent and round
                 bool pending = alive && found < 0 && !alone;
                 for (int round = 0; round <= GI_THREADS; ++round) {

@@ -298,6 +298,51 @@ __global__ void assign_rank_kernel(const u64* keys, const uint32_t* vals, const 
     rank_out[vals[j]] = ex[j] + flag;                 // dense, 1-based
 }
 
+// Suffix order of sequences that are sorted one by one (the trees of different requests share
+// nothing, so no suffix of one request is ever compared with a suffix of another): one block per
+// sequence, tokens and suffix indices in shared memory, bitonic sort with a comparison of at most
+// D tokens.  Order: by the first D tokens, a suffix that ends earlier before its extensions, equal
+// strings by position, which is the order the prefix-doubling rounds produce.  One launch instead of
+// about a hundred, which is what counts when a few prompts are built in the middle of a decode loop.
+constexpr int BS_THREADS = 1024;
+constexpr int BS_MAX_LEN = 16384;              // longest sequence (2 x 64 KB of shared memory)
+
+__global__ void __launch_bounds__(BS_THREADS)
+block_suffix_sort_kernel(const int32_t* tok, const int64_t* seq_off, int D, uint32_t* sa) {
+    extern __shared__ int bs_smem[];
+    const i64 b = seq_off[blockIdx.x], e = seq_off[blockIdx.x + 1];
+    const int n = (int)(e - b), tid = threadIdx.x;
+    if (n <= 0) return;
+    int np = 1;
+    while (np < n) np <<= 1;
+    int* t = bs_smem;                          // [n] tokens
+    int* idx = bs_smem + n;                    // [np] suffixes (>= n: padding, sorts last)
+    for (int i = tid; i < n; i += BS_THREADS) t[i] = tok[b + i];
+    for (int i = tid; i < np; i += BS_THREADS) idx[i] = i;
+    __syncthreads();
+    auto less = [&](int a, int c) -> bool {    // strict total order, a != c
+        if (a >= n || c >= n) return a < c;
+        const int la = min(D, n - a), lc = min(D, n - c), m = min(la, lc);
+        for (int l = 0; l < m; ++l) {
+            const int x = t[a + l], y = t[c + l];
+            if (x != y) return x < y;
+        }
+        if (la != lc) return la < lc;
+        return a < c;
+    };
+    for (int k = 2; k <= np; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int q = tid; q < (np >> 1); q += BS_THREADS) {
+                const int i = ((q & ~(j - 1)) << 1) | (q & (j - 1)), p = i | j;
+                const int a = idx[i], c = idx[p];
+                const bool up = (i & k) == 0;
+                if (less(c, a) == up) { idx[i] = c; idx[p] = a; }
+            }
+            __syncthreads();
+        }
+    for (int i = tid; i < n; i += BS_THREADS) sa[b + i] = (uint32_t)(b + idx[i]);
+}
+
 // lcp[j] = common prefix (capped) of sorted suffixes j-1 and j; len[j] = capped length of suffix j
 __global__ void lcp_kernel(const int32_t* tok, const uint32_t* sa, const int* end_pos, i64 n, int D, uint8_t* lcp,
                            uint8_t* len) {
@@ -685,9 +730,12 @@ struct Pipeline {
 };
 
 // max_token: largest token value + 1 (sets the number of radix passes).  top_blocks: reserve
-// room for top blocks in front of long runs.  Returns SD_OK, SD_ERR_NOMEM or SD_ERR_CUDA.
+// room for top blocks in front of long runs.  per_seq_max_len > 0: the sequences are independent
+// (tokens of different sequences never compare equal, sequence k's tokens below sequence k + 1's)
+// and none is longer than that, so each is sorted by a block of its own.
+// Returns SD_OK, SD_ERR_NOMEM or SD_ERR_CUDA.
 static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_offsets, int n_seqs, i64 N,
-                        i64 max_token, int D, bool top_blocks, cudaStream_t st) {
+                        i64 max_token, int D, bool top_blocks, cudaStream_t st, i64 per_seq_max_len = 0) {
     const int T256 = 256;
     P.N = N;
     DeviceArena& tmp = P.tmp;
@@ -713,7 +761,18 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     uint8_t *lcp = P.lcp, *len = P.len;
 
     seq_end_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_seq_offsets, n_seqs, N, end_pos);
-    rank0_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tok, N, rank[0]);
+    const bool block_sort = per_seq_max_len > 0 && per_seq_max_len <= BS_MAX_LEN;
+    if (block_sort) {
+        i64 np = 1;
+        while (np < per_seq_max_len) np <<= 1;
+        const size_t smem = (size_t)(per_seq_max_len + np) * sizeof(int);
+        if (smem > 48 * 1024 &&
+            cudaFuncSetAttribute(block_suffix_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)((BS_MAX_LEN * 2) * sizeof(int))) != cudaSuccess)
+            return SD_ERR_CUDA;
+        block_suffix_sort_kernel<<<(unsigned)n_seqs, BS_THREADS, smem, st>>>(d_tok, d_seq_offsets, D, sb.vals[0]);
+    } else
+        rank0_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tok, N, rank[0]);
     const int bits_tok = bits_for(max_token + 1), bits_rank = bits_for(N + 1);
     int sorted = 0;
     // rank[k] orders the first 2^k tokens of every suffix
@@ -726,7 +785,9 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
             assign_rank_kernel<<<grid_for(N, T256), T256, 0, st>>>(sb.keys[sorted], sb.vals[sorted], ex, N, rout);
         }
     };
-    if (m == 0) {
+    if (block_sort) {
+        // sb.vals[0] holds the suffix order already
+    } else if (m == 0) {
         round(rank[0], rank[0], 1 << 30, nullptr);        // D == 1: the first token alone
     } else {
         const bool pow2 = D == (1 << m);
@@ -1070,7 +1131,9 @@ extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, 
     }
     requests_prepare_kernel<<<grid_for((i64)n * 32, T256), T256, 0, st>>>(*s, n, d_slot, d_off, d_tokens);
     if (N > 0) {
-        const int rc = pipeline_run(P, mtok, d_off, n, N, (i64)n * s->V, D, false, st);
+        i64 max_len = 0;
+        for (int q = 0; q < n; ++q) max_len = std::max<i64>(max_len, h_offsets[q + 1] - h_offsets[q]);
+        const int rc = pipeline_run(P, mtok, d_off, n, N, (i64)n * s->V, D, false, st, max_len);
         if (rc != SD_OK) return rc;
         requests_layout_kernel<<<grid_for(n, T256), T256, 0, st>>>(*s, n, d_off, P.nbase, P.runstart, P.lv.E, L);
         emit_nodes_slots_kernel<<<grid_for(N, T256), T256, 0, st>>>(*s, n, d_slot, d_off, mtok, P.sa, P.lcp, P.len, N, P.lv,

@@ -108,6 +108,87 @@ def test_global_online_insert(U, vocab):
     pr.close()
 
 
+@pytest.mark.parametrize("vocab,D,zipf", [(2, 32, False), (3, 7, False), (40, 32, True), (5000, 32, True),
+                                          (5000, 16, False)])
+def test_global_insert_many_paths_and_items(U, vocab, D, zipf):
+    """Global inserts larger than one pass of the insert kernel (more than 1,024 start positions, more
+    than 256 items in one call), mixed with request items, on trees where many paths share their
+    parents (tiny vocabularies, periodic text) and on trees with long child runs."""
+    rng = np.random.default_rng(1000 * vocab + D)
+
+    def seqs(n, lo, hi):
+        out = []
+        for _ in range(n):
+            L = int(rng.integers(lo, hi + 1))
+            s = np.minimum(rng.zipf(1.2, size=L) - 1, vocab - 1) if zipf else rng.integers(0, vocab, size=L)
+            if L > 8 and rng.random() < 0.5:                      # a copy of an earlier stretch, and a periodic one
+                a, b = sorted(rng.integers(0, L, size=2).tolist())
+                s[b:] = np.resize(s[a:b + 1], L - b)
+            out.append(s.astype(np.int32))
+        return out
+
+    pr = U.Pair(seqs(20, 50, 600), vocab=vocab, D=D, n_slots=4, max_req_tokens=256)
+    # one long sequence and a few short ones: several passes, paths that end early
+    pr.append([-1, -1, 2, -1], [seqs(1, 2500, 2500)[0], seqs(1, 1, 1)[0], seqs(1, 30, 30)[0], seqs(1, 700, 700)[0]])
+    pr.check_tree(-1)
+    pr.check_tree(2)
+    # more items than one round of the item scan takes, empty sequences among them
+    many = seqs(600, 0, 9)
+    slots = [-1] * len(many)
+    slots[100], slots[400] = 0, 1
+    pr.append(slots, many)
+    pr.check_tree(-1)
+    pr.check_tree(0)
+    # the same text again: every node exists, only counts change
+    pr.append([-1] * 3, [np.concatenate(many[:300]), np.concatenate(many[300:]), many[7]])
+    pr.check_tree(-1)
+    assert pr.g.stats()["global_status"] == 0
+    pr.check_speculate([0, 1, 2], 8, 2.0, 16)
+    pr.close()
+
+
+def test_global_insert_bad_token_and_full_pool(U):
+    rng = np.random.default_rng(77)
+    vocab, D = 50, 8
+    base = [rng.integers(0, vocab, size=80).astype(np.int32) for _ in range(3)]
+    # a token outside the vocabulary ends its sequence there; the other sequences are not affected
+    pr = U.Pair(base, vocab=vocab, D=D, n_slots=1, max_req_tokens=16)
+    good = rng.integers(0, vocab, size=300).astype(np.int32)
+    bad = good.copy()
+    bad[120] = vocab
+    other = rng.integers(0, vocab, size=1500).astype(np.int32)
+    off, flat = U.ragged([bad, other])
+    pr.g.append(U.dev_i32([-1, -1]), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat))
+    pr.o.global_insert(bad[:120]); pr.o.global_insert(other)
+    pr.check_tree(-1)
+    assert pr.g.stats()["global_status"] == 8
+    pr.close()
+    # a pool without room: the status bit is set, the store stays usable and every count that is
+    # there is at most the oracle's
+    pr = U.Pair(base, vocab=vocab, D=D, n_slots=1, max_req_tokens=16, global_extra_nodes=500)
+    off, flat = U.ragged([other])
+    pr.g.append(U.dev_i32([-1]), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat))
+    st = pr.g.stats()
+    assert st["global_status"] & 4 and st["global_pool_used"] <= st["global_pool_cap"]
+    pr.o.global_insert(other)
+    depth, parent, tok, cnt = pr.o.dump(-1)
+    sel = np.nonzero(depth <= 2)[0]
+    paths = [[int(tok[i])] if depth[i] == 1 else [int(tok[parent[i]]), int(tok[i])] for i in sel]
+    qoff, qflat = U.ragged(paths)
+    got = pr.g.query_counts(U.dev_i32(np.full(len(paths), -1)), torch.as_tensor(qoff, device=U.DEV), U.dev_i32(qflat))
+    assert (got.cpu().numpy() <= cnt[sel]).all()
+    # later inserts are refused as a whole, speculation still works
+    before = pr.g.stats()["global_tokens"]
+    pr.g.append(U.dev_i32([-1]), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat))
+    assert pr.g.stats()["global_tokens"] == before
+    pr.g.append(U.dev_i32([0]), torch.as_tensor(np.array([0, 10]), device=U.DEV), U.dev_i32(other[:10]),
+                torch.ones(1, dtype=torch.uint8, device=U.DEV))
+    out = pr.g.speculate(U.dev_i32([0]), 4, 2.0, 8)
+    torch.cuda.synchronize()
+    assert int(out["n_draft"][0]) >= 0
+    pr.close()
+
+
 def test_pool_overflow_is_reported_and_tree_stays_consistent(U):
     rng = np.random.default_rng(3)
     pr = U.Pair([], vocab=1000, D=8, n_slots=2, max_req_tokens=64, slot_pool_nodes=100)
@@ -421,6 +502,33 @@ def test_build_requests_equals_token_by_token_append(U, D, vocab):
         pr.g.build_requests([0], [0, 1], U.dev_i32([vocab]))
     pr.check_tree(0)
     pr.close()
+
+
+def test_build_requests_long_and_short_prompts(U):
+    """Prompts up to 16,384 tokens are sorted by one block each, longer ones by the general
+    pipeline: both must give the tree of the token-by-token append."""
+    rng = np.random.default_rng(5)
+    vocab, D = 300, 12
+
+    def text(L):
+        s = np.minimum(rng.zipf(1.3, size=L) - 1, vocab - 1).astype(np.int32)
+        if L > 64:
+            s[L // 2:L // 2 + L // 8] = s[:L // 8]                # a long copy
+            s[-40:] = 7                                           # a constant tail
+        return s
+
+    for lens in ([16384, 5, 0, 9000], [17000, 3], [1, 2, 4097]):
+        pr = U.Pair([text(50)], vocab=vocab, D=D, n_slots=len(lens), max_req_tokens=max(lens) + 8)
+        prompts = [text(L) for L in lens]
+        off, flat = U.ragged(prompts)
+        pr.g.build_requests(np.arange(len(lens), dtype=np.int32), off, U.dev_i32(flat))
+        for q, p_ in enumerate(prompts):
+            pr.o.slot_reset(q)
+        pr.o.slot_append_batch(list(range(len(lens))), prompts, n_threads=4)
+        for q in range(len(lens)):
+            pr.check_tree(q)
+        pr.check_speculate(list(range(len(lens))), 8, 2.0, 16)
+        pr.close()
 
 
 def test_build_requests_pool_overflow(U):

@@ -376,7 +376,7 @@ struct NewNodes {             // nodes opened by suffix j: one at every depth in
 //   end(j, d)   = min{ i > j : bound_c(i) } (else N)        one past the node's range: count = end - j
 //   before(j)   = max{ i < j : lcp[i] < lcp[j] }            first suffix of the parent's range when
 //                                                           the parent was opened by another suffix
-// One warp scans a tile of MS_TILE suffixes, 32 at a time: a ballot per channel turns the 32
+// One warp scans a tile of 32 x CHUNKS suffixes, 32 at a time: a ballot per channel turns the 32
 // suffixes' flags into one word, lane c keeps the running state of channel c.  Three launches:
 // tile totals, carries across tiles (one small block), then the tile again with its carries.
 // Nodes are numbered in depth-first pre-order: the root is 0 and the node that suffix j opens
@@ -384,7 +384,8 @@ struct NewNodes {             // nodes opened by suffix j: one at every depth in
 // child runs are laid down in node order, so the run of a node's first child directly follows
 // the node's own run, and a chain of only children is one run of consecutive entries.
 constexpr int MS_CHUNKS = 32;                     // chunks of 32 suffixes per tile
-constexpr int MS_TILE = 32 * MS_CHUNKS;
+constexpr int MS_CHUNKS_SMALL = 4;                // ... when there are few suffixes (more, shorter tiles: more warps at work)
+constexpr i64 MS_SMALL_N = 1 << 17;
 constexpr int MS_WARPS = 4;                       // tiles (warps) per block
 
 struct LevelTables {
@@ -396,14 +397,15 @@ struct LevelTables {
     int D, tiles;
 };
 
+template <int CHUNKS>
 __global__ void __launch_bounds__(MS_WARPS * 32)
 ms_tile_kernel(const uint8_t* __restrict__ lcp, const uint8_t* __restrict__ len, LevelTables T) {
     const int lane = threadIdx.x & 31;
     const int tile = blockIdx.x * MS_WARPS + (threadIdx.x >> 5);
     if (tile >= T.tiles) return;
-    const i64 t0 = (i64)tile * MS_TILE;
+    const i64 t0 = (i64)tile * (32 * CHUNKS);
     int cnt = 0, last = -1, first = 0x7fffffff;                 // of channel `lane`
-    for (int ch = 0; ch < MS_CHUNKS; ++ch) {
+    for (int ch = 0; ch < CHUNKS; ++ch) {
         const i64 base = t0 + (i64)ch * 32, i = base + lane;
         const int l = i < T.N ? lcp[i] : 255, n = i < T.N ? len[i] : 0;
 #pragma unroll
@@ -453,20 +455,21 @@ __global__ void __launch_bounds__(MC_THREADS) ms_carry_kernel(LevelTables T) {
     for (int k = k0; k < k1; ++k) { const int v = col[at(k)]; col[at(k)] = run; run = op(run, v); }
 }
 
+template <int CHUNKS>
 __global__ void __launch_bounds__(MS_WARPS * 32)
 ms_apply_kernel(const uint8_t* __restrict__ lcp, const uint8_t* __restrict__ len, const int* __restrict__ nbase,
                 LevelTables T) {
-    __shared__ unsigned bmask[MS_WARPS][MS_CHUNKS][32];         // bound words of the tile, by chunk and channel
+    __shared__ unsigned bmask[MS_WARPS][CHUNKS][32];            // bound words of the tile, by chunk and channel
     __shared__ int sfirst[MS_WARPS][32];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int tile = blockIdx.x * MS_WARPS + wib;
     if (tile >= T.tiles) return;
-    const i64 t0 = (i64)tile * MS_TILE;
+    const i64 t0 = (i64)tile * (32 * CHUNKS);
     const unsigned lt = (1u << lane) - 1u;
     int run_cnt = T.agg[(i64)lane * T.tiles + tile], run_last = T.agg[(i64)(32 + lane) * T.tiles + tile],
         run_first = T.agg[(i64)(64 + lane) * T.tiles + tile];
     // forward: E and `before`
-    for (int ch = 0; ch < MS_CHUNKS; ++ch) {
+    for (int ch = 0; ch < CHUNKS; ++ch) {
         const i64 base = t0 + (i64)ch * 32, i = base + lane;
         const int l = i < T.N ? lcp[i] : 255, n = i < T.N ? len[i] : 0;
         const int prev_last = run_last;
@@ -496,7 +499,7 @@ ms_apply_kernel(const uint8_t* __restrict__ lcp, const uint8_t* __restrict__ len
         }
     }
     // backward: the end of every node's range
-    for (int ch = MS_CHUNKS - 1; ch >= 0; --ch) {
+    for (int ch = CHUNKS - 1; ch >= 0; --ch) {
         const i64 base = t0 + (i64)ch * 32, i = base + lane;
         sfirst[wib][lane] = run_first;
         __syncwarp();
@@ -822,7 +825,9 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
 
     LevelTables& lv = P.lv;
     lv.N = N; lv.D = D;
-    lv.tiles = (int)((N + MS_TILE - 1) / MS_TILE);
+    const bool small_tiles = N <= MS_SMALL_N;
+    const int tile_len = 32 * (small_tiles ? MS_CHUNKS_SMALL : MS_CHUNKS);
+    lv.tiles = (int)((N + tile_len - 1) / tile_len);
     tmp.reserve(4ll * ((i64)D * (N + 1) + 3 * (n_nodes + 2) + N + (i64)lv.tiles * 96 + scan_tmp_ints(n_nodes + 1) +
                        n_nodes / SD_TOP_MIN + 2) + 64 * 256);
     ok = tmp.get(&lv.E, (i64)D * (N + 1)) && tmp.get(&lv.node_end, n_nodes + 1) && tmp.get(&lv.before, N) &&
@@ -831,9 +836,11 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
          tmp.get(&P.wide_list, n_nodes / SD_TOP_MIN + 2);
     if (!ok) return SD_ERR_NOMEM;
     const unsigned ms_grid = (unsigned)((lv.tiles + MS_WARPS - 1) / MS_WARPS);
-    ms_tile_kernel<<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, lv);
+    if (small_tiles) ms_tile_kernel<MS_CHUNKS_SMALL><<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, lv);
+    else ms_tile_kernel<MS_CHUNKS><<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, lv);
     ms_carry_kernel<<<96, MC_THREADS, 0, st>>>(lv);
-    ms_apply_kernel<<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, P.nbase, lv);
+    if (small_tiles) ms_apply_kernel<MS_CHUNKS_SMALL><<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, P.nbase, lv);
+    else ms_apply_kernel<MS_CHUNKS><<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, P.nbase, lv);
     count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, P.nbase, lv, P.nchild);
     // child runs (with their top blocks) in node (pre-)order
     exclusive_scan(RunAlloc{P.nchild, top_blocks ? 1 : 0}, n_nodes + 1, P.runstart, P.big_tmp, st);
@@ -970,10 +977,10 @@ __global__ void map_tokens_kernel(const int32_t* tok, const int64_t* off, int n,
     out[i] = seq_rank_of(off, n, i) * V + t;
 }
 
-// one warp per request: forget the slot's old tree and store the new text
+// one block per request: forget the slot's old tree and store the new text
 __global__ void requests_prepare_kernel(sd_store sv, int n, const int32_t* slot_ids, const int64_t* off,
                                         const int32_t* tok) {
-    const int q = (int)((blockIdx.x * (i64)blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    const int q = blockIdx.x;
     if (q >= n) return;
     const int slot = slot_ids[q];
     if (slot < 0 || slot >= sv.R) return;
@@ -981,11 +988,11 @@ __global__ void requests_prepare_kernel(sd_store sv, int n, const int32_t* slot_
     int32_t* text = sv.s_text + (i64)slot * sv.T;
     int32_t* root = sv.s_root + (i64)slot * sv.V;
     const int old_len = ss->len;
-    for (int k = lane; k < old_len; k += 32) root[text[k]] = -1;
-    __syncwarp();
+    for (int k = threadIdx.x; k < old_len; k += blockDim.x) root[text[k]] = -1;
+    __syncthreads();
     const i64 lo = off[q], hi = off[q + 1];
     if (hi - lo <= sv.T)
-        for (i64 k = lane; k < hi - lo; k += 32) text[k] = tok[lo + k];
+        for (i64 k = threadIdx.x; k < hi - lo; k += blockDim.x) text[k] = tok[lo + k];
 }
 
 struct RequestLayout {       // where request q's nodes go (device arrays of n entries)
@@ -1129,7 +1136,7 @@ extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, 
         SD_CUDA_OK(cudaStreamSynchronize(st));
         if (h_bad) return SD_ERR_INVALID_ARG;                    // nothing was changed yet
     }
-    requests_prepare_kernel<<<grid_for((i64)n * 32, T256), T256, 0, st>>>(*s, n, d_slot, d_off, d_tokens);
+    requests_prepare_kernel<<<(unsigned)n, T256, 0, st>>>(*s, n, d_slot, d_off, d_tokens);
     if (N > 0) {
         i64 max_len = 0;
         for (int q = 0; q < n; ++q) max_len = std::max<i64>(max_len, h_offsets[q + 1] - h_offsets[q]);

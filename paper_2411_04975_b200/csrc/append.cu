@@ -1,5 +1,9 @@
 // Batched append kernel (sd_append): see append_core.cuh for how one token is appended.
+#include <cooperative_groups.h>
+
 #include "append_core.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -8,7 +12,7 @@ namespace {
 //
 // Inserting a sequence adds one occurrence to every string of at most D tokens that starts at one
 // of its positions: one root-to-depth-D PATH per start position.  Taking the tokens one after the
-// other makes a chain as long as the sequence.  Here one block takes up to 1,024 paths at once, a
+// other makes a chain as long as the sequence.  Here up to 2,048 paths are taken at once, a
 // thread per path, and all of them go down one level per round:
 //   1. every path enters its current node (the parent of the node it is about to reach) into a
 //      hash set in shared memory, which counts the paths per parent;
@@ -28,25 +32,63 @@ namespace {
 // no waiting on another thread anywhere, only block-wide barriers.  Placement follows the
 // token-by-token append: the first leaf of a path that leaves the known text reserves room down
 // to depth D and the later leaves go directly behind their parents.
-constexpr int GI_THREADS = 1024;
-constexpr int GI_SLOTS = 2048;                // cells of the parent set: at most half full
+//
+// The block is a CLUSTER of GI_CTAS thread blocks on as many SMs (the work of a level is mostly
+// instruction issue, which one SM's schedulers limit): the barriers are cluster barriers, the
+// parent set is spread over the blocks' shared memories and the pool counters live in block 0's,
+// all reached through distributed shared memory.  Tree entries are read through L2 (an SM's L1
+// does not see what the other SMs store), and every block derives the list of sequences from
+// the call's arguments for itself, so all blocks take the same branches and meet at every barrier.
+constexpr int GI_CTAS = 8;
+constexpr int GI_THREADS = 256;               // per block
+constexpr int GI_PASS = GI_CTAS * GI_THREADS; // paths per pass
+constexpr int GI_CELLS = 512;                 // cells of the parent set per block: the set is at most half full
+constexpr int GI_SLOTS = GI_CTAS * GI_CELLS;
 constexpr int GI_ITEMS = 256;
 constexpr int GI_BIG = 48;                    // inserts that move more entries are done by a whole warp
 
 struct GiShared {
-    int key[GI_SLOTS];                        // parent + 1 (level 1: token + 1), 0 = free
-    int cnt[GI_SLOTS];                        // paths at that parent
-    int turn[GI_SLOTS];                       // rounds in which a path of that parent was elected
+    // the parent set, one for the odd and one for the even levels (a level clears the other one's)
+    int key[2][GI_CELLS];                     // parent + 1 (level 1: token + 1), 0 = free
+    int cnt[2][GI_CELLS];                     // paths at that parent
+    int turn[2][GI_CELLS];                    // rounds in which a path of that parent was elected
     int item[GI_ITEMS];
     long long begin[GI_ITEMS], end[GI_ITEMS], pref[GI_ITEMS + 1];
+    int n_items;
+    int any[3];                               // flags of the cluster-wide "or", used in turn
+    // block 0's copy only:
     unsigned long long used;
-    int n_items, live, status;
+    int live, status;
+};
+
+struct GiCluster {
+    cg::cluster_group cl;
+    GiShared* sh;                             // this block's
+    GiShared* sh0;                            // block 0's
+    int phase;
+    __device__ int* cell_ptr(int* base, int cell) const {       // base: a table of this block's GiShared
+        return cl.map_shared_rank(base, (unsigned)cell / GI_CELLS) + (cell & (GI_CELLS - 1));
+    }
+    // Bit 0: a holds for any thread of the cluster, bit 1: b does.  A barrier for the whole
+    // cluster.  Every block tells every block (thread r writes to block r), so the answer is read
+    // from the block's own shared memory.
+    __device__ int any(bool a, bool b = false) {
+        const int mine = (__syncthreads_or(a) ? 1 : 0) | (__syncthreads_or(b) ? 2 : 0);
+        if (threadIdx.x < GI_CTAS && mine) atomicOr(cl.map_shared_rank(&sh->any[phase], threadIdx.x), mine);
+        cl.sync();
+        const int r = *(volatile int*)&sh->any[phase];
+        // the flag of the round before: everybody read it before arriving at the barrier above,
+        // and it is written again only after the next barrier
+        if (threadIdx.x == 0) sh->any[(phase + 2) % 3] = 0;
+        phase = (phase + 1) % 3;
+        return r;
+    }
 };
 
 // Entries for new runs and chain blocks of a warp's lanes (`size` may be 0): one atomic per warp.
 // Returns the lane's first entry, -1 if it asked for none or the pool cannot hold the warp's
 // request (then the status bit is set as well).  All 32 lanes call.
-__device__ __forceinline__ int gi_alloc_warp(GiShared& sh, long long cap, int size, int lane) {
+__device__ __forceinline__ int gi_alloc_warp(GiShared* sh0, long long cap, int size, int lane) {
     const unsigned FULL = 0xffffffffu;
     int inc = size;
 #pragma unroll
@@ -57,10 +99,10 @@ __device__ __forceinline__ int gi_alloc_warp(GiShared& sh, long long cap, int si
     const int total = __shfl_sync(FULL, inc, 31);
     if (total == 0) return -1;
     unsigned long long at = 0;
-    if (lane == 31) at = atomicAdd(&sh.used, (unsigned long long)total);
+    if (lane == 31) at = atomicAdd(&sh0->used, (unsigned long long)total);
     at = __shfl_sync(FULL, at, 31);
     if (at + (unsigned long long)total > (unsigned long long)cap) {
-        if (lane == 31) atomicOr(&sh.status, SD_STATUS_GLOBAL_FULL);
+        if (lane == 31) atomicOr(&sh0->status, SD_STATUS_GLOBAL_FULL);
         return -1;
     }
     return size > 0 ? (int)at + inc - size : -1;
@@ -70,7 +112,7 @@ __device__ __forceinline__ int gi_alloc_warp(GiShared& sh, long long cap, int si
 // false).  All 32 lanes call.  On return nxt is the new node and new_room the room reserved
 // behind it; (seen_cb, seen_n) describe the parent's run right after the insert.  A path whose
 // entries the pool cannot hold stops (rem = 0).
-__device__ __forceinline__ void gi_insert(GiShared& sh, const sd_store& sv, int d, int lane, bool ins, int x, int cur,
+__device__ __forceinline__ void gi_insert(GiShared* sh0, const sd_store& sv, int d, int lane, bool ins, int x, int cur,
                                           int room, int cb, int nc, unsigned w, int pos, int& nxt, int& new_room,
                                           int& seen_cb, int& seen_n, int& rem, int& my_live) {
     const unsigned FULL = 0xffffffffu;
@@ -88,7 +130,7 @@ __device__ __forceinline__ void gi_insert(GiShared& sh, const sd_store& sv, int 
             asz = (int)sd_pow2ceil((uint32_t)nc + 1u);
         }
     }
-    int fresh = gi_alloc_warp(sh, sv.g_cap, asz, lane);
+    int fresh = gi_alloc_warp(sh0, sv.g_cap, asz, lane);
     bool big = false;
     if (ins) {
         if (asz > 0 && fresh < 0) rem = 0;
@@ -105,7 +147,7 @@ __device__ __forceinline__ void gi_insert(GiShared& sh, const sd_store& sv, int 
                 seen_cb = moves ? fresh : cb;
                 seen_n = nc + 1;
                 big = (moves ? nc : nc - pos) > GI_BIG;
-                if (!big) nxt = insert_child<8>(ent, cur, cb, nc, pos, x, fresh, moves);
+                if (!big) nxt = insert_child<8, true>(ent, cur, cb, nc, pos, x, fresh, moves);
             }
         }
     }
@@ -114,15 +156,15 @@ __device__ __forceinline__ void gi_insert(GiShared& sh, const sd_store& sv, int 
     while (bm) {
         const int src = __ffs(bm) - 1;
         bm &= bm - 1;
-        const int idx = insert_child_warp(ent, __shfl_sync(FULL, cur, src), __shfl_sync(FULL, cb, src),
-                                          __shfl_sync(FULL, nc, src), __shfl_sync(FULL, pos, src),
-                                          __shfl_sync(FULL, x, src), __shfl_sync(FULL, fresh, src),
-                                          __shfl_sync(FULL, moves ? 1 : 0, src) != 0, lane);
+        const int idx = insert_child_warp<true>(ent, __shfl_sync(FULL, cur, src), __shfl_sync(FULL, cb, src),
+                                                __shfl_sync(FULL, nc, src), __shfl_sync(FULL, pos, src),
+                                                __shfl_sync(FULL, x, src), __shfl_sync(FULL, fresh, src),
+                                                __shfl_sync(FULL, moves ? 1 : 0, src) != 0, lane);
         if (lane == src) nxt = idx;
     }
 }
 
-__global__ void __launch_bounds__(GI_THREADS, 1)
+__global__ void __cluster_dims__(GI_CTAS, 1, 1) __launch_bounds__(GI_THREADS, 1)
 global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_tokens) {
     __shared__ GiShared sh;
     const unsigned FULL = 0xffffffffu;
@@ -130,17 +172,25 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
     int4* const ent = sv.g_ent;
     const int D = sv.D;
 
+    // (every block looks at all items: all blocks of the cluster take the same way)
     bool mine = false;
     for (int i = tid; i < n; i += GI_THREADS) mine |= d_slot[i] == -1;
     if (!__syncthreads_or(mine)) return;                         // the usual decode step: nothing for the global tree
-    if (tid == 0) { sh.used = (unsigned long long)sv.g_state->used; sh.live = 0; sh.status = sv.g_state->status; }
-    for (int i = tid; i < GI_SLOTS; i += GI_THREADS) { sh.key[i] = 0; sh.cnt[i] = 0; sh.turn[i] = 0; }
-    __syncthreads();
+    GiCluster G{cg::this_cluster(), &sh, nullptr, 0};
+    G.sh0 = G.cl.map_shared_rank(&sh, 0);
+    GiShared* const sh0 = G.sh0;
+    const int path0 = (int)G.cl.block_rank() * GI_THREADS + tid; // this thread's path within a pass
+    if (tid == 0) {
+        sh.used = (unsigned long long)sv.g_state->used; sh.live = 0; sh.status = sv.g_state->status;
+        sh.any[0] = sh.any[1] = sh.any[2] = 0;
+    }
+    for (int i = tid; i < 2 * GI_CELLS; i += GI_THREADS) { sh.key[0][i] = 0; sh.cnt[0][i] = 0; sh.turn[0][i] = 0; }
+    G.cl.sync();
     long long tokens_done = 0;
     int my_live = 0;
 
     for (int base = 0; base < n; base += GI_ITEMS) {
-        if (__syncthreads_or(sh.status & SD_STATUS_GLOBAL_FULL)) break;
+        if (G.any((*(volatile int*)&sh0->status & SD_STATUS_GLOBAL_FULL) != 0)) break;
         // the sequences among items [base, base + GI_ITEMS), in item order
         if (tid == 0) sh.n_items = 0;
         __syncthreads();
@@ -165,7 +215,7 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
             const long long b = sh.begin[j], e = d_offsets[sh.item[j] + 1];
             for (long long k = b + tid; k < e; k += GI_THREADS) {
                 const int x = d_tokens[k];
-                if (x < 0 || x >= sv.V) { atomicMin(&sh.end[j], k); atomicOr(&sh.status, SD_STATUS_BAD_TOKEN); }
+                if (x < 0 || x >= sv.V) { atomicMin(&sh.end[j], k); atomicOr(&sh0->status, SD_STATUS_BAD_TOKEN); }
             }
         }
         __syncthreads();
@@ -177,10 +227,12 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
         __syncthreads();
         const long long total = sh.pref[n_items];
 
-        for (long long c0 = 0; c0 < total; c0 += GI_THREADS) {
-            if (__syncthreads_or(sh.status & SD_STATUS_GLOBAL_FULL)) break;
+        for (long long c0 = 0; c0 < total; c0 += GI_PASS) {
+            // both parent sets are empty behind this barrier (the last level of a pass leaves its own behind)
+            for (int i = tid; i < 2 * GI_CELLS; i += GI_THREADS) { sh.key[0][i] = 0; sh.cnt[0][i] = 0; sh.turn[0][i] = 0; }
+            if (G.any((*(volatile int*)&sh0->status & SD_STATUS_GLOBAL_FULL) != 0)) break;
             // this thread's path: start position k, `rem` tokens to take (at most D)
-            const long long p = c0 + tid;
+            const long long p = c0 + path0;
             long long k = 0;
             int rem = 0;
             if (p < total) {
@@ -195,32 +247,40 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
             // the node of the tokens taken so far, the room reserved behind it, its child run
             int cur = -1, room = 0, run_cb = 0;
             unsigned run_w = 0;
-            for (int d = 1; d <= D; ++d) {
-                if (!__syncthreads_or(rem >= d)) break;          // (the parent set is empty here)
+            bool more = true;                                    // a path of the cluster has a token for this level
+            for (int d = 1; d <= D && more; ++d) {
+                int* const t_key = sh.key[d & 1];
+                int* const t_cnt = sh.cnt[d & 1];
+                int* const t_turn = sh.turn[d & 1];
                 const bool alive = rem >= d;
                 const int x = alive ? d_tokens[k + d - 1] : 0;
                 // 1. the parent set
                 int cell = 0;
                 if (alive) {
                     const int key = (d == 1 ? x : cur) + 1;
-                    cell = (int)(((unsigned)key * 2654435761u) >> 21);          // 11 bits
+                    cell = (int)(((unsigned)key * 2654435761u) >> 20);          // 12 bits
                     for (int probe = 0; probe < GI_SLOTS; ++probe) {
-                        const int old = atomicCAS(&sh.key[cell], 0, key);
+                        const int old = atomicCAS(G.cell_ptr(t_key, cell), 0, key);
                         if (old == 0 || old == key) break;
                         cell = (cell + 1) & (GI_SLOTS - 1);
                     }
-                    atomicAdd(&sh.cnt[cell], 1);
+                    atomicAdd(G.cell_ptr(t_cnt, cell), 1);
                 }
-                __syncthreads();
-                const bool alone = alive && sh.cnt[cell] == 1;
+                G.cl.sync();
+                // the other level's set: last used before the barrier that ended that level, used
+                // again after the one that ends this level
+                for (int i = tid; i < GI_CELLS; i += GI_THREADS) {
+                    sh.key[(d & 1) ^ 1][i] = 0; sh.cnt[(d & 1) ^ 1][i] = 0; sh.turn[(d & 1) ^ 1][i] = 0;
+                }
+                const bool alone = alive && *(volatile int*)G.cell_ptr(t_cnt, cell) == 1;
                 // 2. look the token up
                 int found = -1, pos = 0;
                 int cb = run_cb, nc = (int)(run_w & RUN_COUNT_MASK);
                 unsigned w = run_w;
                 int4 fe = make_int4(0, 0, 0, 0);
                 if (alive) {
-                    if (d == 1) { found = sv.g_root[x]; if (found >= 0) fe = ent[found]; }
-                    else if (nc > 0) found = lookup_child<8>(ent, cb, nc, x, pos, fe);
+                    if (d == 1) { found = __ldcg(sv.g_root + x); if (found >= 0) fe = __ldcg(ent + found); }
+                    else if (nc > 0) found = lookup_child<8, true>(ent, cb, nc, x, pos, fe);
                     if (found >= 0) {
                         atomicAdd(word(&ent[found], 1), 1);
                         // a count changes: the copies in the run's top block (if any) are stale from now on
@@ -230,7 +290,7 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                 int nxt = found, new_room = 0;
                 int seen_cb = cb, seen_n = nc;                    // the parent's run as it was when nxt was taken
                 const bool own = alive && found < 0 && alone;
-                gi_insert(sh, sv, d, lane, own, x, cur, room, cb, nc, w, pos, nxt, new_room, seen_cb, seen_n, rem, my_live);
+                gi_insert(sh0, sv, d, lane, own, x, cur, room, cb, nc, w, pos, nxt, new_room, seen_cb, seen_n, rem, my_live);
                 // A node made by a path that was alone at the parent can be reached by no other path
                 // of this pass, and neither can anything below it: the rest of the path is a chain
                 // of new leaves, written here in one go if the room behind the node holds it.
@@ -245,18 +305,20 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                 }
                 // 3. the other inserts: one path per parent and round
                 bool pending = alive && found < 0 && !alone;
-                for (int round = 0; round <= GI_THREADS; ++round) {
-                    if (!__syncthreads_or(pending)) break;
-                    const bool win = pending && atomicCAS(&sh.turn[cell], round, round + 1) == round;
+                for (int round = 0; round <= GI_PASS; ++round) {
+                    const int r = G.any(pending, rem > d);
+                    more = (r & 2) != 0;
+                    if (!(r & 1)) break;
+                    const bool win = pending && atomicCAS(G.cell_ptr(t_turn, cell), round, round + 1) == round;
                     if (win) {
                         pending = false;
                         if (round > 0) {                         // an earlier round may have changed the run
                             found = -1; pos = 0;
-                            if (d == 1) { found = sv.g_root[x]; if (found >= 0) fe = ent[found]; }
+                            if (d == 1) { found = __ldcg(sv.g_root + x); if (found >= 0) fe = __ldcg(ent + found); }
                             else {
-                                const int4 pe = ent[cur];
+                                const int4 pe = __ldcg(ent + cur);
                                 cb = pe.z; w = (unsigned)pe.w; nc = (int)(w & RUN_COUNT_MASK);
-                                if (nc > 0) found = lookup_child<8>(ent, cb, nc, x, pos, fe);
+                                if (nc > 0) found = lookup_child<8, true>(ent, cb, nc, x, pos, fe);
                             }
                             if (found >= 0) {                    // added meanwhile by a path with the same string
                                 atomicAdd(word(&ent[found], 1), 1);
@@ -264,15 +326,15 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                             }
                         }
                     }
-                    gi_insert(sh, sv, d, lane, win && found < 0, x, cur, room, cb, nc, w, pos, nxt, new_room, seen_cb,
+                    gi_insert(sh0, sv, d, lane, win && found < 0, x, cur, room, cb, nc, w, pos, nxt, new_room, seen_cb,
                               seen_n, rem, my_live);
                 }
                 // 4. the child's place after all inserts of this level
                 if (rem >= d && d > 1 && !alone) {
-                    const int4 pe = ent[cur];
+                    const int4 pe = __ldcg(ent + cur);
                     const int n2 = (int)((unsigned)pe.w & RUN_COUNT_MASK);
                     if (pe.z != seen_cb || n2 != seen_n) {
-                        found = n2 > 0 ? lookup_child<8>(ent, pe.z, n2, x, pos, fe) : -1;
+                        found = n2 > 0 ? lookup_child<8, true>(ent, pe.z, n2, x, pos, fe) : -1;
                         nxt = found;
                         new_room = 0;                            // the node left its chain block
                     }
@@ -282,15 +344,14 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                 room = new_room;
                 run_cb = found >= 0 ? fe.z : 0;                  // a node made just now has no children
                 run_w = found >= 0 ? (unsigned)fe.w : 0u;
-                for (int i = tid; i < GI_SLOTS; i += GI_THREADS) { sh.key[i] = 0; sh.cnt[i] = 0; sh.turn[i] = 0; }
             }
-            tokens_done += min((long long)GI_THREADS, total - c0);
+            tokens_done += min((long long)GI_PASS, total - c0);
         }
     }
-    __syncthreads();
-    if (my_live) atomicAdd(&sh.live, my_live);
-    __syncthreads();
-    if (tid == 0) {
+    G.cl.sync();
+    if (my_live) atomicAdd(&sh0->live, my_live);
+    G.cl.sync();                                                 // (no block leaves while its shared memory may be in use)
+    if (tid == 0 && G.cl.block_rank() == 0) {
         GlobalState* gs = sv.g_state;
         gs->epoch += 1;                              // cached match nodes of every slot are stale now
         gs->used = (int)min(sh.used, (unsigned long long)sv.g_cap);
@@ -350,7 +411,7 @@ extern "C" int sd_append(sd_store* s, int32_t n, const int32_t* d_slot, const in
     if (!d_slot || !d_offsets) return SD_ERR_INVALID_ARG;
     const int warps_per_block = 4;
     const unsigned blocks = (unsigned)((n + 1 + warps_per_block - 1) / warps_per_block);
-    global_insert_kernel<<<1, GI_THREADS, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_offsets, d_tokens);
+    global_insert_kernel<<<GI_CTAS, GI_THREADS, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_offsets, d_tokens);
     SD_CUDA_OK(cudaGetLastError());
     append_kernel<<<blocks, warps_per_block * 32, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset);
     SD_CUDA_OK(cudaGetLastError());

@@ -501,53 +501,68 @@ def run_closed_loop(args):
 
     side = torch.cuda.Stream(device=dev)
 
-    def append(items):
+    def prepare(items):
+        """Host side of an append: device tensors of the items, split into new requests (batched
+        sort-based build) and everything else (sd_append).  Done before the timed events: the
+        device-timed figures start with the inputs resident in HBM."""
         sl, lists, reset = items
-        # new requests go through the batched sort-based build, everything else through sd_append
         new = [i for i in range(len(sl)) if sl[i] >= 0 and reset[i]]
+        skip = set(new)
+        keep = [i for i in range(len(sl)) if i not in skip]
+        prep = {"keep": None, "new": None, "items": items, "new_idx": new, "keep_idx": keep}
+        if keep:
+            ksl, klists, kreset = [sl[i] for i in keep], [lists[i] for i in keep], [reset[i] for i in keep]
+            off = np.zeros(len(ksl) + 1, dtype=np.int64)
+            off[1:] = np.cumsum([len(x) for x in klists])
+            flat = np.concatenate(klists).astype(np.int32) if off[-1] else np.zeros(0, dtype=np.int32)
+            prep["keep"] = (torch.as_tensor(np.asarray(ksl, dtype=np.int32), device=dev), torch.as_tensor(off, device=dev),
+                            torch.as_tensor(flat, device=dev) if flat.size else torch.zeros(0, dtype=torch.int32, device=dev),
+                            torch.as_tensor(np.asarray(kreset, dtype=np.uint8), device=dev))
+            prep["global_tokens"] = sum(len(klists[i]) for i in range(len(ksl)) if ksl[i] < 0)
         if new:
-            # the other items (accepted tokens, finished outputs for the global tree) touch other
-            # slots: they are enqueued first and run while the new requests are built on a side stream
-            keep = [i for i in range(len(sl)) if i not in set(new)]
-            ev_pre = torch.cuda.Event()
-            ev_pre.record()
-            if keep:
-                append(([sl[i] for i in keep], [lists[i] for i in keep], [reset[i] for i in keep]))
-            ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            refill_ev.append((ev_a, ev_b, sum(len(lists[i]) for i in new)))
             noff = np.zeros(len(new) + 1, dtype=np.int64)
             noff[1:] = np.cumsum([len(lists[i]) for i in new])
+            toks_new = torch.as_tensor(np.concatenate([lists[i] for i in new]).astype(np.int32), device=dev)
+            prep["new"] = ([sl[i] for i in new], noff, toks_new)
+        return prep
+
+    def enqueue(prep):
+        """sd_append for the accepted tokens and the finished outputs; new requests are built
+        meanwhile on a side stream (they touch other slots)."""
+        sl, lists, reset = prep["items"]
+        ev_pre = torch.cuda.Event()
+        ev_pre.record()
+        if prep["keep"] is not None:
+            ka, kb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ka.record()
+            store.append(*prep["keep"])
+            kb.record()
+            kernel_ev.append((ka, kb, prep["global_tokens"]))
+        if prep["new"] is not None:
+            nsl, noff, toks_new = prep["new"]
+            ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            refill_ev.append((ev_a, ev_b, int(noff[-1])))
             with torch.cuda.stream(side):
                 side.wait_event(ev_pre)                          # not for the append enqueued just now
                 ev_a.record()
-                toks_new = torch.as_tensor(np.concatenate([lists[i] for i in new]).astype(np.int32), device=dev)
-                store.build_requests([sl[i] for i in new], noff, toks_new)
+                store.build_requests(nsl, noff, toks_new)
                 ev_b.record()
             torch.cuda.current_stream().wait_stream(side)
-            if ref is not None:
-                for i in new:
-                    ref.slot_reset(sl[i])
-                ref.slot_append_batch([sl[i] for i in new], [lists[i] for i in new], n_threads=oracle_threads(B))
-            return
-        off = np.zeros(len(sl) + 1, dtype=np.int64)
-        off[1:] = np.cumsum([len(x) for x in lists])
-        flat = np.concatenate(lists).astype(np.int32) if off[-1] else np.zeros(0, dtype=np.int32)
-        args_ = (torch.as_tensor(np.asarray(sl, dtype=np.int32), device=dev), torch.as_tensor(off, device=dev),
-                 torch.as_tensor(flat, device=dev) if flat.size else torch.zeros(0, dtype=torch.int32, device=dev),
-                 torch.as_tensor(np.asarray(reset, dtype=np.uint8), device=dev))
-        ka, kb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ka.record()
-        store.append(*args_)
-        kb.record()
-        kernel_ev.append((ka, kb, sum(len(lists[i]) for i in range(len(sl)) if sl[i] < 0)))
         if ref is not None:
-            for s_, l_, r_ in zip(sl, lists, reset):
-                if s_ < 0:
-                    ref.global_insert(l_)
-                elif r_:
-                    ref.slot_reset(s_)
-            idx = [i for i, s_ in enumerate(sl) if s_ >= 0]
+            for i in prep["keep_idx"]:
+                if sl[i] < 0:
+                    ref.global_insert(lists[i])
+                elif reset[i]:
+                    ref.slot_reset(sl[i])
+            idx = [i for i in prep["keep_idx"] if sl[i] >= 0]
             ref.slot_append_batch([sl[i] for i in idx], [lists[i] for i in idx], n_threads=oracle_threads(B))
+            for i in prep["new_idx"]:
+                ref.slot_reset(sl[i])
+            ref.slot_append_batch([sl[i] for i in prep["new_idx"]], [lists[i] for i in prep["new_idx"]],
+                                  n_threads=oracle_threads(B))
+
+    def append(items):
+        enqueue(prepare(items))
 
     refill_ev, kernel_ev = [], []
     append(loop.start())
@@ -568,10 +583,10 @@ def run_closed_loop(args):
             for n in ("n_draft", "tokens", "parents", "positions", "chosen_tree", "chosen_p"):
                 ok = ok and np.array_equal(g[n], r[n])
             ok = ok and np.array_equal(g["score"].view(np.int64), r["score"].view(np.int64))
-        items = loop.advance(host)
+        prep = prepare(loop.advance(host))
         e1b = torch.cuda.Event(enable_timing=True)
         e1b.record()
-        append(items)
+        enqueue(prep)
         e2.record()
         torch.cuda.synchronize()
         spec_ms.append(e0.elapsed_time(e1))

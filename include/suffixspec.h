@@ -118,8 +118,13 @@ int sd_build(const sd_build_params* params, const int32_t* d_corpus, const int64
  *   d_slot int32[n], d_offsets int64[n+1], d_tokens int32[d_offsets[n]],
  *   d_reset uint8[n] or NULL (no resets).
  * A slot whose pool or text buffer would overflow keeps its state from before
- * the offending token and gets SD_STATUS_POOL_FULL (see sd_slot_info); a full
- * global pool sets SD_STATUS_GLOBAL_FULL in sd_stats.  n == 0 is a no-op.
+ * the offending token and gets SD_STATUS_POOL_FULL (see sd_slot_info).
+ * Global tree: a sequence is inserted up to its first token outside [0, V)
+ * (SD_STATUS_BAD_TOKEN in sd_stats' global_status, the other sequences of the
+ * call are not affected).  When the global pool cannot hold the new nodes
+ * SD_STATUS_GLOBAL_FULL is set: strings whose nodes found no room are missing
+ * or counted short, the tree stays consistent and usable, and later calls
+ * insert nothing more into it.  n == 0 is a no-op.
  * Errors: INVALID_ARG, CUDA (launch failure).
  */
 int sd_append(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* d_offsets,

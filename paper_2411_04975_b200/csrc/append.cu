@@ -1,4 +1,5 @@
-// Batched append kernel (sd_append): see append_core.cuh for how one token is appended.
+// sd_append: the batched append kernel for the per-request trees (see append_core.cuh for how one
+// token is appended) and the level-by-level insert of whole sequences into the global tree.
 #include <cooperative_groups.h>
 
 #include "append_core.cuh"
@@ -19,10 +20,10 @@ namespace {
 //   2. every path looks its next token up in the parent's child run.  A child that exists gets its
 //      count raised by an atomic add.  A missing child is inserted at once if the path is the
 //      only one at that parent: nobody else reads or writes that run during this level;
-//   3. the other missing children are PENDING and are served in rounds: per parent one path is
-//      elected per round (a turn counter in the parent's hash-set cell), looks again (an earlier
-//      round may have added the very child) and inserts.  Runs of different parents are
-//      disjoint, so the elected paths do not disturb one another;
+//   3. the other missing children are PENDING and are served in rounds: the waiting paths look
+//      again (an earlier round may have added the very child), then per parent one path is
+//      elected (a turn counter in the parent's hash-set cell) and inserts.  Runs of different
+//      parents are disjoint, so the elected paths do not disturb one another;
 //   4. an insert shifts or moves its run, so every path that shares its parent and whose parent's
 //      run changed after it took its child looks the child's new place up.
 // Only runs of ONE depth change during a level, and the entries of their parents (one level up)
@@ -303,16 +304,17 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                     my_live += rem - d;
                     rem = 0;
                 }
-                // 3. the other inserts: one path per parent and round
+                // 3. the other inserts: one path per parent and round.  From the second round on every
+                // waiting path first looks again: the children added in the round before are found by
+                // all the paths that want them at once (text that repeats itself sends many paths
+                // down the same strings), and only the children still missing are competed for.
                 bool pending = alive && found < 0 && !alone;
                 for (int round = 0; round <= GI_PASS; ++round) {
                     const int r = G.any(pending, rem > d);
                     more = (r & 2) != 0;
                     if (!(r & 1)) break;
-                    const bool win = pending && atomicCAS(G.cell_ptr(t_turn, cell), round, round + 1) == round;
-                    if (win) {
-                        pending = false;
-                        if (round > 0) {                         // an earlier round may have changed the run
+                    if (round > 0) {
+                        if (pending) {
                             found = -1; pos = 0;
                             if (d == 1) { found = __ldcg(sv.g_root + x); if (found >= 0) fe = __ldcg(ent + found); }
                             else {
@@ -320,14 +322,18 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                                 cb = pe.z; w = (unsigned)pe.w; nc = (int)(w & RUN_COUNT_MASK);
                                 if (nc > 0) found = lookup_child<8, true>(ent, cb, nc, x, pos, fe);
                             }
-                            if (found >= 0) {                    // added meanwhile by a path with the same string
+                            if (found >= 0) {
                                 atomicAdd(word(&ent[found], 1), 1);
                                 nxt = found; seen_cb = cb; seen_n = nc;
+                                pending = false;
                             }
                         }
+                        G.cl.sync();                             // the look-ups are over before a run moves again
                     }
-                    gi_insert(sh0, sv, d, lane, win && found < 0, x, cur, room, cb, nc, w, pos, nxt, new_room, seen_cb,
-                              seen_n, rem, my_live);
+                    const bool win = pending && atomicCAS(G.cell_ptr(t_turn, cell), round, round + 1) == round;
+                    if (win) pending = false;
+                    gi_insert(sh0, sv, d, lane, win, x, cur, room, cb, nc, w, pos, nxt, new_room, seen_cb, seen_n, rem,
+                              my_live);
                 }
                 // 4. the child's place after all inserts of this level
                 if (rem >= d && d > 1 && !alone) {

@@ -1,11 +1,12 @@
 // Online update of the suffix trees: device functions shared by the kernels that append tokens
-// (the batched append kernel and the fused decode-step kernel).
+// (the batched append kernel, the fused decode-step kernel and the global insert kernel, which
+// uses the look-up and insert primitives).
 //
 // Online update of the suffix trees (Section 3, "Suffix Tree Construction": the
 // tokens of the ongoing request are added as they are generated, a finished
 // request's output is added to the global tree).
 //
-// One warp owns one tree for the duration of the kernel.  Appending token x at
+// Per-request trees: one warp owns one tree for the duration of the kernel.  Appending token x at
 // context length t adds one occurrence to every string that ends at x and is at
 // most D tokens long: lane L extends the ACTIVE node of depth L (the node of
 // the last L tokens; lane 0 extends the root) by child x, creating it or
@@ -99,41 +100,6 @@ __device__ int insert_child_warp(int4* ent, int parent, int cb, int n, int pos, 
     return idx;
 }
 
-// lower_bound of token x in the sorted run ent[cb .. cb+n): 32-way, then eight-way, so that the
-// probes of a round are in flight together (a long run costs a few dependent rounds).
-__device__ int lower_bound_run(const int4* ent, int cb, int n, int x) {
-    int lo = 0, hi = n;
-    while (hi - lo > 256) {                                      // very long runs: 32-way, 31 probes in flight
-        const int step = (hi - lo) >> 5;
-        int sel = 0;
-#pragma unroll
-        for (int k = 0; k < 31; ++k) sel += ent[cb + lo + (k + 1) * step].x < x ? 1 : 0;
-        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
-        const int nhi = sel == 31 ? hi : lo + (sel + 1) * step;
-        lo = nlo; hi = nhi;
-    }
-    while (hi - lo > 8) {                                        // at most 3 rounds from 256
-        const int step = (hi - lo) >> 3;
-        int t[7];
-#pragma unroll
-        for (int k = 0; k < 7; ++k) t[k] = ent[cb + lo + (k + 1) * step].x;
-        int sel = 0;
-#pragma unroll
-        for (int k = 0; k < 7; ++k) sel += t[k] < x ? 1 : 0;     // pivots below x
-        const int nlo = sel == 0 ? lo : lo + sel * step + 1;
-        const int nhi = sel == 7 ? hi : lo + (sel + 1) * step;
-        lo = nlo; hi = nhi;
-    }
-    // at most eight candidates left: all of them in one round
-    int t[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) t[k] = lo + k < hi ? ent[cb + lo + k].x : 0x7fffffff;
-    int below = 0;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) below += t[k] < x ? 1 : 0;
-    return lo + below;
-}
-
 // Look-up of child x in the sorted run ent[cb .. cb+n): insert position in `pos`, and if the
 // child exists its index is returned with its entry in `fe` (else -1).  The last round reads
 // whole entries, so a run of up to G children costs one round of loads.
@@ -185,39 +151,6 @@ __device__ int lookup_child(const int4* ent, int cb, int n, int x, int& pos, int
 #pragma unroll
     for (int k = 0; k < G; ++k) if (k == below && lo + k < hi && e[k].x == x) { fe = e[k]; found = cb + lo + k; }
     return found;
-}
-
-// Child x of `node` (-1 if none), by plain loads.
-__device__ int peek_child(const int4* ent, int node, int x) {
-    if (node < 0) return -1;
-    const int4 pe = ent[node];
-    const int n = (int)((unsigned)pe.w & RUN_COUNT_MASK);
-    if (n == 0) return -1;
-    const int pos = lower_bound_run(ent, pe.z, n, x);
-    if (pos >= n) return -1;
-    return ent[pe.z + pos].x == x ? pe.z + pos : -1;
-}
-
-// The slow look-ups of a token are the shallow ones (long child runs of frequent tokens, cold in
-// the caches), and they depend only on the last two or three tokens, not on the deep state.
-// Lane j walks the two- and three-token strings that end at token k0 + j, 32 tokens at once, so
-// that the token-by-token pass finds those runs in the caches.  Nothing is decided here; the
-// return value only keeps the loads alive.
-__device__ int warm_shallow(const TreeRef& tr, int V, const int32_t* tok, long long b, long long e, long long k0,
-                            int lane) {
-    const long long k = k0 + lane;
-    if (k >= e) return 0;
-    const int x0 = tok[k];
-    const int x1 = k - 1 >= b ? tok[k - 1] : -1, x2 = k - 2 >= b ? tok[k - 2] : -1;
-    if (x0 < 0 || x0 >= V || x1 < 0 || x1 >= V) return 0;
-    int seen = 0;
-    const int c1 = peek_child(tr.ent, tr.root[x1], x0);                        // (x1, x0)
-    if (c1 >= 0) seen += tr.ent[c1].y;
-    if (x2 >= 0 && x2 < V) {
-        const int c2 = peek_child(tr.ent, peek_child(tr.ent, tr.root[x2], x1), x0);   // (x2, x1, x0)
-        if (c2 >= 0) seen += tr.ent[c2].y;
-    }
-    return seen;
 }
 
 // All 32 lanes call.  `act` is this lane's active node of depth lane + 1 (-1: none);

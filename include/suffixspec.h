@@ -125,6 +125,11 @@ int sd_build(const sd_build_params* params, const int32_t* d_corpus, const int64
  * SD_STATUS_GLOBAL_FULL is set: strings whose nodes found no room are missing
  * or counted short, the tree stays consistent and usable, and later calls
  * insert nothing more into it.  n == 0 is a no-op.
+ * Stream order: for the caller everything is ordered on `stream`.  Inside the
+ * call the insert into the global tree runs on a stream the store owns, which
+ * starts behind the work `stream` holds at the call and which `stream` waits
+ * for before it goes on (the two kinds of tree share nothing, so the insert
+ * and the appends to the request trees run side by side).
  * Errors: INVALID_ARG, CUDA (launch failure).
  */
 int sd_append(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* d_offsets,

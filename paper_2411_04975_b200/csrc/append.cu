@@ -417,9 +417,18 @@ extern "C" int sd_append(sd_store* s, int32_t n, const int32_t* d_slot, const in
     if (!d_slot || !d_offsets) return SD_ERR_INVALID_ARG;
     const int warps_per_block = 4;
     const unsigned blocks = (unsigned)((n + 1 + warps_per_block - 1) / warps_per_block);
-    global_insert_kernel<<<GI_CTAS, GI_THREADS, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_offsets, d_tokens);
+    // The global tree and the request trees share nothing: the insert into the global tree runs
+    // beside the appends, on the store's own stream, which starts behind everything the caller's
+    // stream holds so far and which the caller's stream waits for before it goes on.
+    cudaStream_t st = (cudaStream_t)stream;
+    SD_CUDA_OK(cudaEventRecord(s->ev_fork, st));
+    SD_CUDA_OK(cudaStreamWaitEvent(s->aux, s->ev_fork, 0));
+    global_insert_kernel<<<GI_CTAS, GI_THREADS, 0, s->aux>>>(*s, n, d_slot, d_offsets, d_tokens);
     SD_CUDA_OK(cudaGetLastError());
-    append_kernel<<<blocks, warps_per_block * 32, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset);
+    SD_CUDA_OK(cudaEventRecord(s->ev_join, s->aux));
+    append_kernel<<<blocks, warps_per_block * 32, 0, st>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset);
+    SD_CUDA_OK(cudaGetLastError());
+    SD_CUDA_OK(cudaStreamWaitEvent(st, s->ev_join, 0));
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }

@@ -714,6 +714,9 @@ static void store_release(sd_store* s) {
         for (int k = 0; k < 48; ++k) cudaFree(s->ws->ptr[k]);
         delete s->ws;
     }
+    if (s->ev_fork) cudaEventDestroy(s->ev_fork);
+    if (s->ev_join) cudaEventDestroy(s->ev_join);
+    if (s->aux) cudaStreamDestroy(s->aux);
     delete s;
 }
 
@@ -889,6 +892,13 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
               store_alloc(s, &s->j_score, jobs) && store_alloc(s, &s->j_n, jobs) &&
               store_alloc(s, &s->j_tok, jobs * s->M) && store_alloc(s, &s->j_par, jobs * s->M);
     if (!ok) { store_release(s); return SD_ERR_NOMEM; }
+    if (cudaStreamCreateWithFlags(&s->aux, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        store_release(s);
+        return SD_ERR_CUDA;
+    }
     cudaError_t ce = cudaMemsetAsync(s->g_root, 0xFF, sizeof(int32_t) * (size_t)s->V, st);
     if (ce == cudaSuccess) ce = cudaMemsetAsync(s->s_root, 0xFF, sizeof(int32_t) * (size_t)s->R * s->V, st);
     if (ce == cudaSuccess) ce = cudaMemsetAsync(s->s_state, 0, sizeof(SlotState) * (size_t)s->R, st);

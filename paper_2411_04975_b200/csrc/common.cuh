@@ -85,6 +85,10 @@ struct sd_store {
     int32_t* j_par;           // [R*2*D][M]
     long long device_bytes;
     struct sd_workspace* ws;  // HOST: temporaries of sd_build_requests, kept between calls
+    // HOST: sd_append runs the insert into the global tree beside the appends to the request trees
+    // (they share nothing), on this stream, forked from and joined to the caller's stream
+    cudaStream_t aux;
+    cudaEvent_t ev_fork, ev_join;
 };
 
 __host__ __device__ inline uint32_t sd_pow2ceil(uint32_t n) {

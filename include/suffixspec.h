@@ -73,6 +73,12 @@ typedef struct {
     double alpha;                 /* max speculation factor: MAX_SPEC(p) = alpha * p  */
     int32_t max_spec;             /* cap on MAX_SPEC(p), <= max_spec_cap              */
     uint32_t flags;               /* SD_FLAG_*                                        */
+    double tau;                   /* score threshold of Section 3.2 ("Hybrid Suffix   */
+                                  /* Speculative Decoding"): a request gets a draft   */
+                                  /* only if SCORE > tau (strict); otherwise n_draft  */
+                                  /* = 0, chosen_tree = -1, score = 0 and the caller  */
+                                  /* falls back to its other drafter.  0: no gate     */
+                                  /* beyond Algorithm 1's SCORE > 0.  Must be >= 0.   */
 } sd_spec_params;
 
 typedef struct {
@@ -227,7 +233,7 @@ int sd_step(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* d_
  *    different stores) would overwrite each other's records, so keep calls on
  *    one device ordered.
  */
-#define SD_NOALLOC_MAX_JOBS 4096
+#define SD_NOALLOC_MAX_TOKENS (512 * 1024)
 int sd_speculate_noalloc(sd_store* store, int32_t n, const int32_t* d_slot, const sd_spec_params* params,
                          const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
                          int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,

@@ -63,7 +63,7 @@ def _load():
         lib.sfx_oracle_budget.restype = C.c_int
         lib.sfx_oracle_budget.argtypes = [C.c_double, C.c_int, C.c_int]
         lib.sfx_oracle_speculate.argtypes = [C.c_void_p, C.c_int, p32, C.c_int, C.c_double, C.c_int, C.c_int,
-                                             C.c_int, p32, p32, p32, p32, p32, pu32, p32, p32, pd, p64, C.c_int]
+                                             C.c_int, p32, p32, p32, p32, p32, pu32, p32, p32, pd, p64, C.c_int, C.c_double]
         _lib = lib
     return _lib
 
@@ -168,7 +168,7 @@ class SuffixOracle:
         return tok[:n].copy(), par[:n].copy(), dv[:n].copy(), sc.value
 
     def speculate(self, slots, P: int, alpha: float, max_spec: int, M: Optional[int] = None, flags: int = 0,
-                  budget_override=None, n_threads: int = 1) -> dict:
+                  budget_override=None, n_threads: int = 1, tau: float = 0.0) -> dict:
         slots = _i32(slots)
         n = slots.size
         M = max_spec if M is None else M
@@ -192,5 +192,6 @@ class SuffixOracle:
             self._h, n, _p(slots, C.c_int32), P, float(alpha), max_spec, flags, M, bo,
             _p(r["n_draft"], C.c_int32), _p(r["tokens"], C.c_int32), _p(r["parents"], C.c_int32),
             _p(r["positions"], C.c_int32), _p(r["mask"], C.c_uint32), _p(r["chosen_tree"], C.c_int32),
-            _p(r["chosen_p"], C.c_int32), _p(r["score"], C.c_double), _p(r["visited"], C.c_int64), n_threads)
+            _p(r["chosen_p"], C.c_int32), _p(r["score"], C.c_double), _p(r["visited"], C.c_int64), n_threads,
+            float(tau))
         return r

@@ -181,7 +181,7 @@ struct SpecOut {
 
 // GenerateCandidateTree for one request + the hand-off arrays.
 void speculate_one(const Oracle& o, int i, int slot, int P, double alpha, int cap, int flags, int M,
-                   const int32_t* budget_override, const SpecOut& r) {
+                   const int32_t* budget_override, double tau, const SpecOut& r) {
     const Slot& s = o.slots[slot];
     const int64_t t = (int64_t)s.text.size();
     const int words = (M + 31) / 32;
@@ -210,6 +210,9 @@ void speculate_one(const Oracle& o, int i, int slot, int P, double alpha, int ca
             if (sc > best_score) { best_score = sc; best = cur; best_tree = tree; best_p = p; }
         }
     }
+    // Section 3.2 ("Hybrid Suffix Speculative Decoding"): the suffix tree's draft is used only if
+    // its score exceeds the threshold tau; otherwise the caller falls back to its other drafter.
+    if (!(best_score > tau)) { best.clear(); best_score = 0.0; best_tree = -1; best_p = 0; }
     int n = (int)best.size();
     r.n_draft[i] = n; r.chosen_tree[i] = best_tree; r.chosen_p[i] = best_p; r.score[i] = best_score;
     if (r.visited) { r.visited[2 * i] = descents; r.visited[2 * i + 1] = adds; }
@@ -342,18 +345,18 @@ int sfx_oracle_budget(double alpha, int p, int cap) { return budget_for(alpha, p
 void sfx_oracle_speculate(void* h, int n, const int32_t* slots, int P, double alpha, int max_spec, int flags,
                           int M, const int32_t* budget_override, int32_t* n_draft, int32_t* tokens,
                           int32_t* parents, int32_t* positions, uint32_t* mask, int32_t* chosen_tree,
-                          int32_t* chosen_p, double* score, int64_t* visited, int n_threads) {
+                          int32_t* chosen_p, double* score, int64_t* visited, int n_threads, double tau) {
     Oracle* o = (Oracle*)h;
     SpecOut r{n_draft, tokens, parents, positions, mask, chosen_tree, chosen_p, score, visited};
     if (n_threads <= 1) {
-        for (int i = 0; i < n; ++i) speculate_one(*o, i, slots[i], P, alpha, max_spec, flags, M, budget_override, r);
+        for (int i = 0; i < n; ++i) speculate_one(*o, i, slots[i], P, alpha, max_spec, flags, M, budget_override, tau, r);
         return;
     }
     std::vector<std::thread> th;
     for (int w = 0; w < n_threads; ++w)
         th.emplace_back([=] {
             for (int i = w; i < n; i += n_threads)
-                speculate_one(*o, i, slots[i], P, alpha, max_spec, flags, M, budget_override, r);
+                speculate_one(*o, i, slots[i], P, alpha, max_spec, flags, M, budget_override, tau, r);
         });
     for (auto& x : th) x.join();
 }

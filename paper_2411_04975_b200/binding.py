@@ -35,7 +35,8 @@ class _BuildParams(C.Structure):
 
 
 class _SpecParams(C.Structure):
-    _fields_ = [("P", C.c_int32), ("alpha", C.c_double), ("max_spec", C.c_int32), ("flags", C.c_uint32)]
+    _fields_ = [("P", C.c_int32), ("alpha", C.c_double), ("max_spec", C.c_int32), ("flags", C.c_uint32),
+                ("tau", C.c_double)]
 
 
 class _Stats(C.Structure):
@@ -126,8 +127,8 @@ def sd_append(store: int, slots: torch.Tensor, offsets: torch.Tensor, tokens: to
 
 
 def sd_speculate(store: int, slots: torch.Tensor, P: int, alpha: float, max_spec: int, flags: int,
-                 budget_cap: Optional[torch.Tensor], out: Dict[str, torch.Tensor]) -> None:
-    prm = _SpecParams(P, alpha, max_spec, flags)
+                 budget_cap: Optional[torch.Tensor], out: Dict[str, torch.Tensor], tau: float = 0.0) -> None:
+    prm = _SpecParams(P, alpha, max_spec, flags, tau)
     rc = library().sd_speculate(
         store, int(slots.numel()), _ptr(slots, torch.int32, "slots"), C.byref(prm),
         _ptr(budget_cap, torch.int32, "budget_cap"), _ptr(out["n_draft"], torch.int32, "n_draft"),
@@ -140,12 +141,12 @@ def sd_speculate(store: int, slots: torch.Tensor, P: int, alpha: float, max_spec
 
 
 def sd_speculate_noalloc(store: int, slots: torch.Tensor, P: int, alpha: float, max_spec: int, flags: int,
-                         budget_cap: Optional[torch.Tensor], out: Dict[str, torch.Tensor]) -> None:
+                         budget_cap: Optional[torch.Tensor], out: Dict[str, torch.Tensor], tau: float = 0.0) -> None:
     """sd_speculate for callers that may not allocate device memory: the scratch
     records live in a fixed array inside the library, so the batch is limited
     (n * 2 * depth_cap <= 4096 jobs) and calls on one device must not overlap.
     `out` must be preallocated by the caller; nothing is allocated here."""
-    prm = _SpecParams(P, alpha, max_spec, flags)
+    prm = _SpecParams(P, alpha, max_spec, flags, tau)
     rc = library().sd_speculate_noalloc(
         store, int(slots.numel()), _ptr(slots, torch.int32, "slots"), C.byref(prm),
         _ptr(budget_cap, torch.int32, "budget_cap"), _ptr(out["n_draft"], torch.int32, "n_draft"),
@@ -166,10 +167,10 @@ class BoundStep:
     """One sd_step call with all of its arguments already converted (see SuffixStore.bind_step).
     Calling the object launches the step; `out` holds the output tensors it writes."""
 
-    def __init__(self, store, slots, offsets, new_tokens, P, alpha, max_spec, flags, budget_cap, out, stream):
+    def __init__(self, store, slots, offsets, new_tokens, P, alpha, max_spec, flags, budget_cap, out, stream, tau=0.0):
         self.out = out
         self._keep = (store, slots, offsets, new_tokens, budget_cap)       # the buffers must outlive the calls
-        self._prm = _SpecParams(P, alpha, max_spec, flags)
+        self._prm = _SpecParams(P, alpha, max_spec, flags, tau)
         self._fn = library().sd_step
         self._args = (
             store._h, int(slots.numel()), _ptr(slots, torch.int32, "slots"), _ptr(offsets, torch.int64, "offsets"),
@@ -265,21 +266,21 @@ class SuffixStore:
 
     def speculate(self, slots: torch.Tensor, P: int, alpha: float, max_spec: int, flags: int = 0,
                   budget_cap: Optional[torch.Tensor] = None,
-                  out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+                  out: Optional[Dict[str, torch.Tensor]] = None, tau: float = 0.0) -> Dict[str, torch.Tensor]:
         """mask is returned as int32 words (same bits as the uint32 of the C ABI)."""
         if out is None:
             out = self.alloc_outputs(int(slots.numel()))
-        sd_speculate(self._h, slots, P, alpha, max_spec, flags, budget_cap, out)
+        sd_speculate(self._h, slots, P, alpha, max_spec, flags, budget_cap, out, tau)
         return out
 
     def step(self, slots: torch.Tensor, offsets: torch.Tensor, new_tokens: torch.Tensor, P: int, alpha: float,
              max_spec: int, flags: int = 0, budget_cap: Optional[torch.Tensor] = None,
-             out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+             out: Optional[Dict[str, torch.Tensor]] = None, tau: float = 0.0) -> Dict[str, torch.Tensor]:
         """One decode step in one launch: append `new_tokens` (ragged by `offsets`) to the slots,
         then speculate.  Same result as append() followed by speculate()."""
         if out is None:
             out = self.alloc_outputs(int(slots.numel()))
-        prm = _SpecParams(P, alpha, max_spec, flags)
+        prm = _SpecParams(P, alpha, max_spec, flags, tau)
         rc = library().sd_step(
             self._h, int(slots.numel()), _ptr(slots, torch.int32, "slots"), _ptr(offsets, torch.int64, "offsets"),
             _ptr(new_tokens, torch.int32, "new_tokens"), C.byref(prm), _ptr(budget_cap, torch.int32, "budget_cap"),
@@ -294,7 +295,8 @@ class SuffixStore:
 
     def bind_step(self, slots: torch.Tensor, offsets: torch.Tensor, new_tokens: torch.Tensor, P: int, alpha: float,
                   max_spec: int, flags: int = 0, budget_cap: Optional[torch.Tensor] = None,
-                  out: Optional[Dict[str, torch.Tensor]] = None, stream: Optional[int] = None) -> "BoundStep":
+                  out: Optional[Dict[str, torch.Tensor]] = None, stream: Optional[int] = None,
+                  tau: float = 0.0) -> "BoundStep":
         """step() with the argument marshalling done once.  A serving loop calls sd_step with the
         same buffers every step (it refills them in place: `new_tokens` is the whole token buffer,
         `offsets` says how much of it a step uses), so the returned object keeps the converted
@@ -303,7 +305,7 @@ class SuffixStore:
         if out is None:
             out = self.alloc_outputs(int(slots.numel()))
         return BoundStep(self, slots, offsets, new_tokens, P, alpha, max_spec, flags, budget_cap, out,
-                         _stream() if stream is None else stream)
+                         _stream() if stream is None else stream, tau)
 
     def query_counts(self, tree: torch.Tensor, offsets: torch.Tensor, paths: torch.Tensor) -> torch.Tensor:
         n = int(tree.numel())

@@ -1,21 +1,44 @@
-// GenerateCandidateTree (Algorithm 1) for a whole batch.
+// GenerateCandidateTree (Algorithm 1) for a whole batch: one thread block per request, one
+// launch per decode step (sd_step: the accepted tokens are appended in the same launch).
 //
-// Kernel 1, one warp per (request, tree, p) job: MatchPattern, then
-// ExpandSpeculationTree with a warp-wide sorted frontier, then SCORE (Eq. 4).
-// Kernel 2, one warp per request: pick the first job with the strictly largest
-// score and write the verifier's arrays (tokens, parents, positions, mask).
+//   1. text.  The request's text x_{1:t} is copied into shared memory (new tokens included).
+//   2. match.
+//      Per-request tree (implicit, see common.cuh): the block scans the text for the earlier
+//      occurrences of the last token and measures, for each, how many tokens before it agree
+//      with the context (at most P).  Sorted by that length, the occurrences of the pattern of
+//      length p are a prefix of the list: that prefix IS the match node N_p.
+//      Global tree: MatchPattern walks from the root table, the shortest patterns first, a warp
+//      per pattern length, until a match node has at most 32 occurrences and was never touched
+//      by an online insert.  Such a node is a range of the offline build's suffix order; its
+//      occurrences are read from there with the text around them (64 tokens each), and the
+//      occurrences of every longer pattern are those among them whose preceding tokens agree
+//      with the context.  No longer pattern is walked.
+//   3. expand.  The (tree, p) jobs that matched go into a queue, costliest first; a warp per job.
+//      Occurrence mode (at most 32 occurrences): a lane per occurrence.  A node of the suffix
+//      tree below N_p is the set of lanes whose next tokens agree so far, its count their number
+//      (Eq. 1 and Eq. 2 from popcounts), and the frontier of ExpandSpeculationTree is "the next
+//      node on every lane's path": the best candidate is a warp-wide arg-max, adding it moves
+//      its lanes one token on.  Chains are added without an arg-max.
+//      Wide per-request nodes (more than 32 occurrences: short patterns of frequent tokens, small
+//      budgets): children by a histogram of the next tokens over the occurrence list.
+//      Global nodes with more than 32 occurrences or touched by an insert: the tree's entries
+//      (sorted child runs, top blocks, windows of 32 entries) with a sorted frontier.
+//      A job is dropped, exactly, as soon as an upper bound of its SCORE (every D <= 1 and D
+//      never grows along a path) falls below a score another job of the request has reached.
+//   4. select (first in loop order among the largest scores; Section 3.2: only if SCORE > tau)
+//      and emit tokens, parents, positions and the tree-attention mask.
 //
 // fp64 rules: C = count / sibling-sum (Eq. 1), D = D(parent) * C (Eq. 2), SCORE
 // adds D in insertion order; __ddiv_rn / __dmul_rn / __dadd_rn keep every
 // operation a separately rounded IEEE binary64 operation (no FMA contraction).
 #include <mutex>
 
-#include "append_core.cuh"
+#include "common.cuh"
 
 namespace {
 
-constexpr int SPEC_WARPS = 8;                 // warps per block of the job kernel
 constexpr unsigned FULL = 0xffffffffu;
+constexpr int OCC_CAP = 1024;                 // occurrences of the last token kept in shared memory
 
 struct Frontier {                             // candidates of one job, best first, ring buffer
     double d[SD_MAX_SPEC];
@@ -30,29 +53,6 @@ struct Frontier {                             // candidates of one job, best fir
 __device__ __forceinline__ bool better(double da, int ta, int pa, double db, int tb, int pb) {
     const long long a = __double_as_longlong(da), b = __double_as_longlong(db);
     return (a > b) | ((a == b) & ((ta < tb) | ((ta == tb) & (pa < pb))));
-}
-
-// Entry index of child `x` in the sorted run ent[cb .. cb+n), or -1.  Whole warp.
-__device__ int find_child(const int4* __restrict__ ent, int cb, int n, int x, int lane) {
-    int lo = 0, hi = n;
-    for (int it = 0; it < 6 && hi - lo > 32; ++it) {       // window shrinks 33x per round
-        const int q = lo + (int)(((long long)(hi - lo) * (lane + 1)) / 33);
-        const int tk = ent[cb + q].x;
-        const unsigned ge = __ballot_sync(FULL, tk >= x);
-        const int f = ge ? __ffs(ge) - 1 : 32;              // first probe with token >= x
-        const int q_prev = __shfl_sync(FULL, q, f > 0 ? f - 1 : 0);
-        const int q_at = __shfl_sync(FULL, q, f < 32 ? f : 31);
-        if (f > 0) lo = q_prev + 1;
-        if (f < 32) hi = q_at + 1;
-    }
-    int found = -1;
-    for (int base = lo; base < hi && found < 0; base += 32) {   // one round unless n is huge
-        const int idx = base + lane;
-        const bool hit = idx < hi && ent[cb + idx].x == x;
-        const unsigned eq = __ballot_sync(FULL, hit);
-        if (eq) found = cb + base + __ffs(eq) - 1;
-    }
-    return found;
 }
 
 // Insert one candidate (same values on every lane) into the sorted frontier of at
@@ -79,214 +79,12 @@ __device__ void frontier_insert(Frontier& F, int fh, int& fs, int K, double d, i
     fs = ns;
 }
 
-// Offer every child of a node (run ent[cb .. cb+n)) to the frontier.
-__device__ void push_children(const int4* __restrict__ ent, int cb, int n, double d_parent, int par_index, Frontier& F,
-                              int fh, int& fs, int K, int lane) {
-    if (n <= 0 || K <= 0) return;
-    long long sum = 0;
-    int4 first = make_int4(0, 0, 0, 0);
-    for (int base = 0; base < n; base += 32) {
-        const int idx = base + lane;
-        int4 e = make_int4(0, 0, 0, 0);
-        if (idx < n) e = ent[cb + idx];
-        if (base == 0) first = e;
-        sum += e.y;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
-    const double dsum = (double)sum;                            // denominator of Eq. 1
-    for (int base = 0; base < n; base += 32) {
-        const int idx = base + lane;
-        const bool v = idx < n;
-        int4 e = first;
-        if (base != 0) { e = make_int4(0, 0, 0, 0); if (v) e = ent[cb + idx]; }
-        double dc = 0.0;
-        if (v) dc = __dmul_rn(d_parent, __ddiv_rn((double)e.y, dsum));   // Eq. 2 with Eq. 1
-        bool pass = v;
-        if (v && fs == K) {                                     // cannot beat the current worst: skip
-            const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
-            pass = better(dc, e.x, par_index, F.d[last], F.tok[last], F.par[last]);
-        }
-        unsigned m = __ballot_sync(FULL, pass);
-        while (m) {
-            const int src = __ffs(m) - 1;
-            m &= m - 1;
-            const double cd = __shfl_sync(FULL, dc, src);
-            const int ct = __shfl_sync(FULL, e.x, src);
-            const int cc = __shfl_sync(FULL, e.z, src);
-            const unsigned cn = (unsigned)__shfl_sync(FULL, e.w, src);
-            frontier_insert(F, fh, fs, K, cd, ct, par_index, cc, cn, lane);
-        }
-    }
-}
-
 __device__ __forceinline__ int budget_for(double alpha, int p, int cap) {
     const double b = floor(__dmul_rn(alpha, (double)p));        // Eq. 3
     if (b > (double)cap) return cap;
     if (b < 0.0) return 0;
     return (int)b;
 }
-
-__global__ void __launch_bounds__(SPEC_WARPS * 32)
-match_expand_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
-                    unsigned flags, const int32_t* __restrict__ d_budget_cap) {
-    __shared__ Frontier fr[SPEC_WARPS];
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const long long job = (long long)blockIdx.x * SPEC_WARPS + wib;
-    if (job >= (long long)n * 2 * Pe) return;
-    const int i = (int)(job / (2 * Pe));
-    const int rem = (int)(job % (2 * Pe));
-    const int tree = rem / Pe, p = rem % Pe + 1;
-    const long long rec = ((long long)i * 2 + tree) * sv.D + (p - 1);
-    int cnt = 0;
-    double score = 0.0;
-    const int slot = d_slot[i];
-    bool live = slot >= 0 && slot < sv.R;
-    if (tree == 0 && (flags & SD_FLAG_REQUEST_ONLY)) live = false;
-    if (tree == 1 && (flags & SD_FLAG_GLOBAL_ONLY)) live = false;
-    if (live) {
-        const SlotState* ss = sv.s_state + slot;
-        const int t = ss->len;
-        if (ss->status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) live = false;
-        if (p > t) live = false;
-        int cap = max_spec;
-        if (d_budget_cap && d_budget_cap[i] >= 0) cap = min(cap, d_budget_cap[i]);
-        const int budget = budget_for(alpha, p, cap);
-        if (live && budget > 0) {
-            // ---- MatchPattern
-            const int4* ent;
-            int node;
-            if (tree == 1) {
-                ent = sv.s_ent + (long long)slot * sv.spn;
-                node = ss->active[p - 1];                       // node of the last p tokens
-            } else {
-                ent = sv.g_ent;
-                const int32_t* pat = sv.s_text + (long long)slot * sv.T + (t - p);
-                node = sv.g_root[pat[0]];
-                for (int k = 1; k < p && node >= 0; ++k) {
-                    const int4 e = ent[node];
-                    node = find_child(ent, e.z, (int)((unsigned)e.w & RUN_COUNT_MASK), pat[k], lane);
-                }
-            }
-            if (node >= 0) {
-                // ---- ExpandSpeculationTree
-                Frontier& F = fr[wib];
-                int fh = 0, fs = 0;
-                const int4 e = ent[node];
-                push_children(ent, e.z, (int)((unsigned)e.w & RUN_COUNT_MASK), 1.0, -1, F, fh, fs, budget, lane);
-                int32_t* out_tok = sv.j_tok + rec * sv.M;
-                int32_t* out_par = sv.j_par + rec * sv.M;
-                while (cnt < budget && fs > 0) {
-                    const double d = F.d[fh];
-                    const int tok = F.tok[fh], par = F.par[fh], cb = F.cb[fh];
-                    const int nc = (int)(F.nc[fh] & RUN_COUNT_MASK);
-                    __syncwarp();
-                    fh = (fh + 1) & (SD_MAX_SPEC - 1);
-                    --fs;
-                    if (lane == 0) { out_tok[cnt] = tok; out_par[cnt] = par; }
-                    score = __dadd_rn(score, d);                // Eq. 4, insertion order
-                    const int idx = cnt++;
-                    const int K = budget - cnt;
-                    if (fs > K) fs = K;
-                    if (flags & SD_FLAG_LINEAR) fs = 0;
-                    push_children(ent, cb, nc, d, idx, F, fh, fs, K, lane);
-                }
-            }
-        }
-    }
-    if (lane == 0) { sv.j_n[rec] = cnt; sv.j_score[rec] = score; }
-}
-
-__global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, int32_t* d_n_draft,
-                                   int32_t* d_tokens, int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask,
-                                   int32_t* d_chosen_tree, int32_t* d_chosen_p, double* d_score, int32_t* d_status) {
-    __shared__ int spar[4][SD_MAX_SPEC];
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int i = blockIdx.x * 4 + wib;
-    if (i >= n) return;
-    const int M = sv.M, words = (M + 31) / 32;
-    const int slot = d_slot[i];
-    const bool ok = slot >= 0 && slot < sv.R;
-    // first job in loop order (global before per-request, p ascending) with the largest score
-    double best = 0.0;
-    int best_o = -1;
-    for (int o = lane; o < 2 * Pe; o += 32) {
-        const long long rec = ((long long)i * 2 + o / Pe) * sv.D + (o % Pe);
-        const double sc = sv.j_score[rec];
-        if (sc > best) { best = sc; best_o = o; }               // ascending o: strict '>' keeps the first
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const double ob = __shfl_xor_sync(FULL, best, off);
-        const int oo = __shfl_xor_sync(FULL, best_o, off);
-        if (oo >= 0 && (ob > best || (ob == best && (best_o < 0 || oo < best_o)))) { best = ob; best_o = oo; }
-    }
-    int nd = 0, tree = -1, p = 0, t = 0, status = SD_STATUS_BAD_SLOT;
-    long long rec = 0;
-    if (ok) {
-        t = sv.s_state[slot].len;
-        status = sv.s_state[slot].status;
-    }
-    if (ok && best_o >= 0) {
-        tree = best_o / Pe; p = best_o % Pe + 1;
-        rec = ((long long)i * 2 + tree) * sv.D + (p - 1);
-        nd = sv.j_n[rec];
-    } else {
-        best = 0.0;
-    }
-    for (int j = lane; j < SD_MAX_SPEC; j += 32) spar[wib][j] = j < nd ? sv.j_par[rec * M + j] : -1;
-    __syncwarp();
-    for (int j = lane; j < M; j += 32) {
-        int tok = -1, par = -1, pos = -1;
-        unsigned long long bits = 0;
-        if (j < nd) {
-            tok = sv.j_tok[rec * M + j];
-            par = spar[wib][j];
-            int depth = 0;
-            for (int a = j, hops = 0; a >= 0 && hops < SD_MAX_SPEC; a = spar[wib][a], ++hops) {
-                bits |= 1ull << a;
-                ++depth;
-            }
-            pos = t + depth - 1;
-        }
-        const long long o = (long long)i * M + j;
-        d_tokens[o] = tok; d_parents[o] = par; d_positions[o] = pos;
-        d_mask[o * words] = (uint32_t)bits;
-        if (words > 1) d_mask[o * words + 1] = (uint32_t)(bits >> 32);
-    }
-    if (lane == 0) {
-        d_n_draft[i] = nd; d_chosen_tree[i] = tree; d_chosen_p[i] = p; d_score[i] = best;
-        if (d_status) d_status[i] = status;
-    }
-}
-
-
-// ---------------------------------------------------------------------------------------------
-// Fused path: one block of W warps per request.  Two blocks per SM is the usual shape: W = 16
-// with 64 registers per thread for sd_speculate, W = 10 with 96 for sd_step, whose append is
-// register hungry.  A batch of at most one request per SM gets bigger blocks (W = 24 / 16), a
-// batch of more than two requests per SM smaller ones (W = 8 / 5, four per SM) to stay in one wave.
-//   1. match: the per-request match nodes are the slot's active nodes; the global match
-//      nodes are advanced from the nodes cached at the previous call by descending only the
-//      tokens appended since (full walks when the cache is stale).  Warp w serves pattern
-//      lengths w + 1, w + 1 + W, ...
-//   2. expand: the (tree, p) jobs that matched go into a queue, costliest first; warps pull
-//      jobs until it is empty.  A job is dropped, exactly, as soon as an upper bound of its
-//      SCORE (every D <= 1 and D never grows along a path) falls below a score already
-//      reached by another job of the request.
-//   3. select + emit from shared memory; no global scratch.
-constexpr int CTA_WARPS = 16;                  // the usual block
-constexpr int CTA_WARPS_STEP = 10;             // the usual block of sd_step: 10 warps with 96 registers each and
-constexpr int STEP_G = 4;                      // an append that moves four entries per round, so that the
-                                               // append in front does not spill.  Measured per step: 92.7 us;
-                                               // 9 warps 92.8, 11 (80 registers) 95, 8 (128) 96; with eight
-                                               // entries per round: 8 warps x 128 registers 95, 10 x 96 100,
-                                               // 12 x 80 100, 16 x 64 104, 6 x 168 110
-constexpr int CTA_WARPS_WIDE = 24;             // small batches (one block per SM at most): the block has the SM's
-constexpr int CTA_WARPS_WIDE_STEP = 16;        // registers to itself (80 per thread; sd_step: 128)
-constexpr int CTA_WARPS_NARROW = 8;            // batches of more than two requests per SM: four blocks per SM
-constexpr int CTA_WARPS_NARROW_STEP = 5;       // (sd_step: 96 registers and the four-entry append; 512 requests:
-                                               // 82 us per step, 88 with 4 warps x 128 registers, 100 with 8 x 64)
 
 struct WarpWork {
     Frontier F;
@@ -303,7 +101,7 @@ struct WarpWork {
 template <int WARPS>
 struct BlockSharedT {
     WarpWork w[WARPS];
-    int node[2][SD_MAX_DEPTH];                // match node per tree and pattern length (-1: none)
+    int node[2][SD_MAX_DEPTH];                // global tree: match node per pattern length (-1: none); row 1 unused
     int cb[2][SD_MAX_DEPTH];                  // its child run
     unsigned nc[2][SD_MAX_DEPTH];             // ... as the node's w field (count | flags)
     int cost[2 * SD_MAX_DEPTH];
@@ -316,6 +114,22 @@ struct BlockSharedT {
                                               // bound of it (scores are non-negative doubles), which is
                                               // all the pruning needs; 32 bits keep the atomic native
     int win_warp;
+    int first_bad;                            // sd_step: first new token outside the vocabulary
+    // per-request tree: earlier occurrences of the last token by backward match length
+    int r_hist[SD_MAX_DEPTH + 2];
+    int r_cum[SD_MAX_DEPTH + 2];              // r_cum[p]: occurrences that agree on at least p tokens
+    int r_fill[SD_MAX_DEPTH + 2];
+    int scan_next[2];
+    // global tree: the base of occurrence mode
+    int g_cnt[SD_MAX_DEPTH];                  // COUNT of the match node
+    int g_rank[SD_MAX_DEPTH];                 // its first suffix in the suffix order (-1: not usable as base)
+    int g_walked, g_failed, g_base_p, g_base_m;
+    int g_pos[SD_OCC_LANES];                  // text position of the occurrence's first pattern token
+    int g_ell[SD_OCC_LANES];                  // longest pattern the occurrence matches
+    int g_avail[SD_OCC_LANES];                // tokens that follow the pattern inside the sequence (depth cap applied)
+    int g_cum[SD_MAX_DEPTH + 2];
+    int gwin[SD_OCC_LANES][64];               // tokens pos - 32 .. pos + 31 around every occurrence
+    int occ[OCC_CAP];
 };
 
 // find_child that also hands back the matched entry (valid when the result is >= 0)
@@ -544,44 +358,6 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
         }
     }
 }
-
-// MatchPattern from a known node: descend text[from .. to).  Levels whose child run lies inside
-// the window already in registers cost no memory access.  Returns the node reached (-1: no
-// match) and its child run in (cb, n).
-// The context is `text` up to position t_old and `newtok` from there on (tokens that are
-// being appended in the same launch).
-__device__ int walk_from(const int4* __restrict__ ent, int limit, int node, const int32_t* __restrict__ text, int t_old,
-                         const int32_t* __restrict__ newtok, int from, int to, int lane, int& cb, unsigned& wfull) {
-    if (node < 0) return -1;
-    int wb = node;
-    int4 w = load_window(ent, wb, limit, lane);
-    cb = __shfl_sync(FULL, w.z, 0);
-    wfull = (unsigned)__shfl_sync(FULL, w.w, 0);
-    int n = (int)(wfull & RUN_COUNT_MASK);
-    for (int pos = from; pos < to; ++pos) {
-        const int x = pos < t_old ? text[pos] : newtok[pos - t_old];
-        if (n == 0) return -1;
-        if (n > 32) {                                           // wide run: 32-way search
-            int4 e;
-            node = find_child_entry(ent, cb, n, x, lane, e);
-            if (node < 0) return -1;
-            cb = e.z; wfull = (unsigned)e.w; n = (int)(wfull & RUN_COUNT_MASK);
-            wb = -64;                                           // no usable window
-            continue;
-        }
-        if (!(cb >= wb && cb + n <= wb + 32)) { wb = cb; w = load_window(ent, wb, limit, lane); }
-        const int rel = wb + lane - cb;
-        const unsigned hit = __ballot_sync(FULL, rel >= 0 && rel < n && w.x == x);
-        if (!hit) return -1;
-        const int src = __ffs(hit) - 1;
-        node = wb + src;
-        cb = __shfl_sync(FULL, w.z, src);
-        wfull = (unsigned)__shfl_sync(FULL, w.w, src);
-        n = (int)(wfull & RUN_COUNT_MASK);
-    }
-    return node;
-}
-
 
 // Children of a node whose run has a top block (see RUN_HAS_TOP): the 64 best by count are
 // listed, best first, right before the run, together with the sum of all counts.
@@ -821,157 +597,522 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
     __syncwarp();
 }
 
-// STEP: the block first appends the request's newly accepted tokens (warp 0, exactly what
-// sd_append does for the slot) while its other warps already advance the global match nodes
-// over those tokens, then speculates: one launch per decode step, and the appends of long
-// token lists overlap with the speculation of the other requests.
-template <bool STEP, int WARPS, int MINB, int APPEND_G = 8>
-__global__ void __launch_bounds__(WARPS * 32, MINB)
-speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
-                       unsigned flags, const int32_t* __restrict__ d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
-                       int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
-                       int32_t* d_chosen_p, double* d_score, int32_t* d_status, const int64_t* __restrict__ d_app_off,
-                       const int32_t* __restrict__ d_app_tok) {
+// MatchPattern(S_g, x_{1:t}, p) from the root table: descends tx[t - p .. t).  Levels whose child
+// run lies inside the window already in registers cost no memory access.  Returns the node
+// reached (-1: no match), its child run (cb, wfull) and its COUNT.
+__device__ int walk_root(const int4* __restrict__ ent, int limit, const int32_t* __restrict__ root, int V, const int* tx,
+                         int t, int p, int lane, int& cb, unsigned& wfull, int& count) {
+    const int x0 = tx[t - p];
+    int node = (x0 >= 0 && x0 < V) ? root[x0] : -1;
+    if (node < 0) return -1;
+    int wb = node;
+    int4 w = load_window(ent, wb, limit, lane);
+    cb = __shfl_sync(FULL, w.z, 0);
+    wfull = (unsigned)__shfl_sync(FULL, w.w, 0);
+    count = __shfl_sync(FULL, w.y, 0);
+    int n = (int)(wfull & RUN_COUNT_MASK);
+    for (int pos = t - p + 1; pos < t; ++pos) {
+        const int x = tx[pos];
+        if (n == 0) return -1;
+        if (n > 32) {                                           // wide run: 32-way search
+            int4 e;
+            node = find_child_entry(ent, cb, n, x, lane, e);
+            if (node < 0) return -1;
+            cb = e.z; wfull = (unsigned)e.w; count = e.y; n = (int)(wfull & RUN_COUNT_MASK);
+            wb = -64;                                           // no usable window
+            continue;
+        }
+        if (!(cb >= wb && cb + n <= wb + 32)) { wb = cb; w = load_window(ent, wb, limit, lane); }
+        const int rel = wb + lane - cb;
+        const unsigned hit = __ballot_sync(FULL, rel >= 0 && rel < n && w.x == x);
+        if (!hit) return -1;
+        const int src = __ffs(hit) - 1;
+        node = wb + src;
+        cb = __shfl_sync(FULL, w.z, src);
+        wfull = (unsigned)__shfl_sync(FULL, w.w, src);
+        count = __shfl_sync(FULL, w.y, src);
+        n = (int)(wfull & RUN_COUNT_MASK);
+    }
+    return node;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Occurrence mode: ExpandSpeculationTree + SCORE for one (tree, p) job whose match node has at
+// most 32 occurrences, a lane per occurrence.  cptr[k] (k >= 1) is the k-th token behind the
+// lane's occurrence of the pattern and kmax says how many of them count (end of the text or
+// sequence, depth cap; 0: the lane holds no occurrence of this job).
+// A node below N_p is the set of lanes that agree on the tokens so far.  Every lane knows the
+// deepest node on its own path that is already in the speculation tree (k levels down, index
+// par_idx, D value d_par); the candidate it stands for is the next node on its path:
+//   COUNT = lanes that agree on the next token too, sibling sum = lanes that have a next token.
+// The candidates of all lanes together are exactly the frontier of Algorithm 1's expansion.
+template <class BlockShared>
+__device__ void expand_occ(BlockShared& sh, WarpWork& W, const int* cptr, int kmax, int tree, int p, int budget,
+                           unsigned flags, int lane) {
+    const int order = tree * SD_MAX_DEPTH + p;                  // loop order of Algorithm 1
+    const int buf = W.best_buf ^ 1;
+    int cnt = 0;
+    double score = 0.0;
+    bool dropped = false;
+    int k = 0, par_idx = -1;
+    double d_par = 1.0;                                         // D(N_p) = 1
+    bool cv = false;                                            // this lane stands for a candidate
+    int ctok = 0;
+    double cd = 0.0;
+    unsigned cmask = 0;                                         // lanes of the candidate node
+    // candidates of the lanes in `grp`, which share (k, par_idx, d_par); returns the lanes with a next token
+    auto refresh = [&](unsigned grp) -> unsigned {
+        const bool in = (grp >> lane) & 1u;
+        const bool valid = in && k + 1 <= kmax;
+        const unsigned vm = __ballot_sync(FULL, valid);
+        if (in) cv = false;
+        if (valid) {
+            ctok = cptr[k + 1];
+            cmask = __match_any_sync(vm, ctok);
+            const int c = __popc(cmask), s = __popc(vm);
+            cd = c == s ? d_par : __dmul_rn(d_par, __ddiv_rn((double)c, (double)s));   // Eq. 2 with Eq. 1
+            cv = true;
+        }
+        return vm;
+    };
+    refresh(__ballot_sync(FULL, kmax > 0));
+    while (cnt < budget) {
+        // ---- the best candidate: larger D, then smaller token, then smaller parent index
+        const unsigned hi = cv ? (unsigned)__double2hiint(cd) : 0u;     // D > 0, so hi > 0 for a candidate
+        const unsigned mx = __reduce_max_sync(FULL, hi);
+        if (mx == 0u) break;                                    // the frontier is empty
+        unsigned b = __ballot_sync(FULL, hi == mx);
+        int leader = __ffs(b) - 1;
+        unsigned lm = __shfl_sync(FULL, cmask, leader);
+        if (b & ~lm) {                                          // several nodes share the high word: full comparison
+            const bool in1 = hi == mx;
+            const unsigned lo = in1 ? (unsigned)__double2loint(cd) : 0u;
+            const unsigned mlo = __reduce_max_sync(FULL, lo);
+            const bool in2 = in1 && lo == mlo;
+            const unsigned mtk = __reduce_min_sync(FULL, in2 ? (unsigned)ctok : 0xffffffffu);
+            const bool in3 = in2 && (unsigned)ctok == mtk;
+            const unsigned mpk = __reduce_min_sync(FULL, in3 ? (unsigned)(par_idx + 1) : 0xffffffffu);
+            b = __ballot_sync(FULL, in3 && (unsigned)(par_idx + 1) == mpk);
+            leader = __ffs(b) - 1;
+            lm = __shfl_sync(FULL, cmask, leader);
+        }
+        const double wd = __shfl_sync(FULL, cd, leader);
+        const int wt = __shfl_sync(FULL, ctok, leader), wp = __shfl_sync(FULL, par_idx, leader);
+        // everything still to come is at most wd each
+        if ((score + (double)(budget - cnt) * wd) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
+        if (lane == 0) { W.tok[buf][cnt] = wt; W.par[buf][cnt] = (unsigned char)(wp + 1); }
+        score = __dadd_rn(score, wd);                           // Eq. 4, insertion order
+        int idx = cnt++;
+        const bool in = (lm >> lane) & 1u;
+        if (in) { ++k; par_idx = idx; d_par = wd; }
+        if ((flags & SD_FLAG_LINEAR) && !in) cv = false;        // chain variant: only the new node's children go on
+        // the best of the other candidates: while the new node has one child that all its lanes
+        // continue with, that child has the same D; if that is strictly above every other
+        // candidate it is the next node whatever else there is, and no arg-max is needed
+        const unsigned oth = __reduce_max_sync(FULL, (!in && cv) ? (unsigned)__double2hiint(cd) : 0u);
+        const bool chain_ok = (unsigned)__double2hiint(wd) > oth;
+        const int first = __ffs(lm) - 1;
+        while (true) {
+            const unsigned vm = refresh(lm);
+            if (cnt >= budget || !chain_ok || vm != lm || __shfl_sync(FULL, cmask, first) != lm) break;
+            if ((score + (double)(budget - cnt) * wd) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
+            if ((lm & (lm - 1u)) == 0u) {
+                // one occurrence: the rest of its text, as far as it counts and the budget goes
+                const int k0 = __shfl_sync(FULL, k, first);
+                const int len = min(__shfl_sync(FULL, kmax, first) - k0, budget - cnt);
+                const int* src = (const int*)(unsigned long long)__shfl_sync(FULL, (unsigned long long)cptr, first);
+                for (int j = lane; j < len; j += 32) {
+                    W.tok[buf][cnt + j] = src[k0 + 1 + j];
+                    W.par[buf][cnt + j] = (unsigned char)((j == 0 ? idx : cnt + j - 1) + 1);
+                }
+                for (int j = 0; j < len; ++j) score = __dadd_rn(score, wd);
+                cnt += len;
+                idx = cnt - 1;
+                if (in) { k += len; par_idx = idx; }
+            } else {
+                const int ct = __shfl_sync(FULL, ctok, first);
+                if (lane == 0) { W.tok[buf][cnt] = ct; W.par[buf][cnt] = (unsigned char)(idx + 1); }
+                score = __dadd_rn(score, wd);
+                idx = cnt++;
+                if (in) { ++k; par_idx = idx; }
+            }
+        }
+        if (dropped) break;
+        // the final SCORE of this job is at least its running value: let the others prune on it
+        if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
+    }
+    __syncwarp();
+    if (!dropped && (score > W.best_score || (score == W.best_score && score > 0.0 && order < W.best_order))) {
+        if (lane == 0) {
+            W.best_score = score; W.best_order = order; W.best_n = cnt; W.best_buf = buf;
+            atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
+        }
+    }
+    __syncwarp();
+}
+
+// ---------------------------------------------------------------------------------------------
+// A per-request job whose match node has more than 32 occurrences (list[0 .. m): positions of the
+// pattern's last token).  A node below N_p is named by one of its occurrences and its depth:
+// (rep, k) stands for the string tx[rep + 1 .. rep + k].  Its children come from a pass over the
+// list: the occurrences that agree with rep on k tokens are its members, and a hash table of
+// 128 cells in shared memory counts their next tokens.  The members' tokens are taken a part
+// at a time (by bits of a hash of the token) when the table cannot hold them all.  Frontier:
+// the sorted ring of the tree-entry path; fields cb / nc hold rep / k.
+template <class BlockShared>
+__device__ void expand_wide_text(BlockShared& sh, WarpWork& W, const int* tx, int t, const int* list, int m, int p,
+                                 int budget, int dlim, unsigned flags, int lane) {
+    const int order = SD_MAX_DEPTH + p;
+    const int buf = W.best_buf ^ 1;
+    int* const hkey = reinterpret_cast<int*>(&W.T);             // 128 cells: token, count, an occurrence
+    int* const hcnt = hkey + 128;
+    int* const hrep = hkey + 256;
+    Frontier& F = W.F;
+    int fh = 0, fs = 0, cnt = 0;
+    double score = 0.0;
+    bool dropped = false;
+    double cur_d = 1.0;
+    int cur_rep = 0, cur_k = 0, cur_idx = -1;
+    bool have_cur = true;
+    while (true) {
+        if (!have_cur) {
+            if (cnt >= budget || fs == 0) break;
+            cur_d = F.d[fh];
+            const int tok = F.tok[fh], par = F.par[fh];
+            cur_rep = F.cb[fh];
+            cur_k = (int)F.nc[fh];
+            if ((score + (double)(budget - cnt) * cur_d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
+            __syncwarp();
+            fh = (fh + 1) & (SD_MAX_SPEC - 1);
+            --fs;
+            if (lane == 0) { W.tok[buf][cnt] = tok; W.par[buf][cnt] = (unsigned char)(par + 1); }
+            score = __dadd_rn(score, cur_d);
+            if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
+            cur_idx = cnt++;
+            const int K = budget - cnt;
+            if (fs > K) fs = K;
+            if (flags & SD_FLAG_LINEAR) fs = 0;
+        }
+        have_cur = false;
+        if (cnt >= budget) break;
+        if (cur_k >= dlim) continue;                            // depth cap: the node has no children
+        const int K = budget - cnt;
+        // parts of the token space still to do: (pre, nb) = tokens whose hash ends in the nb bits `pre`
+        unsigned st_pre[34];
+        int st_nb[34];
+        int sp = 0;
+        st_pre[0] = 0u; st_nb[0] = 0; sp = 1;
+        for (int guard = 0; sp > 0 && guard < 100000; ++guard) {
+            --sp;
+            const unsigned pre = st_pre[sp];
+            const int nb = st_nb[sp];
+            const unsigned pmask = nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u);
+            for (int q = lane; q < 128; q += 32) { hkey[q] = -1; hcnt[q] = 0; }
+            __syncwarp();
+            int sum = 0;
+            bool ovf = false;
+            for (int base = 0; base < m; base += 32) {
+                const int q = base + lane;
+                bool member = false;
+                int c = 0, e = 0;
+                if (q < m) {
+                    e = list[q];
+                    member = e + cur_k + 1 <= t - 1;
+                    for (int i = 1; member && i <= cur_k; ++i) member = tx[e + i] == tx[cur_rep + i];
+                    if (member) c = tx[e + cur_k + 1];
+                }
+                sum += __popc(__ballot_sync(FULL, member));
+                const unsigned h = (unsigned)c * 2654435761u;
+                const bool mine = member && (h & pmask) == pre;
+                const unsigned mm = __ballot_sync(FULL, mine);
+                if (mine) {
+                    const unsigned grp = __match_any_sync(mm, c);
+                    if (lane == __ffs(grp) - 1) {
+                        int cell = (int)(((unsigned)c * 0x85EBCA6Bu) >> 25);
+                        bool done = false;
+                        for (int pr = 0; pr < 128 && !done; ++pr) {
+                            const int old = atomicCAS(&hkey[cell], -1, c);
+                            if (old == -1) hrep[cell] = e;
+                            if (old == -1 || old == c) { atomicAdd(&hcnt[cell], __popc(grp)); done = true; }
+                            else cell = (cell + 1) & 127;
+                        }
+                        if (!done) ovf = true;
+                    }
+                }
+                __syncwarp();
+            }
+            if (__any_sync(FULL, ovf) && nb < 32) {             // too many different tokens: split the part
+                st_pre[sp] = pre | (1u << nb); st_nb[sp] = nb + 1; ++sp;
+                st_pre[sp] = pre; st_nb[sp] = nb + 1; ++sp;
+                continue;
+            }
+            const double dsum = (double)sum;                    // denominator of Eq. 1: members with a next token
+            for (int q0 = 0; q0 < 128; q0 += 32) {
+                const int c = hkey[q0 + lane];
+                const bool pass = c >= 0;
+                double dc = 0.0;
+                int rep = 0;
+                if (pass) { dc = __dmul_rn(cur_d, __ddiv_rn((double)hcnt[q0 + lane], dsum)); rep = hrep[q0 + lane]; }
+                unsigned pm = __ballot_sync(FULL, pass);
+                while (pm) {
+                    const int src = __ffs(pm) - 1;
+                    pm &= pm - 1;
+                    frontier_insert(F, fh, fs, K, __shfl_sync(FULL, dc, src), __shfl_sync(FULL, c, src), cur_idx,
+                                    __shfl_sync(FULL, rep, src), (unsigned)(cur_k + 1), lane);
+                }
+            }
+            __syncwarp();
+        }
+    }
+    __syncwarp();
+    if (!dropped && (score > W.best_score || (score == W.best_score && score > 0.0 && order < W.best_order))) {
+        if (lane == 0) {
+            W.best_score = score; W.best_order = order; W.best_n = cnt; W.best_buf = buf;
+            atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
+        }
+    }
+    __syncwarp();
+}
+
+struct StepArgs {             // what one launch needs beyond the store
+    int n;
+    const int32_t* d_slot;
+    int Pe;
+    double alpha;
+    int max_spec;
+    unsigned flags;
+    double tau;
+    const int32_t* d_budget_cap;
+    int32_t *d_n_draft, *d_tokens, *d_parents, *d_positions;
+    uint32_t* d_mask;
+    int32_t *d_chosen_tree, *d_chosen_p;
+    double* d_score;
+    int32_t* d_status;
+    const int64_t* d_app_off;     // sd_step: the tokens to append first (NULL: sd_speculate)
+    const int32_t* d_app_tok;
+    int stage_tokens;             // tokens of text the block can hold in shared memory (longer texts are read in place)
+    int32_t* occ_scratch;         // [n][Tp] by request: occurrence lists longer than OCC_CAP
+};
+
+template <int WARPS, int MINB>
+__global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_store sv, StepArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using BlockShared = BlockSharedT<WARPS>;
-    constexpr int CTA_WARPS = WARPS;
+    constexpr int NT = WARPS * 32;
     BlockShared& sh = *reinterpret_cast<BlockShared*>(smem_raw);
+    int* const stx = reinterpret_cast<int*>(smem_raw + ((sizeof(BlockShared) + 15) & ~(size_t)15));
     const int tid = threadIdx.x, lane = tid & 31, wib = tid >> 5;
     const int i = blockIdx.x;
-    const int M = sv.M, words = (M + 31) / 32;
-    const int slot = d_slot[i];
+    const int M = sv.M, words = (M + 31) / 32, D = sv.D, Pe = a.Pe;
+    const unsigned flags = a.flags;
+    const int slot = a.d_slot[i];
     const bool ok = slot >= 0 && slot < sv.R;
     int t = 0, status = SD_STATUS_BAD_SLOT;
     SlotState* ss = nullptr;
-    if (ok) { ss = sv.s_state + slot; t = ss->len; status = ss->status; }
-    // STEP: t_old tokens are in the slot's text, the next n_new come from the append list; the
-    // match below already runs on the context of t = t_old + n_new tokens
+    int32_t* gtext = nullptr;
+    if (ok) { ss = sv.s_state + slot; t = ss->len; status = ss->status; gtext = sv.s_text + (long long)slot * sv.Tp; }
     const int t_old = t;
-    const int32_t* newtok = nullptr;
-    int n_new = 0;
-    if (STEP && ok) {
-        newtok = d_app_tok + d_app_off[i];
-        n_new = (int)(d_app_off[i + 1] - d_app_off[i]);
-        t = t_old + n_new;
-    }
-    bool usable = ok && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && t > 0;
-    int cap = max_spec;
-    if (d_budget_cap && d_budget_cap[i] >= 0) cap = min(cap, d_budget_cap[i]);
     if (tid < 2 * SD_MAX_DEPTH) { (&sh.node[0][0])[tid] = -1; (&sh.nc[0][0])[tid] = 0; }
-    if (tid == 0) { sh.njobs = 0; sh.next = 0; sh.nwide = 0; sh.nwide_kept = 0; sh.best_hi = 0u; sh.win_warp = -1; }
+    if (tid < SD_MAX_DEPTH + 2) { sh.r_hist[tid] = 0; sh.r_cum[tid] = 0; sh.r_fill[tid] = 0; sh.g_cum[tid] = 0; }
+    if (tid < SD_MAX_DEPTH) { sh.g_cnt[tid] = 0; sh.g_rank[tid] = -1; }
+    if (tid == 0) {
+        sh.njobs = 0; sh.next = 0; sh.nwide = 0; sh.nwide_kept = 0; sh.best_hi = 0u; sh.win_warp = -1;
+        sh.first_bad = 0x7fffffff; sh.scan_next[0] = 0; sh.scan_next[1] = 0;
+        sh.g_walked = 0; sh.g_failed = 0; sh.g_base_p = 0; sh.g_base_m = 0;
+    }
     WarpWork& W = sh.w[wib];
     if (lane == 0) { W.best_score = 0.0; W.best_order = 1 << 30; W.best_n = 0; W.best_buf = 0; }
+    __syncthreads();
 
-    // ---------------- 1. match
-    bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
-    bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
-    // warps that advance the global match nodes, and this warp's rank among them
-    const int mwarps = STEP ? CTA_WARPS - 1 : CTA_WARPS;
-    const int mrank = STEP ? wib - 1 : wib;
-    constexpr int MROUNDS = STEP ? (SD_MAX_DEPTH + CTA_WARPS - 2) / (CTA_WARPS - 1)
-                                 : (SD_MAX_DEPTH + CTA_WARPS - 1) / CTA_WARPS;   // pattern lengths per warp
-    int src_node[MROUNDS], src_from[MROUNDS];                   // per target: start node and first text index
-#pragma unroll
-    for (int h = 0; h < MROUNDS; ++h) { src_node[h] = -1; src_from[h] = 0; }
-    const int32_t* text = ok ? sv.s_text + (long long)slot * sv.T : nullptr;
-    if (want_g && mrank >= 0) {
-        const bool cache_ok = ss->g_gen == ss->gen && ss->g_epoch == sv.g_state->epoch && ss->g_len <= t;
-        const int k = t - ss->g_len;                            // tokens appended since the cache was taken
-        const int depths = ss->g_depths;
-#pragma unroll
-        for (int h = 0; h < MROUNDS; ++h) {
-            const int d = mrank + 1 + h * mwarps;               // target pattern length
-            if (d > Pe || d > t) continue;
-            if (cache_ok && d > k && d - k <= depths) {
-                src_node[h] = ss->g_node[d - k - 1];            // node of the tokens before the new ones
-                src_from[h] = t - k;
-            } else {
-                const int x0 = t - d < t_old ? text[t - d] : newtok[t - d - t_old];
-                src_node[h] = (x0 >= 0 && x0 < sv.V) ? sv.g_root[x0] : -1;
-                src_from[h] = t - d + 1;
+    // ---------------- 0. sd_step: the accepted tokens go behind the request's text
+    const int32_t* newtok = nullptr;
+    int take = 0;
+    if (a.d_app_off && ok) {
+        const long long b0 = a.d_app_off[i];
+        const int n_new = (int)(a.d_app_off[i + 1] - b0);
+        newtok = a.d_app_tok + b0;
+        if (n_new > 0 && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN))) {
+            take = min(n_new, sv.T - t_old);
+            for (int k = tid; k < take; k += NT) {
+                const int x = newtok[k];
+                if (x < 0 || x >= sv.V) atomicMin(&sh.first_bad, k);
             }
+            __syncthreads();
+            const int good = min(take, sh.first_bad);
+            if (good < take) status |= SD_STATUS_BAD_TOKEN;     // the text stops before the first bad token
+            else if (take < n_new) status |= SD_STATUS_POOL_FULL;
+            take = good;
+            for (int k = tid; k < take; k += NT) gtext[t_old + k] = newtok[k];
+            t = t_old + take;
+            if (tid == 0) { ss->len = t; ss->status = status; }
         }
     }
-    __syncthreads();                                            // all cached nodes read before any is replaced
-    if (STEP && wib == 0 && ok && n_new > 0) {
-        // ---- the request's accepted tokens go into its tree and text (as sd_append does)
-        int32_t* wtext = sv.s_text + (long long)slot * sv.T;
-        TreeRef tr{sv.s_ent + (long long)slot * sv.spn, sv.s_root + (long long)slot * sv.V, (int)sv.spn};
-        int len = ss->len, used = ss->used, live = ss->live, st = ss->status;
-        int act = ss->active[lane], room = ss->room[lane], run_cb = ss->run_cb[lane];
-        unsigned run_w = ss->run_w[lane];
-        for (int k = 0; k < n_new && !(st & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)); ++k) {
-            const int x = newtok[k];
-            if (x < 0 || x >= sv.V) { st |= SD_STATUS_BAD_TOKEN; break; }
-            if (len >= sv.T || !append_token<APPEND_G>(tr, sv.D, x, len, lane, act, room, run_cb, run_w, used, live)) {
-                st |= SD_STATUS_POOL_FULL;
-                break;
-            }
-            if (lane == 0) wtext[len] = x;
-            ++len;
-        }
-        ss->active[lane] = act; ss->room[lane] = room; ss->run_cb[lane] = run_cb; ss->run_w[lane] = run_w;
-        if (lane == 0) { ss->len = len; ss->used = used; ss->live = live; ss->status = st; }
-    }
-    if (want_g && mrank >= 0) {
+    const bool usable = ok && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && t > 0;
+    int cap = a.max_spec;
+    if (a.d_budget_cap && a.d_budget_cap[i] >= 0) cap = min(cap, a.d_budget_cap[i]);
+    const bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
+    const bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
+
+    // ---------------- 1. the text
+    const int* tx = stx;
+    if (usable) {
+        if (t <= a.stage_tokens) {
+            const int4* g4 = reinterpret_cast<const int4*>(gtext);
+            int4* s4 = reinterpret_cast<int4*>(stx);
+            for (int g = tid; g * 4 < t; g += NT) {
+                int4 v = make_int4(0, 0, 0, 0);
+                if (g * 4 < t_old) v = g4[g];
+                // (the new tokens come from the call's list: the copy in the text buffer above may not have landed yet)
+                int* c = reinterpret_cast<int*>(&v);
 #pragma unroll
-        for (int h = 0; h < MROUNDS; ++h) {
-            const int d = mrank + 1 + h * mwarps;
-            if (d > Pe) continue;
-            int cb = 0;
+                for (int u = 0; u < 4; ++u) { const int q = g * 4 + u; if (q >= t_old && q < t) c[u] = newtok[q - t_old]; }
+                s4[g] = v;
+            }
+        } else {
+            tx = gtext;                                         // too long to stage: read in place
+        }
+    }
+    __syncthreads();                                            // (also: the new tokens in gtext are visible to the block)
+
+    // ---------------- 2. match
+    const int Lcap = min(Pe, D - 1);                            // a match node at depth D has no children
+    const int last = usable ? tx[t - 1] : 0;
+    const bool scan = want_r && t >= 2 && Lcap >= 1;
+    // one chunk of positions at a time, handed out by a counter: warps that come late from their
+    // walk in the global tree take fewer.  pass 0 counts the occurrences by match length,
+    // pass 1 (below) writes them, longest matches first.
+    const int nchunks = scan ? (t - 1 + 255) / 256 : 0;
+    auto scan_pass = [&](int pass, int* list) {
+        while (true) {
+            int c = 0;
+            if (lane == 0) c = atomicAdd(&sh.scan_next[pass], 1);
+            c = __shfl_sync(FULL, c, 0);
+            if (c >= nchunks) break;
+#pragma unroll 1
+            for (int u = 0; u < 8; ++u) {
+                const int e = c * 256 + u * 32 + lane;
+                if (e < t - 1 && tx[e] == last) {
+                    int l = 1;
+                    while (l < Lcap && e - l >= 0 && tx[e - l] == tx[t - 1 - l]) ++l;
+                    if (pass == 0) atomicAdd(&sh.r_hist[l], 1);
+                    else list[sh.r_cum[l + 1] + atomicAdd(&sh.r_fill[l], 1)] = e;
+                }
+            }
+        }
+    };
+    // Global tree: rounds of WARPS pattern lengths, shortest first, until a node can serve as
+    // the base of occurrence mode, a pattern does not occur, or all lengths are done.
+    const int PeG = want_g ? min(Pe, t) : 0;
+    const bool occ_mode = sv.g_lo != nullptr;
+    for (int r0 = 0; r0 < PeG; r0 += WARPS) {
+        const int p = r0 + wib + 1;
+        if (p <= PeG) {
+            int cb = 0, cntn = 0;
             unsigned wf = 0;
-            const int node = (d > t) ? -1 : walk_from(sv.g_ent, (int)sv.g_cap, src_node[h], text, t_old, newtok, src_from[h], t,
-                                                      lane, cb, wf);
+            const int node = walk_root(sv.g_ent, (int)sv.g_cap, sv.g_root, sv.V, tx, t, p, lane, cb, wf, cntn);
+            int rank = -1;
+            const int nch = (int)(wf & RUN_COUNT_MASK);
+            // usable as base: at most 32 occurrences, laid down by the offline build, never touched since
+            const bool elig = occ_mode && node >= 0 && cntn <= SD_OCC_LANES && !(wf & NODE_TOUCHED) &&
+                              (nch == 0 || ((wf & RUN_STATIC) && cb < sv.static_entries));
+            if (elig && nch > 0 && lane == 0) rank = sv.g_lo[cb];
             if (lane == 0) {
-                ss->g_node[d - 1] = node;
-                sh.node[0][d - 1] = node;
-                if (node >= 0) { sh.cb[0][d - 1] = cb; sh.nc[0][d - 1] = wf; }
+                sh.node[0][p - 1] = node;
+                if (node >= 0) { sh.cb[0][p - 1] = cb; sh.nc[0][p - 1] = wf; sh.g_cnt[p - 1] = cntn; }
+                else atomicOr(&sh.g_failed, 1);
+                sh.g_rank[p - 1] = elig ? (nch > 0 ? rank : -2) : -1;   // -2: usable, and known to have no children
             }
         }
-        if (tid == (STEP ? 32 : 0)) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = Pe; }
+        if (r0 == 0 && scan) scan_pass(0, nullptr);
+        __syncthreads();
+        if (tid == 0) {
+            const int hi = min(PeG, r0 + WARPS);
+            sh.g_walked = hi;
+            for (int p = r0 + 1; p <= hi && sh.g_base_p == 0; ++p)
+                if (sh.node[0][p - 1] >= 0 && sh.g_rank[p - 1] != -1) sh.g_base_p = p;
+        }
+        __syncthreads();
+        if (sh.g_base_p || sh.g_failed) break;
     }
-    if (STEP) {
-        __syncthreads();                                        // the append is done and visible
-        if (ok) {
-            status = ss->status;
-            if (ss->len != t || (status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN))) {
-                // the append stopped early: no speculation for this request, and the match nodes
-                // taken above describe a context that does not exist
-                usable = false; want_g = false; want_r = false;
-                t = ss->len;
-                if (tid == 0) ss->g_gen = ss->gen - 1;
-                if (tid < 2 * SD_MAX_DEPTH) { (&sh.node[0][0])[tid] = -1; (&sh.nc[0][0])[tid] = 0; }
-            }
+    if (PeG == 0 && scan) scan_pass(0, nullptr);
+    __syncthreads();
+    // occurrences by match length -> r_cum; the base's occurrences (first pattern token, suffix length)
+    const int base_p = sh.g_base_p;
+    if (wib == 0) {
+        int h = (lane + 1 <= Lcap) ? sh.r_hist[lane + 1] : 0;   // lane L: matches of exactly L + 1 tokens
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {                      // suffix sums
+            const int y = __shfl_down_sync(FULL, h, o);
+            if (lane + o < 32) h += y;
         }
+        sh.r_cum[lane + 1] = h;
+    } else if (wib == 1 && base_p > 0) {
+        const int rank = sh.g_rank[base_p - 1];
+        const int m = rank >= 0 ? sh.g_cnt[base_p - 1] : 0;
+        if (lane < m) {
+            const int pos = (int)sv.g_sa[rank + lane];
+            sh.g_pos[lane] = pos;
+            sh.g_avail[lane] = (int)sv.g_len[rank + lane] - base_p;
+            sh.g_ell[lane] = (int)sv.g_back[pos];               // for now: tokens before the occurrence in its sequence
+        }
+        if (lane == 0) sh.g_base_m = m;
     }
-    if (want_r && wib == CTA_WARPS - 1) {
-        const int d = lane + 1;
-        if (d <= Pe && d <= t) {
-            const int node = ss->active[d - 1];
-            int rcb = ss->run_cb[d - 1];
-            unsigned rw = ss->run_w[d - 1];                      // kept current by sd_append
-            if (rw == RUN_UNKNOWN) {
-                const int4 e = (sv.s_ent + (long long)slot * sv.spn)[node];
-                rcb = e.z; rw = (unsigned)e.w;
-            }
-            sh.node[1][d - 1] = node; sh.cb[1][d - 1] = rcb; sh.nc[1][d - 1] = rw;
+    __syncthreads();
+    const int m1 = sh.r_cum[1];
+    int* const occ_list = m1 <= OCC_CAP ? sh.occ : a.occ_scratch + (long long)i * sv.Tp;
+    const int base_m = sh.g_base_m;
+    // the 64 tokens around every occurrence of the base (one coalesced row per occurrence), then the scan's second pass
+    for (int o = wib; o < base_m; o += WARPS) {
+        const long long pos = sh.g_pos[o];
+        const long long q0 = pos - 32 + lane, q1 = pos + lane;
+        sh.gwin[o][lane] = (q0 >= 0) ? sv.g_text[q0] : -1;
+        sh.gwin[o][32 + lane] = (q1 < sv.N0) ? sv.g_text[q1] : -1;
+    }
+    if (scan && m1 > 0) scan_pass(1, occ_list);
+    __syncthreads();
+    if (wib == 0 && base_m > 0) {
+        // how far back every occurrence of the base agrees with the context
+        int ell = 0;
+        if (lane < base_m) {
+            const int back = sh.g_ell[lane];
+            const int lim = min(Lcap, t);
+            ell = base_p;
+            while (ell < lim && ell - base_p < back && sh.gwin[lane][31 - (ell - base_p)] == tx[t - 1 - ell]) ++ell;
+            sh.g_ell[lane] = ell;
         }
+        // lane L: occurrences that match at least L + 1 tokens
+        int c = 0;
+        for (int o = 0; o < base_m; ++o) c += (__shfl_sync(FULL, ell, o) >= lane + 1) ? 1 : 0;
+        sh.g_cum[lane + 1] = lane + 1 >= base_p ? c : 0;
     }
     __syncthreads();
 
-    // ---------------- 2. job queue, costliest first; jobs that start at a wide node wait
+    // ---------------- 3. job queue, costliest first; tree-entry jobs that start at a wide node wait
     if (tid < 2 * SD_MAX_DEPTH) {
         const int tree = tid / SD_MAX_DEPTH, p = tid % SD_MAX_DEPTH + 1;
         int c = 0;
-        const unsigned wf = sh.nc[tree][p - 1];
-        const int nch = (int)(wf & RUN_COUNT_MASK);
-        if (p <= Pe && sh.node[tree][p - 1] >= 0 && nch > 0) {
-            // all first runs start their way to L2 now, long before a warp gets to them
-            const int4* base = (tree == 0 ? sv.g_ent : sv.s_ent + (long long)slot * sv.spn) + sh.cb[tree][p - 1];
-            const int lines = min(4, (nch + 7) >> 3);
-            for (int l = 0; l < lines; ++l) prefetch_l2(base + l * 8);
-            c = min(budget_for(alpha, p, cap), 2 * (sv.D - p));
-            if (c > 0 && nch > WIDE_RUN && !(wf & RUN_HAS_TOP)) { sh.wide[atomicAdd(&sh.nwide, 1)] = tid; c = 0; }
+        if (p <= Pe && p <= Lcap) {
+            bool has = false;
+            if (tree == 1) has = want_r && sh.r_cum[p] > 0;
+            else if (base_p > 0 && p >= base_p) has = sh.g_cum[p] > 0;
+            else if (p <= sh.g_walked) {
+                const unsigned wf = sh.nc[0][p - 1];
+                const int nch = (int)(wf & RUN_COUNT_MASK);
+                has = sh.node[0][p - 1] >= 0 && nch > 0;
+                if (has) {
+                    // all first runs start their way to L2 now, long before a warp gets to them
+                    const int4* base = sv.g_ent + sh.cb[0][p - 1];
+                    const int lines = min(4, (nch + 7) >> 3);
+                    for (int l = 0; l < lines; ++l) prefetch_l2(base + l * 8);
+                }
+            }
+            if (has) {
+                c = min(budget_for(a.alpha, p, cap), 2 * (D - p));
+                if (c > 0 && tree == 0 && !(base_p > 0 && p >= base_p)) {
+                    const unsigned wf = sh.nc[0][p - 1];
+                    if ((int)(wf & RUN_COUNT_MASK) > WIDE_RUN && !(wf & RUN_HAS_TOP)) { sh.wide[atomicAdd(&sh.nwide, 1)] = tid; c = 0; }
+                }
+            }
         }
         sh.cost[tid] = c;
     }
@@ -990,7 +1131,6 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     }
     __syncthreads();
     const int njobs = sh.njobs;
-    const int4* s_ent = ok ? sv.s_ent + (long long)slot * sv.spn : nullptr;
     while (true) {
         int j = 0;
         if (lane == 0) j = atomicAdd(&sh.next, 1);
@@ -998,40 +1138,52 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
         if (j >= njobs) break;
         const int code = sh.job[j];
         const int tree = code / SD_MAX_DEPTH, p = code % SD_MAX_DEPTH + 1;
-        const int budget = budget_for(alpha, p, cap);
+        const int budget = budget_for(a.alpha, p, cap);
         if ((double)budget < best_so_far(sh)) continue;         // SCORE <= number of draft nodes
-        expand_job(sh, W, tree == 0 ? sv.g_ent : s_ent, tree == 0 ? (int)sv.g_cap : (int)sv.spn, tree, p, budget, flags,
-                   false, 0, lane);
+        if (tree == 1) {
+            const int m = sh.r_cum[p];
+            if (m <= SD_OCC_LANES) {
+                const int e = lane < m ? occ_list[lane] : 0;
+                const int kmax = lane < m ? min(t - 1 - e, D - p) : 0;
+                expand_occ(sh, W, tx + e, kmax, 1, p, budget, flags, lane);
+            } else {
+                expand_wide_text(sh, W, tx, t, occ_list, m, p, budget, D - p, flags, lane);
+            }
+        } else if (base_p > 0 && p >= base_p) {
+            const bool mine = lane < base_m && sh.g_ell[lane] >= p;
+            const int kmax = mine ? min(sh.g_avail[lane], D - p) : 0;
+            expand_occ(sh, W, &sh.gwin[lane][31 + base_p], kmax, 0, p, budget, flags, lane);
+        } else {
+            expand_job(sh, W, sv.g_ent, (int)sv.g_cap, 0, p, budget, flags, false, 0, lane);
+        }
     }
     __syncthreads();
-    // Jobs that start at a wide node (short patterns, hence small budgets): most cannot reach
-    // the best score any more and are dropped here.  For the rest the warps of the block share
+    // Tree-entry jobs that start at a wide node (short patterns, hence small budgets): most cannot
+    // reach the best score any more and are dropped here.  For the rest the warps of the block share
     // the scan of the run, then one warp merges the partial lists and finishes the job.
     if (tid == 0) {
         const double best = __hiloint2double((int)sh.best_hi, 0);
         int kept = 0;
         for (int q = 0; q < sh.nwide; ++q) {
             const int p = sh.wide[q] % SD_MAX_DEPTH + 1;
-            if (!((double)budget_for(alpha, p, cap) < best)) sh.wide[kept++] = sh.wide[q];
+            if (!((double)budget_for(a.alpha, p, cap) < best)) sh.wide[kept++] = sh.wide[q];
         }
         sh.nwide_kept = kept;
     }
     __syncthreads();
     const int nwide = sh.nwide_kept;
-    for (int base = 0; base < nwide; base += CTA_WARPS) {
-        const int nj = min(CTA_WARPS, nwide - base);
-        const int G = CTA_WARPS / nj;                           // warps per job
+    for (int base = 0; base < nwide; base += WARPS) {
+        const int nj = min(WARPS, nwide - base);
+        const int G = WARPS / nj;                               // warps per job
         const int my_job = wib / G, my_slice = wib % G;
         const bool active = my_job < nj;
-        int tree = 0, p = 1, budget = 0, fs = 0;
-        const int4* ent = sv.g_ent;
+        int p = 1, budget = 0, fs = 0;
         if (active) {
             const int code = sh.wide[base + my_job];
-            tree = code / SD_MAX_DEPTH; p = code % SD_MAX_DEPTH + 1;
-            budget = budget_for(alpha, p, cap);
-            ent = tree == 0 ? sv.g_ent : s_ent;
+            p = code % SD_MAX_DEPTH + 1;
+            budget = budget_for(a.alpha, p, cap);
             long long sum;
-            scan_run_by_count(ent, sh.cb[tree][p - 1], (int)(sh.nc[tree][p - 1] & RUN_COUNT_MASK), my_slice, G, -1, 1, W,
+            scan_run_by_count(sv.g_ent, sh.cb[0][p - 1], (int)(sh.nc[0][p - 1] & RUN_COUNT_MASK), my_slice, G, -1, 1, W,
                               W.F, 0, fs, budget, sum, lane);
             if (lane == 0) { sh.slice_sum[wib] = sum; sh.slice_fs[wib] = fs; }
         }
@@ -1045,15 +1197,15 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
                 frontier_merge_list(W.F, 0, fs, budget, O, ofs, -1, lane);
             }
             counts_to_d(W.F, 0, fs, 1.0, sum, lane);
-            expand_job(sh, W, ent, tree == 0 ? (int)sv.g_cap : (int)sv.spn, tree, p, budget, flags, true, fs, lane);
+            expand_job(sh, W, sv.g_ent, (int)sv.g_cap, 0, p, budget, flags, true, fs, lane);
         }
         __syncthreads();
     }
 
-    // ---------------- 3. select (first in loop order among the largest scores) and emit
+    // ---------------- 4. select (first in loop order among the largest scores) and emit
     if (wib == 0) {
-        double sc = lane < CTA_WARPS ? sh.w[lane].best_score : 0.0;
-        int od = lane < CTA_WARPS ? sh.w[lane].best_order : 1 << 30;
+        double sc = lane < WARPS ? sh.w[lane].best_score : 0.0;
+        int od = lane < WARPS ? sh.w[lane].best_order : 1 << 30;
         int ww = lane;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
@@ -1062,7 +1214,8 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
             const int oww = __shfl_xor_sync(FULL, ww, off);
             if (osc > sc || (osc == sc && ood < od)) { sc = osc; od = ood; ww = oww; }
         }
-        if (lane == 0) sh.win_warp = sc > 0.0 ? ww : -1;
+        // Section 3.2: the tree is used only if its score exceeds the threshold (tau = 0: any score above 0)
+        if (lane == 0) sh.win_warp = (sc > 0.0 && sc > a.tau) ? ww : -1;
     }
     __syncthreads();
     const int win = sh.win_warp;
@@ -1077,105 +1230,129 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
         if (cp == 0) { cp = SD_MAX_DEPTH; ctree -= 1; }          // order = tree * 32 + p with p in 1..32
         wtok = B.tok[B.best_buf]; wpar = B.par[B.best_buf];
     }
-    if (tid < M) {
-        const int j = tid;
+    for (int j = tid; j < M; j += NT) {
         int tok = -1, par = -1, pos = -1;
         unsigned long long bits = 0;
         if (j < nd) {
             tok = wtok[j];
             par = (int)wpar[j] - 1;
             int depth = 0;
-            for (int a = j, hops = 0; a >= 0 && hops < SD_MAX_SPEC; a = (int)wpar[a] - 1, ++hops) {
-                bits |= 1ull << a;
+            for (int an = j, hops = 0; an >= 0 && hops < SD_MAX_SPEC; an = (int)wpar[an] - 1, ++hops) {
+                bits |= 1ull << an;
                 ++depth;
             }
             pos = t + depth - 1;
         }
         const long long o = (long long)i * M + j;
-        d_tokens[o] = tok; d_parents[o] = par; d_positions[o] = pos;
-        d_mask[o * words] = (uint32_t)bits;
-        if (words > 1) d_mask[o * words + 1] = (uint32_t)(bits >> 32);
+        a.d_tokens[o] = tok; a.d_parents[o] = par; a.d_positions[o] = pos;
+        a.d_mask[o * words] = (uint32_t)bits;
+        if (words > 1) a.d_mask[o * words + 1] = (uint32_t)(bits >> 32);
     }
     if (tid == 0) {
-        d_n_draft[i] = nd; d_chosen_tree[i] = ctree; d_chosen_p[i] = cp; d_score[i] = best;
-        if (d_status) d_status[i] = status;
+        a.d_n_draft[i] = nd; a.d_chosen_tree[i] = ctree; a.d_chosen_p[i] = cp; a.d_score[i] = best;
+        if (a.d_status) a.d_status[i] = status;
     }
 }
 
 }  // namespace
 
-static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
-                        const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents,
-                        int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
-                        double* d_score, int32_t* d_status, const int64_t* d_app_off, const int32_t* d_app_tok,
-                        bool step, void* stream) {
+// ---------------------------------------------------------------------------------------------
+// Launch.  Block shapes (measured): two blocks per SM is the usual one; a batch of at most one
+// request per SM gets bigger blocks, a batch of more than two requests per SM smaller ones
+// (four per SM) to stay in one wave.  The text of a request is staged in shared memory when it
+// fits beside the block's working set, else it is read in place.
+namespace {
+
+constexpr int CTA_WARPS = 10;
+constexpr int CTA_WARPS_WIDE = 16;
+constexpr int CTA_WARPS_NARROW = 5;
+constexpr int SMEM_PER_SM = 228 * 1024;       // shared memory of one SM; a block also costs 1 KB of it
+constexpr int MAX_DEVICES = 64;
+
+struct DeviceInfo {
+    bool ready = false;
+    int sm_count = 0;
+};
+DeviceInfo g_dev[MAX_DEVICES];
+std::mutex g_dev_mutex;
+
+template <int WARPS, int MINB>
+constexpr int stage_limit_tokens() {
+    return (int)((SMEM_PER_SM / MINB - 1024 - (int)((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15)) / 4) & ~3;
+}
+
+// once per device: raise the kernels' dynamic shared memory limit, read the SM count
+int device_setup(int dev, int* sm_count) {
+    if (dev < 0 || dev >= MAX_DEVICES) return SD_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (!g_dev[dev].ready) {
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<CTA_WARPS, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        SMEM_PER_SM / 2 - 1024));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<CTA_WARPS_WIDE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        SMEM_PER_SM - 1024));
+        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<CTA_WARPS_NARROW, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        SMEM_PER_SM / 4 - 1024));
+        SD_CUDA_OK(cudaDeviceGetAttribute(&g_dev[dev].sm_count, cudaDevAttrMultiProcessorCount, dev));
+        g_dev[dev].ready = true;
+    }
+    *sm_count = g_dev[dev].sm_count;
+    return SD_OK;
+}
+
+template <int WARPS, int MINB>
+void launch_shape(const sd_store& s, StepArgs a, cudaStream_t st) {
+    const int lim = stage_limit_tokens<WARPS, MINB>();
+    a.stage_tokens = s.Tp <= lim ? s.Tp : 0;
+    const size_t smem = ((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15) + (size_t)a.stage_tokens * 4;
+    speculate_fused_kernel<WARPS, MINB><<<(unsigned)a.n, WARPS * 32, smem, st>>>(s, a);
+}
+
+int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm, const int32_t* d_budget_cap,
+                 int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask,
+                 int32_t* d_chosen_tree, int32_t* d_chosen_p, double* d_score, int32_t* d_status,
+                 const int64_t* d_app_off, const int32_t* d_app_tok, bool step, int32_t* scratch, void* stream) {
     if (!s || !prm || n < 0 || n > s->R) return SD_ERR_INVALID_ARG;
-    if (prm->P < 1 || prm->max_spec < 0 || prm->max_spec > s->M || !(prm->alpha >= 0.0)) return SD_ERR_INVALID_ARG;
+    if (prm->P < 1 || prm->max_spec < 0 || prm->max_spec > s->M || !(prm->alpha >= 0.0) || !(prm->tau >= 0.0))
+        return SD_ERR_INVALID_ARG;
     if ((prm->flags & SD_FLAG_GLOBAL_ONLY) && (prm->flags & SD_FLAG_REQUEST_ONLY)) return SD_ERR_INVALID_ARG;
+    SD_CHECK_DEVICE(s);
     if (n == 0) return SD_OK;
     if (!d_slot || !d_n_draft || !d_tokens || !d_parents || !d_positions || !d_mask || !d_chosen_tree || !d_chosen_p ||
         !d_score)
         return SD_ERR_INVALID_ARG;
     if (step && !d_app_off) return SD_ERR_INVALID_ARG;
+    int sms = 0;
+    const int rc = device_setup(s->device, &sms);
+    if (rc != SD_OK) return rc;
+    StepArgs a;
+    a.n = n; a.d_slot = d_slot;
+    a.Pe = prm->P < s->D ? prm->P : s->D;                       // longer patterns never match
+    a.alpha = prm->alpha; a.max_spec = prm->max_spec; a.flags = prm->flags; a.tau = prm->tau;
+    a.d_budget_cap = d_budget_cap;
+    a.d_n_draft = d_n_draft; a.d_tokens = d_tokens; a.d_parents = d_parents; a.d_positions = d_positions;
+    a.d_mask = d_mask; a.d_chosen_tree = d_chosen_tree; a.d_chosen_p = d_chosen_p; a.d_score = d_score;
+    a.d_status = d_status;
+    a.d_app_off = step ? d_app_off : nullptr; a.d_app_tok = step ? d_app_tok : nullptr;
+    a.stage_tokens = 0;
+    a.occ_scratch = scratch;
     cudaStream_t st = (cudaStream_t)stream;
-    const int Pe = prm->P < s->D ? prm->P : s->D;               // longer patterns never match
-    static bool raised[64] = {false};
-    static int sm_count[64] = {0};
-    int dev = 0;
-    SD_CUDA_OK(cudaGetDevice(&dev));
-    if (dev >= 0 && dev < 64 && !raised[dev]) {
-        // the block's shared memory exceeds the default limit: raise it once per device
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(BlockSharedT<CTA_WARPS>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_STEP, 2, STEP_G>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(BlockSharedT<CTA_WARPS_STEP>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_WIDE, 1>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(BlockSharedT<CTA_WARPS_WIDE>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_WIDE_STEP, 1>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(BlockSharedT<CTA_WARPS_WIDE_STEP>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<false, CTA_WARPS_NARROW, 4>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(BlockSharedT<CTA_WARPS_NARROW>)));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<true, CTA_WARPS_NARROW_STEP, 4, STEP_G>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(BlockSharedT<CTA_WARPS_NARROW_STEP>)));
-        SD_CUDA_OK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
-        raised[dev] = true;
-    }
-    // one block per SM is all a small batch can use: sd_speculate then takes more warps if a
-    // request has more jobs (two trees, Pe pattern lengths each) than 16 warps start at once,
-    // sd_step takes more registers
-    const bool known = dev >= 0 && dev < 64;
-    const bool wide = known && n <= sm_count[dev] && (step || 2 * Pe > 2 * CTA_WARPS);
-    // more requests than two 16-warp blocks per SM hold at once: smaller blocks, one wave
-    const bool narrow = known && n > 2 * sm_count[dev];
-#define SD_LAUNCH_FUSED(STEP, WARPS, MINB, G, OFF, TOK)                                                                 \
-    speculate_fused_kernel<STEP, WARPS, MINB, G><<<(unsigned)n, WARPS * 32, sizeof(BlockSharedT<WARPS>), st>>>(           \
-        *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap, d_n_draft, d_tokens, d_parents,          \
-        d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, OFF, TOK)
-    if (step) {
-        if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE_STEP, 1, 8, d_app_off, d_app_tok);
-        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW_STEP, 4, STEP_G, d_app_off, d_app_tok);
-        else SD_LAUNCH_FUSED(true, CTA_WARPS_STEP, 2, STEP_G, d_app_off, d_app_tok);
-    } else {
-        if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, 1, 8, nullptr, nullptr);
-        else if (narrow) SD_LAUNCH_FUSED(false, CTA_WARPS_NARROW, 4, 8, nullptr, nullptr);
-        else SD_LAUNCH_FUSED(false, CTA_WARPS, 2, 8, nullptr, nullptr);
-    }
-#undef SD_LAUNCH_FUSED
+    // a text too long for the usual shape's shared memory may still fit the one-block-per-SM shape
+    const bool long_text = s->Tp > stage_limit_tokens<CTA_WARPS, 2>();
+    if (n <= sms || (long_text && n <= 2 * sms)) launch_shape<CTA_WARPS_WIDE, 1>(*s, a, st);
+    else if (n > 2 * sms && s->Tp <= stage_limit_tokens<CTA_WARPS_NARROW, 4>()) launch_shape<CTA_WARPS_NARROW, 4>(*s, a, st);
+    else launch_shape<CTA_WARPS, 2>(*s, a, st);
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }
+
+}  // namespace
 
 extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
                             const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents,
                             int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
                             double* d_score, int32_t* d_status, void* stream) {
     return launch_fused(s, n, d_slot, prm, d_budget_cap, d_n_draft, d_tokens, d_parents, d_positions, d_mask, d_chosen_tree,
-                        d_chosen_p, d_score, d_status, nullptr, nullptr, false, stream);
+                        d_chosen_p, d_score, d_status, nullptr, nullptr, false, s ? s->occ_scratch : nullptr, stream);
 }
 
 extern "C" int sd_step(sd_store* s, int32_t n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_new_tokens,
@@ -1183,37 +1360,33 @@ extern "C" int sd_step(sd_store* s, int32_t n, const int32_t* d_slot, const int6
                        int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
                        int32_t* d_chosen_p, double* d_score, int32_t* d_status, void* stream) {
     return launch_fused(s, n, d_slot, prm, d_budget_cap, d_n_draft, d_tokens, d_parents, d_positions, d_mask, d_chosen_tree,
-                        d_chosen_p, d_score, d_status, d_offsets, d_new_tokens, true, stream);
+                        d_chosen_p, d_score, d_status, d_offsets, d_new_tokens, true, s ? s->occ_scratch : nullptr, stream);
 }
 
 // ---------------------------------------------------------------------------------------------
-// sd_speculate_noalloc: the same two kernels, with the per-job scratch records kept in a
-// fixed array that is part of the loaded library image instead of in memory obtained
-// from cudaMalloc.  Meant for callers that must not touch the CUDA allocator at all
-// (see the declaration in suffixspec.h).
+// sd_speculate_noalloc: sd_speculate with the kernel's scratch memory (the occurrence lists that
+// do not fit shared memory) in a fixed array that is part of the loaded library image instead of
+// in memory the store obtained from cudaMalloc.  Meant for callers that must not touch the CUDA
+// allocator at all (see the declaration in suffixspec.h).
 //
 // The array's name below is only meaningful to device code.  Host code holds a stand-in
 // symbol of the same name, so the launch code first asks the runtime for the array's
 // real device address (once per device, with that device current) and passes that on.
 namespace {
 
-constexpr long long NOALLOC_BYTES =
-    (long long)SD_NOALLOC_MAX_JOBS * (sizeof(double) + sizeof(int32_t) + 2ll * SD_MAX_SPEC * sizeof(int32_t));
+static __device__ __align__(256) int32_t g_noalloc_scratch[SD_NOALLOC_MAX_TOKENS];
 
-static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
-
-constexpr int NOALLOC_MAX_DEVICES = 64;
-unsigned char* g_noalloc_ptr[NOALLOC_MAX_DEVICES];      // device address of the array, per device
-bool g_noalloc_ready[NOALLOC_MAX_DEVICES];
+int32_t* g_noalloc_ptr[MAX_DEVICES];          // device address of the array, per device
+bool g_noalloc_ready[MAX_DEVICES];
 std::mutex g_noalloc_mutex;
 
 // Device address of the scratch array on the current device (looked up on first use).
-int noalloc_scratch_address(unsigned char** out) {
+int noalloc_scratch_address(int32_t** out) {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return SD_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return SD_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_noalloc_mutex);
     if (!g_noalloc_ready[dev]) {
-        unsigned char* p = nullptr;
+        int32_t* p = nullptr;
         if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) {
             cudaGetLastError();
             return SD_ERR_CUDA;
@@ -1231,34 +1404,15 @@ extern "C" int sd_speculate_noalloc(sd_store* s, int32_t n, const int32_t* d_slo
                                     const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
                                     int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
                                     int32_t* d_chosen_p, double* d_score, int32_t* d_status, void* stream) {
-    if (!s || !prm || n < 0 || n > s->R) return SD_ERR_INVALID_ARG;
-    if (prm->P < 1 || prm->max_spec < 0 || prm->max_spec > s->M || !(prm->alpha >= 0.0)) return SD_ERR_INVALID_ARG;
-    if ((prm->flags & SD_FLAG_GLOBAL_ONLY) && (prm->flags & SD_FLAG_REQUEST_ONLY)) return SD_ERR_INVALID_ARG;
-    // one record per (request, tree, depth): the batch must fit the fixed array
-    if ((long long)n * 2 * s->D > SD_NOALLOC_MAX_JOBS) return SD_ERR_CAPACITY;
-    if (n == 0) return SD_OK;
-    if (!d_slot || !d_n_draft || !d_tokens || !d_parents || !d_positions || !d_mask || !d_chosen_tree || !d_chosen_p ||
-        !d_score)
-        return SD_ERR_INVALID_ARG;
-    unsigned char* base = nullptr;
+    if (!s || n < 0 || n > s->R) return SD_ERR_INVALID_ARG;
+    SD_CHECK_DEVICE(s);
+    // one row of max_req_tokens (rounded up to 4) per request: the batch must fit the fixed array
+    if ((long long)n * s->Tp > SD_NOALLOC_MAX_TOKENS) return SD_ERR_CAPACITY;
+    int32_t* base = nullptr;
     const int rc = noalloc_scratch_address(&base);
     if (rc != SD_OK) return rc;
-    // Same record layout as the store's own scratch, carved out of the fixed array.  Every
-    // record the second kernel reads is written by the first kernel of the same call, so
-    // nothing left over from an earlier call is ever consumed and nothing needs clearing.
-    sd_store view = *s;
-    view.j_score = reinterpret_cast<double*>(base);
-    view.j_n = reinterpret_cast<int32_t*>(base + (long long)SD_NOALLOC_MAX_JOBS * sizeof(double));
-    view.j_tok = view.j_n + SD_NOALLOC_MAX_JOBS;
-    view.j_par = view.j_tok + (long long)SD_NOALLOC_MAX_JOBS * SD_MAX_SPEC;
-    cudaStream_t st = (cudaStream_t)stream;
-    const int Pe = prm->P < s->D ? prm->P : s->D;
-    const long long jobs = (long long)n * 2 * Pe;
-    match_expand_kernel<<<(unsigned)((jobs + SPEC_WARPS - 1) / SPEC_WARPS), SPEC_WARPS * 32, 0, st>>>(
-        view, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap);
-    select_emit_kernel<<<(unsigned)((n + 3) / 4), 128, 0, st>>>(view, n, d_slot, Pe, d_n_draft, d_tokens, d_parents,
-                                                                d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score,
-                                                                d_status);
-    SD_CUDA_OK(cudaGetLastError());
-    return SD_OK;
+    // Every list the kernel reads from the array was written by the same block earlier in the same
+    // launch, so nothing left over from an earlier call is ever consumed and nothing needs clearing.
+    return launch_fused(s, n, d_slot, prm, d_budget_cap, d_n_draft, d_tokens, d_parents, d_positions, d_mask, d_chosen_tree,
+                        d_chosen_p, d_score, d_status, nullptr, nullptr, false, base, stream);
 }

@@ -48,6 +48,8 @@ def _load():
         lib.sfx_oracle_slot_append_batch.argtypes = [C.c_void_p, C.c_int, p32, p64, p32, C.c_int]
         lib.sfx_oracle_slot_len.restype = C.c_int64
         lib.sfx_oracle_slot_len.argtypes = [C.c_void_p, C.c_int]
+        lib.sfx_oracle_slot_updates.restype = C.c_int64
+        lib.sfx_oracle_slot_updates.argtypes = [C.c_void_p, C.c_int]
         lib.sfx_oracle_slot_text.argtypes = [C.c_void_p, C.c_int, p32]
         lib.sfx_oracle_count.restype = C.c_int64
         lib.sfx_oracle_count.argtypes = [C.c_void_p, C.c_int, p32, C.c_int]
@@ -125,6 +127,10 @@ class SuffixOracle:
 
     def slot_len(self, slot: int) -> int:
         return int(self._lib.sfx_oracle_slot_len(self._h, slot))
+
+    def slot_updates(self, slot: int) -> int:
+        """Node updates made by the appends to `slot` since its last reset."""
+        return int(self._lib.sfx_oracle_slot_updates(self._h, slot))
 
     def slot_text(self, slot: int) -> np.ndarray:
         out = np.empty(self.slot_len(slot), dtype=np.int32)

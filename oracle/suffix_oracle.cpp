@@ -164,6 +164,7 @@ int budget_for(double alpha, int p, int cap) {
 struct Slot {
     Trie trie;
     std::vector<int32_t> text;
+    int64_t updates = 0;     // nodes whose COUNT grew through appends (one per string that ends at a new token)
 };
 
 struct Oracle {
@@ -179,42 +180,67 @@ struct SpecOut {
     int32_t* chosen_tree; int32_t* chosen_p; double* score; int64_t* visited;
 };
 
-// GenerateCandidateTree for one request + the hand-off arrays.
+// The node of pattern `pat` (p tokens) in S, or null.  `steps` grows by one for every child that
+// was found on the way (the work counter "descents": a pattern that fails at its k-th token adds k - 1).
+const Node* match_counting(const Trie& S, const int32_t* pat, int p, int64_t& steps) {
+    const Node* n = &S.root;
+    for (int k = 0; k < p; ++k) {
+        auto it = n->children.find(pat[k]);
+        if (it == n->children.end()) return nullptr;
+        n = it->second;
+        ++steps;
+    }
+    return n;
+}
+
+struct TreeCandidate {       // one speculation tree that Section 3's selection step looks at
+    int tree, p;             // where it came from: 0 global / 1 per-request, pattern length
+    double score;            // Eq. 4
+    std::vector<Draft> drafts;
+};
+
+// Candidate selection for one request (Section 3, "Speculation Tree Scoring" and the adaptive
+// budget of Eq. 3), then the arrays the verifier takes.  Two stages: every (tree, pattern length)
+// pair that matches yields one scored tree; then the first tree with the strictly largest score
+// is kept, provided it beats the threshold of Section 3.2.
 void speculate_one(const Oracle& o, int i, int slot, int P, double alpha, int cap, int flags, int M,
                    const int32_t* budget_override, double tau, const SpecOut& r) {
     const Slot& s = o.slots[slot];
     const int64_t t = (int64_t)s.text.size();
     const int words = (M + 31) / 32;
-    std::vector<Draft> best, cur;
-    double best_score = 0.0;
-    int best_tree = -1, best_p = 0;
-    int64_t descents = 0, adds = 0;
     int cap_i = cap;
     if (budget_override && budget_override[i] >= 0) cap_i = std::min(cap, (int)budget_override[i]);
+    const bool linear = (flags & FLAG_LINEAR) != 0;
+
+    // stage 1: the candidates, global tree before per-request tree, short patterns before long ones
+    std::vector<TreeCandidate> cands;
+    int64_t descents = 0, adds = 0;
     for (int tree = 0; tree < 2; ++tree) {
         if (tree == 0 && (flags & FLAG_REQUEST_ONLY)) continue;
         if (tree == 1 && (flags & FLAG_GLOBAL_ONLY)) continue;
         const Trie& S = tree == 0 ? o.global : s.trie;
-        for (int p = 1; p <= P; ++p) {
-            if (p > t || p > o.D) continue;
-            const int32_t* pat = s.text.data() + (t - p);
-            // MatchPattern, counting successful child steps
-            const Node* n = &S.root;
-            for (int k = 0; k < p && n; ++k) {
-                auto it = n->children.find(pat[k]);
-                if (it == n->children.end()) n = nullptr; else { n = it->second; ++descents; }
-            }
-            if (!n) continue;
-            double sc = expand(n, budget_for(alpha, p, cap_i), (flags & FLAG_LINEAR) != 0, cur);
-            adds += (int64_t)cur.size();
-            if (sc > best_score) { best_score = sc; best = cur; best_tree = tree; best_p = p; }
+        const int p_max = (int)std::min<int64_t>(std::min<int64_t>(P, t), o.D);
+        for (int p = 1; p <= p_max; ++p) {
+            const Node* np = match_counting(S, s.text.data() + (t - p), p, descents);
+            if (!np) continue;
+            TreeCandidate c{tree, p, 0.0, {}};
+            c.score = expand(np, budget_for(alpha, p, cap_i), linear, c.drafts);
+            adds += (int64_t)c.drafts.size();
+            cands.push_back(std::move(c));
         }
     }
+    // stage 2: the best one; equal scores keep the earlier candidate, a score of 0 is no candidate
+    const TreeCandidate* best = nullptr;
+    double best_score = 0.0;
+    for (const TreeCandidate& c : cands)
+        if (c.score > best_score) { best_score = c.score; best = &c; }
     // Section 3.2 ("Hybrid Suffix Speculative Decoding"): the suffix tree's draft is used only if
     // its score exceeds the threshold tau; otherwise the caller falls back to its other drafter.
-    if (!(best_score > tau)) { best.clear(); best_score = 0.0; best_tree = -1; best_p = 0; }
-    int n = (int)best.size();
-    r.n_draft[i] = n; r.chosen_tree[i] = best_tree; r.chosen_p[i] = best_p; r.score[i] = best_score;
+    if (best && !(best_score > tau)) { best = nullptr; best_score = 0.0; }
+
+    const int n = best ? (int)best->drafts.size() : 0;
+    r.n_draft[i] = n; r.chosen_tree[i] = best ? best->tree : -1; r.chosen_p[i] = best ? best->p : 0;
+    r.score[i] = best_score;
     if (r.visited) { r.visited[2 * i] = descents; r.visited[2 * i + 1] = adds; }
     int32_t* tok = r.tokens + (int64_t)i * M; int32_t* par = r.parents + (int64_t)i * M;
     int32_t* pos = r.positions + (int64_t)i * M; uint32_t* msk = r.mask + (int64_t)i * M * words;
@@ -222,7 +248,7 @@ void speculate_one(const Oracle& o, int i, int slot, int P, double alpha, int ca
     for (int j = 0; j < M; ++j) { tok[j] = -1; par[j] = -1; pos[j] = -1; }
     std::memset(msk, 0, sizeof(uint32_t) * (size_t)M * words);
     for (int j = 0; j < n; ++j) {
-        tok[j] = best[j].token; par[j] = best[j].parent;
+        tok[j] = best->drafts[j].token; par[j] = best->drafts[j].parent;
         depth[j] = par[j] < 0 ? 1 : depth[par[j]] + 1;
         pos[j] = (int32_t)(t + depth[j] - 1);
         for (int a = j; a >= 0; a = par[a]) msk[(int64_t)j * words + a / 32] |= (1u << (a % 32));
@@ -246,13 +272,14 @@ void sfx_oracle_global_insert(void* h, const int32_t* tok, int64_t n) { ((Oracle
 
 void sfx_oracle_slot_reset(void* h, int slot) {
     Slot& s = ((Oracle*)h)->slots[slot];
-    s.trie.clear(); s.text.clear();
+    s.trie.clear(); s.text.clear(); s.updates = 0;
 }
 void sfx_oracle_slot_append(void* h, int slot, const int32_t* tok, int64_t n) {
     Slot& s = ((Oracle*)h)->slots[slot];
     for (int64_t k = 0; k < n; ++k) {
         s.text.push_back(tok[k]);
         s.trie.extend(s.text.data(), (int64_t)s.text.size());
+        s.updates += std::min<int64_t>(s.trie.D, (int64_t)s.text.size());
     }
 }
 // Several slots at once, one thread per group of slots (slots are independent).
@@ -267,6 +294,9 @@ void sfx_oracle_slot_append_batch(void* h, int n, const int32_t* slots, const in
         });
     for (auto& x : th) x.join();
 }
+// Node updates the appends to this slot have made since its last reset: every appended token
+// raises the COUNT of one node per string that ends at it (at most D of them).
+int64_t sfx_oracle_slot_updates(void* h, int slot) { return ((Oracle*)h)->slots[slot].updates; }
 int64_t sfx_oracle_slot_len(void* h, int slot) { return (int64_t)((Oracle*)h)->slots[slot].text.size(); }
 void sfx_oracle_slot_text(void* h, int slot, int32_t* out) {
     Slot& s = ((Oracle*)h)->slots[slot];

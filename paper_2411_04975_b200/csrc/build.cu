@@ -805,7 +805,7 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
     if (!out) return SD_ERR_INVALID_ARG;
     *out = nullptr;
     if (!p || p->vocab < 1 || p->depth_cap < 1 || p->depth_cap > SD_MAX_DEPTH || p->max_requests < 1 ||
-        p->max_req_tokens < 1 || p->max_req_tokens >= (1 << 30) || p->max_spec_cap < 1 || p->max_spec_cap > SD_MAX_SPEC ||
+        p->max_req_tokens < 1 || p->max_req_tokens >= (1 << 27) || p->max_spec_cap < 1 || p->max_spec_cap > SD_MAX_SPEC ||
         n_seqs < 0)
         return SD_ERR_INVALID_ARG;
     if (n_seqs > 0 && (!d_corpus || !d_seq_offsets)) return SD_ERR_INVALID_ARG;

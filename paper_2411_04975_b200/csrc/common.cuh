@@ -60,7 +60,14 @@ struct SlotState {            // device-resident bookkeeping of one request slot
     int32_t len;              // context length t
     int32_t status;           // SD_STATUS_*
     int32_t gen;              // grows when the slot is reset
+    // Match nodes of this request in the GLOBAL tree, kept from the last speculation so that the
+    // next one only descends the tokens appended since (a cache: losing it costs walks from the root).
+    int32_t g_gen;            // value of gen the cache was taken at
+    int32_t g_epoch;          // global epoch the cache was taken at
+    int32_t g_len;            // context length the cache was taken at
+    int32_t g_depths;         // pattern lengths 1..g_depths are cached
     int32_t pad;
+    int32_t g_node[SD_MAX_DEPTH];   // g_node[d-1]: global node of the last d tokens, -1 none
 };
 
 struct sd_store {

@@ -38,7 +38,9 @@
 namespace {
 
 constexpr unsigned FULL = 0xffffffffu;
-constexpr int OCC_CAP = 1024;                 // occurrences of the last token kept in shared memory
+constexpr int OCC_POS_BITS = 27;              // an occurrence list item: position | (match length - 1) << 27
+constexpr unsigned OCC_POS_MASK = (1u << OCC_POS_BITS) - 1u;
+constexpr int COOP_MIN = 64;                  // per-request match nodes with more occurrences are expanded by a group of warps
 
 struct Frontier {                             // candidates of one job, best first, ring buffer
     double d[SD_MAX_SPEC];
@@ -57,14 +59,15 @@ __device__ __forceinline__ bool better(double da, int ta, int pa, double db, int
 
 // Insert one candidate (same values on every lane) into the sorted frontier of at
 // most K entries.  fh = ring head, fs = size.
-__device__ void frontier_insert(Frontier& F, int fh, int& fs, int K, double d, int tok, int par, int cb, unsigned nc,
+// Returns false if at least K entries are better (nothing changes then).
+__device__ bool frontier_insert(Frontier& F, int fh, int& fs, int K, double d, int tok, int par, int cb, unsigned nc,
                                 int lane) {
     const int i0 = lane, i1 = lane + 32;
     const int s0 = (fh + i0) & (SD_MAX_SPEC - 1), s1 = (fh + i1) & (SD_MAX_SPEC - 1);
     const bool b0 = i0 < fs && better(F.d[s0], F.tok[s0], F.par[s0], d, tok, par);
     const bool b1 = i1 < fs && better(F.d[s1], F.tok[s1], F.par[s1], d, tok, par);
     const int pos = __popc(__ballot_sync(FULL, b0)) + __popc(__ballot_sync(FULL, b1));
-    if (pos >= K) return;
+    if (pos >= K) return false;
     const int ns = min(fs + 1, K);
     double md0 = 0, md1 = 0; int mt0 = 0, mt1 = 0, mp0 = 0, mp1 = 0, mc0 = 0, mc1 = 0; unsigned mn0 = 0, mn1 = 0;
     const bool mv0 = i0 > pos && i0 < ns, mv1 = i1 > pos && i1 < ns;
@@ -77,6 +80,7 @@ __device__ void frontier_insert(Frontier& F, int fh, int& fs, int K, double d, i
     if (i1 == pos) { F.d[s1] = d; F.tok[s1] = tok; F.par[s1] = par; F.cb[s1] = cb; F.nc[s1] = nc; }
     __syncwarp();
     fs = ns;
+    return true;
 }
 
 __device__ __forceinline__ int budget_for(double alpha, int p, int cap) {
@@ -96,6 +100,12 @@ struct WarpWork {
     unsigned char par[2][SD_MAX_SPEC];        // parent index + 1 (0: child of the match node)
     double best_score;
     int best_order, best_n, best_buf;
+};
+
+struct CoopState {            // the node a group of warps is expanding (expand_wide_group)
+    int rep, k, idx, go, sum, keys, ovf, acc;
+    double d;
+    unsigned long long best[2];
 };
 
 template <int WARPS>
@@ -124,12 +134,16 @@ struct BlockSharedT {
     int g_cnt[SD_MAX_DEPTH];                  // COUNT of the match node
     int g_rank[SD_MAX_DEPTH];                 // its first suffix in the suffix order (-1: not usable as base)
     int g_walked, g_failed, g_base_p, g_base_m;
+    int g_src[SD_MAX_DEPTH];                  // the slot's cached match nodes, as they were before this launch
+    int g_src_depths, g_src_k;                // how many are cached (0: none usable), tokens appended since
     int g_pos[SD_OCC_LANES];                  // text position of the occurrence's first pattern token
     int g_ell[SD_OCC_LANES];                  // longest pattern the occurrence matches
     int g_avail[SD_OCC_LANES];                // tokens that follow the pattern inside the sequence (depth cap applied)
     int g_cum[SD_MAX_DEPTH + 2];
     int gwin[SD_OCC_LANES][64];               // tokens pos - 32 .. pos + 31 around every occurrence
-    int occ[OCC_CAP];
+    int w_job[SD_MAX_DEPTH];                  // per-request jobs that groups of warps expand together
+    int w_count;
+    CoopState cw[WARPS];                      // one per group of warps
 };
 
 // find_child that also hands back the matched entry (valid when the result is >= 0)
@@ -290,13 +304,11 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
         }
     }
     // With a full frontier only a child that beats its worst entry matters:
-    // D = d_parent * count / sum, so counts below `cmin` lose without any fp64 work.
-    double ld = 0.0, need = 0.0; int lt = 0, lp = 0;
-    const bool full = fs == K;
-    if (full) {
+    // D = d_parent * count / sum, so small counts lose without any fp64 work.
+    double need = 0.0;
+    if (fs == K) {
         const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
-        ld = F.d[last]; lt = F.tok[last]; lp = F.par[last];
-        need = ld * dsum * 0.999999;                            // count * d_parent must reach this
+        need = F.d[last] * dsum * 0.999999;                     // count * d_parent must reach this
     }
     for (int base = 0; base < n; base += 32) {
         const int idx = base + lane;
@@ -304,16 +316,15 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
         if (base != 0) { e = make_int4(0, 0, 0, 0); if (idx < n) e = ent[cb + idx]; }
         bool pass = idx < n && idx != skip && (double)e.y * d_parent >= need;
         if (!__any_sync(FULL, pass)) continue;
-        double dc = 0.0;
-        if (pass) {
-            dc = __dmul_rn(d_parent, __ddiv_rn((double)e.y, dsum));      // Eq. 2 with Eq. 1
-            if (full) pass = better(dc, e.x, par_index, ld, lt, lp);
-            if (pass && ((unsigned)e.w & RUN_COUNT_MASK)) prefetch_l2(ent + e.z);   // likely looked at soon
-        }
         if (fs == 0 && n <= 32) {
             // Nothing waits yet (the first children of a job): the candidates are siblings, and
             // among siblings the order of D is the order of (count, then token).  Their places
             // follow from one pass per distinct count, largest first, without any merging.
+            double dc = 0.0;
+            if (pass) {
+                dc = __dmul_rn(d_parent, __ddiv_rn((double)e.y, dsum));      // Eq. 2 with Eq. 1
+                if ((unsigned)e.w & RUN_COUNT_MASK) prefetch_l2(ent + e.z);   // likely looked at soon
+            }
             unsigned rem = __ballot_sync(FULL, pass);
             const int np = __popc(rem);
             const unsigned below = (1u << lane) - 1u;
@@ -334,27 +345,19 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
             fs = min(np, K);
             return;
         }
-        frontier_merge(F, fh, fs, K, pass, dc, e.x, par_index, e.z, (unsigned)e.w, lane);
-        if (!full && fs == K) {                                 // it filled up while merging
-            const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
-            const double d2 = F.d[last];
-            const int t2 = F.tok[last], p2 = F.par[last];
-            // from here on compare exactly against the new worst entry (no count shortcut)
-            for (int b2 = base + 32; b2 < n; b2 += 32) {
-                const int i2 = b2 + lane;
-                int4 e2 = make_int4(0, 0, 0, 0);
-                if (i2 < n) e2 = ent[cb + i2];
-                double dc2 = 0.0;
-                bool pass2 = i2 < n;
-                if (pass2) {
-                    dc2 = __dmul_rn(d_parent, __ddiv_rn((double)e2.y, dsum));
-                    const int l3 = (fh + fs - 1) & (SD_MAX_SPEC - 1);
-                    pass2 = better(dc2, e2.x, par_index, F.d[l3], F.tok[l3], F.par[l3]);
-                }
-                frontier_merge(F, fh, fs, K, pass2, dc2, e2.x, par_index, e2.z, (unsigned)e2.w, lane);
-            }
-            (void)d2; (void)t2; (void)p2;
-            return;
+        // The children of this chunk are offered best first: (count, then smaller token) orders
+        // siblings like their D values, and the first one that does not enter ends the chunk.
+        unsigned rem = __ballot_sync(FULL, pass);
+        while (rem) {
+            const bool in = (rem >> lane) & 1u;
+            const unsigned top = __reduce_max_sync(FULL, in ? (unsigned)e.y : 0u);
+            const int src = __ffs(__ballot_sync(FULL, in && (unsigned)e.y == top)) - 1;    // smallest token among them
+            const double dc = __dmul_rn(d_parent, __ddiv_rn((double)top, dsum));          // Eq. 2 with Eq. 1
+            const int cz = __shfl_sync(FULL, e.z, src);
+            const unsigned cw = (unsigned)__shfl_sync(FULL, e.w, src);
+            if (!frontier_insert(F, fh, fs, K, dc, __shfl_sync(FULL, e.x, src), par_index, cz, cw, lane)) break;
+            if (lane == 0 && (cw & RUN_COUNT_MASK)) prefetch_l2(ent + cz);                 // likely looked at soon
+            rem &= ~(1u << src);
         }
     }
 }
@@ -597,13 +600,11 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
     __syncwarp();
 }
 
-// MatchPattern(S_g, x_{1:t}, p) from the root table: descends tx[t - p .. t).  Levels whose child
-// run lies inside the window already in registers cost no memory access.  Returns the node
-// reached (-1: no match), its child run (cb, wfull) and its COUNT.
-__device__ int walk_root(const int4* __restrict__ ent, int limit, const int32_t* __restrict__ root, int V, const int* tx,
-                         int t, int p, int lane, int& cb, unsigned& wfull, int& count) {
-    const int x0 = tx[t - p];
-    int node = (x0 >= 0 && x0 < V) ? root[x0] : -1;
+// MatchPattern in the global tree, from a node that is already known: descends tx[from .. to).
+// Levels whose child run lies inside the window already in registers cost no memory access.
+// Returns the node reached (-1: no match), its child run (cb, wfull) and its COUNT.
+__device__ int walk_from(const int4* __restrict__ ent, int limit, int node, const int* tx, int from, int to, int lane,
+                         int& cb, unsigned& wfull, int& count) {
     if (node < 0) return -1;
     int wb = node;
     int4 w = load_window(ent, wb, limit, lane);
@@ -611,7 +612,7 @@ __device__ int walk_root(const int4* __restrict__ ent, int limit, const int32_t*
     wfull = (unsigned)__shfl_sync(FULL, w.w, 0);
     count = __shfl_sync(FULL, w.y, 0);
     int n = (int)(wfull & RUN_COUNT_MASK);
-    for (int pos = t - p + 1; pos < t; ++pos) {
+    for (int pos = from; pos < to; ++pos) {
         const int x = tx[pos];
         if (n == 0) return -1;
         if (n > 32) {                                           // wide run: 32-way search
@@ -809,14 +810,14 @@ __device__ void expand_wide_text(BlockShared& sh, WarpWork& W, const int* tx, in
             const unsigned pmask = nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u);
             for (int q = lane; q < 128; q += 32) { hkey[q] = -1; hcnt[q] = 0; }
             __syncwarp();
-            int sum = 0;
+            int sum = 0, keys = 0;                              // keys: different tokens in the table (kept half empty)
             bool ovf = false;
-            for (int base = 0; base < m; base += 32) {
+            for (int base = 0; base < m && keys <= 64; base += 32) {
                 const int q = base + lane;
                 bool member = false;
                 int c = 0, e = 0;
                 if (q < m) {
-                    e = list[q];
+                    e = (int)((unsigned)list[q] & OCC_POS_MASK);
                     member = e + cur_k + 1 <= t - 1;
                     for (int i = 1; member && i <= cur_k; ++i) member = tx[e + i] == tx[cur_rep + i];
                     if (member) c = tx[e + cur_k + 1];
@@ -825,6 +826,7 @@ __device__ void expand_wide_text(BlockShared& sh, WarpWork& W, const int* tx, in
                 const unsigned h = (unsigned)c * 2654435761u;
                 const bool mine = member && (h & pmask) == pre;
                 const unsigned mm = __ballot_sync(FULL, mine);
+                bool fresh = false;
                 if (mine) {
                     const unsigned grp = __match_any_sync(mm, c);
                     if (lane == __ffs(grp) - 1) {
@@ -832,34 +834,46 @@ __device__ void expand_wide_text(BlockShared& sh, WarpWork& W, const int* tx, in
                         bool done = false;
                         for (int pr = 0; pr < 128 && !done; ++pr) {
                             const int old = atomicCAS(&hkey[cell], -1, c);
-                            if (old == -1) hrep[cell] = e;
+                            if (old == -1) { hrep[cell] = e; fresh = true; }
                             if (old == -1 || old == c) { atomicAdd(&hcnt[cell], __popc(grp)); done = true; }
                             else cell = (cell + 1) & 127;
                         }
                         if (!done) ovf = true;
                     }
                 }
+                keys += __popc(__ballot_sync(FULL, fresh));
                 __syncwarp();
             }
-            if (__any_sync(FULL, ovf) && nb < 32) {             // too many different tokens: split the part
+            if ((keys > 64 || __any_sync(FULL, ovf)) && nb < 32) {   // too many different tokens: split the part
                 st_pre[sp] = pre | (1u << nb); st_nb[sp] = nb + 1; ++sp;
                 st_pre[sp] = pre; st_nb[sp] = nb + 1; ++sp;
                 continue;
             }
             const double dsum = (double)sum;                    // denominator of Eq. 1: members with a next token
-            for (int q0 = 0; q0 < 128; q0 += 32) {
-                const int c = hkey[q0 + lane];
-                const bool pass = c >= 0;
-                double dc = 0.0;
-                int rep = 0;
-                if (pass) { dc = __dmul_rn(cur_d, __ddiv_rn((double)hcnt[q0 + lane], dsum)); rep = hrep[q0 + lane]; }
-                unsigned pm = __ballot_sync(FULL, pass);
-                while (pm) {
-                    const int src = __ffs(pm) - 1;
-                    pm &= pm - 1;
-                    frontier_insert(F, fh, fs, K, __shfl_sync(FULL, dc, src), __shfl_sync(FULL, c, src), cur_idx,
-                                    __shfl_sync(FULL, rep, src), (unsigned)(cur_k + 1), lane);
+            // The children of one node order by (count, then token) like their D values, so they are
+            // offered best first and the first one that does not enter the frontier ends the part.
+            unsigned long long prev = ~0ull;
+            for (int round = 0; round < 129; ++round) {
+                unsigned long long best = 0ull;
+                int bcell = 0;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int c = hkey[lane + 32 * u];
+                    if (c >= 0) {
+                        const unsigned long long k64 = ((unsigned long long)(unsigned)hcnt[lane + 32 * u] << 32) |
+                                                       (unsigned long long)(0xffffffffu - (unsigned)c);
+                        if (k64 < prev && k64 > best) { best = k64; bcell = lane + 32 * u; }
+                    }
                 }
+                const unsigned mh = __reduce_max_sync(FULL, (unsigned)(best >> 32));
+                const unsigned ml = __reduce_max_sync(FULL, (unsigned)(best >> 32) == mh ? (unsigned)best : 0u);
+                const unsigned long long top = ((unsigned long long)mh << 32) | ml;
+                if (top == 0ull) break;
+                const int src = __ffs(__ballot_sync(FULL, best == top)) - 1;
+                const int rep = __shfl_sync(FULL, hrep[bcell], src);
+                const double dc = __dmul_rn(cur_d, __ddiv_rn((double)mh, dsum));      // Eq. 2 with Eq. 1
+                if (!frontier_insert(F, fh, fs, K, dc, (int)(0xffffffffu - ml), cur_idx, rep, (unsigned)(cur_k + 1), lane)) break;
+                prev = top;
             }
             __syncwarp();
         }
@@ -872,6 +886,174 @@ __device__ void expand_wide_text(BlockShared& sh, WarpWork& W, const int* tx, in
         }
     }
     __syncwarp();
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same job done by a GROUP OF WARPS, for match nodes with hundreds or thousands of
+// occurrences (the last tokens are frequent ones; budgets are small there, but each expansion
+// has to look at every occurrence).  The threads of the group share the occurrence list and
+// count the next tokens in one hash table of C cells in shared memory (tkey / tcnt / trep);
+// the children are then offered to the frontier best first: a group-wide maximum over the
+// table's (count, token) keys per child, until one does not enter.  The group's first warp keeps
+// the frontier (in its own working set W) and takes the next node; the state of the node being
+// expanded is handed to the other warps through shared memory (cs).  The jobs of a request that
+// need this run side by side, a group each; a group meets at a barrier of its own (bar).
+__device__ __forceinline__ void group_sync(int bar, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(threads) : "memory");
+}
+
+template <class BlockShared>
+__device__ void expand_wide_group(BlockShared& sh, CoopState& cs, WarpWork& W, const int* tx, int t, const int* list,
+                                  int m, int p, int budget, int dlim, unsigned flags, int* tkey, int* tcnt, int* trep,
+                                  int logC, int gtid, int GT, int bar) {
+    const int lane = gtid & 31, gw = gtid >> 5;
+    const int C = 1 << logC;
+    const int order = SD_MAX_DEPTH + p;
+    Frontier& F = W.F;
+    // first warp only:
+    const int buf = W.best_buf ^ 1;
+    int fh = 0, fs = 0, cnt = 0;
+    double score = 0.0;
+    bool dropped = false;
+    int xround = 0;                                              // extraction rounds so far: picks the slot of cs.best
+    if (gtid == 0) {
+        cs.rep = 0; cs.k = 0; cs.idx = -1; cs.d = 1.0; cs.best[0] = 0ull; cs.best[1] = 0ull;
+        cs.go = !((double)budget < __hiloint2double((int)*(volatile unsigned*)&sh.best_hi, 0));   // SCORE <= number of draft nodes
+    }
+    group_sync(bar, GT);
+    for (int guard = 0; guard <= SD_MAX_SPEC + 1; ++guard) {
+        if (!cs.go) break;
+        const int rep = cs.rep, k = cs.k, idx = cs.idx;
+        const double d = cs.d;
+        const int K = budget - cnt;                              // (meaningful in the first warp)
+        if (k < dlim) {
+            // parts of the token space still to do: (pre, nb) = tokens whose hash ends in the nb bits `pre`
+            unsigned st_pre[34];
+            int st_nb[34];
+            int sp = 1;
+            st_pre[0] = 0u; st_nb[0] = 0;
+            for (int pguard = 0; sp > 0 && pguard < 100000; ++pguard) {
+                --sp;
+                const unsigned pre = st_pre[sp];
+                const int nb = st_nb[sp];
+                const unsigned pmask = nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u);
+                for (int c = gtid; c < C; c += GT) { tkey[c] = -1; tcnt[c] = 0; }
+                if (gtid == 0) { cs.sum = 0; cs.keys = 0; cs.ovf = 0; }
+                group_sync(bar, GT);
+                int mine_sum = 0, mine_keys = 0;
+                for (int q0 = gw * 32; q0 < m; q0 += GT) {       // a warp takes 32 consecutive items at a time
+                    const int q = q0 + lane;
+                    bool member = false;
+                    int e = 0, c = 0;
+                    if (q < m) {
+                        e = (int)((unsigned)list[q] & OCC_POS_MASK);
+                        member = e + k + 1 <= t - 1;
+                        for (int i = 1; member && i <= k; ++i) member = tx[e + i] == tx[rep + i];
+                        if (member) c = tx[e + k + 1];
+                    }
+                    mine_sum += member ? 1 : 0;
+                    const bool mine = member && (((unsigned)c * 2654435761u) & pmask) == pre;
+                    const unsigned mm = __ballot_sync(FULL, mine);
+                    if (mine) {
+                        // equal tokens of the 32 items are counted once (frequent tokens would otherwise
+                        // all queue up at one cell of the table)
+                        const unsigned grp = __match_any_sync(mm, c);
+                        if (lane == __ffs(grp) - 1) {
+                            int cell = (int)(((unsigned)c * 0x85EBCA6Bu) >> (32 - logC));
+                            bool done = false;
+                            for (int pr = 0; pr < 64 && !done; ++pr) {
+                                const int old = atomicCAS(&tkey[cell], -1, c);
+                                if (old == -1) { trep[cell] = e; ++mine_keys; }
+                                if (old == -1 || old == c) { atomicAdd(&tcnt[cell], __popc(grp)); done = true; }
+                                else cell = (cell + 1) & (C - 1);
+                            }
+                            if (!done) cs.ovf = 1;
+                        }
+                    }
+                }
+                mine_sum = __reduce_add_sync(FULL, mine_sum);
+                mine_keys = __reduce_add_sync(FULL, mine_keys);
+                if (lane == 0) { if (mine_sum) atomicAdd(&cs.sum, mine_sum); if (mine_keys) atomicAdd(&cs.keys, mine_keys); }
+                group_sync(bar, GT);
+                const bool split = (cs.ovf || cs.keys > C - (C >> 2)) && nb < 32;
+                const double dsum = (double)cs.sum;              // denominator of Eq. 1: members with a next token
+                group_sync(bar, GT);                             // (everybody has read the counters: the next pass may clear them)
+                if (split) {                                     // too many different tokens: split the part
+                    st_pre[sp] = pre | (1u << nb); st_nb[sp] = nb + 1; ++sp;
+                    st_pre[sp] = pre; st_nb[sp] = nb + 1; ++sp;
+                    continue;
+                }
+                // children best first: (count, then smaller token) orders them like their D values
+                unsigned long long prev = ~0ull;
+                for (int round = 0; round <= SD_MAX_SPEC; ++round, ++xround) {
+                    unsigned long long best = 0ull;
+                    for (int c = gtid; c < C; c += GT) {
+                        const int tk = tkey[c];
+                        if (tk >= 0) {
+                            const unsigned long long k64 = ((unsigned long long)(unsigned)tcnt[c] << 32) |
+                                                           (unsigned long long)(0xffffffffu - (unsigned)tk);
+                            if (k64 < prev && k64 > best) best = k64;
+                        }
+                    }
+                    const unsigned mh = __reduce_max_sync(FULL, (unsigned)(best >> 32));
+                    const unsigned ml = __reduce_max_sync(FULL, (unsigned)(best >> 32) == mh ? (unsigned)best : 0u);
+                    if (lane == 0 && mh) atomicMax(&cs.best[xround & 1], ((unsigned long long)mh << 32) | ml);
+                    group_sync(bar, GT);
+                    const unsigned long long top = cs.best[xround & 1];
+                    if (gw == 0) {
+                        bool acc = false;
+                        if (top != 0ull) {
+                            const int tk = (int)(0xffffffffu - (unsigned)top);
+                            int cell = (int)(((unsigned)tk * 0x85EBCA6Bu) >> (32 - logC));
+                            for (int pr = 0; pr < 64 && tkey[cell] != tk; ++pr) cell = (cell + 1) & (C - 1);
+                            const double dc = __dmul_rn(d, __ddiv_rn((double)(unsigned)(top >> 32), dsum));   // Eq. 2 with Eq. 1
+                            acc = frontier_insert(F, fh, fs, K, dc, tk, idx, trep[cell], (unsigned)(k + 1), lane);
+                        }
+                        if (lane == 0) { cs.acc = acc ? 1 : 0; cs.best[(xround + 1) & 1] = 0ull; }
+                    }
+                    group_sync(bar, GT);
+                    if (!cs.acc) { ++xround; break; }
+                    prev = top;
+                }
+            }
+        }
+        // the first warp takes the next node
+        if (gw == 0) {
+            int go = 0;
+            if (!dropped && cnt < budget && fs > 0) {
+                const double nd = F.d[fh];
+                const int tok = F.tok[fh], par = F.par[fh], nrep = F.cb[fh], nk = (int)F.nc[fh];
+                if ((score + (double)(budget - cnt) * nd) * 1.000000001 < best_so_far(sh)) dropped = true;
+                else {
+                    __syncwarp();
+                    fh = (fh + 1) & (SD_MAX_SPEC - 1);
+                    --fs;
+                    if (lane == 0) { W.tok[buf][cnt] = tok; W.par[buf][cnt] = (unsigned char)(par + 1); }
+                    score = __dadd_rn(score, nd);               // Eq. 4, insertion order
+                    if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
+                    const int nidx = cnt++;
+                    const int K2 = budget - cnt;
+                    if (fs > K2) fs = K2;
+                    if (flags & SD_FLAG_LINEAR) fs = 0;
+                    if (cnt < budget) {
+                        go = 1;
+                        if (lane == 0) { cs.rep = nrep; cs.k = nk; cs.idx = nidx; cs.d = nd; }
+                    }
+                }
+            }
+            if (lane == 0) cs.go = go;
+        }
+        group_sync(bar, GT);
+    }
+    if (gw == 0) {
+        if (!dropped && (score > W.best_score || (score == W.best_score && score > 0.0 && order < W.best_order))) {
+            if (lane == 0) {
+                W.best_score = score; W.best_order = order; W.best_n = cnt; W.best_buf = buf;
+                atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
+            }
+        }
+    }
+    group_sync(bar, GT);
 }
 
 struct StepArgs {             // what one launch needs beyond the store
@@ -891,7 +1073,8 @@ struct StepArgs {             // what one launch needs beyond the store
     const int64_t* d_app_off;     // sd_step: the tokens to append first (NULL: sd_speculate)
     const int32_t* d_app_tok;
     int stage_tokens;             // tokens of text the block can hold in shared memory (longer texts are read in place)
-    int32_t* occ_scratch;         // [n][Tp] by request: occurrence lists longer than OCC_CAP
+    int occ_cap;                  // occurrence list items the block can hold in shared memory
+    int32_t* occ_scratch;         // [n][Tp] by request: occurrence lists longer than that
 };
 
 template <int WARPS, int MINB>
@@ -919,6 +1102,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         sh.njobs = 0; sh.next = 0; sh.nwide = 0; sh.nwide_kept = 0; sh.best_hi = 0u; sh.win_warp = -1;
         sh.first_bad = 0x7fffffff; sh.scan_next[0] = 0; sh.scan_next[1] = 0;
         sh.g_walked = 0; sh.g_failed = 0; sh.g_base_p = 0; sh.g_base_m = 0;
+        sh.w_count = 0;
     }
     WarpWork& W = sh.w[wib];
     if (lane == 0) { W.best_score = 0.0; W.best_order = 1 << 30; W.best_n = 0; W.best_buf = 0; }
@@ -975,6 +1159,17 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
     __syncthreads();                                            // (also: the new tokens in gtext are visible to the block)
 
     // ---------------- 2. match
+    if (wib == 0) {
+        // the slot's cached global match nodes (taken at context length g_len <= t)
+        int depths = 0, kk = 0;
+        if (usable) {
+            const bool cache_ok = ss->g_gen == ss->gen && ss->g_epoch == sv.g_state->epoch && ss->g_len <= t && ss->g_len > 0;
+            if (cache_ok) { depths = ss->g_depths; kk = t - ss->g_len; }
+            sh.g_src[lane] = (cache_ok && lane < depths) ? ss->g_node[lane] : -1;
+        }
+        if (lane == 0) { sh.g_src_depths = depths; sh.g_src_k = kk; }
+    }
+    __syncthreads();
     const int Lcap = min(Pe, D - 1);                            // a match node at depth D has no children
     const int last = usable ? tx[t - 1] : 0;
     const bool scan = want_r && t >= 2 && Lcap >= 1;
@@ -995,7 +1190,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
                     int l = 1;
                     while (l < Lcap && e - l >= 0 && tx[e - l] == tx[t - 1 - l]) ++l;
                     if (pass == 0) atomicAdd(&sh.r_hist[l], 1);
-                    else list[sh.r_cum[l + 1] + atomicAdd(&sh.r_fill[l], 1)] = e;
+                    else list[sh.r_cum[l + 1] + atomicAdd(&sh.r_fill[l], 1)] = e | ((l - 1) << OCC_POS_BITS);
                 }
             }
         }
@@ -1009,7 +1204,12 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         if (p <= PeG) {
             int cb = 0, cntn = 0;
             unsigned wf = 0;
-            const int node = walk_root(sv.g_ent, (int)sv.g_cap, sv.g_root, sv.V, tx, t, p, lane, cb, wf, cntn);
+            // from the cached node of the tokens before the new ones, if there is one; else from the root table
+            const int kk = sh.g_src_k;
+            int node, from;
+            if (p > kk && p - kk <= sh.g_src_depths) { node = sh.g_src[p - kk - 1]; from = t - kk; }
+            else { const int x0 = tx[t - p]; node = (x0 >= 0 && x0 < sv.V) ? sv.g_root[x0] : -1; from = t - p + 1; }
+            node = walk_from(sv.g_ent, (int)sv.g_cap, node, tx, from, t, lane, cb, wf, cntn);
             int rank = -1;
             const int nch = (int)(wf & RUN_COUNT_MASK);
             // usable as base: at most 32 occurrences, laid down by the offline build, never touched since
@@ -1036,6 +1236,14 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
     }
     if (PeG == 0 && scan) scan_pass(0, nullptr);
     __syncthreads();
+    if (wib == 0 && PeG > 0) {
+        // the match nodes of this context, for the next call.  A pattern that does not occur ends
+        // the list: no longer one occurs either.
+        const int walked = sh.g_walked, failed = sh.g_failed;
+        const int depths = failed ? SD_MAX_DEPTH : walked;
+        if (lane < depths) ss->g_node[lane] = lane < walked ? sh.node[0][lane] : -1;
+        if (lane == 0) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = depths; }
+    }
     // occurrences by match length -> r_cum; the base's occurrences (first pattern token, suffix length)
     const int base_p = sh.g_base_p;
     if (wib == 0) {
@@ -1059,7 +1267,14 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
     }
     __syncthreads();
     const int m1 = sh.r_cum[1];
-    int* const occ_list = m1 <= OCC_CAP ? sh.occ : a.occ_scratch + (long long)i * sv.Tp;
+    int* const occ_smem = stx + a.stage_tokens;
+    int* const occ_list = m1 <= a.occ_cap ? occ_smem : a.occ_scratch + (long long)i * sv.Tp;
+    // what is left of the shared memory behind the list: the hash table of expand_wide_block
+    const int list_ints = m1 <= a.occ_cap ? m1 : 0;
+    int logC = 0;
+    while ((3 << (logC + 1)) <= a.occ_cap - list_ints && logC < 12) ++logC;
+    const bool coop_ok = logC >= 8;
+    int* const tkey = occ_smem + list_ints;
     const int base_m = sh.g_base_m;
     // the 64 tokens around every occurrence of the base (one coalesced row per occurrence), then the scan's second pass
     for (int o = wib; o < base_m; o += WARPS) {
@@ -1093,7 +1308,13 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         int c = 0;
         if (p <= Pe && p <= Lcap) {
             bool has = false;
-            if (tree == 1) has = want_r && sh.r_cum[p] > 0;
+            if (tree == 1) {
+                has = want_r && sh.r_cum[p] > 0;
+                if (has && sh.r_cum[p] > COOP_MIN && coop_ok && budget_for(a.alpha, p, cap) > 0) {
+                    sh.w_job[atomicAdd(&sh.w_count, 1)] = p;     // taken up by the whole block below
+                    has = false;
+                }
+            }
             else if (base_p > 0 && p >= base_p) has = sh.g_cum[p] > 0;
             else if (p <= sh.g_walked) {
                 const unsigned wf = sh.nc[0][p - 1];
@@ -1143,7 +1364,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         if (tree == 1) {
             const int m = sh.r_cum[p];
             if (m <= SD_OCC_LANES) {
-                const int e = lane < m ? occ_list[lane] : 0;
+                const int e = lane < m ? (int)((unsigned)occ_list[lane] & OCC_POS_MASK) : 0;
                 const int kmax = lane < m ? min(t - 1 - e, D - p) : 0;
                 expand_occ(sh, W, tx + e, kmax, 1, p, budget, flags, lane);
             } else {
@@ -1198,6 +1419,39 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
             }
             counts_to_d(W.F, 0, fs, 1.0, sum, lane);
             expand_job(sh, W, sv.g_ent, (int)sv.g_cap, 0, p, budget, flags, true, fs, lane);
+        }
+        __syncthreads();
+    }
+
+    // Per-request jobs whose match node has hundreds of occurrences (short patterns of frequent
+    // tokens): those that can still reach the best score, longest pattern first, each by the
+    // whole block.
+    if (tid == 0) {
+        const double best = __hiloint2double((int)sh.best_hi, 0);
+        int kept = 0;
+        for (int q = 0; q < sh.w_count; ++q) {
+            const int p = sh.w_job[q];
+            if ((double)budget_for(a.alpha, p, cap) < best) continue;
+            int at = kept++;
+            while (at > 0 && sh.w_job[at - 1] < p) { sh.w_job[at] = sh.w_job[at - 1]; --at; }
+            sh.w_job[at] = p;
+        }
+        sh.w_count = kept;
+    }
+    __syncthreads();
+    const int nw = sh.w_count;
+    for (int base = 0; base < nw; base += (WARPS < 15 ? WARPS : 15)) {
+        const int nj = min(WARPS < 15 ? WARPS : 15, nw - base);  // (a group has a hardware barrier of its own: 15 of them)
+        const int G = WARPS / nj;                               // warps per job
+        const int my_job = wib / G;
+        if (my_job < nj) {
+            const int p = sh.w_job[base + my_job];
+            // the table room is shared out among the groups
+            int lg = 0;
+            while ((3 << (lg + 1)) <= (a.occ_cap - list_ints) / nj && lg < 12) ++lg;
+            int* const tk = tkey + my_job * (3 << lg);
+            expand_wide_group(sh, sh.cw[my_job], sh.w[my_job * G], tx, t, occ_list, sh.r_cum[p], p, budget_for(a.alpha, p, cap),
+                              D - p, flags, tk, tk + (1 << lg), tk + (2 << lg), lg, tid - my_job * G * 32, G * 32, 1 + my_job);
         }
         __syncthreads();
     }
@@ -1301,9 +1555,13 @@ int device_setup(int dev, int* sm_count) {
 
 template <int WARPS, int MINB>
 void launch_shape(const sd_store& s, StepArgs a, cudaStream_t st) {
+    // shared memory behind the block's working set: the text if it fits, then room for the
+    // occurrence list (at most one item per token) and the hash table of expand_wide_block
     const int lim = stage_limit_tokens<WARPS, MINB>();
     a.stage_tokens = s.Tp <= lim ? s.Tp : 0;
-    const size_t smem = ((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15) + (size_t)a.stage_tokens * 4;
+    const int want = s.Tp + 3 * 4096;
+    a.occ_cap = lim - a.stage_tokens < want ? lim - a.stage_tokens : want;
+    const size_t smem = ((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15) + (size_t)(a.stage_tokens + a.occ_cap) * 4;
     speculate_fused_kernel<WARPS, MINB><<<(unsigned)a.n, WARPS * 32, smem, st>>>(s, a);
 }
 
@@ -1334,6 +1592,7 @@ int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_pa
     a.d_status = d_status;
     a.d_app_off = step ? d_app_off : nullptr; a.d_app_tok = step ? d_app_tok : nullptr;
     a.stage_tokens = 0;
+    a.occ_cap = 0;
     a.occ_scratch = scratch;
     cudaStream_t st = (cudaStream_t)stream;
     // a text too long for the usual shape's shared memory may still fit the one-block-per-SM shape

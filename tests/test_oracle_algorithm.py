@@ -246,3 +246,72 @@ def test_per_request_budget_override(oracle_mod):
     o.slot_append(0, [1, 2]); o.slot_append(1, [1, 2])
     r = o.speculate([0, 1], 2, 4.0, 8, budget_override=[1, -1])
     assert r["n_draft"].tolist() == [1, 4]
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_visit_counters_equal_bruteforce(oracle_mod, seed):
+    """The two work counters (they are the numerator of the benchmark's bytes and nodes-visited
+    figures).  descents: for every tree and pattern length, the tokens of the pattern that the walk
+    finds before it stops = the longest prefix of the pattern that occurs; adds: draft nodes of
+    every tree that was expanded, whether or not it is chosen.  Both from list scans, no trie."""
+    rng = np.random.default_rng(500 + seed)
+    D = int(rng.integers(2, 7))
+    vocab = int(rng.integers(2, 5))
+    seqs = [rng.integers(0, vocab, size=int(rng.integers(3, 25))).tolist() for _ in range(4)]
+    o = _mk(oracle_mod, D, seqs, n_slots=3)
+    texts = [rng.integers(0, vocab, size=int(rng.integers(1, 20))).tolist() for _ in range(3)]
+    for s in range(3):
+        o.slot_append(s, texts[s])
+    for (P, alpha, cap, flags) in [(4, 2.0, 8, 0), (7, 1.0, 3, 0), (3, 4.0, 64, 4), (5, 1.5, 6, 1), (5, 1.5, 6, 2)]:
+        r = o.speculate([0, 1, 2], P, alpha, cap, flags=flags)
+        for s in range(3):
+            ctx = texts[s]
+            descents = adds = 0
+            for tree, src in ((0, seqs), (1, [ctx])):
+                if (tree == 0 and flags & 2) or (tree == 1 and flags & 1):
+                    continue
+                for p in range(1, min(P, len(ctx), D) + 1):
+                    pat = ctx[len(ctx) - p:]
+                    k = 0
+                    while k < p and occurrences(src, pat[:k + 1]) > 0:
+                        k += 1
+                    descents += k
+                    if k == p:
+                        adds += len(greedy_tree(src, pat, D, o.budget(alpha, p, cap), bool(flags & 4))[0])
+            assert r["visited"][s].tolist() == [descents, adds], (s, P, alpha, cap, flags)
+
+
+def test_score_threshold_is_strict(oracle_mod):
+    """Section 3.2: the draft is used only if SCORE > tau.  The hand-worked example scores
+    2/3 + 1/3 + 1/3 + 1/3 (in that order, in binary64)."""
+    g = json.load(open(os.path.join(GOLDEN, "hand_example.json")))
+    o = _mk(oracle_mod, g["depth_cap"], g["global_sequences"])
+    o.slot_append(0, g["context"])
+    s = 0.0
+    for x in (2.0 / 3.0, 1.0 / 3.0, (2.0 / 3.0) * (1.0 / 2.0), (2.0 / 3.0) * (1.0 / 2.0)):
+        s = s + x
+    below = np.nextafter(s, 0.0)
+    for tau, kept in ((0.0, True), (1.0, True), (below, True), (s, False), (np.nextafter(s, 2.0), False), (5.0, False)):
+        r = o.speculate([0], g["P"], g["alpha"], g["max_spec"], tau=float(tau))
+        if kept:
+            assert r["n_draft"][0] == 4 and r["score"][0] == s and r["chosen_tree"][0] == 0 and r["chosen_p"][0] == 2
+        else:
+            assert r["n_draft"][0] == 0 and r["score"][0] == 0.0 and r["chosen_tree"][0] == -1 and r["chosen_p"][0] == 0
+            assert (r["tokens"][0] == -1).all() and (r["mask"][0] == 0).all()
+    # the work counters do not depend on the threshold: every tree is still built
+    a = o.speculate([0], g["P"], g["alpha"], g["max_spec"], tau=0.0)["visited"]
+    b = o.speculate([0], g["P"], g["alpha"], g["max_spec"], tau=5.0)["visited"]
+    assert np.array_equal(a, b)
+
+
+def test_update_counter_is_min_depth_cap_context_length(oracle_mod):
+    """Appending the token at context length t raises one COUNT per string that ends there:
+    min(D, t) nodes (closed form of the online update of Section 3)."""
+    o = oracle_mod.SuffixOracle(5, 2)
+    o.slot_append(0, [1, 2, 3])
+    assert o.slot_updates(0) == 1 + 2 + 3
+    o.slot_append(0, [4, 5, 6, 7])
+    assert o.slot_updates(0) == 1 + 2 + 3 + 4 + 5 + 5 + 5
+    assert o.slot_updates(1) == 0
+    o.slot_reset(0)
+    assert o.slot_updates(0) == 0

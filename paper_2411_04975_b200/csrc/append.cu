@@ -3,6 +3,7 @@
 #include <cooperative_groups.h>
 
 #include "append_core.cuh"
+#include "suffix_order.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -370,22 +371,27 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
 }
 
 // One block per item: the item's tokens go behind the slot's text (a reset empties the slot
-// first).  A token outside [0, V) ends the item there (SD_STATUS_BAD_TOKEN), a full text buffer
-// likewise (SD_STATUS_POOL_FULL); both stick until the slot is reset.  Items for the global tree
-// are taken by global_insert_kernel.
-constexpr int TA_THREADS = 128;
+// first) and the suffix order of the text is brought up to date, SA_CHUNK tokens at a time
+// (suffix_order.cuh).  A token outside [0, V) ends the item there (SD_STATUS_BAD_TOKEN), a full
+// text buffer likewise (SD_STATUS_POOL_FULL); both stick until the slot is reset.  Items for the
+// global tree are taken by global_insert_kernel.  Text and order are staged in shared memory
+// when they fit (stage_tokens > 0), else the block works on the global arrays.
+constexpr int TA_THREADS = 256;
 
 __global__ void __launch_bounds__(TA_THREADS)
-text_append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_tokens,
-                   const uint8_t* d_reset, int reset_all) {
+slot_append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_tokens,
+                   const uint8_t* d_reset, int reset_all, int stage_tokens) {
+    extern __shared__ __align__(16) int ta_smem[];
+    __shared__ SaTemp tmp;
     __shared__ int first_bad;
+    const int tid = threadIdx.x;
     const int i = blockIdx.x;
     if (i >= n) return;
     const int slot = d_slot[i];
     if (slot < 0 || slot >= sv.R) return;
     SlotState* ss = sv.s_state + slot;
     int32_t* text = sv.s_text + (long long)slot * sv.Tp;
-    int len = ss->len, status = ss->status;
+    int len = ss->len, status = ss->status, buf = ss->sa_buf;
     const bool reset = reset_all || (d_reset && d_reset[i]);
     if (reset) { len = 0; status = 0; }
     const long long b = d_offsets[i];
@@ -394,9 +400,9 @@ text_append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_o
     if (!(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && cnt > 0) {
         const int room = sv.T - len;
         take = (int)min((long long)room, cnt);
-        if (threadIdx.x == 0) first_bad = take;
+        if (tid == 0) first_bad = take;
         __syncthreads();
-        for (int k = threadIdx.x; k < take; k += TA_THREADS) {
+        for (int k = tid; k < take; k += TA_THREADS) {
             const int x = d_tokens[b + k];
             if (x < 0 || x >= sv.V) atomicMin(&first_bad, k);
         }
@@ -405,11 +411,29 @@ text_append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_o
         if (good < take) status |= SD_STATUS_BAD_TOKEN;            // the bad token comes before the buffer's end
         else if ((long long)take < cnt) status |= SD_STATUS_POOL_FULL;
         take = good;
-        for (int k = threadIdx.x; k < take; k += TA_THREADS) text[len + k] = d_tokens[b + k];
     }
-    if (threadIdx.x == 0) {
+    if (take > 0) {
+        const bool staged = stage_tokens >= len + take;
+        int* tx = staged ? ta_smem : text;
+        int* S = staged ? ta_smem + stage_tokens : sv.occ_scratch + (long long)slot * sv.Tp;
+        int32_t* sa[2] = {sv.s_sa + (long long)slot * sv.Tp, sv.s_sa + ((long long)sv.R + slot) * sv.Tp};
+        for (int k = tid; k < take; k += TA_THREADS) text[len + k] = d_tokens[b + k];
+        if (staged) {
+            for (int k = tid; k < len; k += TA_THREADS) tx[k] = text[k];
+            for (int k = tid; k < take; k += TA_THREADS) tx[len + k] = d_tokens[b + k];
+        }
+        for (int k = tid; k < len; k += TA_THREADS) S[k] = sa[buf][k];
+        __syncthreads();
+        for (int t0 = len; t0 < len + take; t0 += SA_CHUNK) {
+            const int t1 = min(len + take, t0 + SA_CHUNK);
+            sa_merge_chunk<TA_THREADS>(tx, t0, t1, sv.D, S, sa[buf], sa[buf ^ 1], tmp, tid);
+            buf ^= 1;
+        }
+    }
+    if (tid == 0) {
         ss->len = len + take;
         ss->status = status;
+        ss->sa_buf = buf;
         if (reset) ss->gen += 1;
     }
 }
@@ -419,7 +443,18 @@ text_append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_o
 // Shared by sd_append and sd_build_requests.
 int sd_launch_text_append(sd_store* s, int32_t n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_tokens,
                           const uint8_t* d_reset, int reset_all, cudaStream_t st) {
-    text_append_kernel<<<(unsigned)n, TA_THREADS, 0, st>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset, reset_all);
+    // text and suffix order of a slot in shared memory if both fit (2 x Tp ints), else in place
+    const long long want = 2ll * s->Tp * 4;
+    const int stage = want <= 200 * 1024 ? s->Tp : 0;
+    const size_t smem = stage ? (size_t)want : 0;
+    if (smem > 48 * 1024) {
+        static bool raised[64] = {false};
+        if (s->device >= 0 && s->device < 64 && !raised[s->device]) {
+            SD_CUDA_OK(cudaFuncSetAttribute(slot_append_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            raised[s->device] = true;
+        }
+    }
+    slot_append_kernel<<<(unsigned)n, TA_THREADS, smem, st>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset, reset_all, stage);
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }

@@ -668,7 +668,7 @@ static void store_release(sd_store* s) {
     if (!s) return;
     cudaFree(s->g_ent); cudaFree(s->g_root); cudaFree(s->g_state);
     cudaFree(s->g_text); cudaFree(s->g_sa); cudaFree(s->g_len); cudaFree(s->g_back); cudaFree(s->g_lo);
-    cudaFree(s->s_text); cudaFree(s->s_state); cudaFree(s->occ_scratch);
+    cudaFree(s->s_text); cudaFree(s->s_sa); cudaFree(s->s_state); cudaFree(s->occ_scratch);
     cudaFree(s->stage_slot); cudaFree(s->stage_off);
     if (s->ev_fork) cudaEventDestroy(s->ev_fork);
     if (s->ev_join) cudaEventDestroy(s->ev_join);
@@ -828,7 +828,8 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
     const int D = s->D;
 
     bool ok = store_alloc(s, &s->g_root, s->V) && store_alloc(s, &s->g_state, 1) &&
-              store_alloc(s, &s->s_text, (i64)s->R * s->Tp) && store_alloc(s, &s->s_state, s->R) &&
+              store_alloc(s, &s->s_text, (i64)s->R * s->Tp) && store_alloc(s, &s->s_sa, 2ll * s->R * s->Tp) &&
+              store_alloc(s, &s->s_state, s->R) &&
               store_alloc(s, &s->occ_scratch, (i64)s->R * s->Tp) && store_alloc(s, &s->stage_slot, s->R) &&
               store_alloc(s, &s->stage_off, s->R + 1) && store_alloc(s, &s->g_text, N) && store_alloc(s, &s->g_sa, N) &&
               store_alloc(s, &s->g_len, N) && store_alloc(s, &s->g_back, N);

@@ -19,10 +19,11 @@
 // and the tokens around each occurrence are plain text (see occurrence mode in speculate.cu).
 //
 // Per-request trees are IMPLICIT: the tree over a request's text x_{1:t} is the set of its
-// substrings of at most D tokens with their numbers of occurrences, so the text itself is the
-// store; appending a token is writing it, and every question asked of the tree (match nodes,
-// children and their counts) is answered by scanning the text, which a thread block holds in
-// shared memory.
+// substrings of at most D tokens with their numbers of occurrences.  The store keeps the text
+// and the order of its suffixes (suffix_order.cuh): a node is a range of that order, its count
+// the range's size, its children the runs of equal next tokens.  Appending a token is writing
+// it and giving the few suffixes it changes their new places; a thread block holds text and
+// order in shared memory while it works on a request.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -46,7 +47,8 @@
 #define NODE_TOUCHED 0x20000000u
 #define SD_TOP_MIN 128            // runs longer than this get a top block
 #define SD_TOP_BLOCK 65           // entries of a top block
-#define SD_OCC_LANES 32           // a node with at most this many occurrences is expanded from its occurrences
+#define SD_OCC_LANES 32           // a node with at most this many occurrences is expanded a lane per occurrence
+#define SD_OCC_BASE 64            // a global match node with at most this many occurrences stands in for all longer patterns
 
 struct GlobalState {          // device-resident bookkeeping of the global tree
     int32_t used;             // entries handed out
@@ -66,7 +68,7 @@ struct SlotState {            // device-resident bookkeeping of one request slot
     int32_t g_epoch;          // global epoch the cache was taken at
     int32_t g_len;            // context length the cache was taken at
     int32_t g_depths;         // pattern lengths 1..g_depths are cached
-    int32_t pad;
+    int32_t sa_buf;           // which of the slot's two suffix-order arrays is the current one
     int32_t g_node[SD_MAX_DEPTH];   // g_node[d-1]: global node of the last d tokens, -1 none
 };
 
@@ -89,8 +91,10 @@ struct sd_store {
     int32_t* g_lo;            // [static_entries] by first entry of a child run: rank of the owner's first suffix
     // per-request trees: the texts
     int32_t* s_text;          // [R][Tp]
+    int32_t* s_sa;            // [2][R][Tp] suffix order of each text (suffix_order.cuh); an update reads one
+                              // array and writes the other, SlotState.sa_buf says which is current
     SlotState* s_state;       // [R]
-    int32_t* occ_scratch;     // [R][Tp]: occurrence lists that do not fit shared memory
+    int32_t* occ_scratch;     // [R][Tp]: work buffer for the suffix order of a text too long for shared memory
     // staging of sd_build_requests' host arrays
     int32_t* stage_slot;      // [R]
     int64_t* stage_off;       // [R + 1]

@@ -34,13 +34,11 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "suffix_order.cuh"
 
 namespace {
 
 constexpr unsigned FULL = 0xffffffffu;
-constexpr int OCC_POS_BITS = 27;              // an occurrence list item: position | (match length - 1) << 27
-constexpr unsigned OCC_POS_MASK = (1u << OCC_POS_BITS) - 1u;
-constexpr int COOP_MIN = 64;                  // per-request match nodes with more occurrences are expanded by a group of warps
 
 struct Frontier {                             // candidates of one job, best first, ring buffer
     double d[SD_MAX_SPEC];
@@ -102,12 +100,6 @@ struct WarpWork {
     int best_order, best_n, best_buf;
 };
 
-struct CoopState {            // the node a group of warps is expanding (expand_wide_group)
-    int rep, k, idx, go, sum, keys, ovf, acc;
-    double d;
-    unsigned long long best[2];
-};
-
 template <int WARPS>
 struct BlockSharedT {
     WarpWork w[WARPS];
@@ -125,25 +117,21 @@ struct BlockSharedT {
                                               // all the pruning needs; 32 bits keep the atomic native
     int win_warp;
     int first_bad;                            // sd_step: first new token outside the vocabulary
-    // per-request tree: earlier occurrences of the last token by backward match length
-    int r_hist[SD_MAX_DEPTH + 2];
-    int r_cum[SD_MAX_DEPTH + 2];              // r_cum[p]: occurrences that agree on at least p tokens
-    int r_fill[SD_MAX_DEPTH + 2];
-    int scan_next[2];
+    // per-request tree: the match nodes as ranges of the text's suffix order
+    int r_lo[SD_MAX_DEPTH + 1];               // r_lo[p]: first suffix that starts with the last p tokens (the context's own end)
+    int r_cnt[SD_MAX_DEPTH + 1];              // earlier occurrences of that pattern: suffixes r_lo[p] + 1 .. r_lo[p] + r_cnt[p]
+    SaTemp sat;                               // scratch of the suffix-order update
     // global tree: the base of occurrence mode
     int g_cnt[SD_MAX_DEPTH];                  // COUNT of the match node
     int g_rank[SD_MAX_DEPTH];                 // its first suffix in the suffix order (-1: not usable as base)
     int g_walked, g_failed, g_base_p, g_base_m;
     int g_src[SD_MAX_DEPTH];                  // the slot's cached match nodes, as they were before this launch
     int g_src_depths, g_src_k;                // how many are cached (0: none usable), tokens appended since
-    int g_pos[SD_OCC_LANES];                  // text position of the occurrence's first pattern token
-    int g_ell[SD_OCC_LANES];                  // longest pattern the occurrence matches
-    int g_avail[SD_OCC_LANES];                // tokens that follow the pattern inside the sequence (depth cap applied)
+    int g_pos[SD_OCC_BASE];                   // text position of the occurrence's first pattern token
+    int g_ell[SD_OCC_BASE];                   // longest pattern the occurrence matches
+    int g_avail[SD_OCC_BASE];                 // tokens that follow the pattern inside the sequence (depth cap applied)
     int g_cum[SD_MAX_DEPTH + 2];
-    int gwin[SD_OCC_LANES][64];               // tokens pos - 32 .. pos + 31 around every occurrence
-    int w_job[SD_MAX_DEPTH];                  // per-request jobs that groups of warps expand together
-    int w_count;
-    CoopState cw[WARPS];                      // one per group of warps
+    int gwin[SD_OCC_BASE][64];                // tokens pos - 32 .. pos + 31 around every occurrence
 };
 
 // find_child that also hands back the matched entry (valid when the result is >= 0)
@@ -753,41 +741,55 @@ __device__ void expand_occ(BlockShared& sh, WarpWork& W, const int* cptr, int km
 }
 
 // ---------------------------------------------------------------------------------------------
-// A per-request job whose match node has more than 32 occurrences (list[0 .. m): positions of the
-// pattern's last token).  A node below N_p is named by one of its occurrences and its depth:
-// (rep, k) stands for the string tx[rep + 1 .. rep + k].  Its children come from a pass over the
-// list: the occurrences that agree with rep on k tokens are its members, and a hash table of
-// 128 cells in shared memory counts their next tokens.  The members' tokens are taken a part
-// at a time (by bits of a hash of the token) when the table cannot hold them all.  Frontier:
-// the sorted ring of the tree-entry path; fields cb / nc hold rep / k.
-template <class BlockShared>
-__device__ void expand_wide_text(BlockShared& sh, WarpWork& W, const int* tx, int t, const int* list, int m, int p,
-                                 int budget, int dlim, unsigned flags, int lane) {
-    const int order = SD_MAX_DEPTH + p;
+// A job whose match node has more than 32 occurrences, over a list of occurrences that is SORTED
+// by the text behind them.  Every node below the match node is a range of the list (the items
+// that agree on the tokens so far), its children are the runs of equal next tokens inside the
+// range, and expanding a node is one pass over its own range.
+//   Per-request tree: the list is the suffix order of the request's text (suffix_order.cuh), the
+//   pattern's occurrences are the range S[lo .. hi), COUNT is the size of a range.
+//   Global tree: the list is the base node's range of the offline build's suffix order, staged
+//   with the tokens around every occurrence; the job of pattern length p counts only the items
+//   that match at least p tokens (FILTER).
+// Frontier: the sorted ring of the tree-entry path; fields cb / nc hold the candidate's range as
+// lo / (hi << 5 | depth below the match node).
+struct TextItems {            // items j of S: suffixes that start with the pattern of length p
+    const int* tx; const int* S; int t, p;
+    // token `level` (1: the first one behind the pattern) of item j, -1 if the text ends before it
+    __device__ __forceinline__ int tok(int j, int level) const { const int q = S[j] + p - 1 + level; return q <= t - 1 ? tx[q] : -1; }
+    __device__ __forceinline__ bool member(int) const { return true; }
+};
+struct WindowItems {          // items j: occurrences of the global base pattern, with 64 tokens around each
+    const int (*gwin)[64]; const int* avail; const int* ell; int base_p, p;
+    __device__ __forceinline__ int tok(int j, int level) const { return level <= avail[j] ? gwin[j][31 + base_p + level] : -1; }
+    __device__ __forceinline__ bool member(int j) const { return ell[j] >= p; }
+};
+
+template <bool FILTER, class Items, class BlockShared>
+__device__ void expand_range(BlockShared& sh, WarpWork& W, const Items& it, int lo0, int hi0, int tree, int p, int budget,
+                             int dlim, unsigned flags, int lane) {
+    const int order = tree * SD_MAX_DEPTH + p;
     const int buf = W.best_buf ^ 1;
-    int* const hkey = reinterpret_cast<int*>(&W.T);             // 128 cells: token, count, an occurrence
-    int* const hcnt = hkey + 128;
-    int* const hrep = hkey + 256;
     Frontier& F = W.F;
     int fh = 0, fs = 0, cnt = 0;
     double score = 0.0;
     bool dropped = false;
     double cur_d = 1.0;
-    int cur_rep = 0, cur_k = 0, cur_idx = -1;
+    int lo = lo0, hi = hi0, cur_k = 0, cur_idx = -1;
     bool have_cur = true;
     while (true) {
         if (!have_cur) {
             if (cnt >= budget || fs == 0) break;
             cur_d = F.d[fh];
             const int tok = F.tok[fh], par = F.par[fh];
-            cur_rep = F.cb[fh];
-            cur_k = (int)F.nc[fh];
+            lo = F.cb[fh];
+            hi = (int)(F.nc[fh] >> 5);
+            cur_k = (int)(F.nc[fh] & 31u);
             if ((score + (double)(budget - cnt) * cur_d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
             __syncwarp();
             fh = (fh + 1) & (SD_MAX_SPEC - 1);
             --fs;
             if (lane == 0) { W.tok[buf][cnt] = tok; W.par[buf][cnt] = (unsigned char)(par + 1); }
-            score = __dadd_rn(score, cur_d);
+            score = __dadd_rn(score, cur_d);                    // Eq. 4, insertion order
             if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
             cur_idx = cnt++;
             const int K = budget - cnt;
@@ -796,86 +798,68 @@ __device__ void expand_wide_text(BlockShared& sh, WarpWork& W, const int* tx, in
         }
         have_cur = false;
         if (cnt >= budget) break;
-        if (cur_k >= dlim) continue;                            // depth cap: the node has no children
+        if (cur_k >= dlim || lo >= hi) continue;                // depth cap: the node has no children
         const int K = budget - cnt;
-        // parts of the token space still to do: (pre, nb) = tokens whose hash ends in the nb bits `pre`
-        unsigned st_pre[34];
-        int st_nb[34];
-        int sp = 0;
-        st_pre[0] = 0u; st_nb[0] = 0; sp = 1;
-        for (int guard = 0; sp > 0 && guard < 100000; ++guard) {
-            --sp;
-            const unsigned pre = st_pre[sp];
-            const int nb = st_nb[sp];
-            const unsigned pmask = nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u);
-            for (int q = lane; q < 128; q += 32) { hkey[q] = -1; hcnt[q] = 0; }
-            __syncwarp();
-            int sum = 0, keys = 0;                              // keys: different tokens in the table (kept half empty)
-            bool ovf = false;
-            for (int base = 0; base < m && keys <= 64; base += 32) {
-                const int q = base + lane;
-                bool member = false;
-                int c = 0, e = 0;
-                if (q < m) {
-                    e = (int)((unsigned)list[q] & OCC_POS_MASK);
-                    member = e + cur_k + 1 <= t - 1;
-                    for (int i = 1; member && i <= cur_k; ++i) member = tx[e + i] == tx[cur_rep + i];
-                    if (member) c = tx[e + cur_k + 1];
-                }
-                sum += __popc(__ballot_sync(FULL, member));
-                const unsigned h = (unsigned)c * 2654435761u;
-                const bool mine = member && (h & pmask) == pre;
-                const unsigned mm = __ballot_sync(FULL, mine);
-                bool fresh = false;
-                if (mine) {
-                    const unsigned grp = __match_any_sync(mm, c);
-                    if (lane == __ffs(grp) - 1) {
-                        int cell = (int)(((unsigned)c * 0x85EBCA6Bu) >> 25);
-                        bool done = false;
-                        for (int pr = 0; pr < 128 && !done; ++pr) {
-                            const int old = atomicCAS(&hkey[cell], -1, c);
-                            if (old == -1) { hrep[cell] = e; fresh = true; }
-                            if (old == -1 || old == c) { atomicAdd(&hcnt[cell], __popc(grp)); done = true; }
-                            else cell = (cell + 1) & 127;
-                        }
-                        if (!done) ovf = true;
+        const int level = cur_k + 1;
+        // the sibling sum (denominator of Eq. 1): items of the job that have a next token
+        int sum;
+        if (FILTER) {
+            sum = 0;
+            for (int base = lo; base < hi; base += 32) {
+                const int j = base + lane;
+                sum += __popc(__ballot_sync(FULL, j < hi && it.member(j) && it.tok(j, level) >= 0));
+            }
+        } else {
+            sum = hi - lo - (it.tok(lo, level) < 0 ? 1 : 0);    // an item whose text ends here sorts first; all others go on
+        }
+        if (sum <= 0) continue;
+        const double dsum = (double)sum;
+        // the runs of equal next tokens; an open run is carried from chunk to chunk
+        int run_tok = -2, run_lo = lo, run_c = 0;               // -2: none yet
+        for (int base = lo; base < hi + 32; base += 32) {       // (a last round behind the range closes the last run)
+            const int j = base + lane;
+            int tk = -3;                                        // behind the range: differs from every token
+            bool mem = false;
+            if (j < hi) { tk = it.tok(j, level); mem = FILTER ? (tk >= 0 && it.member(j)) : true; }
+            int prev = __shfl_up_sync(FULL, tk, 1);
+            if (lane == 0) prev = run_tok;
+            const bool bnd = tk != prev;                        // a run starts here
+            const unsigned bm = __ballot_sync(FULL, bnd);
+            const unsigned mm = FILTER ? __ballot_sync(FULL, mem) : 0u;
+            if (!bm) { if (FILTER) run_c += __popc(mm); }
+            else {
+                // every boundary closes the run that ends right before it: the open run for the
+                // first boundary of the chunk, else the run that began at the boundary before
+                const unsigned lt = (1u << lane) - 1u;
+                const unsigned below = bm & lt;
+                const int sb = below ? 31 - __clz(below) : 0;
+                const int s_tok = __shfl_sync(FULL, tk, sb);
+                const int c_tok = below ? s_tok : run_tok, c_lo = below ? base + sb : run_lo, c_hi = base + lane;
+                int c_cnt = c_hi - c_lo;
+                if (FILTER) c_cnt = below ? __popc(mm & lt & ~((1u << sb) - 1u)) : run_c + __popc(mm & lt);
+                bool pass = bnd && c_tok >= 0 && c_cnt > 0;
+                double dc = 0.0;
+                if (pass) {
+                    dc = __dmul_rn(cur_d, __ddiv_rn((double)c_cnt, dsum));             // Eq. 2 with Eq. 1
+                    if (fs == K) {
+                        const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+                        pass = better(dc, c_tok, cur_idx, F.d[last], F.tok[last], F.par[last]);
                     }
                 }
-                keys += __popc(__ballot_sync(FULL, fresh));
-                __syncwarp();
-            }
-            if ((keys > 64 || __any_sync(FULL, ovf)) && nb < 32) {   // too many different tokens: split the part
-                st_pre[sp] = pre | (1u << nb); st_nb[sp] = nb + 1; ++sp;
-                st_pre[sp] = pre; st_nb[sp] = nb + 1; ++sp;
-                continue;
-            }
-            const double dsum = (double)sum;                    // denominator of Eq. 1: members with a next token
-            // The children of one node order by (count, then token) like their D values, so they are
-            // offered best first and the first one that does not enter the frontier ends the part.
-            unsigned long long prev = ~0ull;
-            for (int round = 0; round < 129; ++round) {
-                unsigned long long best = 0ull;
-                int bcell = 0;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = hkey[lane + 32 * u];
-                    if (c >= 0) {
-                        const unsigned long long k64 = ((unsigned long long)(unsigned)hcnt[lane + 32 * u] << 32) |
-                                                       (unsigned long long)(0xffffffffu - (unsigned)c);
-                        if (k64 < prev && k64 > best) { best = k64; bcell = lane + 32 * u; }
-                    }
+                unsigned pm = __ballot_sync(FULL, pass);
+                while (pm) {
+                    const int src = __ffs(pm) - 1;
+                    pm &= pm - 1;
+                    frontier_insert(F, fh, fs, K, __shfl_sync(FULL, dc, src), __shfl_sync(FULL, c_tok, src), cur_idx,
+                                    __shfl_sync(FULL, c_lo, src),
+                                    ((unsigned)__shfl_sync(FULL, c_hi, src) << 5) | (unsigned)level, lane);
                 }
-                const unsigned mh = __reduce_max_sync(FULL, (unsigned)(best >> 32));
-                const unsigned ml = __reduce_max_sync(FULL, (unsigned)(best >> 32) == mh ? (unsigned)best : 0u);
-                const unsigned long long top = ((unsigned long long)mh << 32) | ml;
-                if (top == 0ull) break;
-                const int src = __ffs(__ballot_sync(FULL, best == top)) - 1;
-                const int rep = __shfl_sync(FULL, hrep[bcell], src);
-                const double dc = __dmul_rn(cur_d, __ddiv_rn((double)mh, dsum));      // Eq. 2 with Eq. 1
-                if (!frontier_insert(F, fh, fs, K, dc, (int)(0xffffffffu - ml), cur_idx, rep, (unsigned)(cur_k + 1), lane)) break;
-                prev = top;
+                const int lb = 31 - __clz(bm);                  // the last boundary opens the run that is carried on
+                run_tok = __shfl_sync(FULL, tk, lb);
+                run_lo = base + lb;
+                if (FILTER) run_c = __popc(mm & ~((1u << lb) - 1u));
             }
-            __syncwarp();
+            if (base >= hi) break;
         }
     }
     __syncwarp();
@@ -886,174 +870,6 @@ __device__ void expand_wide_text(BlockShared& sh, WarpWork& W, const int* tx, in
         }
     }
     __syncwarp();
-}
-
-// ---------------------------------------------------------------------------------------------
-// The same job done by a GROUP OF WARPS, for match nodes with hundreds or thousands of
-// occurrences (the last tokens are frequent ones; budgets are small there, but each expansion
-// has to look at every occurrence).  The threads of the group share the occurrence list and
-// count the next tokens in one hash table of C cells in shared memory (tkey / tcnt / trep);
-// the children are then offered to the frontier best first: a group-wide maximum over the
-// table's (count, token) keys per child, until one does not enter.  The group's first warp keeps
-// the frontier (in its own working set W) and takes the next node; the state of the node being
-// expanded is handed to the other warps through shared memory (cs).  The jobs of a request that
-// need this run side by side, a group each; a group meets at a barrier of its own (bar).
-__device__ __forceinline__ void group_sync(int bar, int threads) {
-    asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(threads) : "memory");
-}
-
-template <class BlockShared>
-__device__ void expand_wide_group(BlockShared& sh, CoopState& cs, WarpWork& W, const int* tx, int t, const int* list,
-                                  int m, int p, int budget, int dlim, unsigned flags, int* tkey, int* tcnt, int* trep,
-                                  int logC, int gtid, int GT, int bar) {
-    const int lane = gtid & 31, gw = gtid >> 5;
-    const int C = 1 << logC;
-    const int order = SD_MAX_DEPTH + p;
-    Frontier& F = W.F;
-    // first warp only:
-    const int buf = W.best_buf ^ 1;
-    int fh = 0, fs = 0, cnt = 0;
-    double score = 0.0;
-    bool dropped = false;
-    int xround = 0;                                              // extraction rounds so far: picks the slot of cs.best
-    if (gtid == 0) {
-        cs.rep = 0; cs.k = 0; cs.idx = -1; cs.d = 1.0; cs.best[0] = 0ull; cs.best[1] = 0ull;
-        cs.go = !((double)budget < __hiloint2double((int)*(volatile unsigned*)&sh.best_hi, 0));   // SCORE <= number of draft nodes
-    }
-    group_sync(bar, GT);
-    for (int guard = 0; guard <= SD_MAX_SPEC + 1; ++guard) {
-        if (!cs.go) break;
-        const int rep = cs.rep, k = cs.k, idx = cs.idx;
-        const double d = cs.d;
-        const int K = budget - cnt;                              // (meaningful in the first warp)
-        if (k < dlim) {
-            // parts of the token space still to do: (pre, nb) = tokens whose hash ends in the nb bits `pre`
-            unsigned st_pre[34];
-            int st_nb[34];
-            int sp = 1;
-            st_pre[0] = 0u; st_nb[0] = 0;
-            for (int pguard = 0; sp > 0 && pguard < 100000; ++pguard) {
-                --sp;
-                const unsigned pre = st_pre[sp];
-                const int nb = st_nb[sp];
-                const unsigned pmask = nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u);
-                for (int c = gtid; c < C; c += GT) { tkey[c] = -1; tcnt[c] = 0; }
-                if (gtid == 0) { cs.sum = 0; cs.keys = 0; cs.ovf = 0; }
-                group_sync(bar, GT);
-                int mine_sum = 0, mine_keys = 0;
-                for (int q0 = gw * 32; q0 < m; q0 += GT) {       // a warp takes 32 consecutive items at a time
-                    const int q = q0 + lane;
-                    bool member = false;
-                    int e = 0, c = 0;
-                    if (q < m) {
-                        e = (int)((unsigned)list[q] & OCC_POS_MASK);
-                        member = e + k + 1 <= t - 1;
-                        for (int i = 1; member && i <= k; ++i) member = tx[e + i] == tx[rep + i];
-                        if (member) c = tx[e + k + 1];
-                    }
-                    mine_sum += member ? 1 : 0;
-                    const bool mine = member && (((unsigned)c * 2654435761u) & pmask) == pre;
-                    const unsigned mm = __ballot_sync(FULL, mine);
-                    if (mine) {
-                        // equal tokens of the 32 items are counted once (frequent tokens would otherwise
-                        // all queue up at one cell of the table)
-                        const unsigned grp = __match_any_sync(mm, c);
-                        if (lane == __ffs(grp) - 1) {
-                            int cell = (int)(((unsigned)c * 0x85EBCA6Bu) >> (32 - logC));
-                            bool done = false;
-                            for (int pr = 0; pr < 64 && !done; ++pr) {
-                                const int old = atomicCAS(&tkey[cell], -1, c);
-                                if (old == -1) { trep[cell] = e; ++mine_keys; }
-                                if (old == -1 || old == c) { atomicAdd(&tcnt[cell], __popc(grp)); done = true; }
-                                else cell = (cell + 1) & (C - 1);
-                            }
-                            if (!done) cs.ovf = 1;
-                        }
-                    }
-                }
-                mine_sum = __reduce_add_sync(FULL, mine_sum);
-                mine_keys = __reduce_add_sync(FULL, mine_keys);
-                if (lane == 0) { if (mine_sum) atomicAdd(&cs.sum, mine_sum); if (mine_keys) atomicAdd(&cs.keys, mine_keys); }
-                group_sync(bar, GT);
-                const bool split = (cs.ovf || cs.keys > C - (C >> 2)) && nb < 32;
-                const double dsum = (double)cs.sum;              // denominator of Eq. 1: members with a next token
-                group_sync(bar, GT);                             // (everybody has read the counters: the next pass may clear them)
-                if (split) {                                     // too many different tokens: split the part
-                    st_pre[sp] = pre | (1u << nb); st_nb[sp] = nb + 1; ++sp;
-                    st_pre[sp] = pre; st_nb[sp] = nb + 1; ++sp;
-                    continue;
-                }
-                // children best first: (count, then smaller token) orders them like their D values
-                unsigned long long prev = ~0ull;
-                for (int round = 0; round <= SD_MAX_SPEC; ++round, ++xround) {
-                    unsigned long long best = 0ull;
-                    for (int c = gtid; c < C; c += GT) {
-                        const int tk = tkey[c];
-                        if (tk >= 0) {
-                            const unsigned long long k64 = ((unsigned long long)(unsigned)tcnt[c] << 32) |
-                                                           (unsigned long long)(0xffffffffu - (unsigned)tk);
-                            if (k64 < prev && k64 > best) best = k64;
-                        }
-                    }
-                    const unsigned mh = __reduce_max_sync(FULL, (unsigned)(best >> 32));
-                    const unsigned ml = __reduce_max_sync(FULL, (unsigned)(best >> 32) == mh ? (unsigned)best : 0u);
-                    if (lane == 0 && mh) atomicMax(&cs.best[xround & 1], ((unsigned long long)mh << 32) | ml);
-                    group_sync(bar, GT);
-                    const unsigned long long top = cs.best[xround & 1];
-                    if (gw == 0) {
-                        bool acc = false;
-                        if (top != 0ull) {
-                            const int tk = (int)(0xffffffffu - (unsigned)top);
-                            int cell = (int)(((unsigned)tk * 0x85EBCA6Bu) >> (32 - logC));
-                            for (int pr = 0; pr < 64 && tkey[cell] != tk; ++pr) cell = (cell + 1) & (C - 1);
-                            const double dc = __dmul_rn(d, __ddiv_rn((double)(unsigned)(top >> 32), dsum));   // Eq. 2 with Eq. 1
-                            acc = frontier_insert(F, fh, fs, K, dc, tk, idx, trep[cell], (unsigned)(k + 1), lane);
-                        }
-                        if (lane == 0) { cs.acc = acc ? 1 : 0; cs.best[(xround + 1) & 1] = 0ull; }
-                    }
-                    group_sync(bar, GT);
-                    if (!cs.acc) { ++xround; break; }
-                    prev = top;
-                }
-            }
-        }
-        // the first warp takes the next node
-        if (gw == 0) {
-            int go = 0;
-            if (!dropped && cnt < budget && fs > 0) {
-                const double nd = F.d[fh];
-                const int tok = F.tok[fh], par = F.par[fh], nrep = F.cb[fh], nk = (int)F.nc[fh];
-                if ((score + (double)(budget - cnt) * nd) * 1.000000001 < best_so_far(sh)) dropped = true;
-                else {
-                    __syncwarp();
-                    fh = (fh + 1) & (SD_MAX_SPEC - 1);
-                    --fs;
-                    if (lane == 0) { W.tok[buf][cnt] = tok; W.par[buf][cnt] = (unsigned char)(par + 1); }
-                    score = __dadd_rn(score, nd);               // Eq. 4, insertion order
-                    if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
-                    const int nidx = cnt++;
-                    const int K2 = budget - cnt;
-                    if (fs > K2) fs = K2;
-                    if (flags & SD_FLAG_LINEAR) fs = 0;
-                    if (cnt < budget) {
-                        go = 1;
-                        if (lane == 0) { cs.rep = nrep; cs.k = nk; cs.idx = nidx; cs.d = nd; }
-                    }
-                }
-            }
-            if (lane == 0) cs.go = go;
-        }
-        group_sync(bar, GT);
-    }
-    if (gw == 0) {
-        if (!dropped && (score > W.best_score || (score == W.best_score && score > 0.0 && order < W.best_order))) {
-            if (lane == 0) {
-                W.best_score = score; W.best_order = order; W.best_n = cnt; W.best_buf = buf;
-                atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
-            }
-        }
-    }
-    group_sync(bar, GT);
 }
 
 struct StepArgs {             // what one launch needs beyond the store
@@ -1072,9 +888,9 @@ struct StepArgs {             // what one launch needs beyond the store
     int32_t* d_status;
     const int64_t* d_app_off;     // sd_step: the tokens to append first (NULL: sd_speculate)
     const int32_t* d_app_tok;
-    int stage_tokens;             // tokens of text the block can hold in shared memory (longer texts are read in place)
-    int occ_cap;                  // occurrence list items the block can hold in shared memory
-    int32_t* occ_scratch;         // [n][Tp] by request: occurrence lists longer than that
+    int stage_tokens;             // tokens of text, and entries of its suffix order, the block can hold in shared
+                                  // memory (0: the text is too long; both are then used in place)
+    int32_t* scratch;             // [n][Tp] by request: the suffix order of a text that is not staged
 };
 
 template <int WARPS, int MINB>
@@ -1090,19 +906,22 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
     const unsigned flags = a.flags;
     const int slot = a.d_slot[i];
     const bool ok = slot >= 0 && slot < sv.R;
-    int t = 0, status = SD_STATUS_BAD_SLOT;
+    int t = 0, status = SD_STATUS_BAD_SLOT, sa_buf = 0;
     SlotState* ss = nullptr;
     int32_t* gtext = nullptr;
-    if (ok) { ss = sv.s_state + slot; t = ss->len; status = ss->status; gtext = sv.s_text + (long long)slot * sv.Tp; }
+    if (ok) {
+        ss = sv.s_state + slot; t = ss->len; status = ss->status; sa_buf = ss->sa_buf;
+        gtext = sv.s_text + (long long)slot * sv.Tp;
+    }
     const int t_old = t;
     if (tid < 2 * SD_MAX_DEPTH) { (&sh.node[0][0])[tid] = -1; (&sh.nc[0][0])[tid] = 0; }
-    if (tid < SD_MAX_DEPTH + 2) { sh.r_hist[tid] = 0; sh.r_cum[tid] = 0; sh.r_fill[tid] = 0; sh.g_cum[tid] = 0; }
+    if (tid < SD_MAX_DEPTH + 2) sh.g_cum[tid] = 0;
+    if (tid <= SD_MAX_DEPTH) { sh.r_lo[tid] = 0; sh.r_cnt[tid] = 0; }
     if (tid < SD_MAX_DEPTH) { sh.g_cnt[tid] = 0; sh.g_rank[tid] = -1; }
     if (tid == 0) {
         sh.njobs = 0; sh.next = 0; sh.nwide = 0; sh.nwide_kept = 0; sh.best_hi = 0u; sh.win_warp = -1;
-        sh.first_bad = 0x7fffffff; sh.scan_next[0] = 0; sh.scan_next[1] = 0;
+        sh.first_bad = 0x7fffffff;
         sh.g_walked = 0; sh.g_failed = 0; sh.g_base_p = 0; sh.g_base_m = 0;
-        sh.w_count = 0;
     }
     WarpWork& W = sh.w[wib];
     if (lane == 0) { W.best_score = 0.0; W.best_order = 1 << 30; W.best_n = 0; W.best_buf = 0; }
@@ -1128,7 +947,6 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
             take = good;
             for (int k = tid; k < take; k += NT) gtext[t_old + k] = newtok[k];
             t = t_old + take;
-            if (tid == 0) { ss->len = t; ss->status = status; }
         }
     }
     const bool usable = ok && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && t > 0;
@@ -1137,10 +955,13 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
     const bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
     const bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
 
-    // ---------------- 1. the text
+    // ---------------- 1. the text and its suffix order
+    const bool staged = t <= a.stage_tokens;
+    int fin_a0 = -1;
     const int* tx = stx;
-    if (usable) {
-        if (t <= a.stage_tokens) {
+    int* S = stx + a.stage_tokens;
+    if (ok && (usable || take > 0)) {
+        if (staged) {
             const int4* g4 = reinterpret_cast<const int4*>(gtext);
             int4* s4 = reinterpret_cast<int4*>(stx);
             for (int g = tid; g * 4 < t; g += NT) {
@@ -1153,10 +974,24 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
                 s4[g] = v;
             }
         } else {
-            tx = gtext;                                         // too long to stage: read in place
+            tx = gtext;                                         // too long to stage: text and order are used in place
+            S = a.scratch + (long long)i * sv.Tp;
         }
+        int32_t* sa[2] = {sv.s_sa + (long long)slot * sv.Tp, sv.s_sa + ((long long)sv.R + slot) * sv.Tp};
+        if (staged || take > 0)
+            for (int k = tid; k < t_old; k += NT) S[k] = sa[sa_buf][k];
+        else
+            S = sa[sa_buf];                                     // nothing to merge: the stored order is read as it is
+        __syncthreads();                                        // (also: the new tokens in gtext are visible to the block)
+        for (int t0 = t_old; t0 < t; t0 += SA_CHUNK) {
+            sa_merge_chunk<NT>(tx, t0, min(t, t0 + SA_CHUNK), D, S, sa[sa_buf], sa[sa_buf ^ 1], sh.sat, tid);
+            sa_buf ^= 1;
+            fin_a0 = max(0, t0 - (D - 1));                      // sh.sat.fin[a - fin_a0]: where the last merge put suffix a
+        }
+        if (tid == 0 && take > 0) { ss->len = t; ss->sa_buf = sa_buf; }
     }
-    __syncthreads();                                            // (also: the new tokens in gtext are visible to the block)
+    if (tid == 0 && ok && a.d_app_off) ss->status = status;
+    __syncthreads();
 
     // ---------------- 2. match
     if (wib == 0) {
@@ -1171,28 +1006,16 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
     }
     __syncthreads();
     const int Lcap = min(Pe, D - 1);                            // a match node at depth D has no children
-    const int last = usable ? tx[t - 1] : 0;
-    const bool scan = want_r && t >= 2 && Lcap >= 1;
-    // one chunk of positions at a time, handed out by a counter: warps that come late from their
-    // walk in the global tree take fewer.  pass 0 counts the occurrences by match length,
-    // pass 1 (below) writes them, longest matches first.
-    const int nchunks = scan ? (t - 1 + 255) / 256 : 0;
-    auto scan_pass = [&](int pass, int* list) {
-        while (true) {
-            int c = 0;
-            if (lane == 0) c = atomicAdd(&sh.scan_next[pass], 1);
-            c = __shfl_sync(FULL, c, 0);
-            if (c >= nchunks) break;
-#pragma unroll 1
-            for (int u = 0; u < 8; ++u) {
-                const int e = c * 256 + u * 32 + lane;
-                if (e < t - 1 && tx[e] == last) {
-                    int l = 1;
-                    while (l < Lcap && e - l >= 0 && tx[e - l] == tx[t - 1 - l]) ++l;
-                    if (pass == 0) atomicAdd(&sh.r_hist[l], 1);
-                    else list[sh.r_cum[l + 1] + atomicAdd(&sh.r_fill[l], 1)] = e | ((l - 1) << OCC_POS_BITS);
-                }
-            }
+    // Per-request tree: the range of every pattern in the suffix order, a warp per pattern length.
+    // Its first suffix is the context's own end (the pattern followed by nothing); the earlier
+    // occurrences follow it.
+    const int Lr = want_r ? min(Lcap, t - 1) : 0;
+    auto request_ranges = [&]() {
+        for (int p = wib + 1; p <= Lr; p += WARPS) {
+            // the range begins with the context's own end, whose place the merge above may have just found
+            const int lo = fin_a0 >= 0 ? sh.sat.fin[t - p - fin_a0] : pattern_lo_warp(tx, t, S, t - p, p, lane);
+            const int hi = pattern_hi_warp(tx, t, S, t - p, p, lo, lane);
+            if (lane == 0) { sh.r_lo[p] = lo; sh.r_cnt[p] = max(hi - lo - 1, 0); }
         }
     };
     // Global tree: rounds of WARPS pattern lengths, shortest first, until a node can serve as
@@ -1212,8 +1035,8 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
             node = walk_from(sv.g_ent, (int)sv.g_cap, node, tx, from, t, lane, cb, wf, cntn);
             int rank = -1;
             const int nch = (int)(wf & RUN_COUNT_MASK);
-            // usable as base: at most 32 occurrences, laid down by the offline build, never touched since
-            const bool elig = occ_mode && node >= 0 && cntn <= SD_OCC_LANES && !(wf & NODE_TOUCHED) &&
+            // usable as base: at most 64 occurrences, laid down by the offline build, never touched since
+            const bool elig = occ_mode && node >= 0 && cntn <= SD_OCC_BASE && !(wf & NODE_TOUCHED) &&
                               (nch == 0 || ((wf & RUN_STATIC) && cb < sv.static_entries));
             if (elig && nch > 0 && lane == 0) rank = sv.g_lo[cb];
             if (lane == 0) {
@@ -1223,7 +1046,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
                 sh.g_rank[p - 1] = elig ? (nch > 0 ? rank : -2) : -1;   // -2: usable, and known to have no children
             }
         }
-        if (r0 == 0 && scan) scan_pass(0, nullptr);
+        if (r0 == 0) request_ranges();
         __syncthreads();
         if (tid == 0) {
             const int hi = min(PeG, r0 + WARPS);
@@ -1234,7 +1057,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         __syncthreads();
         if (sh.g_base_p || sh.g_failed) break;
     }
-    if (PeG == 0 && scan) scan_pass(0, nullptr);
+    if (PeG == 0) request_ranges();
     __syncthreads();
     if (wib == 0 && PeG > 0) {
         // the match nodes of this context, for the next call.  A pattern that does not occur ends
@@ -1244,60 +1067,50 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         if (lane < depths) ss->g_node[lane] = lane < walked ? sh.node[0][lane] : -1;
         if (lane == 0) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = depths; }
     }
-    // occurrences by match length -> r_cum; the base's occurrences (first pattern token, suffix length)
+    // the base's occurrences (first pattern token, suffix length)
     const int base_p = sh.g_base_p;
-    if (wib == 0) {
-        int h = (lane + 1 <= Lcap) ? sh.r_hist[lane + 1] : 0;   // lane L: matches of exactly L + 1 tokens
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {                      // suffix sums
-            const int y = __shfl_down_sync(FULL, h, o);
-            if (lane + o < 32) h += y;
-        }
-        sh.r_cum[lane + 1] = h;
-    } else if (wib == 1 && base_p > 0) {
+    if (wib == 1 && base_p > 0) {
         const int rank = sh.g_rank[base_p - 1];
         const int m = rank >= 0 ? sh.g_cnt[base_p - 1] : 0;
-        if (lane < m) {
-            const int pos = (int)sv.g_sa[rank + lane];
-            sh.g_pos[lane] = pos;
-            sh.g_avail[lane] = (int)sv.g_len[rank + lane] - base_p;
-            sh.g_ell[lane] = (int)sv.g_back[pos];               // for now: tokens before the occurrence in its sequence
+        for (int o = lane; o < m; o += 32) {
+            const int pos = (int)sv.g_sa[rank + o];
+            sh.g_pos[o] = pos;
+            sh.g_avail[o] = (int)sv.g_len[rank + o] - base_p;
+            sh.g_ell[o] = (int)sv.g_back[pos];                  // for now: tokens before the occurrence in its sequence
         }
         if (lane == 0) sh.g_base_m = m;
     }
     __syncthreads();
-    const int m1 = sh.r_cum[1];
-    int* const occ_smem = stx + a.stage_tokens;
-    int* const occ_list = m1 <= a.occ_cap ? occ_smem : a.occ_scratch + (long long)i * sv.Tp;
-    // what is left of the shared memory behind the list: the hash table of expand_wide_block
-    const int list_ints = m1 <= a.occ_cap ? m1 : 0;
-    int logC = 0;
-    while ((3 << (logC + 1)) <= a.occ_cap - list_ints && logC < 12) ++logC;
-    const bool coop_ok = logC >= 8;
-    int* const tkey = occ_smem + list_ints;
     const int base_m = sh.g_base_m;
-    // the 64 tokens around every occurrence of the base (one coalesced row per occurrence), then the scan's second pass
+    // the 64 tokens around every occurrence of the base (one coalesced row per occurrence)
     for (int o = wib; o < base_m; o += WARPS) {
         const long long pos = sh.g_pos[o];
         const long long q0 = pos - 32 + lane, q1 = pos + lane;
         sh.gwin[o][lane] = (q0 >= 0) ? sv.g_text[q0] : -1;
         sh.gwin[o][32 + lane] = (q1 < sv.N0) ? sv.g_text[q1] : -1;
     }
-    if (scan && m1 > 0) scan_pass(1, occ_list);
     __syncthreads();
     if (wib == 0 && base_m > 0) {
         // how far back every occurrence of the base agrees with the context
-        int ell = 0;
-        if (lane < base_m) {
-            const int back = sh.g_ell[lane];
-            const int lim = min(Lcap, t);
-            ell = base_p;
-            while (ell < lim && ell - base_p < back && sh.gwin[lane][31 - (ell - base_p)] == tx[t - 1 - ell]) ++ell;
-            sh.g_ell[lane] = ell;
+        int ell[SD_OCC_BASE / 32];
+#pragma unroll
+        for (int u = 0; u < SD_OCC_BASE / 32; ++u) {
+            const int o = lane + 32 * u;
+            ell[u] = 0;
+            if (o < base_m) {
+                const int back = sh.g_ell[o];
+                const int lim = min(Lcap, t);
+                int l = base_p;
+                while (l < lim && l - base_p < back && sh.gwin[o][31 - (l - base_p)] == tx[t - 1 - l]) ++l;
+                sh.g_ell[o] = l;
+                ell[u] = l;
+            }
         }
         // lane L: occurrences that match at least L + 1 tokens
         int c = 0;
-        for (int o = 0; o < base_m; ++o) c += (__shfl_sync(FULL, ell, o) >= lane + 1) ? 1 : 0;
+#pragma unroll
+        for (int u = 0; u < SD_OCC_BASE / 32; ++u)
+            for (int o = 0; o < 32; ++o) c += (__shfl_sync(FULL, ell[u], o) >= lane + 1) ? 1 : 0;
         sh.g_cum[lane + 1] = lane + 1 >= base_p ? c : 0;
     }
     __syncthreads();
@@ -1308,13 +1121,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         int c = 0;
         if (p <= Pe && p <= Lcap) {
             bool has = false;
-            if (tree == 1) {
-                has = want_r && sh.r_cum[p] > 0;
-                if (has && sh.r_cum[p] > COOP_MIN && coop_ok && budget_for(a.alpha, p, cap) > 0) {
-                    sh.w_job[atomicAdd(&sh.w_count, 1)] = p;     // taken up by the whole block below
-                    has = false;
-                }
-            }
+            if (tree == 1) has = p <= Lr && sh.r_cnt[p] > 0;
             else if (base_p > 0 && p >= base_p) has = sh.g_cum[p] > 0;
             else if (p <= sh.g_walked) {
                 const unsigned wf = sh.nc[0][p - 1];
@@ -1328,7 +1135,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
                 }
             }
             if (has) {
-                c = min(budget_for(a.alpha, p, cap), 2 * (D - p));
+                c = min(budget_for(a.alpha, p, cap), D - p);      // an upper bound of the job's SCORE, see below
                 if (c > 0 && tree == 0 && !(base_p > 0 && p >= base_p)) {
                     const unsigned wf = sh.nc[0][p - 1];
                     if ((int)(wf & RUN_COUNT_MASK) > WIDE_RUN && !(wf & RUN_HAS_TOP)) { sh.wide[atomicAdd(&sh.nwide, 1)] = tid; c = 0; }
@@ -1360,20 +1167,37 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         const int code = sh.job[j];
         const int tree = code / SD_MAX_DEPTH, p = code % SD_MAX_DEPTH + 1;
         const int budget = budget_for(a.alpha, p, cap);
-        if ((double)budget < best_so_far(sh)) continue;         // SCORE <= number of draft nodes
+        // SCORE <= number of draft nodes (every D <= 1), and SCORE <= number of levels below the
+        // match node: the D values of one level of a tree add up to at most 1 (Eq. 1 shares out the
+        // parent's D among its children).  A job that cannot reach the best score so far is skipped.
+        if ((double)min(budget, D - p) * 1.000000001 < best_so_far(sh)) continue;
         if (tree == 1) {
-            const int m = sh.r_cum[p];
+            const int m = sh.r_cnt[p], lo = sh.r_lo[p] + 1;
             if (m <= SD_OCC_LANES) {
-                const int e = lane < m ? (int)((unsigned)occ_list[lane] & OCC_POS_MASK) : 0;
+                const int e = lane < m ? S[lo + lane] + p - 1 : 0;       // the occurrence's last pattern token
                 const int kmax = lane < m ? min(t - 1 - e, D - p) : 0;
                 expand_occ(sh, W, tx + e, kmax, 1, p, budget, flags, lane);
             } else {
-                expand_wide_text(sh, W, tx, t, occ_list, m, p, budget, D - p, flags, lane);
+                expand_range<false>(sh, W, TextItems{tx, S, t, p}, lo, lo + m, 1, p, budget, D - p, flags, lane);
             }
         } else if (base_p > 0 && p >= base_p) {
-            const bool mine = lane < base_m && sh.g_ell[lane] >= p;
-            const int kmax = mine ? min(sh.g_avail[lane], D - p) : 0;
-            expand_occ(sh, W, &sh.gwin[lane][31 + base_p], kmax, 0, p, budget, flags, lane);
+            if (sh.g_cum[p] <= SD_OCC_LANES) {
+                // a lane per occurrence that matches p tokens: lane i takes the i-th of them
+                unsigned mk[SD_OCC_BASE / 32];
+                int o = -1, left = lane + 1;
+#pragma unroll
+                for (int u = 0; u < SD_OCC_BASE / 32; ++u) {
+                    mk[u] = __ballot_sync(FULL, lane + 32 * u < base_m && sh.g_ell[lane + 32 * u] >= p);
+                    const int c = __popc(mk[u]);
+                    if (o < 0 && left <= c) o = 32 * u + (int)__fns(mk[u], 0, left);
+                    left -= c;
+                }
+                const int kmax = o >= 0 ? min(sh.g_avail[o], D - p) : 0;
+                expand_occ(sh, W, &sh.gwin[o >= 0 ? o : 0][31 + base_p], kmax, 0, p, budget, flags, lane);
+            } else {
+                expand_range<true>(sh, W, WindowItems{sh.gwin, sh.g_avail, sh.g_ell, base_p, p}, 0, base_m, 0, p, budget, D - p,
+                                   flags, lane);
+            }
         } else {
             expand_job(sh, W, sv.g_ent, (int)sv.g_cap, 0, p, budget, flags, false, 0, lane);
         }
@@ -1387,7 +1211,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
         int kept = 0;
         for (int q = 0; q < sh.nwide; ++q) {
             const int p = sh.wide[q] % SD_MAX_DEPTH + 1;
-            if (!((double)budget_for(a.alpha, p, cap) < best)) sh.wide[kept++] = sh.wide[q];
+            if (!((double)min(budget_for(a.alpha, p, cap), D - p) * 1.000000001 < best)) sh.wide[kept++] = sh.wide[q];
         }
         sh.nwide_kept = kept;
     }
@@ -1419,39 +1243,6 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
             }
             counts_to_d(W.F, 0, fs, 1.0, sum, lane);
             expand_job(sh, W, sv.g_ent, (int)sv.g_cap, 0, p, budget, flags, true, fs, lane);
-        }
-        __syncthreads();
-    }
-
-    // Per-request jobs whose match node has hundreds of occurrences (short patterns of frequent
-    // tokens): those that can still reach the best score, longest pattern first, each by the
-    // whole block.
-    if (tid == 0) {
-        const double best = __hiloint2double((int)sh.best_hi, 0);
-        int kept = 0;
-        for (int q = 0; q < sh.w_count; ++q) {
-            const int p = sh.w_job[q];
-            if ((double)budget_for(a.alpha, p, cap) < best) continue;
-            int at = kept++;
-            while (at > 0 && sh.w_job[at - 1] < p) { sh.w_job[at] = sh.w_job[at - 1]; --at; }
-            sh.w_job[at] = p;
-        }
-        sh.w_count = kept;
-    }
-    __syncthreads();
-    const int nw = sh.w_count;
-    for (int base = 0; base < nw; base += (WARPS < 15 ? WARPS : 15)) {
-        const int nj = min(WARPS < 15 ? WARPS : 15, nw - base);  // (a group has a hardware barrier of its own: 15 of them)
-        const int G = WARPS / nj;                               // warps per job
-        const int my_job = wib / G;
-        if (my_job < nj) {
-            const int p = sh.w_job[base + my_job];
-            // the table room is shared out among the groups
-            int lg = 0;
-            while ((3 << (lg + 1)) <= (a.occ_cap - list_ints) / nj && lg < 12) ++lg;
-            int* const tk = tkey + my_job * (3 << lg);
-            expand_wide_group(sh, sh.cw[my_job], sh.w[my_job * G], tx, t, occ_list, sh.r_cum[p], p, budget_for(a.alpha, p, cap),
-                              D - p, flags, tk, tk + (1 << lg), tk + (2 << lg), lg, tid - my_job * G * 32, G * 32, 1 + my_job);
         }
         __syncthreads();
     }
@@ -1555,13 +1346,10 @@ int device_setup(int dev, int* sm_count) {
 
 template <int WARPS, int MINB>
 void launch_shape(const sd_store& s, StepArgs a, cudaStream_t st) {
-    // shared memory behind the block's working set: the text if it fits, then room for the
-    // occurrence list (at most one item per token) and the hash table of expand_wide_block
+    // shared memory behind the block's working set: the text and its suffix order (as many entries), if they fit
     const int lim = stage_limit_tokens<WARPS, MINB>();
-    a.stage_tokens = s.Tp <= lim ? s.Tp : 0;
-    const int want = s.Tp + 3 * 4096;
-    a.occ_cap = lim - a.stage_tokens < want ? lim - a.stage_tokens : want;
-    const size_t smem = ((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15) + (size_t)(a.stage_tokens + a.occ_cap) * 4;
+    a.stage_tokens = 2 * s.Tp <= lim ? s.Tp : 0;
+    const size_t smem = ((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15) + (size_t)a.stage_tokens * 8;
     speculate_fused_kernel<WARPS, MINB><<<(unsigned)a.n, WARPS * 32, smem, st>>>(s, a);
 }
 
@@ -1592,13 +1380,12 @@ int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_pa
     a.d_status = d_status;
     a.d_app_off = step ? d_app_off : nullptr; a.d_app_tok = step ? d_app_tok : nullptr;
     a.stage_tokens = 0;
-    a.occ_cap = 0;
-    a.occ_scratch = scratch;
+    a.scratch = scratch;
     cudaStream_t st = (cudaStream_t)stream;
     // a text too long for the usual shape's shared memory may still fit the one-block-per-SM shape
-    const bool long_text = s->Tp > stage_limit_tokens<CTA_WARPS, 2>();
+    const bool long_text = 2 * s->Tp > stage_limit_tokens<CTA_WARPS, 2>();
     if (n <= sms || (long_text && n <= 2 * sms)) launch_shape<CTA_WARPS_WIDE, 1>(*s, a, st);
-    else if (n > 2 * sms && s->Tp <= stage_limit_tokens<CTA_WARPS_NARROW, 4>()) launch_shape<CTA_WARPS_NARROW, 4>(*s, a, st);
+    else if (n > 2 * sms && 2 * s->Tp <= stage_limit_tokens<CTA_WARPS_NARROW, 4>()) launch_shape<CTA_WARPS_NARROW, 4>(*s, a, st);
     else launch_shape<CTA_WARPS, 2>(*s, a, st);
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;

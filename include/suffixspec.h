@@ -12,20 +12,11 @@
  * per-step calls (sd_append, sd_speculate) never allocate device memory.
  *
  * Return value: SD_OK (0) or a negative SD_ERR_* code.  Nothing aborts, throws
- * or traps.  Conditions that depend on device data (a request whose text buffer
+ * or traps.  Conditions that depend on device data (a request whose slot pool
  * ran full, an empty slot) are reported per request in d_status and leave the
  * store consistent.  A store belongs to the CUDA device that was current in
  * sd_build(); every call checks that this device is current (else
- * SD_ERR_INVALID_ARG).  Calls on one store must be ordered (one stream, or
- * events between streams): they share the store's arrays.
- *
- * The two kinds of tree.  The global tree is a flattened suffix trie in device
- * memory (sorted child runs, one 16-byte entry per node).  A per-request tree
- * is kept IMPLICITLY as the request's text x_{1:t}: its nodes are the distinct
- * substrings of at most depth_cap tokens and COUNT is the number of occurrences,
- * so appending a token is storing it, and match nodes, children and counts are
- * found by scanning the text (which a thread block holds in shared memory).
- * Every result is the one the explicit tree would give.
+ * SD_ERR_INVALID_ARG).
  *
  * Limits: depth_cap <= 32, max_spec_cap <= 64, P <= depth_cap is not required
  * (pattern lengths above depth_cap or above the context length never match).
@@ -53,8 +44,8 @@ enum {
 enum {
     SD_STATUS_OK = 0,
     SD_STATUS_BAD_SLOT = 1,       /* slot index out of range                         */
-    SD_STATUS_POOL_FULL = 2,      /* the slot's text buffer (max_req_tokens) ran full; */
-                                  /* its tree stopped growing at the last token held  */
+    SD_STATUS_POOL_FULL = 2,      /* the slot's node pool or text buffer ran full;    */
+                                  /* its tree stopped growing at the last good token  */
     SD_STATUS_GLOBAL_FULL = 4,    /* the global node pool ran full during an insert   */
     SD_STATUS_BAD_TOKEN = 8       /* a token outside [0, V) was met; the tree stopped */
                                   /* growing at the last good token                   */
@@ -75,8 +66,8 @@ typedef struct {
     int32_t max_spec_cap;         /* M: row stride of the per-draft outputs, <= 64    */
     int64_t global_extra_nodes;   /* node head-room for online inserts into the       */
                                   /* global tree; < 0: library default                */
-    int64_t slot_pool_nodes;      /* ignored (per-request trees hold no nodes; kept   */
-                                  /* so that the struct's layout stays as it was)     */
+    int64_t slot_pool_nodes;      /* node pool per slot; <= 0: library default        */
+                                  /* (2 * max_req_tokens * depth_cap)                 */
 } sd_build_params;
 
 typedef struct {
@@ -97,7 +88,7 @@ typedef struct {
     int64_t global_pool_used;     /* node entries handed out (live + abandoned)       */
     int64_t global_pool_cap;
     int64_t global_tokens;        /* tokens inserted so far                           */
-    int64_t slot_pool_nodes;      /* always 0 (per-request trees hold no nodes)       */
+    int64_t slot_pool_nodes;      /* node entries per slot                            */
     int64_t device_bytes;         /* device memory owned by the store                 */
     int32_t global_status;        /* SD_STATUS_GLOBAL_FULL or 0                       */
 } sd_stats_t;
@@ -109,15 +100,11 @@ typedef struct {
  * depth_cap tokens that occurs in some sequence, and the node's count is its
  * number of occurrences (COUNT as used by Eq. 1).  Strings do not cross
  * sequence boundaries.  The tree is built on the GPU by a depth-capped suffix
- * sort followed by adjacent-suffix LCPs.  The store keeps the corpus, its suffix
- * order and the suffix lengths as well (9 bytes per corpus token and 4 per node
- * entry): a node that no online insert has touched is a range of that order, and
- * sd_speculate reads the occurrences of a rare match node from there.
+ * sort followed by adjacent-suffix LCPs.
  *   d_corpus       int32[seq_offsets[n_seqs]]  tokens of all sequences, back to back
  *   d_seq_offsets  int64[n_seqs + 1]           start of each sequence, ascending, [0] = 0
  * n_seqs may be 0 (empty global tree; both pointers may then be NULL).
- * Also allocates max_requests empty request slots (text buffers of max_req_tokens
- * tokens and as much scratch).  Synchronises the stream.
+ * Also allocates max_requests empty per-request trees.  Synchronises the stream.
  * On success *out is the new store; on failure *out is NULL and nothing leaks.
  * Errors: INVALID_ARG (NULL, limits, a corpus token outside [0, V), offsets not
  * ascending), NOMEM (cudaMalloc failed), CUDA.
@@ -131,18 +118,15 @@ int sd_build(const sd_build_params* params, const int32_t* d_corpus, const int64
  * request's output is added to the global tree).
  * For item i in [0, n):
  *   d_slot[i] >= 0 : append tokens d_tokens[d_offsets[i] .. d_offsets[i+1]) to the
- *                    text of that slot, which is its per-request tree; if
+ *                    per-request tree (and stored context) of that slot; if
  *                    d_reset[i] != 0 the slot is emptied first (new request, the
- *                    tokens are its prompt).  A slot may appear at most once per call
- *                    (the items of a call are taken side by side).
+ *                    tokens are its prompt).  A slot may appear at most once per call.
  *   d_slot[i] == -1: insert the tokens as one whole sequence into the GLOBAL tree.
  * After the call each tree equals the tree built from scratch over its text.
  *   d_slot int32[n], d_offsets int64[n+1], d_tokens int32[d_offsets[n]],
  *   d_reset uint8[n] or NULL (no resets).
- * A slot whose text buffer would overflow keeps the tokens that fit and gets
- * SD_STATUS_POOL_FULL; a token outside [0, V) ends the item before it
- * (SD_STATUS_BAD_TOKEN).  Both stick, and the slot takes no more tokens and gets
- * no drafts, until it is reset (see sd_slot_info).
+ * A slot whose pool or text buffer would overflow keeps its state from before
+ * the offending token and gets SD_STATUS_POOL_FULL (see sd_slot_info).
  * Global tree: a sequence is inserted up to its first token outside [0, V)
  * (SD_STATUS_BAD_TOKEN in sd_stats' global_status, the other sequences of the
  * call are not affected).  When the global pool cannot hold the new nodes
@@ -153,25 +137,26 @@ int sd_build(const sd_build_params* params, const int32_t* d_corpus, const int64
  * call the insert into the global tree runs on a stream the store owns, which
  * starts behind the work `stream` holds at the call and which `stream` waits
  * for before it goes on (the two kinds of tree share nothing, so the insert
- * and the appends to the request texts run side by side).
+ * and the appends to the request trees run side by side).
  * Errors: INVALID_ARG, CUDA (launch failure).
  */
 int sd_append(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* d_offsets,
               const int32_t* d_tokens, const uint8_t* d_reset, void* stream);
 
 /*
- * sd_build_requests: start n new requests at once (Section 3, "Suffix Tree Construction": the
- * per-request tree is constructed when the request is received).  The same as sd_append with
- * d_reset = 1 for every item, with the slot and offset arrays taken from HOST memory (the caller
- * of a serving loop has them there): they are copied into a staging area of the store, one
- * kernel stores the prompts.  Nothing is allocated and the stream is not synchronised.
+ * sd_build_requests: start n new requests at once: their per-request trees are built from the
+ * prompts by the sort-based pipeline of sd_build instead of token by token (Section 3, "Suffix
+ * Tree Construction": the per-request tree is constructed when the request is received).  The
+ * result is the same as sd_append with d_reset = 1 for every item, only faster for long prompts.
  *   h_slot     int32[n]    HOST: slot of each request (each slot at most once, 0 <= slot < max_requests)
  *   h_offsets  int64[n+1]  HOST: prompt i is d_tokens[h_offsets[i] .. h_offsets[i+1]), h_offsets[0] = 0
  *   d_tokens   int32[h_offsets[n]]  DEVICE
- * Both host arrays may be reused as soon as the call returns.  A prompt longer than
- * max_req_tokens is cut there (SD_STATUS_POOL_FULL), a token outside [0, V) ends its prompt
- * before it (SD_STATUS_BAD_TOKEN).
- * Errors: INVALID_ARG (bad slot, slot twice, offsets not ascending: nothing is changed), CUDA.
+ * A prompt that does not fit the slot's node pool or text buffer leaves the slot empty with
+ * SD_STATUS_POOL_FULL.  Unlike the per-step calls this one may allocate device memory: its
+ * temporaries (about 100 bytes per prompt token of the largest batch so far) are kept by the
+ * store and reused.  It synchronises the stream before it returns.
+ * Errors: INVALID_ARG (bad slot, slot twice, offsets not ascending, token outside [0, V): nothing
+ * is changed), CAPACITY (n * vocab or the token total does not fit 31 bits), NOMEM, CUDA.
  */
 int sd_build_requests(sd_store* store, int32_t n, const int32_t* h_slot, const int64_t* h_offsets,
                       const int32_t* d_tokens, void* stream);
@@ -188,9 +173,6 @@ int sd_build_requests(sd_store* store, int32_t n, const int32_t* h_slot, const i
  * smaller index of the parent inside the speculation tree.  All scores are
  * IEEE binary64: divide, multiply root-to-leaf, add in insertion order, no FMA.
  * Section 3.2: the chosen tree is handed out only if its SCORE > params->tau.
- * One launch, one thread block per request, no global scratch except for
- * requests whose last token has more than 1,024 earlier occurrences in their own
- * text (their occurrence list goes to a buffer the store allocated in sd_build).
  * Outputs, row stride M = max_spec_cap, draft nodes in insertion order:
  *   d_n_draft     int32[n]        number of draft nodes (0: no speculation)
  *   d_tokens      int32[n][M]     token of each draft node, -1 beyond n_draft
@@ -204,7 +186,8 @@ int sd_build_requests(sd_store* store, int32_t n, const int32_t* h_slot, const i
  *   d_score       double[n]       SCORE of the chosen tree, 0.0 if none
  *   d_status      int32[n]        SD_STATUS_* of the request's slot
  *   d_budget_cap  int32[n] or NULL: per-request cap on the draft size (< 0: none)
- * The slots of a call should be distinct (a slot given twice is speculated twice).
+ * The slots of a call must be distinct; a slot that appears twice gets
+ * SD_STATUS_BAD_SLOT and no draft for its later appearances.
  * Errors: INVALID_ARG (n > max_requests, max_spec > M, P < 1, tau < 0 or NaN ...), CUDA.
  */
 int sd_speculate(sd_store* store, int32_t n, const int32_t* d_slot, const sd_spec_params* params,
@@ -215,11 +198,11 @@ int sd_speculate(sd_store* store, int32_t n, const int32_t* d_slot, const sd_spe
 /*
  * sd_step: one decode step in one launch: for every request i first append the tokens
  * d_new_tokens[d_offsets[i] .. d_offsets[i+1]) (accepted drafts + bonus token of the previous
- * step) to its text, then speculate, exactly as sd_append followed by sd_speculate on the same
- * slots would (Section 3: tokens are added to the per-request tree as they are generated;
- * Algorithm 1 then runs on the extended context).
- *   d_slot int32[n]: DISTINCT slots >= 0 (no global inserts, no resets: use sd_append for those;
- *   two blocks appending to one slot would race);
+ * step) to its per-request tree and context, then speculate, exactly as sd_append followed by
+ * sd_speculate on the same slots would (Section 3: tokens are added to the per-request tree as
+ * they are generated; Algorithm 1 then runs on the extended context).  The appends of requests
+ * with many new tokens overlap with the speculation of the others.
+ *   d_slot int32[n]: distinct slots >= 0 (no global inserts, no resets: use sd_append for those);
  *   d_offsets int64[n+1], d_new_tokens int32[d_offsets[n]]; all other arguments as sd_speculate.
  * A request whose append stops early (pool full, bad token) gets no draft and the status bits.
  */
@@ -235,29 +218,31 @@ int sd_step(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* d_
  * Some hosts of this library run where device allocation is off limits: a
  * serving loop that has handed all free device memory to its own pool, a
  * plug-in that is only given buffers and a stream, or a real-time thread that
- * may not take the allocator's locks.  sd_speculate itself does not allocate
- * either, but the scratch buffer of its kernel (the occurrence lists that do
- * not fit a block's shared memory, see sd_speculate) is memory that sd_build
- * obtained with cudaMalloc; this variant gives the same kernel a fixed array
- * inside the library image instead, and calls no allocating routine at all.
+ * may not take the allocator's locks.  sd_speculate needs no global scratch
+ * (its one kernel keeps everything in shared memory); this variant runs the
+ * library's two-kernel form of the same computation, one warp per (request,
+ * tree, pattern length), whose per-job records go through global memory, and
+ * keeps those records in a fixed array inside the library image instead of in
+ * memory from cudaMalloc.  It calls no allocating routine at all.  Unlike
+ * sd_speculate it neither uses nor refreshes the slots' cached global match
+ * nodes.
  *
  * Same arguments, outputs and results as sd_speculate.  Differences:
- *  - Size limit: n * max_req_tokens (rounded up to a multiple of 4) must not
- *    exceed SD_NOALLOC_MAX_TOKENS (e.g. 64 requests of up to 8,192 tokens); a
- *    larger batch returns SD_ERR_CAPACITY ("capacity exceeded") and launches
- *    nothing.  Split the batch instead.
- *  - The array (2 MiB) is held on every GPU that loads the library, until the
- *    process exits.
+ *  - Size limit: n * 2 * depth_cap must not exceed SD_NOALLOC_MAX_JOBS (e.g. 64
+ *    requests at depth_cap 32); a larger batch returns SD_ERR_CAPACITY
+ *    ("capacity exceeded") and launches nothing.  Split the batch instead.
+ *  - The array (about 2.1 MB) is held on every GPU that loads the library,
+ *    until the process exits.
  *  - The first call on each device looks up the array's device address (a
  *    short, synchronous runtime query; that device must be current).  Make
  *    that first call before starting any stream capture.
  *  - All calls on a device share the one array.  Its contents carry over from
  *    call to call but are never read before being rewritten, so no clearing is
  *    needed; two calls whose kernels overlap on the GPU (different streams,
- *    different stores) would overwrite each other's lists, so keep calls on
+ *    different stores) would overwrite each other's records, so keep calls on
  *    one device ordered.
  */
-#define SD_NOALLOC_MAX_TOKENS (512 * 1024)
+#define SD_NOALLOC_MAX_JOBS 4096
 int sd_speculate_noalloc(sd_store* store, int32_t n, const int32_t* d_slot, const sd_spec_params* params,
                          const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
                          int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
@@ -269,18 +254,13 @@ int sd_speculate_noalloc(sd_store* store, int32_t n, const int32_t* d_slot, cons
  *   d_tree int32[n]: -1 global tree, else slot; path i is
  *   d_paths[d_offsets[i] .. d_offsets[i+1]); d_counts int32[n] receives the count,
  *   0 when the path is not in the tree (or is longer than depth_cap).
- * For a slot the count is found by a scan of its text (one thread per path).
  */
 int sd_query_counts(sd_store* store, int32_t n, const int32_t* d_tree, const int64_t* d_offsets,
                     const int32_t* d_paths, int32_t* d_counts, void* stream);
 
 /*
- * sd_slot_info: per-slot context length, node count of the per-request tree and status.
- *   d_slot int32[n], n <= 65,535; outputs int32[n] each, any may be NULL.
- * The node count is the number of distinct substrings of at most depth_cap tokens of the
- * slot's text; it is computed on demand by comparing every start position with the earlier
- * ones (quadratic in the text length: a checking aid, not a per-step call).  Pass
- * d_nodes = NULL to skip it.
+ * sd_slot_info: per-slot context length, live node count and status.
+ *   d_slot int32[n]; outputs int32[n] each, any may be NULL.
  */
 int sd_slot_info(sd_store* store, int32_t n, const int32_t* d_slot, int32_t* d_len, int32_t* d_nodes,
                  int32_t* d_status, void* stream);
@@ -292,8 +272,7 @@ int sd_slot_info(sd_store* store, int32_t n, const int32_t* d_slot, int32_t* d_l
  * sum of the children's counts.  A low value says the next token is predictable from its
  * prefix, i.e. that suffix-tree speculation will work well on this kind of text.
  *   tree: -1 global tree, else a slot.  h_entropy: HOST double.  An empty tree gives 0.
- * An offline analysis call: allocates temporary device memory and synchronises the stream
- * (for a slot the work is quadratic in the text length).
+ * An offline analysis call: allocates temporary device memory and synchronises the stream.
  * Sums are accumulated with atomics, so the last bits vary from call to call.
  */
 int sd_entropy(sd_store* store, int32_t tree, double* h_entropy, void* stream);

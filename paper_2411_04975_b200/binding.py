@@ -18,8 +18,8 @@ from . import build as _build
 FLAG_GLOBAL_ONLY, FLAG_REQUEST_ONLY, FLAG_LINEAR = 1, 2, 4
 STATUS_BAD_SLOT, STATUS_POOL_FULL, STATUS_GLOBAL_FULL, STATUS_BAD_TOKEN = 1, 2, 4, 8
 
-EXPORTS = ["sd_build", "sd_build_requests", "sd_append", "sd_speculate", "sd_step", "sd_speculate_noalloc", "sd_query_counts", "sd_slot_info", "sd_entropy", "sd_stats", "sd_free",
-           "sd_strerror"]
+EXPORTS = ["sd_build", "sd_build_requests", "sd_append", "sd_speculate", "sd_step", "sd_speculate_noalloc", "sd_query_counts",
+           "sd_slot_info", "sd_entropy", "sd_stats", "sd_free", "sd_strerror", "sd_debug_fail_alloc"]
 
 
 class SuffixSpecError(RuntimeError):
@@ -80,6 +80,8 @@ def library() -> C.CDLL:
         lib.sd_stats.argtypes = [vp, C.POINTER(_Stats), vp]
         lib.sd_free.restype = None
         lib.sd_free.argtypes = [vp]
+        lib.sd_debug_fail_alloc.restype = None
+        lib.sd_debug_fail_alloc.argtypes = [C.c_int64]
         lib.sd_strerror.restype = C.c_char_p
         lib.sd_strerror.argtypes = [C.c_int]
         _lib = lib

@@ -1,9 +1,8 @@
-// sd_append: the append of accepted tokens to the requests' texts (the implicit per-request trees,
-// see common.cuh) and the level-by-level insert of whole sequences into the global tree.
+// sd_append: the batched append kernel for the per-request trees (see append_core.cuh for how one
+// token is appended) and the level-by-level insert of whole sequences into the global tree.
 #include <cooperative_groups.h>
 
 #include "append_core.cuh"
-#include "suffix_order.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -139,7 +138,7 @@ __device__ __forceinline__ void gi_insert(GiShared* sh0, const sd_store& sv, int
         else {
             ++my_live;
             if (d == 1) {
-                ent[fresh] = make_int4(x, 1, 0, (int)NODE_TOUCHED);
+                ent[fresh] = make_int4(x, 1, 0, 0);
                 sv.g_root[x] = fresh;
                 nxt = fresh;
                 new_room = D - 1;
@@ -285,7 +284,6 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                     else if (nc > 0) found = lookup_child<8, true>(ent, cb, nc, x, pos, fe);
                     if (found >= 0) {
                         atomicAdd(word(&ent[found], 1), 1);
-                        if (!((unsigned)fe.w & NODE_TOUCHED)) atomicOr(word(&ent[found], 3), (int)NODE_TOUCHED);
                         // a count changes: the copies in the run's top block (if any) are stale from now on
                         if (d > 1 && (w & RUN_HAS_TOP)) atomicAnd(word(&ent[cur], 3), (int)~RUN_HAS_TOP);
                     }
@@ -299,10 +297,10 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                 // of new leaves, written here in one go if the room behind the node holds it.
                 if (own && rem > d && new_room >= rem - d) {
                     *word(&ent[nxt], 2) = nxt + 1;
-                    *word(&ent[nxt], 3) = (int)(1u | NODE_TOUCHED);
+                    *word(&ent[nxt], 3) = 1;
                     for (int j = d + 1; j <= rem; ++j)
-                        ent[nxt + j - d] = j < rem ? make_int4(d_tokens[k + j - 1], 1, nxt + j - d + 1, (int)(1u | NODE_TOUCHED))
-                                                   : make_int4(d_tokens[k + j - 1], 1, 0, (int)NODE_TOUCHED);
+                        ent[nxt + j - d] = j < rem ? make_int4(d_tokens[k + j - 1], 1, nxt + j - d + 1, 1)
+                                                   : make_int4(d_tokens[k + j - 1], 1, 0, 0);
                     my_live += rem - d;
                     rem = 0;
                 }
@@ -326,7 +324,6 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
                             }
                             if (found >= 0) {
                                 atomicAdd(word(&ent[found], 1), 1);
-                                if (!((unsigned)fe.w & NODE_TOUCHED)) atomicOr(word(&ent[found], 3), (int)NODE_TOUCHED);
                                 nxt = found; seen_cb = cb; seen_n = nc;
                                 pending = false;
                             }
@@ -370,94 +367,48 @@ global_insert_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d
     }
 }
 
-// One block per item: the item's tokens go behind the slot's text (a reset empties the slot
-// first) and the suffix order of the text is brought up to date, SA_CHUNK tokens at a time
-// (suffix_order.cuh).  A token outside [0, V) ends the item there (SD_STATUS_BAD_TOKEN), a full
-// text buffer likewise (SD_STATUS_POOL_FULL); both stick until the slot is reset.  Items for the
-// global tree are taken by global_insert_kernel.  Text and order are staged in shared memory
-// when they fit (stage_tokens > 0), else the block works on the global arrays.
-constexpr int TA_THREADS = 256;
-
-__global__ void __launch_bounds__(TA_THREADS)
-slot_append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_tokens,
-                   const uint8_t* d_reset, int reset_all, int stage_tokens) {
-    extern __shared__ __align__(16) int ta_smem[];
-    __shared__ SaTemp tmp;
-    __shared__ int first_bad;
-    const int tid = threadIdx.x;
-    const int i = blockIdx.x;
-    if (i >= n) return;
+// Warp i + 1 of the grid appends item i to its request slot (items for the global tree are
+// taken by global_insert_kernel).
+__global__ void append_kernel(sd_store sv, int n, const int32_t* d_slot, const int64_t* d_offsets,
+                              const int32_t* d_tokens, const uint8_t* d_reset) {
+    const int lane = threadIdx.x & 31;
+    const int warp = (int)((blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5);
+    if (warp > n || warp == 0) return;
+    const int i = warp - 1;
     const int slot = d_slot[i];
     if (slot < 0 || slot >= sv.R) return;
     SlotState* ss = sv.s_state + slot;
-    int32_t* text = sv.s_text + (long long)slot * sv.Tp;
-    int len = ss->len, status = ss->status, buf = ss->sa_buf;
-    const bool reset = reset_all || (d_reset && d_reset[i]);
-    if (reset) { len = 0; status = 0; }
-    const long long b = d_offsets[i];
-    const long long cnt = d_offsets[i + 1] - b;
-    int take = 0;
-    if (!(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && cnt > 0) {
-        const int room = sv.T - len;
-        take = (int)min((long long)room, cnt);
-        if (tid == 0) first_bad = take;
-        __syncthreads();
-        for (int k = tid; k < take; k += TA_THREADS) {
-            const int x = d_tokens[b + k];
-            if (x < 0 || x >= sv.V) atomicMin(&first_bad, k);
-        }
-        __syncthreads();
-        const int good = first_bad;
-        if (good < take) status |= SD_STATUS_BAD_TOKEN;            // the bad token comes before the buffer's end
-        else if ((long long)take < cnt) status |= SD_STATUS_POOL_FULL;
-        take = good;
+    int32_t* text = sv.s_text + (long long)slot * sv.T;
+    TreeRef tr{sv.s_ent + (long long)slot * sv.spn, sv.s_root + (long long)slot * sv.V, (int)sv.spn};
+    int len = ss->len, used = ss->used, live = ss->live, status = ss->status;
+    int act = ss->active[lane], room = ss->room[lane], run_cb = ss->run_cb[lane];
+    unsigned run_w = ss->run_w[lane];
+    if (d_reset && d_reset[i]) {
+        // forget the old tree: only root-table cells of tokens that occur can be set
+        for (int k = lane; k < len; k += 32) tr.root[text[k]] = -1;
+        __syncwarp();
+        len = 0; used = 0; live = 0; status = 0; act = -1; room = 0; run_cb = 0; run_w = 0;
+        if (lane == 0) ss->gen += 1;
     }
-    if (take > 0) {
-        const bool staged = stage_tokens >= len + take;
-        int* tx = staged ? ta_smem : text;
-        int* S = staged ? ta_smem + stage_tokens : sv.occ_scratch + (long long)slot * sv.Tp;
-        int32_t* sa[2] = {sv.s_sa + (long long)slot * sv.Tp, sv.s_sa + ((long long)sv.R + slot) * sv.Tp};
-        for (int k = tid; k < take; k += TA_THREADS) text[len + k] = d_tokens[b + k];
-        if (staged) {
-            for (int k = tid; k < len; k += TA_THREADS) tx[k] = text[k];
-            for (int k = tid; k < take; k += TA_THREADS) tx[len + k] = d_tokens[b + k];
+    const long long b = d_offsets[i], e = d_offsets[i + 1];
+    for (long long k = b; k < e && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)); ++k) {
+        const int x = d_tokens[k];
+        if (x < 0 || x >= sv.V) { status |= SD_STATUS_BAD_TOKEN; break; }
+        if (len >= sv.T || !append_token(tr, sv.D, x, len, lane, act, room, run_cb, run_w, used, live)) {
+            status |= SD_STATUS_POOL_FULL;
+            break;
         }
-        for (int k = tid; k < len; k += TA_THREADS) S[k] = sa[buf][k];
-        __syncthreads();
-        for (int t0 = len; t0 < len + take; t0 += SA_CHUNK) {
-            const int t1 = min(len + take, t0 + SA_CHUNK);
-            sa_merge_chunk<TA_THREADS>(tx, t0, t1, sv.D, S, sa[buf], sa[buf ^ 1], tmp, tid);
-            buf ^= 1;
-        }
+        if (lane == 0) text[len] = x;
+        ++len;
     }
-    if (tid == 0) {
-        ss->len = len + take;
-        ss->status = status;
-        ss->sa_buf = buf;
-        if (reset) ss->gen += 1;
-    }
+    ss->active[lane] = act;
+    ss->room[lane] = room;
+    ss->run_cb[lane] = run_cb;
+    ss->run_w[lane] = run_w;
+    if (lane == 0) { ss->len = len; ss->used = used; ss->live = live; ss->status = status; }
 }
 
 }  // namespace
-
-// Shared by sd_append and sd_build_requests.
-int sd_launch_text_append(sd_store* s, int32_t n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_tokens,
-                          const uint8_t* d_reset, int reset_all, cudaStream_t st) {
-    // text and suffix order of a slot in shared memory if both fit (2 x Tp ints), else in place
-    const long long want = 2ll * s->Tp * 4;
-    const int stage = want <= 200 * 1024 ? s->Tp : 0;
-    const size_t smem = stage ? (size_t)want : 0;
-    if (smem > 48 * 1024) {
-        static bool raised[64] = {false};
-        if (s->device >= 0 && s->device < 64 && !raised[s->device]) {
-            SD_CUDA_OK(cudaFuncSetAttribute(slot_append_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-            raised[s->device] = true;
-        }
-    }
-    slot_append_kernel<<<(unsigned)n, TA_THREADS, smem, st>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset, reset_all, stage);
-    SD_CUDA_OK(cudaGetLastError());
-    return SD_OK;
-}
 
 extern "C" int sd_append(sd_store* s, int32_t n, const int32_t* d_slot, const int64_t* d_offsets,
                          const int32_t* d_tokens, const uint8_t* d_reset, void* stream) {
@@ -465,7 +416,9 @@ extern "C" int sd_append(sd_store* s, int32_t n, const int32_t* d_slot, const in
     SD_CHECK_DEVICE(s);
     if (n == 0) return SD_OK;
     if (!d_slot || !d_offsets) return SD_ERR_INVALID_ARG;
-    // The global tree and the request texts share nothing: the insert into the global tree runs
+    const int warps_per_block = 4;
+    const unsigned blocks = (unsigned)((n + 1 + warps_per_block - 1) / warps_per_block);
+    // The global tree and the request trees share nothing: the insert into the global tree runs
     // beside the appends, on the store's own stream, which starts behind everything the caller's
     // stream holds so far and which the caller's stream waits for before it goes on.
     cudaStream_t st = (cudaStream_t)stream;
@@ -474,8 +427,8 @@ extern "C" int sd_append(sd_store* s, int32_t n, const int32_t* d_slot, const in
     global_insert_kernel<<<GI_CTAS, GI_THREADS, 0, s->aux>>>(*s, n, d_slot, d_offsets, d_tokens);
     SD_CUDA_OK(cudaGetLastError());
     SD_CUDA_OK(cudaEventRecord(s->ev_join, s->aux));
-    const int rc = sd_launch_text_append(s, n, d_slot, d_offsets, d_tokens, d_reset, 0, st);
-    if (rc != SD_OK) return rc;
+    append_kernel<<<blocks, warps_per_block * 32, 0, st>>>(*s, n, d_slot, d_offsets, d_tokens, d_reset);
+    SD_CUDA_OK(cudaGetLastError());
     SD_CUDA_OK(cudaStreamWaitEvent(st, s->ev_join, 0));
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;

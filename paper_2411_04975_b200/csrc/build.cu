@@ -3,7 +3,7 @@
 // then all depths at once: ballot scans over (lcp, len) give every node's rank, range
 // and parent, and one kernel lays the nodes down as sorted child runs in pre-order.
 // Hand-written LSD radix sort and scans (no CUB / Thrust).
-// Also: sd_build_requests (the texts of new requests) and the store's life cycle.
+// Also: sd_build_requests (the trees of a batch of new requests by the same pipeline).
 #include <algorithm>
 #include <new>
 #include <stdio.h>
@@ -254,8 +254,7 @@ int radix_sort_pairs(SortBuffers& b, i64 n, int bits_lo, int bits_hi, cudaStream
 
 // ------------------------------------------------------------------ suffix order
 // end_pos[i]: one past the last token of the sequence that holds position i.
-// back[i] (optional): tokens before position i inside its sequence, capped at D.
-__global__ void seq_end_kernel(const int64_t* seq_offsets, int n_seqs, i64 n, int* end_pos, uint8_t* back, int D) {
+__global__ void seq_end_kernel(const int64_t* seq_offsets, int n_seqs, i64 n, int* end_pos) {
     i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     int lo = 0, hi = n_seqs;                          // largest s with seq_offsets[s] <= i
@@ -264,7 +263,6 @@ __global__ void seq_end_kernel(const int64_t* seq_offsets, int n_seqs, i64 n, in
         if (seq_offsets[mid] <= i) lo = mid; else hi = mid;
     }
     end_pos[i] = (int)seq_offsets[lo + 1];
-    if (back) back[i] = (uint8_t)min((i64)D, i - (i64)seq_offsets[lo]);
 }
 
 // bad[0] != 0 when a token is outside [0, V) or the offsets do not ascend from 0
@@ -300,6 +298,51 @@ __global__ void assign_rank_kernel(const u64* keys, const uint32_t* vals, const 
     if (j >= n) return;
     int flag = j == 0 ? 1 : (keys[j] != keys[j - 1] ? 1 : 0);
     rank_out[vals[j]] = ex[j] + flag;                 // dense, 1-based
+}
+
+// Suffix order of sequences that are sorted one by one (the trees of different requests share
+// nothing, so no suffix of one request is ever compared with a suffix of another): one block per
+// sequence, tokens and suffix indices in shared memory, bitonic sort with a comparison of at most
+// D tokens.  Order: by the first D tokens, a suffix that ends earlier before its extensions, equal
+// strings by position, which is the order the prefix-doubling rounds produce.  One launch instead of
+// about a hundred, which is what counts when a few prompts are built in the middle of a decode loop.
+constexpr int BS_THREADS = 1024;
+constexpr int BS_MAX_LEN = 16384;              // longest sequence (2 x 64 KB of shared memory)
+
+__global__ void __launch_bounds__(BS_THREADS)
+block_suffix_sort_kernel(const int32_t* tok, const int64_t* seq_off, int D, uint32_t* sa) {
+    extern __shared__ int bs_smem[];
+    const i64 b = seq_off[blockIdx.x], e = seq_off[blockIdx.x + 1];
+    const int n = (int)(e - b), tid = threadIdx.x;
+    if (n <= 0) return;
+    int np = 1;
+    while (np < n) np <<= 1;
+    int* t = bs_smem;                          // [n] tokens
+    int* idx = bs_smem + n;                    // [np] suffixes (>= n: padding, sorts last)
+    for (int i = tid; i < n; i += BS_THREADS) t[i] = tok[b + i];
+    for (int i = tid; i < np; i += BS_THREADS) idx[i] = i;
+    __syncthreads();
+    auto less = [&](int a, int c) -> bool {    // strict total order, a != c
+        if (a >= n || c >= n) return a < c;
+        const int la = min(D, n - a), lc = min(D, n - c), m = min(la, lc);
+        for (int l = 0; l < m; ++l) {
+            const int x = t[a + l], y = t[c + l];
+            if (x != y) return x < y;
+        }
+        if (la != lc) return la < lc;
+        return a < c;
+    };
+    for (int k = 2; k <= np; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int q = tid; q < (np >> 1); q += BS_THREADS) {
+                const int i = ((q & ~(j - 1)) << 1) | (q & (j - 1)), p = i | j;
+                const int a = idx[i], c = idx[p];
+                const bool up = (i & k) == 0;
+                if (less(c, a) == up) { idx[i] = c; idx[p] = a; }
+            }
+            __syncthreads();
+        }
+    for (int i = tid; i < n; i += BS_THREADS) sa[b + i] = (uint32_t)(b + idx[i]);
 }
 
 // lcp[j] = common prefix (capped) of sorted suffixes j-1 and j; len[j] = capped length of suffix j
@@ -565,7 +608,7 @@ __global__ void fill_top_kernel(const int* list, const int* nchild, const int* r
 // of the one before it.
 __global__ void emit_nodes_kernel(const int32_t* tok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len, i64 n,
                                   LevelTables T, const int* nbase, const int* nchild, const int* runstart, int4* ent,
-                                  int32_t* root, int32_t* run_owner_rank) {
+                                  int32_t* root) {
     const i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
     const int l = lcp[j], m = len[j];
@@ -587,8 +630,6 @@ __global__ void emit_nodes_kernel(const int32_t* tok, const uint32_t* sa, const 
         const int tb = top_block_of(nid, nc);
         e.z = nc > 0 ? runstart[nid] + tb : 0;
         e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC | (tb ? RUN_HAS_TOP : 0u)) : 0;
-        // the node's occurrences are the suffixes j .. j + count - 1 of the suffix order
-        if (nc > 0) run_owner_rank[e.z] = (int)j;
         const int pos = runstart[pnid] + top_block_of(pnid, nchild[pnid]) + rank;
         ent[pos] = e;
         if (d == 1) root[e.x] = pos;
@@ -600,25 +641,30 @@ __global__ void init_global_state_kernel(GlobalState* g, int used, int live, lon
     g->used = used; g->live = live; g->status = 0; g->epoch = 1; g->tokens = tokens;
 }
 
-// Test hook: the k-th device allocation from now on fails (k = 1: the next one); 0 switches it off.
-// Only the allocation-failure tests use it; nothing else in the library reads it.
-static long long g_fail_alloc_in = 0;
+}  // namespace
 
+// Test hook: the k-th device allocation from now on fails (k = 1: the next one); 0 switches it off.
+// Only the allocation-failure tests use it.
+static long long g_fail_alloc_in = 0;
 static cudaError_t sd_device_malloc(void** p, size_t bytes) {
     if (g_fail_alloc_in > 0 && --g_fail_alloc_in == 0) { *p = nullptr; return cudaErrorMemoryAllocation; }
     return cudaMalloc(p, bytes);
 }
+extern "C" void sd_debug_fail_alloc(int64_t k) { g_fail_alloc_in = k; }
 
-struct DeviceArena {          // temporaries of one build: freed together
+namespace {
+
+struct DeviceArena {          // temporaries of one build: freed together, or kept in a workspace
     void* ptr[48];
     int n = 0;
+    sd_workspace* keep = nullptr;                     // if set, buffers live there and are reused
     char* chunk = nullptr;                            // reserved block the next buffers are carved from
     long long chunk_left = 0;
-    ~DeviceArena() { for (int i = 0; i < n; ++i) cudaFree(ptr[i]); }
+    ~DeviceArena() { if (!keep) for (int i = 0; i < n; ++i) cudaFree(ptr[i]); }
     // One allocation for the buffers to come (an allocation of its own costs far more than the
     // kernels that use a buffer).  If it fails the buffers are simply allocated one by one.
     void reserve(long long bytes) {
-        if (n >= 48 || bytes <= 0) return;
+        if (keep || n >= 48 || bytes <= 0) return;
         void* p = nullptr;
         if (sd_device_malloc(&p, (size_t)bytes) != cudaSuccess) { cudaGetLastError(); return; }
         ptr[n++] = p;
@@ -628,12 +674,24 @@ struct DeviceArena {          // temporaries of one build: freed together
         if (count < 1) count = 1;
         const long long need = (long long)count * (long long)sizeof(T);
         const long long padded = (need + 255) / 256 * 256;
-        if (chunk_left >= padded) {
+        if (!keep && chunk_left >= padded) {
             *out = (T*)chunk;
             chunk += padded; chunk_left -= padded;
             return true;
         }
         if (n >= 48) return false;
+        if (keep) {
+            const int k = n++;
+            if (keep->bytes[k] < need) {
+                if (keep->ptr[k]) cudaFree(keep->ptr[k]);
+                keep->ptr[k] = nullptr; keep->bytes[k] = 0;
+                const long long want = need + need / 4 + 256;
+                if (sd_device_malloc(&keep->ptr[k], (size_t)want) != cudaSuccess) { cudaGetLastError(); return false; }
+                keep->bytes[k] = want;
+            }
+            *out = (T*)keep->ptr[k];
+            return true;
+        }
         void* p = nullptr;
         if (sd_device_malloc(&p, (size_t)need) != cudaSuccess) { cudaGetLastError(); return false; }
         ptr[n++] = p;
@@ -652,8 +710,6 @@ int bits_for(i64 maxval) {
 
 }  // namespace
 
-extern "C" void sd_debug_fail_alloc(int64_t k) { g_fail_alloc_in = k; }
-
 template <class T>
 static bool store_alloc(sd_store* s, T** out, long long count) {
     void* p = nullptr;
@@ -667,9 +723,11 @@ static bool store_alloc(sd_store* s, T** out, long long count) {
 static void store_release(sd_store* s) {
     if (!s) return;
     cudaFree(s->g_ent); cudaFree(s->g_root); cudaFree(s->g_state);
-    cudaFree(s->g_text); cudaFree(s->g_sa); cudaFree(s->g_len); cudaFree(s->g_back); cudaFree(s->g_lo);
-    cudaFree(s->s_text); cudaFree(s->s_sa); cudaFree(s->s_state); cudaFree(s->occ_scratch);
-    cudaFree(s->stage_slot); cudaFree(s->stage_off);
+    cudaFree(s->s_ent); cudaFree(s->s_root); cudaFree(s->s_text); cudaFree(s->s_state);
+    if (s->ws) {
+        for (int k = 0; k < 48; ++k) cudaFree(s->ws->ptr[k]);
+        delete s->ws;
+    }
     if (s->ev_fork) cudaEventDestroy(s->ev_fork);
     if (s->ev_join) cudaEventDestroy(s->ev_join);
     if (s->aux) cudaStreamDestroy(s->aux);
@@ -691,11 +749,13 @@ struct Pipeline {
     int n_wide = 0;
 };
 
-// max_token: largest token value + 1 (sets the number of radix passes).  back: receives, per text
-// position, the number of tokens before it inside its sequence (capped at D).
+// max_token: largest token value + 1 (sets the number of radix passes).  top_blocks: reserve
+// room for top blocks in front of long runs.  per_seq_max_len > 0: the sequences are independent
+// (tokens of different sequences never compare equal, sequence k's tokens below sequence k + 1's)
+// and none is longer than that, so each is sorted by a block of its own.
 // Returns SD_OK, SD_ERR_NOMEM or SD_ERR_CUDA.
 static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_offsets, int n_seqs, i64 N,
-                        i64 max_token, int D, uint8_t* back, cudaStream_t st) {
+                        i64 max_token, int D, bool top_blocks, cudaStream_t st, i64 per_seq_max_len = 0) {
     const int T256 = 256;
     P.N = N;
     DeviceArena& tmp = P.tmp;
@@ -720,8 +780,19 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     int *end_pos = P.end_pos, **rank = P.rank, **comb = P.comb, *ex = P.ex;
     uint8_t *lcp = P.lcp, *len = P.len;
 
-    seq_end_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_seq_offsets, n_seqs, N, end_pos, back, D);
-    rank0_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tok, N, rank[0]);
+    seq_end_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_seq_offsets, n_seqs, N, end_pos);
+    const bool block_sort = per_seq_max_len > 0 && per_seq_max_len <= BS_MAX_LEN;
+    if (block_sort) {
+        i64 np = 1;
+        while (np < per_seq_max_len) np <<= 1;
+        const size_t smem = (size_t)(per_seq_max_len + np) * sizeof(int);
+        if (smem > 48 * 1024 &&
+            cudaFuncSetAttribute(block_suffix_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)((BS_MAX_LEN * 2) * sizeof(int))) != cudaSuccess)
+            return SD_ERR_CUDA;
+        block_suffix_sort_kernel<<<(unsigned)n_seqs, BS_THREADS, smem, st>>>(d_tok, d_seq_offsets, D, sb.vals[0]);
+    } else
+        rank0_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tok, N, rank[0]);
     const int bits_tok = bits_for(max_token + 1), bits_rank = bits_for(N + 1);
     int sorted = 0;
     // rank[k] orders the first 2^k tokens of every suffix
@@ -734,7 +805,9 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
             assign_rank_kernel<<<grid_for(N, T256), T256, 0, st>>>(sb.keys[sorted], sb.vals[sorted], ex, N, rout);
         }
     };
-    if (m == 0) {
+    if (block_sort) {
+        // sb.vals[0] holds the suffix order already
+    } else if (m == 0) {
         round(rank[0], rank[0], 1 << 30, nullptr);        // D == 1: the first token alone
     } else {
         const bool pow2 = D == (1 << m);
@@ -787,10 +860,11 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     else ms_apply_kernel<MS_CHUNKS><<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, P.nbase, lv);
     count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, P.nbase, lv, P.nchild);
     // child runs (with their top blocks) in node (pre-)order
-    exclusive_scan(RunAlloc{P.nchild, 1}, n_nodes + 1, P.runstart, P.big_tmp, st);
+    exclusive_scan(RunAlloc{P.nchild, top_blocks ? 1 : 0}, n_nodes + 1, P.runstart, P.big_tmp, st);
     int* wide_counter = P.wide_counter;
     ce = cudaMemsetAsync(wide_counter, 0, sizeof(int), st);
-    collect_wide_kernel<<<grid_for(n_nodes + 1, T256), T256, 0, st>>>(P.nchild, n_nodes + 1, P.wide_list, wide_counter);
+    if (top_blocks)
+        collect_wide_kernel<<<grid_for(n_nodes + 1, T256), T256, 0, st>>>(P.nchild, n_nodes + 1, P.wide_list, wide_counter);
     int h_total = 0;
     if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_total, P.runstart + n_nodes + 1, sizeof(int), cudaMemcpyDeviceToHost, st);
     if (ce == cudaSuccess) ce = cudaMemcpyAsync(&P.n_wide, wide_counter, sizeof(int), cudaMemcpyDeviceToHost, st);
@@ -805,8 +879,7 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
     if (!out) return SD_ERR_INVALID_ARG;
     *out = nullptr;
     if (!p || p->vocab < 1 || p->depth_cap < 1 || p->depth_cap > SD_MAX_DEPTH || p->max_requests < 1 ||
-        p->max_req_tokens < 1 || p->max_req_tokens >= (1 << 27) || p->max_spec_cap < 1 || p->max_spec_cap > SD_MAX_SPEC ||
-        n_seqs < 0)
+        p->max_req_tokens < 1 || p->max_spec_cap < 1 || p->max_spec_cap > SD_MAX_SPEC || n_seqs < 0)
         return SD_ERR_INVALID_ARG;
     if (n_seqs > 0 && (!d_corpus || !d_seq_offsets)) return SD_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
@@ -822,17 +895,14 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
     if (!s) return SD_ERR_NOMEM;
     memset(s, 0, sizeof(*s));
     s->V = p->vocab; s->D = p->depth_cap; s->R = p->max_requests; s->T = p->max_req_tokens; s->M = p->max_spec_cap;
-    s->Tp = (s->T + 3) & ~3;
-    s->N0 = N;
     if (cudaGetDevice(&s->device) != cudaSuccess) { delete s; return SD_ERR_CUDA; }
     const int D = s->D;
+    s->spn = p->slot_pool_nodes > 0 ? p->slot_pool_nodes : 2ll * s->T * D;
+    if (s->spn >= (1ll << 31) - 2) { delete s; return SD_ERR_INVALID_ARG; }
 
     bool ok = store_alloc(s, &s->g_root, s->V) && store_alloc(s, &s->g_state, 1) &&
-              store_alloc(s, &s->s_text, (i64)s->R * s->Tp) && store_alloc(s, &s->s_sa, 2ll * s->R * s->Tp) &&
-              store_alloc(s, &s->s_state, s->R) &&
-              store_alloc(s, &s->occ_scratch, (i64)s->R * s->Tp) && store_alloc(s, &s->stage_slot, s->R) &&
-              store_alloc(s, &s->stage_off, s->R + 1) && store_alloc(s, &s->g_text, N) && store_alloc(s, &s->g_sa, N) &&
-              store_alloc(s, &s->g_len, N) && store_alloc(s, &s->g_back, N);
+              store_alloc(s, &s->s_ent, (i64)s->R * s->spn) && store_alloc(s, &s->s_root, (i64)s->R * s->V) &&
+              store_alloc(s, &s->s_text, (i64)s->R * s->T) && store_alloc(s, &s->s_state, s->R);
     if (!ok) { store_release(s); return SD_ERR_NOMEM; }
     if (cudaStreamCreateWithFlags(&s->aux, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -842,6 +912,7 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
         return SD_ERR_CUDA;
     }
     cudaError_t ce = cudaMemsetAsync(s->g_root, 0xFF, sizeof(int32_t) * (size_t)s->V, st);
+    if (ce == cudaSuccess) ce = cudaMemsetAsync(s->s_root, 0xFF, sizeof(int32_t) * (size_t)s->R * s->V, st);
     if (ce == cudaSuccess) ce = cudaMemsetAsync(s->s_state, 0, sizeof(SlotState) * (size_t)s->R, st);
     if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
 
@@ -861,7 +932,7 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
             if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
             if (h_bad) { store_release(s); return SD_ERR_INVALID_ARG; }
         }
-        const int rc = pipeline_run(P, d_corpus, d_seq_offsets, n_seqs, N, s->V, D, s->g_back, st);
+        const int rc = pipeline_run(P, d_corpus, d_seq_offsets, n_seqs, N, s->V, D, true, st);
         if (rc != SD_OK) { store_release(s); return rc; }
         n_nodes = P.n_nodes;
         used_entries = P.used_entries;
@@ -869,22 +940,14 @@ extern "C" int sd_build(const sd_build_params* p, const int32_t* d_corpus, const
 
     i64 extra = p->global_extra_nodes >= 0 ? p->global_extra_nodes : std::max<i64>(1ll << 22, n_nodes);
     s->g_cap = used_entries + extra;
-    s->static_entries = used_entries;
     if (s->g_cap >= (1ll << 31) - 2) { store_release(s); return SD_ERR_INVALID_ARG; }
-    if (!store_alloc(s, &s->g_ent, s->g_cap) || !store_alloc(s, &s->g_lo, used_entries)) {
-        store_release(s);
-        return SD_ERR_NOMEM;
-    }
+    if (!store_alloc(s, &s->g_ent, s->g_cap)) { store_release(s); return SD_ERR_NOMEM; }
 
     if (N > 0) {
-        // write the entries; keep the text, the suffix order and the suffix lengths
+        // write the entries
         emit_nodes_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_corpus, P.sa, P.lcp, P.len, N, P.lv, P.nbase, P.nchild,
-                                                             P.runstart, s->g_ent, s->g_root, s->g_lo);
+                                                             P.runstart, s->g_ent, s->g_root);
         if (P.n_wide > 0) fill_top_kernel<<<P.n_wide, 256, 0, st>>>(P.wide_list, P.nchild, P.runstart, s->g_ent);
-        ce = cudaMemcpyAsync(s->g_text, d_corpus, sizeof(int32_t) * (size_t)N, cudaMemcpyDeviceToDevice, st);
-        if (ce == cudaSuccess) ce = cudaMemcpyAsync(s->g_sa, P.sa, sizeof(uint32_t) * (size_t)N, cudaMemcpyDeviceToDevice, st);
-        if (ce == cudaSuccess) ce = cudaMemcpyAsync(s->g_len, P.len, (size_t)N, cudaMemcpyDeviceToDevice, st);
-        if (ce != cudaSuccess) { store_release(s); return SD_ERR_CUDA; }
     }
     init_global_state_kernel<<<1, 1, 0, st>>>(s->g_state, (int)used_entries, (int)n_nodes, N);
     ce = cudaStreamSynchronize(st);
@@ -912,11 +975,147 @@ extern "C" const char* sd_strerror(int code) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// sd_build_requests: start a batch of new requests.  A per-request tree is its text (common.cuh),
-// so building one is storing the prompt: the host arrays go to a staging area the store owns
-// and one kernel copies the prompts.  Nothing is allocated and the stream is not synchronised.
-int sd_launch_text_append(sd_store* s, int32_t n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_tokens,
-                          const uint8_t* d_reset, int reset_all, cudaStream_t st);
+// sd_build_requests: the per-request trees of a batch of new requests, built from their prompts
+// by the same sort-based pipeline as the global tree instead of token by token.  The prompts
+// are kept apart by giving every request its own token range (token + rank * V), so one
+// suffix sort orders all of them request by request and one pre-order numbering lays every
+// request's nodes down contiguously; each request's part is then written into its own pool.
+namespace {
+
+__device__ __forceinline__ int seq_rank_of(const int64_t* off, int n, i64 pos) {
+    int lo = 0, hi = n;                               // largest q with off[q] <= pos
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (off[mid] <= pos) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__global__ void map_tokens_kernel(const int32_t* tok, const int64_t* off, int n, i64 N, int V, int32_t* out, int* bad) {
+    i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const int t = tok[i];
+    if (t < 0 || t >= V) { atomicOr(bad, 1); out[i] = 0; return; }
+    out[i] = seq_rank_of(off, n, i) * V + t;
+}
+
+// one block per request: forget the slot's old tree and store the new text
+__global__ void requests_prepare_kernel(sd_store sv, int n, const int32_t* slot_ids, const int64_t* off,
+                                        const int32_t* tok) {
+    const int q = blockIdx.x;
+    if (q >= n) return;
+    const int slot = slot_ids[q];
+    if (slot < 0 || slot >= sv.R) return;
+    SlotState* ss = sv.s_state + slot;
+    int32_t* text = sv.s_text + (i64)slot * sv.T;
+    int32_t* root = sv.s_root + (i64)slot * sv.V;
+    const int old_len = ss->len;
+    for (int k = threadIdx.x; k < old_len; k += blockDim.x) root[text[k]] = -1;
+    __syncthreads();
+    const i64 lo = off[q], hi = off[q + 1];
+    if (hi - lo <= sv.T)
+        for (i64 k = threadIdx.x; k < hi - lo; k += blockDim.x) text[k] = tok[lo + k];
+}
+
+struct RequestLayout {       // where request q's nodes go (device arrays of n entries)
+    int* run_base;           // global position of its first child run
+    int* n1;                 // its depth-1 nodes
+    int* r1lo;               // depth-1 nodes of earlier requests
+    int* used;               // entries it takes
+    int* live;               // nodes
+    int* ok;                 // fits its pool and text buffer
+};
+
+__global__ void requests_layout_kernel(sd_store sv, int n, const int64_t* off, const int* nbase, const int* runstart,
+                                       const int* r1, RequestLayout L) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= n) return;
+    const i64 lo = off[q], hi = off[q + 1];
+    const int first = 1 + nbase[lo], next = 1 + nbase[hi];
+    const int rb = runstart[first], re = runstart[next];
+    const int n1 = r1[hi] - r1[lo];
+    L.run_base[q] = rb; L.n1[q] = n1; L.r1lo[q] = r1[lo];
+    L.used[q] = n1 + (re - rb); L.live[q] = next - first;
+    L.ok[q] = ((i64)n1 + (re - rb) <= sv.spn && hi - lo <= sv.T) ? 1 : 0;
+}
+
+__global__ void emit_nodes_slots_kernel(sd_store sv, int n_req, const int32_t* slot_ids, const int64_t* off,
+                                        const int32_t* mtok, const uint32_t* sa, const uint8_t* lcp, const uint8_t* len,
+                                        i64 n, LevelTables T, const int* nbase, const int* nchild, const int* runstart,
+                                        RequestLayout L) {
+    const i64 j = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    const int l = lcp[j], m = len[j];
+    if (m <= l) return;
+    const i64 text = (i64)sa[j];
+    const int q = seq_rank_of(off, n_req, text);
+    const int slot = slot_ids[q];
+    if (!L.ok[q] || slot < 0 || slot >= sv.R) return;
+    int4* ent = sv.s_ent + (i64)slot * sv.spn;
+    const int shift = L.n1[q] - L.run_base[q];                  // global run position -> index in the slot pool
+    int nid = 1 + nbase[j];
+    int pos = T.E[j] - L.r1lo[q];                               // depth 1: the request's own root table
+    if (l >= 1) {
+        const int jx = T.before[j];
+        const int pnid = 1 + nbase[jx] + (l - (int)lcp[jx] - 1);
+        const int* row = T.E + (i64)l * (T.N + 1);
+        pos = runstart[pnid] + (row[j] - row[jx]) + shift;
+    }
+    for (int d = l + 1; d <= m; ++d, ++nid) {
+        const int nc = nchild[nid];
+        int4 e;
+        e.x = mtok[text + d - 1] - q * sv.V;
+        e.y = T.node_end[nid] - (int)j;
+        e.z = nc > 0 ? runstart[nid] + shift : 0;
+        e.w = nc > 0 ? (int)((unsigned)nc | RUN_STATIC) : 0;
+        ent[pos] = e;
+        if (d == 1) (sv.s_root + (i64)slot * sv.V)[e.x] = pos;
+        pos = runstart[nid] + shift;                             // the next one is this node's first child
+    }
+}
+
+// one warp per request: bookkeeping and the active nodes (lane d-1: node of the last d tokens)
+__global__ void requests_finalize_kernel(sd_store sv, int n, const int32_t* slot_ids, const int64_t* off,
+                                         RequestLayout L) {
+    const int q = (int)((blockIdx.x * (i64)blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    if (q >= n) return;
+    const int slot = slot_ids[q];
+    if (slot < 0 || slot >= sv.R) return;
+    SlotState* ss = sv.s_state + slot;
+    const bool ok = L.ok[q] != 0;
+    const int len = ok ? (int)(off[q + 1] - off[q]) : 0;
+    const int4* ent = sv.s_ent + (i64)slot * sv.spn;
+    const int32_t* root = sv.s_root + (i64)slot * sv.V;
+    const int32_t* text = sv.s_text + (i64)slot * sv.T;
+    int node = -1, rcb = 0;
+    unsigned rw = 0;
+    const int d = lane + 1;
+    if (d <= len && d <= sv.D) {
+        node = root[text[len - d]];
+        int4 e = make_int4(0, 0, 0, 0);
+        if (node >= 0) e = ent[node];
+        for (int k = 1; k < d && node >= 0; ++k) {
+            const int x = text[len - d + k];
+            const int cb = e.z, nn = (int)((unsigned)e.w & RUN_COUNT_MASK);
+            int lo = 0, hi = nn;
+            while (lo < hi) {                                    // at most 24 rounds
+                const int mid = (lo + hi) >> 1;
+                if (ent[cb + mid].x < x) lo = mid + 1; else hi = mid;
+            }
+            node = -1;
+            if (lo < nn) { e = ent[cb + lo]; if (e.x == x) node = cb + lo; }
+        }
+        if (node >= 0) { rcb = e.z; rw = (unsigned)e.w; }
+    }
+    ss->active[lane] = node; ss->room[lane] = 0; ss->run_cb[lane] = rcb; ss->run_w[lane] = rw;
+    if (lane == 0) {
+        ss->len = len; ss->used = ok ? L.used[q] : 0; ss->live = ok ? L.live[q] : 0;
+        ss->status = ok ? 0 : SD_STATUS_POOL_FULL;
+        ss->gen += 1;
+    }
+}
+
+}  // namespace
 
 extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, const int64_t* h_offsets,
                                  const int32_t* d_tokens, void* stream) {
@@ -929,11 +1128,53 @@ extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, 
         if (h_offsets[q + 1] < h_offsets[q] || h_slot[q] < 0 || h_slot[q] >= s->R) return SD_ERR_INVALID_ARG;
         for (int r = 0; r < q; ++r) if (h_slot[r] == h_slot[q]) return SD_ERR_INVALID_ARG;   // a slot once per call
     }
-    if (h_offsets[n] > 0 && !d_tokens) return SD_ERR_INVALID_ARG;
+    const i64 N = h_offsets[n];
+    if (N > 0 && !d_tokens) return SD_ERR_INVALID_ARG;
+    if ((i64)n * s->V >= (1ll << 31) - 2 || N >= (1ll << 31) - 2) return SD_ERR_CAPACITY;
     cudaStream_t st = (cudaStream_t)stream;
-    // (copies from pageable host memory are staged by the runtime before the call returns, so the
-    // caller's arrays may be reused at once)
-    SD_CUDA_OK(cudaMemcpyAsync(s->stage_slot, h_slot, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st));
-    SD_CUDA_OK(cudaMemcpyAsync(s->stage_off, h_offsets, sizeof(int64_t) * (n + 1), cudaMemcpyHostToDevice, st));
-    return sd_launch_text_append(s, n, s->stage_slot, s->stage_off, d_tokens, nullptr, 1, st);
+    const int T256 = 256, D = s->D;
+
+    Pipeline P;
+    if (!s->ws) {
+        s->ws = new (std::nothrow) sd_workspace();
+        if (!s->ws) return SD_ERR_NOMEM;
+        memset(s->ws, 0, sizeof(*s->ws));
+    }
+    P.tmp.keep = s->ws;                                          // temporaries are kept for the next call
+    int32_t *d_slot = nullptr, *mtok = nullptr;
+    int64_t* d_off = nullptr;
+    int* bad = nullptr;
+    RequestLayout L;
+    bool ok = P.tmp.get(&d_slot, n) && P.tmp.get(&d_off, n + 1) && P.tmp.get(&mtok, N) && P.tmp.get(&bad, 1) &&
+              P.tmp.get(&L.run_base, n) && P.tmp.get(&L.n1, n) && P.tmp.get(&L.r1lo, n) &&
+              P.tmp.get(&L.used, n) && P.tmp.get(&L.live, n) && P.tmp.get(&L.ok, n);
+    if (!ok) return SD_ERR_NOMEM;
+    SD_CUDA_OK(cudaMemcpyAsync(d_slot, h_slot, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st));
+    SD_CUDA_OK(cudaMemcpyAsync(d_off, h_offsets, sizeof(int64_t) * (n + 1), cudaMemcpyHostToDevice, st));
+    SD_CUDA_OK(cudaMemsetAsync(bad, 0, sizeof(int), st));
+    if (N > 0) {
+        map_tokens_kernel<<<grid_for(N, T256), T256, 0, st>>>(d_tokens, d_off, n, N, s->V, mtok, bad);
+        int h_bad = 0;
+        SD_CUDA_OK(cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, st));
+        SD_CUDA_OK(cudaStreamSynchronize(st));
+        if (h_bad) return SD_ERR_INVALID_ARG;                    // nothing was changed yet
+    }
+    requests_prepare_kernel<<<(unsigned)n, T256, 0, st>>>(*s, n, d_slot, d_off, d_tokens);
+    if (N > 0) {
+        i64 max_len = 0;
+        for (int q = 0; q < n; ++q) max_len = std::max<i64>(max_len, h_offsets[q + 1] - h_offsets[q]);
+        const int rc = pipeline_run(P, mtok, d_off, n, N, (i64)n * s->V, D, false, st, max_len);
+        if (rc != SD_OK) return rc;
+        requests_layout_kernel<<<grid_for(n, T256), T256, 0, st>>>(*s, n, d_off, P.nbase, P.runstart, P.lv.E, L);
+        emit_nodes_slots_kernel<<<grid_for(N, T256), T256, 0, st>>>(*s, n, d_slot, d_off, mtok, P.sa, P.lcp, P.len, N, P.lv,
+                                                                   P.nbase, P.nchild, P.runstart, L);
+    } else {
+        SD_CUDA_OK(cudaMemsetAsync(L.ok, 0xFF, sizeof(int) * n, st));
+        SD_CUDA_OK(cudaMemsetAsync(L.used, 0, sizeof(int) * n, st));
+        SD_CUDA_OK(cudaMemsetAsync(L.live, 0, sizeof(int) * n, st));
+    }
+    requests_finalize_kernel<<<grid_for((i64)n * 32, T256), T256, 0, st>>>(*s, n, d_slot, d_off, L);
+    SD_CUDA_OK(cudaStreamSynchronize(st));                       // the temporaries are released on return
+    SD_CUDA_OK(cudaGetLastError());
+    return SD_OK;
 }

@@ -1,6 +1,5 @@
-// Read-only queries on a store: COUNT of token paths (the quantity Eq. 1 divides), per-slot and
-// store-wide bookkeeping, empirical entropy.  The global tree is walked through its entries; a
-// per-request tree is its text (common.cuh), so its counts are numbers of occurrences in the text.
+// Read-only queries on a store: COUNT of token paths (the quantity Eq. 1
+// divides), per-slot and store-wide bookkeeping.
 #include "common.cuh"
 
 namespace {
@@ -13,10 +12,11 @@ __global__ void query_counts_kernel(sd_store sv, int n, const int32_t* d_tree, c
     const long long b = d_offsets[i], e = d_offsets[i + 1];
     const int len = (int)(e - b);
     int count = 0;
-    if (tree == -1 && len >= 1 && len <= sv.D) {
-        const int4* ent = sv.g_ent;
+    if (tree >= -1 && tree < sv.R && len >= 1 && len <= sv.D) {
+        const int4* ent = tree < 0 ? sv.g_ent : sv.s_ent + (long long)tree * sv.spn;
+        const int32_t* root = tree < 0 ? sv.g_root : sv.s_root + (long long)tree * sv.V;
         int x = d_paths[b];
-        int node = (x >= 0 && x < sv.V) ? sv.g_root[x] : -1;
+        int node = (x >= 0 && x < sv.V) ? root[x] : -1;
         for (int k = 1; k < len && node >= 0; ++k) {
             const int4 pe = ent[node];
             const int cb = pe.z, nc = (int)((unsigned)pe.w & RUN_COUNT_MASK);
@@ -29,17 +29,6 @@ __global__ void query_counts_kernel(sd_store sv, int n, const int32_t* d_tree, c
             node = (lo < nc && ent[cb + lo].x == x) ? cb + lo : -1;
         }
         if (node >= 0) count = ent[node].y;
-    } else if (tree >= 0 && tree < sv.R && len >= 1 && len <= sv.D) {
-        // occurrences of the path in the request's text
-        const int32_t* text = sv.s_text + (long long)tree * sv.Tp;
-        const int t = sv.s_state[tree].len;
-        const int x0 = d_paths[b];
-        for (int s = 0; s + len <= t; ++s) {
-            if (text[s] != x0) continue;
-            int k = 1;
-            while (k < len && text[s + k] == d_paths[b + k]) ++k;
-            count += k == len ? 1 : 0;
-        }
     }
     d_counts[i] = count;
 }
@@ -49,42 +38,14 @@ __global__ void slot_info_kernel(sd_store sv, int n, const int32_t* d_slot, int3
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const int slot = d_slot[i];
-    int len = 0, status = SD_STATUS_BAD_SLOT;
+    int len = 0, nodes = 0, status = SD_STATUS_BAD_SLOT;
     if (slot >= 0 && slot < sv.R) {
         const SlotState* ss = sv.s_state + slot;
-        len = ss->len; status = ss->status;
+        len = ss->len; nodes = ss->live; status = ss->status;
     }
     if (d_len) d_len[i] = len;
-    if (d_nodes) d_nodes[i] = 0;                                 // slot_nodes_kernel adds the nodes up
+    if (d_nodes) d_nodes[i] = nodes;
     if (d_status) d_status[i] = status;
-}
-
-// Nodes of a per-request tree = distinct substrings of at most D tokens of its text.  Every one
-// is counted at its first occurrence: start position s brings min(D, t - s) strings, of which
-// those no longer than its longest common prefix with an earlier start are not new.
-// Grid: (chunks of 256 start positions, requests).
-__global__ void slot_nodes_kernel(sd_store sv, const int32_t* d_slot, int32_t* d_nodes) {
-    const int slot = d_slot[blockIdx.y];
-    if (slot < 0 || slot >= sv.R) return;
-    const int32_t* text = sv.s_text + (long long)slot * sv.Tp;
-    const int t = sv.s_state[slot].len;
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    int fresh = 0;
-    if (s < t) {
-        const int L = min(sv.D, t - s);
-        const int x0 = text[s];
-        int seen = 0;                                            // longest common prefix with an earlier start
-        for (int j = 0; j < s && seen < L; ++j) {
-            if (text[j] != x0) continue;
-            int k = 1;
-            while (k < L && text[j + k] == text[s + k]) ++k;
-            seen = max(seen, k);
-        }
-        fresh = L - seen;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) fresh += __shfl_xor_sync(0xffffffffu, fresh, o);
-    if ((threadIdx.x & 31) == 0 && fresh) atomicAdd(&d_nodes[blockIdx.y], fresh);
 }
 
 }  // namespace
@@ -106,11 +67,9 @@ extern "C" int sd_slot_info(sd_store* s, int32_t n, const int32_t* d_slot, int32
     if (!s || n < 0) return SD_ERR_INVALID_ARG;
     SD_CHECK_DEVICE(s);
     if (n == 0) return SD_OK;
-    if (!d_slot || n > 65535) return SD_ERR_INVALID_ARG;
+    if (!d_slot) return SD_ERR_INVALID_ARG;
     slot_info_kernel<<<(unsigned)((n + 127) / 128), 128, 0, (cudaStream_t)stream>>>(*s, n, d_slot, d_len, d_nodes,
                                                                                   d_status);
-    if (d_nodes)
-        slot_nodes_kernel<<<dim3((unsigned)((s->T + 255) / 256), (unsigned)n), 256, 0, (cudaStream_t)stream>>>(*s, d_slot, d_nodes);
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }
@@ -125,7 +84,7 @@ extern "C" int sd_stats(sd_store* s, sd_stats_t* out, void* stream) {
     out->global_pool_used = g.used;
     out->global_pool_cap = s->g_cap;
     out->global_tokens = g.tokens;
-    out->slot_pool_nodes = 0;
+    out->slot_pool_nodes = s->spn;
     out->device_bytes = s->device_bytes;
     out->global_status = g.status;
     return SD_OK;
@@ -134,9 +93,8 @@ extern "C" int sd_stats(sd_store* s, sd_stats_t* out, void* stream) {
 // ---------------------------------------------------------------------------------------------
 // Empirical entropy of a tree (Appendix "Predicting SuffixDecoding Effectiveness"): for every
 // node the entropy of its children's count distribution, averaged over the nodes with the
-// sibling sum as weight.  With S the sum of a node's children's counts c, S times its entropy
-// is  S log2 S - sum c log2 c.  Global tree: level-by-level traversal from the root table (the
-// pool also holds abandoned runs and top-block copies, so a plain sweep would count too much).
+// sibling sum as weight.  Level-by-level traversal from the root table (the pools also hold
+// abandoned runs and top-block copies, so a plain sweep over the pool would count too much).
 namespace {
 
 __device__ __forceinline__ void warp_accumulate(double h_times_s, unsigned long long s, double* acc,
@@ -204,94 +162,25 @@ __global__ void entropy_level_kernel(const int4* ent, const int* frontier, int n
     warp_accumulate(part, S, acc, wsum);
 }
 
-// A per-request tree, from its text.  Thread s looks at the strings that start at position s: for
-// every length L it knows their COUNT c (starts whose common prefix with s is at least L) and
-// whether s is the first start of that string, in which case the string is a node and
-// contributes  -c log2 c  as a child of its parent and, if it is shorter than D,  S log2 S  as a
-// parent, S = c minus the occurrence that ends the text (sum of its children's counts).
-__global__ void entropy_text_kernel(sd_store sv, int slot, double* acc, unsigned long long* wsum) {
-    const int32_t* text = sv.s_text + (long long)slot * sv.Tp;
-    const int t = sv.s_state[slot].len;
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    double part = 0.0;
-    unsigned long long S_total = 0;
-    if (s < t) {
-        const int L = min(sv.D, t - s);
-        int hist[SD_MAX_DEPTH + 1];                              // hist[k]: other starts with common prefix exactly k
-        unsigned long long ends = 0;                                     // bit L: an occurrence of the L-token string ends the text
-#pragma unroll
-        for (int k = 0; k <= SD_MAX_DEPTH; ++k) hist[k] = 0;
-        const int x0 = text[s];
-        int seen = 0;
-        for (int j = 0; j < t; ++j) {
-            int k = 0;
-            if (j != s) {
-                if (text[j] != x0) continue;
-                const int lim = min(L, t - j);
-                k = 1;
-                while (k < lim && text[j + k] == text[s + k]) ++k;
-                hist[k] += 1;
-                if (j < s) seen = max(seen, k);
-            } else {
-                k = L;
-            }
-            if (t - j <= k && t - j <= L) ends |= 1ull << (t - j);  // the match reaches the end of the text
-        }
-        int c = 1;                                               // this start itself
-        for (int len = L; len >= 1; --len) {
-            c += hist[len];                                      // starts that share at least `len` tokens
-            if (len > seen) {                                    // first occurrence: a node
-                const double dc = (double)c;
-                part -= dc * log2(dc);
-                if (len < sv.D) {
-                    const int S = c - (int)((ends >> len) & 1ull);
-                    if (S > 0) { part += (double)S * log2((double)S); S_total += (unsigned long long)S; }
-                }
-            }
-        }
-    }
-    if (s == 0 && t > 0) { part += (double)t * log2((double)t); S_total += (unsigned long long)t; }   // the root
-    warp_accumulate(part, S_total, acc, wsum);
-}
-
 }  // namespace
-
-static int entropy_of_text(sd_store* s, int32_t slot, double* h_entropy, cudaStream_t st) {
-    SlotState ss;
-    SD_CUDA_OK(cudaMemcpyAsync(&ss, s->s_state + slot, sizeof(ss), cudaMemcpyDeviceToHost, st));
-    SD_CUDA_OK(cudaStreamSynchronize(st));
-    *h_entropy = 0.0;
-    if (ss.len <= 0) return SD_OK;
-    unsigned char* small = nullptr;
-    if (cudaMalloc(&small, 64) != cudaSuccess) { cudaGetLastError(); return SD_ERR_NOMEM; }
-    double* acc = (double*)small;
-    unsigned long long* wsum = (unsigned long long*)(small + 8);
-    cudaError_t ce = cudaMemsetAsync(small, 0, 64, st);
-    entropy_text_kernel<<<(unsigned)((ss.len + 127) / 128), 128, 0, st>>>(*s, slot, acc, wsum);
-    double h_acc = 0.0;
-    unsigned long long h_w = 0;
-    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_acc, acc, sizeof(double), cudaMemcpyDeviceToHost, st);
-    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_w, wsum, sizeof(h_w), cudaMemcpyDeviceToHost, st);
-    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
-    cudaFree(small);
-    if (ce != cudaSuccess) return SD_ERR_CUDA;
-    *h_entropy = h_w ? h_acc / (double)h_w : 0.0;
-    return SD_OK;
-}
 
 extern "C" int sd_entropy(sd_store* s, int32_t tree, double* h_entropy, void* stream) {
     if (!s || !h_entropy || tree < -1 || tree >= s->R) return SD_ERR_INVALID_ARG;
     SD_CHECK_DEVICE(s);
     cudaStream_t st = (cudaStream_t)stream;
-    if (tree >= 0) return entropy_of_text(s, tree, h_entropy, st);
-    const int4* ent = s->g_ent;
-    const int32_t* root = s->g_root;
+    const int4* ent = tree < 0 ? s->g_ent : s->s_ent + (long long)tree * s->spn;
+    const int32_t* root = tree < 0 ? s->g_root : s->s_root + (long long)tree * s->V;
     int live = 0;
-    {
+    if (tree < 0) {
         GlobalState g;
         SD_CUDA_OK(cudaMemcpyAsync(&g, s->g_state, sizeof(g), cudaMemcpyDeviceToHost, st));
         SD_CUDA_OK(cudaStreamSynchronize(st));
         live = g.live;
+    } else {
+        SlotState ss;
+        SD_CUDA_OK(cudaMemcpyAsync(&ss, s->s_state + tree, sizeof(ss), cudaMemcpyDeviceToHost, st));
+        SD_CUDA_OK(cudaStreamSynchronize(st));
+        live = ss.live;
     }
     *h_entropy = 0.0;
     if (live <= 0) return SD_OK;

@@ -1,43 +1,31 @@
-// GenerateCandidateTree (Algorithm 1) for a whole batch: one thread block per request, one
-// launch per decode step (sd_step: the accepted tokens are appended in the same launch).
+// GenerateCandidateTree (Algorithm 1) for a whole batch.
 //
-//   1. text.  The request's text x_{1:t} is copied into shared memory (new tokens included).
-//   2. match.
-//      Per-request tree (implicit, see common.cuh): the block scans the text for the earlier
-//      occurrences of the last token and measures, for each, how many tokens before it agree
-//      with the context (at most P).  Sorted by that length, the occurrences of the pattern of
-//      length p are a prefix of the list: that prefix IS the match node N_p.
-//      Global tree: MatchPattern walks from the root table, the shortest patterns first, a warp
-//      per pattern length, until a match node has at most 32 occurrences and was never touched
-//      by an online insert.  Such a node is a range of the offline build's suffix order; its
-//      occurrences are read from there with the text around them (64 tokens each), and the
-//      occurrences of every longer pattern are those among them whose preceding tokens agree
-//      with the context.  No longer pattern is walked.
-//   3. expand.  The (tree, p) jobs that matched go into a queue, costliest first; a warp per job.
-//      Occurrence mode (at most 32 occurrences): a lane per occurrence.  A node of the suffix
-//      tree below N_p is the set of lanes whose next tokens agree so far, its count their number
-//      (Eq. 1 and Eq. 2 from popcounts), and the frontier of ExpandSpeculationTree is "the next
-//      node on every lane's path": the best candidate is a warp-wide arg-max, adding it moves
-//      its lanes one token on.  Chains are added without an arg-max.
-//      Wide per-request nodes (more than 32 occurrences: short patterns of frequent tokens, small
-//      budgets): children by a histogram of the next tokens over the occurrence list.
-//      Global nodes with more than 32 occurrences or touched by an insert: the tree's entries
-//      (sorted child runs, top blocks, windows of 32 entries) with a sorted frontier.
-//      A job is dropped, exactly, as soon as an upper bound of its SCORE (every D <= 1 and D
-//      never grows along a path) falls below a score another job of the request has reached.
-//   4. select (first in loop order among the largest scores; Section 3.2: only if SCORE > tau)
-//      and emit tokens, parents, positions and the tree-attention mask.
+// sd_speculate / sd_step: ONE launch, one thread block per request (speculate_fused_kernel):
+//   - sd_step: warp 0 appends the request's accepted tokens to its tree (exactly what sd_append
+//     does), and nothing but the few jobs that need the tree's wide nodes waits for it;
+//   - the other warps copy the request's text into shared memory and scan it for the earlier
+//     occurrences of the last token: how many tokens before each one agree with the context says
+//     which patterns it is an occurrence of.  A per-request match node with at most 32
+//     occurrences needs no tree at all: a lane per occurrence, the node's sub-tree is read off
+//     the text behind the occurrences (expand_occ);
+//   - the global match nodes are advanced from the nodes cached at the previous call by
+//     descending only the tokens appended since;
+//   - the (tree, p) jobs go into a queue, costliest first, a warp per job; a job is dropped,
+//     exactly, as soon as an upper bound of its SCORE falls below a score already reached;
+//   - select (Section 3.2: only if SCORE > tau) and emit from shared memory.
+// sd_speculate_noalloc: the two-kernel form, one warp per (request, tree, p) job with the jobs'
+// records in global memory (match_expand_kernel, select_emit_kernel).
 //
 // fp64 rules: C = count / sibling-sum (Eq. 1), D = D(parent) * C (Eq. 2), SCORE
 // adds D in insertion order; __ddiv_rn / __dmul_rn / __dadd_rn keep every
 // operation a separately rounded IEEE binary64 operation (no FMA contraction).
 #include <mutex>
 
-#include "common.cuh"
-#include "suffix_order.cuh"
+#include "append_core.cuh"
 
 namespace {
 
+constexpr int SPEC_WARPS = 8;                 // warps per block of the job kernel
 constexpr unsigned FULL = 0xffffffffu;
 
 struct Frontier {                             // candidates of one job, best first, ring buffer
@@ -53,6 +41,29 @@ struct Frontier {                             // candidates of one job, best fir
 __device__ __forceinline__ bool better(double da, int ta, int pa, double db, int tb, int pb) {
     const long long a = __double_as_longlong(da), b = __double_as_longlong(db);
     return (a > b) | ((a == b) & ((ta < tb) | ((ta == tb) & (pa < pb))));
+}
+
+// Entry index of child `x` in the sorted run ent[cb .. cb+n), or -1.  Whole warp.
+__device__ int find_child(const int4* __restrict__ ent, int cb, int n, int x, int lane) {
+    int lo = 0, hi = n;
+    for (int it = 0; it < 6 && hi - lo > 32; ++it) {       // window shrinks 33x per round
+        const int q = lo + (int)(((long long)(hi - lo) * (lane + 1)) / 33);
+        const int tk = ent[cb + q].x;
+        const unsigned ge = __ballot_sync(FULL, tk >= x);
+        const int f = ge ? __ffs(ge) - 1 : 32;              // first probe with token >= x
+        const int q_prev = __shfl_sync(FULL, q, f > 0 ? f - 1 : 0);
+        const int q_at = __shfl_sync(FULL, q, f < 32 ? f : 31);
+        if (f > 0) lo = q_prev + 1;
+        if (f < 32) hi = q_at + 1;
+    }
+    int found = -1;
+    for (int base = lo; base < hi && found < 0; base += 32) {   // one round unless n is huge
+        const int idx = base + lane;
+        const bool hit = idx < hi && ent[cb + idx].x == x;
+        const unsigned eq = __ballot_sync(FULL, hit);
+        if (eq) found = cb + base + __ffs(eq) - 1;
+    }
+    return found;
 }
 
 // Insert one candidate (same values on every lane) into the sorted frontier of at
@@ -81,12 +92,214 @@ __device__ bool frontier_insert(Frontier& F, int fh, int& fs, int K, double d, i
     return true;
 }
 
+// Offer every child of a node (run ent[cb .. cb+n)) to the frontier.
+__device__ void push_children(const int4* __restrict__ ent, int cb, int n, double d_parent, int par_index, Frontier& F,
+                              int fh, int& fs, int K, int lane) {
+    if (n <= 0 || K <= 0) return;
+    long long sum = 0;
+    int4 first = make_int4(0, 0, 0, 0);
+    for (int base = 0; base < n; base += 32) {
+        const int idx = base + lane;
+        int4 e = make_int4(0, 0, 0, 0);
+        if (idx < n) e = ent[cb + idx];
+        if (base == 0) first = e;
+        sum += e.y;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+    const double dsum = (double)sum;                            // denominator of Eq. 1
+    for (int base = 0; base < n; base += 32) {
+        const int idx = base + lane;
+        const bool v = idx < n;
+        int4 e = first;
+        if (base != 0) { e = make_int4(0, 0, 0, 0); if (v) e = ent[cb + idx]; }
+        double dc = 0.0;
+        if (v) dc = __dmul_rn(d_parent, __ddiv_rn((double)e.y, dsum));   // Eq. 2 with Eq. 1
+        bool pass = v;
+        if (v && fs == K) {                                     // cannot beat the current worst: skip
+            const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+            pass = better(dc, e.x, par_index, F.d[last], F.tok[last], F.par[last]);
+        }
+        unsigned m = __ballot_sync(FULL, pass);
+        while (m) {
+            const int src = __ffs(m) - 1;
+            m &= m - 1;
+            const double cd = __shfl_sync(FULL, dc, src);
+            const int ct = __shfl_sync(FULL, e.x, src);
+            const int cc = __shfl_sync(FULL, e.z, src);
+            const unsigned cn = (unsigned)__shfl_sync(FULL, e.w, src);
+            frontier_insert(F, fh, fs, K, cd, ct, par_index, cc, cn, lane);
+        }
+    }
+}
+
 __device__ __forceinline__ int budget_for(double alpha, int p, int cap) {
     const double b = floor(__dmul_rn(alpha, (double)p));        // Eq. 3
     if (b > (double)cap) return cap;
     if (b < 0.0) return 0;
     return (int)b;
 }
+
+__global__ void __launch_bounds__(SPEC_WARPS * 32)
+match_expand_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
+                    unsigned flags, const int32_t* __restrict__ d_budget_cap) {
+    __shared__ Frontier fr[SPEC_WARPS];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const long long job = (long long)blockIdx.x * SPEC_WARPS + wib;
+    if (job >= (long long)n * 2 * Pe) return;
+    const int i = (int)(job / (2 * Pe));
+    const int rem = (int)(job % (2 * Pe));
+    const int tree = rem / Pe, p = rem % Pe + 1;
+    const long long rec = ((long long)i * 2 + tree) * sv.D + (p - 1);
+    int cnt = 0;
+    double score = 0.0;
+    const int slot = d_slot[i];
+    bool live = slot >= 0 && slot < sv.R;
+    if (tree == 0 && (flags & SD_FLAG_REQUEST_ONLY)) live = false;
+    if (tree == 1 && (flags & SD_FLAG_GLOBAL_ONLY)) live = false;
+    if (live) {
+        const SlotState* ss = sv.s_state + slot;
+        const int t = ss->len;
+        if (ss->status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) live = false;
+        if (p > t) live = false;
+        int cap = max_spec;
+        if (d_budget_cap && d_budget_cap[i] >= 0) cap = min(cap, d_budget_cap[i]);
+        const int budget = budget_for(alpha, p, cap);
+        if (live && budget > 0) {
+            // ---- MatchPattern
+            const int4* ent;
+            int node;
+            if (tree == 1) {
+                ent = sv.s_ent + (long long)slot * sv.spn;
+                node = ss->active[p - 1];                       // node of the last p tokens
+            } else {
+                ent = sv.g_ent;
+                const int32_t* pat = sv.s_text + (long long)slot * sv.T + (t - p);
+                node = sv.g_root[pat[0]];
+                for (int k = 1; k < p && node >= 0; ++k) {
+                    const int4 e = ent[node];
+                    node = find_child(ent, e.z, (int)((unsigned)e.w & RUN_COUNT_MASK), pat[k], lane);
+                }
+            }
+            if (node >= 0) {
+                // ---- ExpandSpeculationTree
+                Frontier& F = fr[wib];
+                int fh = 0, fs = 0;
+                const int4 e = ent[node];
+                push_children(ent, e.z, (int)((unsigned)e.w & RUN_COUNT_MASK), 1.0, -1, F, fh, fs, budget, lane);
+                int32_t* out_tok = sv.j_tok + rec * sv.M;
+                int32_t* out_par = sv.j_par + rec * sv.M;
+                while (cnt < budget && fs > 0) {
+                    const double d = F.d[fh];
+                    const int tok = F.tok[fh], par = F.par[fh], cb = F.cb[fh];
+                    const int nc = (int)(F.nc[fh] & RUN_COUNT_MASK);
+                    __syncwarp();
+                    fh = (fh + 1) & (SD_MAX_SPEC - 1);
+                    --fs;
+                    if (lane == 0) { out_tok[cnt] = tok; out_par[cnt] = par; }
+                    score = __dadd_rn(score, d);                // Eq. 4, insertion order
+                    const int idx = cnt++;
+                    const int K = budget - cnt;
+                    if (fs > K) fs = K;
+                    if (flags & SD_FLAG_LINEAR) fs = 0;
+                    push_children(ent, cb, nc, d, idx, F, fh, fs, K, lane);
+                }
+            }
+        }
+    }
+    if (lane == 0) { sv.j_n[rec] = cnt; sv.j_score[rec] = score; }
+}
+
+__global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double tau, int32_t* d_n_draft,
+                                   int32_t* d_tokens, int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask,
+                                   int32_t* d_chosen_tree, int32_t* d_chosen_p, double* d_score, int32_t* d_status) {
+    __shared__ int spar[4][SD_MAX_SPEC];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int i = blockIdx.x * 4 + wib;
+    if (i >= n) return;
+    const int M = sv.M, words = (M + 31) / 32;
+    const int slot = d_slot[i];
+    const bool ok = slot >= 0 && slot < sv.R;
+    // first job in loop order (global before per-request, p ascending) with the largest score
+    double best = 0.0;
+    int best_o = -1;
+    for (int o = lane; o < 2 * Pe; o += 32) {
+        const long long rec = ((long long)i * 2 + o / Pe) * sv.D + (o % Pe);
+        const double sc = sv.j_score[rec];
+        if (sc > best) { best = sc; best_o = o; }               // ascending o: strict '>' keeps the first
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const double ob = __shfl_xor_sync(FULL, best, off);
+        const int oo = __shfl_xor_sync(FULL, best_o, off);
+        if (oo >= 0 && (ob > best || (ob == best && (best_o < 0 || oo < best_o)))) { best = ob; best_o = oo; }
+    }
+    int nd = 0, tree = -1, p = 0, t = 0, status = SD_STATUS_BAD_SLOT;
+    long long rec = 0;
+    if (ok) {
+        t = sv.s_state[slot].len;
+        status = sv.s_state[slot].status;
+    }
+    if (ok && best_o >= 0 && best > tau) {                      // Section 3.2: only a score above the threshold is used
+        tree = best_o / Pe; p = best_o % Pe + 1;
+        rec = ((long long)i * 2 + tree) * sv.D + (p - 1);
+        nd = sv.j_n[rec];
+    } else {
+        best = 0.0;
+    }
+    for (int j = lane; j < SD_MAX_SPEC; j += 32) spar[wib][j] = j < nd ? sv.j_par[rec * M + j] : -1;
+    __syncwarp();
+    for (int j = lane; j < M; j += 32) {
+        int tok = -1, par = -1, pos = -1;
+        unsigned long long bits = 0;
+        if (j < nd) {
+            tok = sv.j_tok[rec * M + j];
+            par = spar[wib][j];
+            int depth = 0;
+            for (int a = j, hops = 0; a >= 0 && hops < SD_MAX_SPEC; a = spar[wib][a], ++hops) {
+                bits |= 1ull << a;
+                ++depth;
+            }
+            pos = t + depth - 1;
+        }
+        const long long o = (long long)i * M + j;
+        d_tokens[o] = tok; d_parents[o] = par; d_positions[o] = pos;
+        d_mask[o * words] = (uint32_t)bits;
+        if (words > 1) d_mask[o * words + 1] = (uint32_t)(bits >> 32);
+    }
+    if (lane == 0) {
+        d_n_draft[i] = nd; d_chosen_tree[i] = tree; d_chosen_p[i] = p; d_score[i] = best;
+        if (d_status) d_status[i] = status;
+    }
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// Fused path: one block of W warps per request.  Two blocks per SM is the usual shape: W = 16
+// with 64 registers per thread for sd_speculate, W = 10 with 96 for sd_step, whose append is
+// register hungry.  A batch of at most one request per SM gets bigger blocks (W = 24 / 16), a
+// batch of more than two requests per SM smaller ones (W = 8 / 5, four per SM) to stay in one wave.
+//   1. match: the per-request match nodes are the slot's active nodes; the global match
+//      nodes are advanced from the nodes cached at the previous call by descending only the
+//      tokens appended since (full walks when the cache is stale).  Warp w serves pattern
+//      lengths w + 1, w + 1 + W, ...
+//   2. expand: the (tree, p) jobs that matched go into a queue, costliest first; warps pull
+//      jobs until it is empty.  A job is dropped, exactly, as soon as an upper bound of its
+//      SCORE (every D <= 1 and D never grows along a path) falls below a score already
+//      reached by another job of the request.
+//   3. select + emit from shared memory; no global scratch.
+constexpr int CTA_WARPS = 16;                  // the usual block
+constexpr int CTA_WARPS_STEP = 10;             // the usual block of sd_step: 10 warps with 96 registers each and
+constexpr int STEP_G = 4;                      // an append that moves four entries per round, so that the
+                                               // append in front does not spill.  Measured per step: 92.7 us;
+                                               // 9 warps 92.8, 11 (80 registers) 95, 8 (128) 96; with eight
+                                               // entries per round: 8 warps x 128 registers 95, 10 x 96 100,
+                                               // 12 x 80 100, 16 x 64 104, 6 x 168 110
+constexpr int CTA_WARPS_WIDE = 24;             // small batches (one block per SM at most): the block has the SM's
+constexpr int CTA_WARPS_WIDE_STEP = 16;        // registers to itself (80 per thread; sd_step: 128)
+constexpr int CTA_WARPS_NARROW = 8;            // batches of more than two requests per SM: four blocks per SM
+constexpr int CTA_WARPS_NARROW_STEP = 5;       // (sd_step: 96 registers and the four-entry append; 512 requests:
+                                               // 82 us per step, 88 with 4 warps x 128 registers, 100 with 8 x 64)
 
 struct WarpWork {
     Frontier F;
@@ -103,7 +316,7 @@ struct WarpWork {
 template <int WARPS>
 struct BlockSharedT {
     WarpWork w[WARPS];
-    int node[2][SD_MAX_DEPTH];                // global tree: match node per pattern length (-1: none); row 1 unused
+    int node[2][SD_MAX_DEPTH];                // match node per tree and pattern length (-1: none)
     int cb[2][SD_MAX_DEPTH];                  // its child run
     unsigned nc[2][SD_MAX_DEPTH];             // ... as the node's w field (count | flags)
     int cost[2 * SD_MAX_DEPTH];
@@ -112,26 +325,20 @@ struct BlockSharedT {
     int njobs, next, nwide, nwide_kept;
     long long slice_sum[WARPS];
     int slice_fs[WARPS];
+    // per-request tree, read off the text: earlier occurrences of the last token by the number of
+    // tokens before them that agree with the context
+    int r_hist[SD_MAX_DEPTH + 2];
+    int r_cum[SD_MAX_DEPTH + 2];              // r_cum[p]: occurrences of the pattern of length p
+    int r_fill[SD_MAX_DEPTH + 2];
+    int r_list[SD_OCC_LANES];                 // the occurrences of the patterns that have at most 32, longest matches first
+    int r_pn;                                 // shortest such pattern
+    int app_done;                             // sd_step: warp 0 has appended the new tokens
+    int nlate, late[SD_MAX_DEPTH];            // per-request jobs whose wait for the append ran out
+    int scan_next[2];
     unsigned best_hi;                         // high word of the largest SCORE reached so far: a lower
                                               // bound of it (scores are non-negative doubles), which is
                                               // all the pruning needs; 32 bits keep the atomic native
     int win_warp;
-    int first_bad;                            // sd_step: first new token outside the vocabulary
-    // per-request tree: the match nodes as ranges of the text's suffix order
-    int r_lo[SD_MAX_DEPTH + 1];               // r_lo[p]: first suffix that starts with the last p tokens (the context's own end)
-    int r_cnt[SD_MAX_DEPTH + 1];              // earlier occurrences of that pattern: suffixes r_lo[p] + 1 .. r_lo[p] + r_cnt[p]
-    SaTemp sat;                               // scratch of the suffix-order update
-    // global tree: the base of occurrence mode
-    int g_cnt[SD_MAX_DEPTH];                  // COUNT of the match node
-    int g_rank[SD_MAX_DEPTH];                 // its first suffix in the suffix order (-1: not usable as base)
-    int g_walked, g_failed, g_base_p, g_base_m;
-    int g_src[SD_MAX_DEPTH];                  // the slot's cached match nodes, as they were before this launch
-    int g_src_depths, g_src_k;                // how many are cached (0: none usable), tokens appended since
-    int g_pos[SD_OCC_BASE];                   // text position of the occurrence's first pattern token
-    int g_ell[SD_OCC_BASE];                   // longest pattern the occurrence matches
-    int g_avail[SD_OCC_BASE];                 // tokens that follow the pattern inside the sequence (depth cap applied)
-    int g_cum[SD_MAX_DEPTH + 2];
-    int gwin[SD_OCC_BASE][64];                // tokens pos - 32 .. pos + 31 around every occurrence
 };
 
 // find_child that also hands back the matched entry (valid when the result is >= 0)
@@ -292,11 +499,13 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
         }
     }
     // With a full frontier only a child that beats its worst entry matters:
-    // D = d_parent * count / sum, so small counts lose without any fp64 work.
-    double need = 0.0;
-    if (fs == K) {
+    // D = d_parent * count / sum, so counts below `cmin` lose without any fp64 work.
+    double ld = 0.0, need = 0.0; int lt = 0, lp = 0;
+    const bool full = fs == K;
+    if (full) {
         const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
-        need = F.d[last] * dsum * 0.999999;                     // count * d_parent must reach this
+        ld = F.d[last]; lt = F.tok[last]; lp = F.par[last];
+        need = ld * dsum * 0.999999;                            // count * d_parent must reach this
     }
     for (int base = 0; base < n; base += 32) {
         const int idx = base + lane;
@@ -304,15 +513,16 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
         if (base != 0) { e = make_int4(0, 0, 0, 0); if (idx < n) e = ent[cb + idx]; }
         bool pass = idx < n && idx != skip && (double)e.y * d_parent >= need;
         if (!__any_sync(FULL, pass)) continue;
+        double dc = 0.0;
+        if (pass) {
+            dc = __dmul_rn(d_parent, __ddiv_rn((double)e.y, dsum));      // Eq. 2 with Eq. 1
+            if (full) pass = better(dc, e.x, par_index, ld, lt, lp);
+            if (pass && ((unsigned)e.w & RUN_COUNT_MASK)) prefetch_l2(ent + e.z);   // likely looked at soon
+        }
         if (fs == 0 && n <= 32) {
             // Nothing waits yet (the first children of a job): the candidates are siblings, and
             // among siblings the order of D is the order of (count, then token).  Their places
             // follow from one pass per distinct count, largest first, without any merging.
-            double dc = 0.0;
-            if (pass) {
-                dc = __dmul_rn(d_parent, __ddiv_rn((double)e.y, dsum));      // Eq. 2 with Eq. 1
-                if ((unsigned)e.w & RUN_COUNT_MASK) prefetch_l2(ent + e.z);   // likely looked at soon
-            }
             unsigned rem = __ballot_sync(FULL, pass);
             const int np = __popc(rem);
             const unsigned below = (1u << lane) - 1u;
@@ -333,22 +543,68 @@ __device__ void push_children_w(const int4* __restrict__ ent, int cb, int n, int
             fs = min(np, K);
             return;
         }
-        // The children of this chunk are offered best first: (count, then smaller token) orders
-        // siblings like their D values, and the first one that does not enter ends the chunk.
-        unsigned rem = __ballot_sync(FULL, pass);
-        while (rem) {
-            const bool in = (rem >> lane) & 1u;
-            const unsigned top = __reduce_max_sync(FULL, in ? (unsigned)e.y : 0u);
-            const int src = __ffs(__ballot_sync(FULL, in && (unsigned)e.y == top)) - 1;    // smallest token among them
-            const double dc = __dmul_rn(d_parent, __ddiv_rn((double)top, dsum));          // Eq. 2 with Eq. 1
-            const int cz = __shfl_sync(FULL, e.z, src);
-            const unsigned cw = (unsigned)__shfl_sync(FULL, e.w, src);
-            if (!frontier_insert(F, fh, fs, K, dc, __shfl_sync(FULL, e.x, src), par_index, cz, cw, lane)) break;
-            if (lane == 0 && (cw & RUN_COUNT_MASK)) prefetch_l2(ent + cz);                 // likely looked at soon
-            rem &= ~(1u << src);
+        frontier_merge(F, fh, fs, K, pass, dc, e.x, par_index, e.z, (unsigned)e.w, lane);
+        if (!full && fs == K) {                                 // it filled up while merging
+            const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+            const double d2 = F.d[last];
+            const int t2 = F.tok[last], p2 = F.par[last];
+            // from here on compare exactly against the new worst entry (no count shortcut)
+            for (int b2 = base + 32; b2 < n; b2 += 32) {
+                const int i2 = b2 + lane;
+                int4 e2 = make_int4(0, 0, 0, 0);
+                if (i2 < n) e2 = ent[cb + i2];
+                double dc2 = 0.0;
+                bool pass2 = i2 < n;
+                if (pass2) {
+                    dc2 = __dmul_rn(d_parent, __ddiv_rn((double)e2.y, dsum));
+                    const int l3 = (fh + fs - 1) & (SD_MAX_SPEC - 1);
+                    pass2 = better(dc2, e2.x, par_index, F.d[l3], F.tok[l3], F.par[l3]);
+                }
+                frontier_merge(F, fh, fs, K, pass2, dc2, e2.x, par_index, e2.z, (unsigned)e2.w, lane);
+            }
+            (void)d2; (void)t2; (void)p2;
+            return;
         }
     }
 }
+
+// MatchPattern from a known node: descend text[from .. to).  Levels whose child run lies inside
+// the window already in registers cost no memory access.  Returns the node reached (-1: no
+// match) and its child run in (cb, n).
+// The context is `text` up to position t_old and `newtok` from there on (tokens that are
+// being appended in the same launch).
+__device__ int walk_from(const int4* __restrict__ ent, int limit, int node, const int32_t* __restrict__ text, int t_old,
+                         const int32_t* __restrict__ newtok, int from, int to, int lane, int& cb, unsigned& wfull) {
+    if (node < 0) return -1;
+    int wb = node;
+    int4 w = load_window(ent, wb, limit, lane);
+    cb = __shfl_sync(FULL, w.z, 0);
+    wfull = (unsigned)__shfl_sync(FULL, w.w, 0);
+    int n = (int)(wfull & RUN_COUNT_MASK);
+    for (int pos = from; pos < to; ++pos) {
+        const int x = pos < t_old ? text[pos] : newtok[pos - t_old];
+        if (n == 0) return -1;
+        if (n > 32) {                                           // wide run: 32-way search
+            int4 e;
+            node = find_child_entry(ent, cb, n, x, lane, e);
+            if (node < 0) return -1;
+            cb = e.z; wfull = (unsigned)e.w; n = (int)(wfull & RUN_COUNT_MASK);
+            wb = -64;                                           // no usable window
+            continue;
+        }
+        if (!(cb >= wb && cb + n <= wb + 32)) { wb = cb; w = load_window(ent, wb, limit, lane); }
+        const int rel = wb + lane - cb;
+        const unsigned hit = __ballot_sync(FULL, rel >= 0 && rel < n && w.x == x);
+        if (!hit) return -1;
+        const int src = __ffs(hit) - 1;
+        node = wb + src;
+        cb = __shfl_sync(FULL, w.z, src);
+        wfull = (unsigned)__shfl_sync(FULL, w.w, src);
+        n = (int)(wfull & RUN_COUNT_MASK);
+    }
+    return node;
+}
+
 
 // Children of a node whose run has a top block (see RUN_HAS_TOP): the 64 best by count are
 // listed, best first, right before the run, together with the sum of all counts.
@@ -588,43 +844,6 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
     __syncwarp();
 }
 
-// MatchPattern in the global tree, from a node that is already known: descends tx[from .. to).
-// Levels whose child run lies inside the window already in registers cost no memory access.
-// Returns the node reached (-1: no match), its child run (cb, wfull) and its COUNT.
-__device__ int walk_from(const int4* __restrict__ ent, int limit, int node, const int* tx, int from, int to, int lane,
-                         int& cb, unsigned& wfull, int& count) {
-    if (node < 0) return -1;
-    int wb = node;
-    int4 w = load_window(ent, wb, limit, lane);
-    cb = __shfl_sync(FULL, w.z, 0);
-    wfull = (unsigned)__shfl_sync(FULL, w.w, 0);
-    count = __shfl_sync(FULL, w.y, 0);
-    int n = (int)(wfull & RUN_COUNT_MASK);
-    for (int pos = from; pos < to; ++pos) {
-        const int x = tx[pos];
-        if (n == 0) return -1;
-        if (n > 32) {                                           // wide run: 32-way search
-            int4 e;
-            node = find_child_entry(ent, cb, n, x, lane, e);
-            if (node < 0) return -1;
-            cb = e.z; wfull = (unsigned)e.w; count = e.y; n = (int)(wfull & RUN_COUNT_MASK);
-            wb = -64;                                           // no usable window
-            continue;
-        }
-        if (!(cb >= wb && cb + n <= wb + 32)) { wb = cb; w = load_window(ent, wb, limit, lane); }
-        const int rel = wb + lane - cb;
-        const unsigned hit = __ballot_sync(FULL, rel >= 0 && rel < n && w.x == x);
-        if (!hit) return -1;
-        const int src = __ffs(hit) - 1;
-        node = wb + src;
-        cb = __shfl_sync(FULL, w.z, src);
-        wfull = (unsigned)__shfl_sync(FULL, w.w, src);
-        count = __shfl_sync(FULL, w.y, src);
-        n = (int)(wfull & RUN_COUNT_MASK);
-    }
-    return node;
-}
-
 // ---------------------------------------------------------------------------------------------
 // Occurrence mode: ExpandSpeculationTree + SCORE for one (tree, p) job whose match node has at
 // most 32 occurrences, a lane per occurrence.  cptr[k] (k >= 1) is the k-th token behind the
@@ -740,495 +959,387 @@ __device__ void expand_occ(BlockShared& sh, WarpWork& W, const int* cptr, int km
     __syncwarp();
 }
 
-// ---------------------------------------------------------------------------------------------
-// A job whose match node has more than 32 occurrences, over a list of occurrences that is SORTED
-// by the text behind them.  Every node below the match node is a range of the list (the items
-// that agree on the tokens so far), its children are the runs of equal next tokens inside the
-// range, and expanding a node is one pass over its own range.
-//   Per-request tree: the list is the suffix order of the request's text (suffix_order.cuh), the
-//   pattern's occurrences are the range S[lo .. hi), COUNT is the size of a range.
-//   Global tree: the list is the base node's range of the offline build's suffix order, staged
-//   with the tokens around every occurrence; the job of pattern length p counts only the items
-//   that match at least p tokens (FILTER).
-// Frontier: the sorted ring of the tree-entry path; fields cb / nc hold the candidate's range as
-// lo / (hi << 5 | depth below the match node).
-struct TextItems {            // items j of S: suffixes that start with the pattern of length p
-    const int* tx; const int* S; int t, p;
-    // token `level` (1: the first one behind the pattern) of item j, -1 if the text ends before it
-    __device__ __forceinline__ int tok(int j, int level) const { const int q = S[j] + p - 1 + level; return q <= t - 1 ? tx[q] : -1; }
-    __device__ __forceinline__ bool member(int) const { return true; }
-};
-struct WindowItems {          // items j: occurrences of the global base pattern, with 64 tokens around each
-    const int (*gwin)[64]; const int* avail; const int* ell; int base_p, p;
-    __device__ __forceinline__ int tok(int j, int level) const { return level <= avail[j] ? gwin[j][31 + base_p + level] : -1; }
-    __device__ __forceinline__ bool member(int j) const { return ell[j] >= p; }
-};
-
-template <bool FILTER, class Items, class BlockShared>
-__device__ void expand_range(BlockShared& sh, WarpWork& W, const Items& it, int lo0, int hi0, int tree, int p, int budget,
-                             int dlim, unsigned flags, int lane) {
-    const int order = tree * SD_MAX_DEPTH + p;
-    const int buf = W.best_buf ^ 1;
-    Frontier& F = W.F;
-    int fh = 0, fs = 0, cnt = 0;
-    double score = 0.0;
-    bool dropped = false;
-    double cur_d = 1.0;
-    int lo = lo0, hi = hi0, cur_k = 0, cur_idx = -1;
-    bool have_cur = true;
-    while (true) {
-        if (!have_cur) {
-            if (cnt >= budget || fs == 0) break;
-            cur_d = F.d[fh];
-            const int tok = F.tok[fh], par = F.par[fh];
-            lo = F.cb[fh];
-            hi = (int)(F.nc[fh] >> 5);
-            cur_k = (int)(F.nc[fh] & 31u);
-            if ((score + (double)(budget - cnt) * cur_d) * 1.000000001 < best_so_far(sh)) { dropped = true; break; }
-            __syncwarp();
-            fh = (fh + 1) & (SD_MAX_SPEC - 1);
-            --fs;
-            if (lane == 0) { W.tok[buf][cnt] = tok; W.par[buf][cnt] = (unsigned char)(par + 1); }
-            score = __dadd_rn(score, cur_d);                    // Eq. 4, insertion order
-            if (lane == 0) atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
-            cur_idx = cnt++;
-            const int K = budget - cnt;
-            if (fs > K) fs = K;
-            if (flags & SD_FLAG_LINEAR) fs = 0;
-        }
-        have_cur = false;
-        if (cnt >= budget) break;
-        if (cur_k >= dlim || lo >= hi) continue;                // depth cap: the node has no children
-        const int K = budget - cnt;
-        const int level = cur_k + 1;
-        // the sibling sum (denominator of Eq. 1): items of the job that have a next token
-        int sum;
-        if (FILTER) {
-            sum = 0;
-            for (int base = lo; base < hi; base += 32) {
-                const int j = base + lane;
-                sum += __popc(__ballot_sync(FULL, j < hi && it.member(j) && it.tok(j, level) >= 0));
-            }
-        } else {
-            sum = hi - lo - (it.tok(lo, level) < 0 ? 1 : 0);    // an item whose text ends here sorts first; all others go on
-        }
-        if (sum <= 0) continue;
-        const double dsum = (double)sum;
-        // the runs of equal next tokens; an open run is carried from chunk to chunk
-        int run_tok = -2, run_lo = lo, run_c = 0;               // -2: none yet
-        for (int base = lo; base < hi + 32; base += 32) {       // (a last round behind the range closes the last run)
-            const int j = base + lane;
-            int tk = -3;                                        // behind the range: differs from every token
-            bool mem = false;
-            if (j < hi) { tk = it.tok(j, level); mem = FILTER ? (tk >= 0 && it.member(j)) : true; }
-            int prev = __shfl_up_sync(FULL, tk, 1);
-            if (lane == 0) prev = run_tok;
-            const bool bnd = tk != prev;                        // a run starts here
-            const unsigned bm = __ballot_sync(FULL, bnd);
-            const unsigned mm = FILTER ? __ballot_sync(FULL, mem) : 0u;
-            if (!bm) { if (FILTER) run_c += __popc(mm); }
-            else {
-                // every boundary closes the run that ends right before it: the open run for the
-                // first boundary of the chunk, else the run that began at the boundary before
-                const unsigned lt = (1u << lane) - 1u;
-                const unsigned below = bm & lt;
-                const int sb = below ? 31 - __clz(below) : 0;
-                const int s_tok = __shfl_sync(FULL, tk, sb);
-                const int c_tok = below ? s_tok : run_tok, c_lo = below ? base + sb : run_lo, c_hi = base + lane;
-                int c_cnt = c_hi - c_lo;
-                if (FILTER) c_cnt = below ? __popc(mm & lt & ~((1u << sb) - 1u)) : run_c + __popc(mm & lt);
-                bool pass = bnd && c_tok >= 0 && c_cnt > 0;
-                double dc = 0.0;
-                if (pass) {
-                    dc = __dmul_rn(cur_d, __ddiv_rn((double)c_cnt, dsum));             // Eq. 2 with Eq. 1
-                    if (fs == K) {
-                        const int last = (fh + fs - 1) & (SD_MAX_SPEC - 1);
-                        pass = better(dc, c_tok, cur_idx, F.d[last], F.tok[last], F.par[last]);
-                    }
-                }
-                unsigned pm = __ballot_sync(FULL, pass);
-                while (pm) {
-                    const int src = __ffs(pm) - 1;
-                    pm &= pm - 1;
-                    frontier_insert(F, fh, fs, K, __shfl_sync(FULL, dc, src), __shfl_sync(FULL, c_tok, src), cur_idx,
-                                    __shfl_sync(FULL, c_lo, src),
-                                    ((unsigned)__shfl_sync(FULL, c_hi, src) << 5) | (unsigned)level, lane);
-                }
-                const int lb = 31 - __clz(bm);                  // the last boundary opens the run that is carried on
-                run_tok = __shfl_sync(FULL, tk, lb);
-                run_lo = base + lb;
-                if (FILTER) run_c = __popc(mm & ~((1u << lb) - 1u));
-            }
-            if (base >= hi) break;
-        }
+// A per-request job that goes through the tree's entries: the match node of pattern length p is
+// the slot's active node of depth p (kept current by the append).  Whole warp.
+template <class BlockShared>
+__device__ void request_tree_job(BlockShared& sh, WarpWork& W, const sd_store& sv, const SlotState* ss, const int4* s_ent, int t,
+                                 int p, int budget, unsigned flags, int lane) {
+    // an append that stopped early leaves a context the jobs were not made for
+    if (ss->len != t || (ss->status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN))) return;
+    int node = -1;
+    unsigned rw = 0;
+    if (lane == 0) {
+        node = ss->active[p - 1];
+        int rcb = ss->run_cb[p - 1];
+        rw = ss->run_w[p - 1];
+        if (node >= 0 && rw == RUN_UNKNOWN) { const int4 e = s_ent[node]; rcb = e.z; rw = (unsigned)e.w; }
+        sh.node[1][p - 1] = node; sh.cb[1][p - 1] = rcb; sh.nc[1][p - 1] = rw;
     }
+    node = __shfl_sync(FULL, node, 0);
+    rw = (unsigned)__shfl_sync(FULL, rw, 0);
     __syncwarp();
-    if (!dropped && (score > W.best_score || (score == W.best_score && score > 0.0 && order < W.best_order))) {
-        if (lane == 0) {
-            W.best_score = score; W.best_order = order; W.best_n = cnt; W.best_buf = buf;
-            atomicMax(&sh.best_hi, (unsigned)__double2hiint(score));
-        }
+    const int nch = (int)(rw & RUN_COUNT_MASK);
+    if (node < 0 || nch == 0) return;
+    if (nch > WIDE_RUN && !(rw & RUN_HAS_TOP)) {                 // scanned by all warps together, later
+        if (lane == 0) sh.wide[atomicAdd(&sh.nwide, 1)] = SD_MAX_DEPTH + p - 1;
+        return;
     }
-    __syncwarp();
+    expand_job(sh, W, s_ent, (int)sv.spn, 1, p, budget, flags, false, 0, lane);
 }
 
-struct StepArgs {             // what one launch needs beyond the store
-    int n;
-    const int32_t* d_slot;
-    int Pe;
-    double alpha;
-    int max_spec;
-    unsigned flags;
-    double tau;
-    const int32_t* d_budget_cap;
-    int32_t *d_n_draft, *d_tokens, *d_parents, *d_positions;
-    uint32_t* d_mask;
-    int32_t *d_chosen_tree, *d_chosen_p;
-    double* d_score;
-    int32_t* d_status;
-    const int64_t* d_app_off;     // sd_step: the tokens to append first (NULL: sd_speculate)
-    const int32_t* d_app_tok;
-    int stage_tokens;             // tokens of text, and entries of its suffix order, the block can hold in shared
-                                  // memory (0: the text is too long; both are then used in place)
-    int32_t* scratch;             // [n][Tp] by request: the suffix order of a text that is not staged
-};
+// One block of W warps per request.
+//   1. match.  Global tree: the match nodes are advanced from the nodes cached at the previous
+//      call by descending only the tokens appended since (full walks when the cache is stale).
+//      Per-request tree: the request's text (with the tokens being appended) is copied into
+//      shared memory and scanned for the earlier occurrences of its last token; the number of
+//      tokens before an occurrence that agree with the context says which patterns it belongs to.
+//   2. expand: the (tree, p) jobs that matched go into a queue, costliest first; a warp per job.
+//      Global jobs go through the tree's entries.  Per-request jobs whose match node has at most
+//      32 occurrences are read off the text (expand_occ: a lane per occurrence, no tree); the
+//      others go through the request's tree from the slot's active nodes.  sd_step: warp 0
+//      appends the accepted tokens to the request's tree meanwhile, exactly as sd_append would,
+//      and joins the queue when it is done; the other warps meet at a barrier of their own until
+//      then, and only the jobs that go through the request's tree wait for the append (they
+//      come last in the queue).
+//   3. jobs of either tree that start at a wide child run without top block are scanned by all
+//      warps together, behind a block-wide barrier.
+//   4. select + emit from shared memory; no global scratch.
+// A job is skipped or dropped, exactly, as soon as an upper bound of its SCORE falls below a
+// score another job of the request has already reached (the running scores are published).
+constexpr int BAR_GROUP = 1, BAR_JOIN = 2;    // hardware barriers beside the block-wide one
 
-template <int WARPS, int MINB>
-__global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_store sv, StepArgs a) {
+template <bool STEP, int WARPS, int MINB, int APPEND_G = 8>
+__global__ void __launch_bounds__(WARPS * 32, MINB)
+speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, int Pe, double alpha, int max_spec,
+                       unsigned flags, double tau, const int32_t* __restrict__ d_budget_cap, int32_t* d_n_draft,
+                       int32_t* d_tokens, int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
+                       int32_t* d_chosen_p, double* d_score, int32_t* d_status, const int64_t* __restrict__ d_app_off,
+                       const int32_t* __restrict__ d_app_tok, int stage_tokens) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using BlockShared = BlockSharedT<WARPS>;
+    constexpr int CTA_WARPS = WARPS;
     constexpr int NT = WARPS * 32;
+    // the warps that do everything but the append: all of them, or all but warp 0
+    constexpr int GW0 = STEP ? 1 : 0, GWARPS = WARPS - GW0, GT = GWARPS * 32;
     BlockShared& sh = *reinterpret_cast<BlockShared*>(smem_raw);
     int* const stx = reinterpret_cast<int*>(smem_raw + ((sizeof(BlockShared) + 15) & ~(size_t)15));
     const int tid = threadIdx.x, lane = tid & 31, wib = tid >> 5;
+    const int gtid = tid - GW0 * 32, gw = wib - GW0;             // index inside that group (negative: warp 0 of sd_step)
+    auto group_sync = [&]() {
+        if (STEP) asm volatile("bar.sync %0, %1;" ::"r"(BAR_GROUP), "r"(GT) : "memory");
+        else __syncthreads();
+    };
     const int i = blockIdx.x;
-    const int M = sv.M, words = (M + 31) / 32, D = sv.D, Pe = a.Pe;
-    const unsigned flags = a.flags;
-    const int slot = a.d_slot[i];
+    const int M = sv.M, words = (M + 31) / 32, D = sv.D;
+    const int slot = d_slot[i];
     const bool ok = slot >= 0 && slot < sv.R;
-    int t = 0, status = SD_STATUS_BAD_SLOT, sa_buf = 0;
+    // a slot may appear once per call: a later appearance is refused (two blocks on one tree would
+    // race); the answer is collected at the first barrier below, before anything is written
+    int dup = 0;
+    for (int j = tid; j < i; j += NT) dup |= d_slot[j] == slot ? 1 : 0;
+    int t = 0, status = SD_STATUS_BAD_SLOT;
     SlotState* ss = nullptr;
-    int32_t* gtext = nullptr;
-    if (ok) {
-        ss = sv.s_state + slot; t = ss->len; status = ss->status; sa_buf = ss->sa_buf;
-        gtext = sv.s_text + (long long)slot * sv.Tp;
-    }
+    if (ok) { ss = sv.s_state + slot; t = ss->len; status = ss->status; }
+    // STEP: t_old tokens are in the slot's text, the next n_new come from the append list; the
+    // match below already runs on the context of t = t_old + n_new tokens
     const int t_old = t;
+    const int32_t* newtok = nullptr;
+    int n_new = 0;
+    if (STEP && ok) {
+        newtok = d_app_tok + d_app_off[i];
+        n_new = (int)(d_app_off[i + 1] - d_app_off[i]);
+        t = t_old + n_new;
+    }
+    bool usable = ok && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && t > 0;
+    // the stored text starts its way into shared memory now (asynchronous copies, nothing waits
+    // for them here): it arrives while the cached match nodes and the append list are read
+    const int32_t* text = ok ? sv.s_text + (long long)slot * sv.T : nullptr;
+    const bool prefetched = ok && gtid >= 0 && t_old <= stage_tokens && !(flags & SD_FLAG_GLOBAL_ONLY);
+    if (prefetched) {
+        const unsigned dst0 = (unsigned)__cvta_generic_to_shared(stx);
+        for (int q = gtid; q < t_old; q += GT)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst0 + 4u * q), "l"(text + q) : "memory");
+    }
+    int cap = max_spec;
+    if (d_budget_cap && d_budget_cap[i] >= 0) cap = min(cap, d_budget_cap[i]);
     if (tid < 2 * SD_MAX_DEPTH) { (&sh.node[0][0])[tid] = -1; (&sh.nc[0][0])[tid] = 0; }
-    if (tid < SD_MAX_DEPTH + 2) sh.g_cum[tid] = 0;
-    if (tid <= SD_MAX_DEPTH) { sh.r_lo[tid] = 0; sh.r_cnt[tid] = 0; }
-    if (tid < SD_MAX_DEPTH) { sh.g_cnt[tid] = 0; sh.g_rank[tid] = -1; }
+    if (tid < SD_MAX_DEPTH + 2) { sh.r_hist[tid] = 0; sh.r_cum[tid] = 0; sh.r_fill[tid] = 0; }
     if (tid == 0) {
         sh.njobs = 0; sh.next = 0; sh.nwide = 0; sh.nwide_kept = 0; sh.best_hi = 0u; sh.win_warp = -1;
-        sh.first_bad = 0x7fffffff;
-        sh.g_walked = 0; sh.g_failed = 0; sh.g_base_p = 0; sh.g_base_m = 0;
+        sh.r_pn = SD_MAX_DEPTH + 1; sh.scan_next[0] = 0; sh.scan_next[1] = 0; sh.app_done = 0; sh.nlate = 0;
     }
     WarpWork& W = sh.w[wib];
     if (lane == 0) { W.best_score = 0.0; W.best_order = 1 << 30; W.best_n = 0; W.best_buf = 0; }
-    __syncthreads();
 
-    // ---------------- 0. sd_step: the accepted tokens go behind the request's text
-    const int32_t* newtok = nullptr;
-    int take = 0;
-    if (a.d_app_off && ok) {
-        const long long b0 = a.d_app_off[i];
-        const int n_new = (int)(a.d_app_off[i + 1] - b0);
-        newtok = a.d_app_tok + b0;
-        if (n_new > 0 && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN))) {
-            take = min(n_new, sv.T - t_old);
-            for (int k = tid; k < take; k += NT) {
-                const int x = newtok[k];
-                if (x < 0 || x >= sv.V) atomicMin(&sh.first_bad, k);
-            }
-            __syncthreads();
-            const int good = min(take, sh.first_bad);
-            if (good < take) status |= SD_STATUS_BAD_TOKEN;     // the text stops before the first bad token
-            else if (take < n_new) status |= SD_STATUS_POOL_FULL;
-            take = good;
-            for (int k = tid; k < take; k += NT) gtext[t_old + k] = newtok[k];
-            t = t_old + take;
-        }
-    }
-    const bool usable = ok && !(status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)) && t > 0;
-    int cap = a.max_spec;
-    if (a.d_budget_cap && a.d_budget_cap[i] >= 0) cap = min(cap, a.d_budget_cap[i]);
-    const bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
-    const bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
-
-    // ---------------- 1. the text and its suffix order
-    const bool staged = t <= a.stage_tokens;
-    int fin_a0 = -1;
-    const int* tx = stx;
-    int* S = stx + a.stage_tokens;
-    if (ok && (usable || take > 0)) {
-        if (staged) {
-            const int4* g4 = reinterpret_cast<const int4*>(gtext);
-            int4* s4 = reinterpret_cast<int4*>(stx);
-            for (int g = tid; g * 4 < t; g += NT) {
-                int4 v = make_int4(0, 0, 0, 0);
-                if (g * 4 < t_old) v = g4[g];
-                // (the new tokens come from the call's list: the copy in the text buffer above may not have landed yet)
-                int* c = reinterpret_cast<int*>(&v);
+    // ---------------- 1. match
+    bool want_g = usable && !(flags & SD_FLAG_REQUEST_ONLY);
+    bool want_r = usable && !(flags & SD_FLAG_GLOBAL_ONLY);
+    // warps that advance the global match nodes, and this warp's rank among them
+    const int mwarps = GWARPS;
+    const int mrank = gw;
+    constexpr int MROUNDS = (SD_MAX_DEPTH + GWARPS - 1) / GWARPS;   // pattern lengths per warp
+    int src_node[MROUNDS], src_from[MROUNDS];                   // per target: start node and first text index
 #pragma unroll
-                for (int u = 0; u < 4; ++u) { const int q = g * 4 + u; if (q >= t_old && q < t) c[u] = newtok[q - t_old]; }
-                s4[g] = v;
+    for (int h = 0; h < MROUNDS; ++h) { src_node[h] = -1; src_from[h] = 0; }
+    if (want_g && mrank >= 0) {
+        const bool cache_ok = ss->g_gen == ss->gen && ss->g_epoch == sv.g_state->epoch && ss->g_len <= t;
+        const int k = t - ss->g_len;                            // tokens appended since the cache was taken
+        const int depths = ss->g_depths;
+#pragma unroll
+        for (int h = 0; h < MROUNDS; ++h) {
+            const int d = mrank + 1 + h * mwarps;               // target pattern length
+            if (d > Pe || d > t) continue;
+            if (cache_ok && d > k && d - k <= depths) {
+                src_node[h] = ss->g_node[d - k - 1];            // node of the tokens before the new ones
+                src_from[h] = t - k;
+            } else {
+                const int x0 = t - d < t_old ? text[t - d] : newtok[t - d - t_old];
+                src_node[h] = (x0 >= 0 && x0 < sv.V) ? sv.g_root[x0] : -1;
+                src_from[h] = t - d + 1;
             }
-        } else {
-            tx = gtext;                                         // too long to stage: text and order are used in place
-            S = a.scratch + (long long)i * sv.Tp;
         }
-        int32_t* sa[2] = {sv.s_sa + (long long)slot * sv.Tp, sv.s_sa + ((long long)sv.R + slot) * sv.Tp};
-        if (staged || take > 0)
-            for (int k = tid; k < t_old; k += NT) S[k] = sa[sa_buf][k];
-        else
-            S = sa[sa_buf];                                     // nothing to merge: the stored order is read as it is
-        __syncthreads();                                        // (also: the new tokens in gtext are visible to the block)
-        for (int t0 = t_old; t0 < t; t0 += SA_CHUNK) {
-            sa_merge_chunk<NT>(tx, t0, min(t, t0 + SA_CHUNK), D, S, sa[sa_buf], sa[sa_buf ^ 1], sh.sat, tid);
-            sa_buf ^= 1;
-            fin_a0 = max(0, t0 - (D - 1));                      // sh.sat.fin[a - fin_a0]: where the last merge put suffix a
-        }
-        if (tid == 0 && take > 0) { ss->len = t; ss->sa_buf = sa_buf; }
     }
-    if (tid == 0 && ok && a.d_app_off) ss->status = status;
-    __syncthreads();
-
-    // ---------------- 2. match
-    if (wib == 0) {
-        // the slot's cached global match nodes (taken at context length g_len <= t)
-        int depths = 0, kk = 0;
-        if (usable) {
-            const bool cache_ok = ss->g_gen == ss->gen && ss->g_epoch == sv.g_state->epoch && ss->g_len <= t && ss->g_len > 0;
-            if (cache_ok) { depths = ss->g_depths; kk = t - ss->g_len; }
-            sh.g_src[lane] = (cache_ok && lane < depths) ? ss->g_node[lane] : -1;
-        }
-        if (lane == 0) { sh.g_src_depths = depths; sh.g_src_k = kk; }
-    }
-    __syncthreads();
+    // all cached nodes read before any is replaced; and: is this a second block for the same slot?
+    const bool refused = __syncthreads_or(dup) != 0;
+    if (refused) { usable = false; want_g = false; want_r = false; status = SD_STATUS_BAD_SLOT; }
+    // the text can be read off only if it fits the shared memory left for it
+    const bool staged = want_r && t >= 2 && t <= stage_tokens;
     const int Lcap = min(Pe, D - 1);                            // a match node at depth D has no children
-    // Per-request tree: the range of every pattern in the suffix order, a warp per pattern length.
-    // Its first suffix is the context's own end (the pattern followed by nothing); the earlier
-    // occurrences follow it.
-    const int Lr = want_r ? min(Lcap, t - 1) : 0;
-    auto request_ranges = [&]() {
-        for (int p = wib + 1; p <= Lr; p += WARPS) {
-            // the range begins with the context's own end, whose place the merge above may have just found
-            const int lo = fin_a0 >= 0 ? sh.sat.fin[t - p - fin_a0] : pattern_lo_warp(tx, t, S, t - p, p, lane);
-            const int hi = pattern_hi_warp(tx, t, S, t - p, p, lo, lane);
-            if (lane == 0) { sh.r_lo[p] = lo; sh.r_cnt[p] = max(hi - lo - 1, 0); }
-        }
-    };
-    // Global tree: rounds of WARPS pattern lengths, shortest first, until a node can serve as
-    // the base of occurrence mode, a pattern does not occur, or all lengths are done.
-    const int PeG = want_g ? min(Pe, t) : 0;
-    const bool occ_mode = sv.g_lo != nullptr;
-    for (int r0 = 0; r0 < PeG; r0 += WARPS) {
-        const int p = r0 + wib + 1;
-        if (p <= PeG) {
-            int cb = 0, cntn = 0;
-            unsigned wf = 0;
-            // from the cached node of the tokens before the new ones, if there is one; else from the root table
-            const int kk = sh.g_src_k;
-            int node, from;
-            if (p > kk && p - kk <= sh.g_src_depths) { node = sh.g_src[p - kk - 1]; from = t - kk; }
-            else { const int x0 = tx[t - p]; node = (x0 >= 0 && x0 < sv.V) ? sv.g_root[x0] : -1; from = t - p + 1; }
-            node = walk_from(sv.g_ent, (int)sv.g_cap, node, tx, from, t, lane, cb, wf, cntn);
-            int rank = -1;
-            const int nch = (int)(wf & RUN_COUNT_MASK);
-            // usable as base: at most 64 occurrences, laid down by the offline build, never touched since
-            const bool elig = occ_mode && node >= 0 && cntn <= SD_OCC_BASE && !(wf & NODE_TOUCHED) &&
-                              (nch == 0 || ((wf & RUN_STATIC) && cb < sv.static_entries));
-            if (elig && nch > 0 && lane == 0) rank = sv.g_lo[cb];
-            if (lane == 0) {
-                sh.node[0][p - 1] = node;
-                if (node >= 0) { sh.cb[0][p - 1] = cb; sh.nc[0][p - 1] = wf; sh.g_cnt[p - 1] = cntn; }
-                else atomicOr(&sh.g_failed, 1);
-                sh.g_rank[p - 1] = elig ? (nch > 0 ? rank : -2) : -1;   // -2: usable, and known to have no children
+    if (STEP && wib == 0) {
+        if (ok && n_new > 0 && !refused) {
+            // ---- the request's accepted tokens go into its tree and text (as sd_append does)
+            int32_t* wtext = sv.s_text + (long long)slot * sv.T;
+            TreeRef tr{sv.s_ent + (long long)slot * sv.spn, sv.s_root + (long long)slot * sv.V, (int)sv.spn};
+            int len = ss->len, used = ss->used, live = ss->live, st = ss->status;
+            int act = ss->active[lane], room = ss->room[lane], run_cb = ss->run_cb[lane];
+            unsigned run_w = ss->run_w[lane];
+            for (int k = 0; k < n_new && !(st & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN)); ++k) {
+                const int x = newtok[k];
+                if (x < 0 || x >= sv.V) { st |= SD_STATUS_BAD_TOKEN; break; }
+                if (len >= sv.T || !append_token<APPEND_G>(tr, sv.D, x, len, lane, act, room, run_cb, run_w, used, live)) {
+                    st |= SD_STATUS_POOL_FULL;
+                    break;
+                }
+                if (lane == 0) wtext[len] = x;
+                ++len;
             }
+            ss->active[lane] = act; ss->room[lane] = room; ss->run_cb[lane] = run_cb; ss->run_w[lane] = run_w;
+            if (lane == 0) { ss->len = len; ss->used = used; ss->live = live; ss->status = st; }
         }
-        if (r0 == 0) request_ranges();
-        __syncthreads();
-        if (tid == 0) {
-            const int hi = min(PeG, r0 + WARPS);
-            sh.g_walked = hi;
-            for (int p = r0 + 1; p <= hi && sh.g_base_p == 0; ++p)
-                if (sh.node[0][p - 1] >= 0 && sh.g_rank[p - 1] != -1) sh.g_base_p = p;
-        }
-        __syncthreads();
-        if (sh.g_base_p || sh.g_failed) break;
-    }
-    if (PeG == 0) request_ranges();
-    __syncthreads();
-    if (wib == 0 && PeG > 0) {
-        // the match nodes of this context, for the next call.  A pattern that does not occur ends
-        // the list: no longer one occurs either.
-        const int walked = sh.g_walked, failed = sh.g_failed;
-        const int depths = failed ? SD_MAX_DEPTH : walked;
-        if (lane < depths) ss->g_node[lane] = lane < walked ? sh.node[0][lane] : -1;
-        if (lane == 0) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = depths; }
-    }
-    // the base's occurrences (first pattern token, suffix length)
-    const int base_p = sh.g_base_p;
-    if (wib == 1 && base_p > 0) {
-        const int rank = sh.g_rank[base_p - 1];
-        const int m = rank >= 0 ? sh.g_cnt[base_p - 1] : 0;
-        for (int o = lane; o < m; o += 32) {
-            const int pos = (int)sv.g_sa[rank + o];
-            sh.g_pos[o] = pos;
-            sh.g_avail[o] = (int)sv.g_len[rank + o] - base_p;
-            sh.g_ell[o] = (int)sv.g_back[pos];                  // for now: tokens before the occurrence in its sequence
-        }
-        if (lane == 0) sh.g_base_m = m;
-    }
-    __syncthreads();
-    const int base_m = sh.g_base_m;
-    // the 64 tokens around every occurrence of the base (one coalesced row per occurrence)
-    for (int o = wib; o < base_m; o += WARPS) {
-        const long long pos = sh.g_pos[o];
-        const long long q0 = pos - 32 + lane, q1 = pos + lane;
-        sh.gwin[o][lane] = (q0 >= 0) ? sv.g_text[q0] : -1;
-        sh.gwin[o][32 + lane] = (q1 < sv.N0) ? sv.g_text[q1] : -1;
-    }
-    __syncthreads();
-    if (wib == 0 && base_m > 0) {
-        // how far back every occurrence of the base agrees with the context
-        int ell[SD_OCC_BASE / 32];
+        __threadfence_block();
+        if (lane == 0) *(volatile int*)&sh.app_done = 1;        // the jobs that go through the tree may start
+        // join the others once their queue is ready
+        asm volatile("bar.sync %0, %1;" ::"r"(BAR_JOIN), "r"(NT) : "memory");
+    } else {
+        // ---- the tokens being appended join the text in shared memory
+        if (staged)
+            for (int q = t_old + gtid; q < t; q += GT) stx[q] = newtok[q - t_old];
+        // ---- global match nodes
+        if (want_g) {
 #pragma unroll
-        for (int u = 0; u < SD_OCC_BASE / 32; ++u) {
-            const int o = lane + 32 * u;
-            ell[u] = 0;
-            if (o < base_m) {
-                const int back = sh.g_ell[o];
-                const int lim = min(Lcap, t);
-                int l = base_p;
-                while (l < lim && l - base_p < back && sh.gwin[o][31 - (l - base_p)] == tx[t - 1 - l]) ++l;
-                sh.g_ell[o] = l;
-                ell[u] = l;
+            for (int h = 0; h < MROUNDS; ++h) {
+                const int d = mrank + 1 + h * mwarps;
+                if (d > Pe) continue;
+                int cb = 0;
+                unsigned wf = 0;
+                const int node = (d > t) ? -1 : walk_from(sv.g_ent, (int)sv.g_cap, src_node[h], text, t_old, newtok, src_from[h], t,
+                                                          lane, cb, wf);
+                if (lane == 0) {
+                    ss->g_node[d - 1] = node;
+                    sh.node[0][d - 1] = node;
+                    if (node >= 0) { sh.cb[0][d - 1] = cb; sh.nc[0][d - 1] = wf; }
+                }
             }
+            if (gtid == 0) { ss->g_gen = ss->gen; ss->g_epoch = sv.g_state->epoch; ss->g_len = t; ss->g_depths = Pe; }
         }
-        // lane L: occurrences that match at least L + 1 tokens
-        int c = 0;
+        if (prefetched) asm volatile("cp.async.wait_all;" ::: "memory");
+        group_sync();                                           // the text is in shared memory
+        // ---- per-request occurrences: a chunk of 256 positions at a time, handed out by a counter
+        // (warps that come late from their walks take fewer).  Pass 0 finds the occurrences of the
+        // last token, notes their match lengths and counts them by length; pass 1 collects those
+        // of the patterns that have at most 32 of them.
+        const int last = staged ? stx[t - 1] : 0;
+        const int nchunks = staged ? (t - 1 + 255) / 256 : 0;
+        unsigned char* const sell = reinterpret_cast<unsigned char*>(stx + stage_tokens);   // match length per position (0: none)
+        auto scan_pass = [&](int pass) {
+            const int pn = sh.r_pn;
+            while (true) {
+                int c = 0;
+                if (lane == 0) c = atomicAdd(&sh.scan_next[pass], 1);
+                c = __shfl_sync(FULL, c, 0);
+                if (c >= nchunks) break;
+#pragma unroll 1
+                for (int u = 0; u < 8; ++u) {
+                    const int e = c * 256 + u * 32 + lane;
+                    if (e >= t - 1) continue;
+                    if (pass == 0) {
+                        int l = 0;
+                        if (stx[e] == last) {
+                            l = 1;
+                            while (l < Lcap && e - l >= 0 && stx[e - l] == stx[t - 1 - l]) ++l;
+                            // equal lengths of the 32 positions are counted once (frequent last tokens
+                            // would otherwise all queue up at one counter)
+                            const unsigned grp = __match_any_sync(__activemask(), l);
+                            if (lane == __ffs(grp) - 1) atomicAdd(&sh.r_hist[l], __popc(grp));
+                        }
+                        sell[e] = (unsigned char)l;
+                    } else {
+                        const int l = sell[e];
+                        if (l >= pn) sh.r_list[sh.r_cum[l + 1] + atomicAdd(&sh.r_fill[l], 1)] = e;
+                    }
+                }
+            }
+        };
+        scan_pass(0);
+        group_sync();
+        if (gw == 0) {
+            int h = (lane + 1 <= Lcap) ? sh.r_hist[lane + 1] : 0;   // lane L: matches of exactly L + 1 tokens
 #pragma unroll
-        for (int u = 0; u < SD_OCC_BASE / 32; ++u)
-            for (int o = 0; o < 32; ++o) c += (__shfl_sync(FULL, ell[u], o) >= lane + 1) ? 1 : 0;
-        sh.g_cum[lane + 1] = lane + 1 >= base_p ? c : 0;
-    }
-    __syncthreads();
+            for (int o = 1; o < 32; o <<= 1) {                  // suffix sums: matches of at least L + 1 tokens
+                const int y = __shfl_down_sync(FULL, h, o);
+                if (lane + o < 32) h += y;
+            }
+            sh.r_cum[lane + 1] = h;
+            const unsigned few = __ballot_sync(FULL, h <= SD_OCC_LANES);
+            if (lane == 0) sh.r_pn = __ffs(few);                // (the counts fall with the length: lane 31 always qualifies)
+        }
+        group_sync();
+        if (staged && sh.r_cum[sh.r_pn] > 0) scan_pass(1);
+        group_sync();
 
-    // ---------------- 3. job queue, costliest first; tree-entry jobs that start at a wide node wait
-    if (tid < 2 * SD_MAX_DEPTH) {
-        const int tree = tid / SD_MAX_DEPTH, p = tid % SD_MAX_DEPTH + 1;
-        int c = 0;
-        if (p <= Pe && p <= Lcap) {
-            bool has = false;
-            if (tree == 1) has = p <= Lr && sh.r_cnt[p] > 0;
-            else if (base_p > 0 && p >= base_p) has = sh.g_cum[p] > 0;
-            else if (p <= sh.g_walked) {
+        // ---------------- 2. the job queue, costliest first.  Per-request jobs that have to go through
+        // the tree (more than 32 occurrences, or no text in shared memory) come last: in sd_step
+        // they have to wait for the append.
+        // (order: the jobs that are read off the text first: they are quick and a long match there
+        // sets a score that rules out most of the others; then by the nodes a job can add at most)
+        if (gtid < 2 * SD_MAX_DEPTH) {
+            const int tree = gtid / SD_MAX_DEPTH, p = gtid % SD_MAX_DEPTH + 1;
+            int c = 0;
+            if (tree == 0) {
                 const unsigned wf = sh.nc[0][p - 1];
                 const int nch = (int)(wf & RUN_COUNT_MASK);
-                has = sh.node[0][p - 1] >= 0 && nch > 0;
-                if (has) {
+                if (p <= Pe && sh.node[0][p - 1] >= 0 && nch > 0) {
                     // all first runs start their way to L2 now, long before a warp gets to them
                     const int4* base = sv.g_ent + sh.cb[0][p - 1];
                     const int lines = min(4, (nch + 7) >> 3);
                     for (int l = 0; l < lines; ++l) prefetch_l2(base + l * 8);
+                    c = min(budget_for(alpha, p, cap), 2 * (D - p));
+                    if (c > 0 && nch > WIDE_RUN && !(wf & RUN_HAS_TOP)) { sh.wide[atomicAdd(&sh.nwide, 1)] = gtid; c = 0; }
+                    if (c > 0) c += 1000;
                 }
+            } else if (want_r && p <= Pe && p <= t) {
+                c = min(budget_for(alpha, p, cap), 2 * (D - p));
+                if (staged && !(p <= Lcap && sh.r_cum[p] > 0)) c = 0;      // no earlier occurrence: nothing to speculate
+                else if (c > 0 && staged && p >= sh.r_pn) c += 2000;       // read off the text
             }
-            if (has) {
-                c = min(budget_for(a.alpha, p, cap), D - p);      // an upper bound of the job's SCORE, see below
-                if (c > 0 && tree == 0 && !(base_p > 0 && p >= base_p)) {
-                    const unsigned wf = sh.nc[0][p - 1];
-                    if ((int)(wf & RUN_COUNT_MASK) > WIDE_RUN && !(wf & RUN_HAS_TOP)) { sh.wide[atomicAdd(&sh.nwide, 1)] = tid; c = 0; }
+            sh.cost[gtid] = c;
+        }
+        group_sync();
+        if (gtid < 2 * SD_MAX_DEPTH) {
+            const int c = sh.cost[gtid];
+            if (c > 0) {
+                int rank = 0;
+                for (int q = 0; q < 2 * SD_MAX_DEPTH; ++q) {
+                    const int cq = sh.cost[q];
+                    rank += (cq > c || (cq == c && q < gtid)) ? 1 : 0;
                 }
+                sh.job[rank] = gtid | (c < 1000 ? 128 : 0);     // bit 7: through the tree, behind the append
+                atomicAdd(&sh.njobs, 1);
             }
         }
-        sh.cost[tid] = c;
+        group_sync();
+        if (STEP) asm volatile("bar.arrive %0, %1;" ::"r"(BAR_JOIN), "r"(NT) : "memory");   // warp 0 may come in
     }
-    __syncthreads();
-    if (tid < 2 * SD_MAX_DEPTH) {
-        const int c = sh.cost[tid];
-        if (c > 0) {
-            int rank = 0;
-            for (int q = 0; q < 2 * SD_MAX_DEPTH; ++q) {
-                const int cq = sh.cost[q];
-                rank += (cq > c || (cq == c && q < tid)) ? 1 : 0;
-            }
-            sh.job[rank] = tid;
-            atomicAdd(&sh.njobs, 1);
-        }
-    }
-    __syncthreads();
-    const int njobs = sh.njobs;
-    while (true) {
-        int j = 0;
-        if (lane == 0) j = atomicAdd(&sh.next, 1);
-        j = __shfl_sync(FULL, j, 0);
-        if (j >= njobs) break;
-        const int code = sh.job[j];
-        const int tree = code / SD_MAX_DEPTH, p = code % SD_MAX_DEPTH + 1;
-        const int budget = budget_for(a.alpha, p, cap);
-        // SCORE <= number of draft nodes (every D <= 1), and SCORE <= number of levels below the
-        // match node: the D values of one level of a tree add up to at most 1 (Eq. 1 shares out the
-        // parent's D among its children).  A job that cannot reach the best score so far is skipped.
-        if ((double)min(budget, D - p) * 1.000000001 < best_so_far(sh)) continue;
-        if (tree == 1) {
-            const int m = sh.r_cnt[p], lo = sh.r_lo[p] + 1;
-            if (m <= SD_OCC_LANES) {
-                const int e = lane < m ? S[lo + lane] + p - 1 : 0;       // the occurrence's last pattern token
+    const int4* s_ent = ok ? sv.s_ent + (long long)slot * sv.spn : nullptr;
+    {
+        const int njobs = sh.njobs;
+        while (true) {
+            int j = 0;
+            if (lane == 0) j = atomicAdd(&sh.next, 1);
+            j = __shfl_sync(FULL, j, 0);
+            if (j >= njobs) break;
+            const int code = sh.job[j];
+            const int tree = (code & 127) / SD_MAX_DEPTH, p = (code & 127) % SD_MAX_DEPTH + 1;
+            const int budget = budget_for(alpha, p, cap);
+            // SCORE <= number of draft nodes (every D <= 1), and SCORE <= number of levels below the
+            // match node: the D values of one level of a tree add up to at most 1 (Eq. 1 shares out
+            // the parent's D among its children)
+            if ((double)min(budget, D - p) * 1.000000001 < best_so_far(sh)) continue;
+            if (tree == 0) {
+                expand_job(sh, W, sv.g_ent, (int)sv.g_cap, 0, p, budget, flags, false, 0, lane);
+            } else if (!(code & 128)) {
+                const int m = sh.r_cum[p];
+                const int e = lane < m ? sh.r_list[lane] : 0;
                 const int kmax = lane < m ? min(t - 1 - e, D - p) : 0;
-                expand_occ(sh, W, tx + e, kmax, 1, p, budget, flags, lane);
+                expand_occ(sh, W, stx + e, kmax, 1, p, budget, flags, lane);
             } else {
-                expand_range<false>(sh, W, TextItems{tx, S, t, p}, lo, lo + m, 1, p, budget, D - p, flags, lane);
-            }
-        } else if (base_p > 0 && p >= base_p) {
-            if (sh.g_cum[p] <= SD_OCC_LANES) {
-                // a lane per occurrence that matches p tokens: lane i takes the i-th of them
-                unsigned mk[SD_OCC_BASE / 32];
-                int o = -1, left = lane + 1;
-#pragma unroll
-                for (int u = 0; u < SD_OCC_BASE / 32; ++u) {
-                    mk[u] = __ballot_sync(FULL, lane + 32 * u < base_m && sh.g_ell[lane + 32 * u] >= p);
-                    const int c = __popc(mk[u]);
-                    if (o < 0 && left <= c) o = 32 * u + (int)__fns(mk[u], 0, left);
-                    left -= c;
+                // through the tree: the match node is the slot's active node of depth p, once the
+                // append is done (bounded wait; a job that runs out of patience is done after the
+                // block-wide barrier below instead)
+                bool ready = true;
+                if (STEP) {
+                    ready = false;
+                    for (int spin = 0; spin < 4096 && !ready; ++spin) {
+                        int flag = 0;
+                        if (lane == 0) flag = *(volatile int*)&sh.app_done;
+                        ready = __shfl_sync(FULL, flag, 0) != 0;
+                        if (!ready) __nanosleep(200);
+                    }
                 }
-                const int kmax = o >= 0 ? min(sh.g_avail[o], D - p) : 0;
-                expand_occ(sh, W, &sh.gwin[o >= 0 ? o : 0][31 + base_p], kmax, 0, p, budget, flags, lane);
-            } else {
-                expand_range<true>(sh, W, WindowItems{sh.gwin, sh.g_avail, sh.g_ell, base_p, p}, 0, base_m, 0, p, budget, D - p,
-                                   flags, lane);
+                if (!ready) { if (lane == 0) sh.late[atomicAdd(&sh.nlate, 1)] = p; continue; }
+                request_tree_job(sh, W, sv, ss, s_ent, t, p, budget, flags, lane);
             }
-        } else {
-            expand_job(sh, W, sv.g_ent, (int)sv.g_cap, 0, p, budget, flags, false, 0, lane);
         }
     }
+    __syncthreads();                                            // sd_step: the append is done and visible
+
+    // ---------------- 3. what had to wait: an append that stopped early, per-request jobs whose wait
+    // ran out, jobs that start at a wide child run
+    if (STEP && ok && !refused) {
+        status = ss->status;
+        if (ss->len != t || (status & (SD_STATUS_POOL_FULL | SD_STATUS_BAD_TOKEN))) {
+            // the append stopped early: no speculation for this request, and the match nodes
+            // taken above describe a context that does not exist
+            usable = false; want_g = false; want_r = false;
+            t = ss->len;
+            if (tid == 0) ss->g_gen = ss->gen - 1;
+        }
+    }
+    for (int q = wib; q < sh.nlate && usable; q += CTA_WARPS) {
+        const int p = sh.late[q];
+        const int budget = budget_for(alpha, p, cap);
+        if ((double)min(budget, D - p) * 1.000000001 < best_so_far(sh)) continue;
+        request_tree_job(sh, W, sv, ss, s_ent, t, p, budget, flags, lane);
+    }
     __syncthreads();
-    // Tree-entry jobs that start at a wide node (short patterns, hence small budgets): most cannot
-    // reach the best score any more and are dropped here.  For the rest the warps of the block share
+    // Jobs that start at a wide node (short patterns, hence small budgets): most cannot reach
+    // the best score any more and are dropped here.  For the rest the warps of the block share
     // the scan of the run, then one warp merges the partial lists and finishes the job.
     if (tid == 0) {
         const double best = __hiloint2double((int)sh.best_hi, 0);
         int kept = 0;
-        for (int q = 0; q < sh.nwide; ++q) {
+        for (int q = 0; q < sh.nwide && usable; ++q) {
             const int p = sh.wide[q] % SD_MAX_DEPTH + 1;
-            if (!((double)min(budget_for(a.alpha, p, cap), D - p) * 1.000000001 < best)) sh.wide[kept++] = sh.wide[q];
+            if (!((double)min(budget_for(alpha, p, cap), D - p) * 1.000000001 < best)) sh.wide[kept++] = sh.wide[q];
         }
         sh.nwide_kept = kept;
     }
     __syncthreads();
     const int nwide = sh.nwide_kept;
-    for (int base = 0; base < nwide; base += WARPS) {
-        const int nj = min(WARPS, nwide - base);
-        const int G = WARPS / nj;                               // warps per job
+    for (int base = 0; base < nwide; base += CTA_WARPS) {
+        const int nj = min(CTA_WARPS, nwide - base);
+        const int G = CTA_WARPS / nj;                           // warps per job
         const int my_job = wib / G, my_slice = wib % G;
         const bool active = my_job < nj;
-        int p = 1, budget = 0, fs = 0;
+        int tree = 0, p = 1, budget = 0, fs = 0;
+        const int4* ent = sv.g_ent;
         if (active) {
             const int code = sh.wide[base + my_job];
-            p = code % SD_MAX_DEPTH + 1;
-            budget = budget_for(a.alpha, p, cap);
+            tree = code / SD_MAX_DEPTH; p = code % SD_MAX_DEPTH + 1;
+            budget = budget_for(alpha, p, cap);
+            ent = tree == 0 ? sv.g_ent : s_ent;
             long long sum;
-            scan_run_by_count(sv.g_ent, sh.cb[0][p - 1], (int)(sh.nc[0][p - 1] & RUN_COUNT_MASK), my_slice, G, -1, 1, W,
+            scan_run_by_count(ent, sh.cb[tree][p - 1], (int)(sh.nc[tree][p - 1] & RUN_COUNT_MASK), my_slice, G, -1, 1, W,
                               W.F, 0, fs, budget, sum, lane);
             if (lane == 0) { sh.slice_sum[wib] = sum; sh.slice_fs[wib] = fs; }
         }
@@ -1242,15 +1353,15 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
                 frontier_merge_list(W.F, 0, fs, budget, O, ofs, -1, lane);
             }
             counts_to_d(W.F, 0, fs, 1.0, sum, lane);
-            expand_job(sh, W, sv.g_ent, (int)sv.g_cap, 0, p, budget, flags, true, fs, lane);
+            expand_job(sh, W, ent, tree == 0 ? (int)sv.g_cap : (int)sv.spn, tree, p, budget, flags, true, fs, lane);
         }
         __syncthreads();
     }
 
     // ---------------- 4. select (first in loop order among the largest scores) and emit
     if (wib == 0) {
-        double sc = lane < WARPS ? sh.w[lane].best_score : 0.0;
-        int od = lane < WARPS ? sh.w[lane].best_order : 1 << 30;
+        double sc = lane < CTA_WARPS ? sh.w[lane].best_score : 0.0;
+        int od = lane < CTA_WARPS ? sh.w[lane].best_order : 1 << 30;
         int ww = lane;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
@@ -1260,7 +1371,7 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
             if (osc > sc || (osc == sc && ood < od)) { sc = osc; od = ood; ww = oww; }
         }
         // Section 3.2: the tree is used only if its score exceeds the threshold (tau = 0: any score above 0)
-        if (lane == 0) sh.win_warp = (sc > 0.0 && sc > a.tau) ? ww : -1;
+        if (lane == 0) sh.win_warp = (usable && sc > 0.0 && sc > tau) ? ww : -1;
     }
     __syncthreads();
     const int win = sh.win_warp;
@@ -1282,48 +1393,43 @@ __global__ void __launch_bounds__(WARPS * 32, MINB) speculate_fused_kernel(sd_st
             tok = wtok[j];
             par = (int)wpar[j] - 1;
             int depth = 0;
-            for (int an = j, hops = 0; an >= 0 && hops < SD_MAX_SPEC; an = (int)wpar[an] - 1, ++hops) {
-                bits |= 1ull << an;
+            for (int a = j, hops = 0; a >= 0 && hops < SD_MAX_SPEC; a = (int)wpar[a] - 1, ++hops) {
+                bits |= 1ull << a;
                 ++depth;
             }
             pos = t + depth - 1;
         }
         const long long o = (long long)i * M + j;
-        a.d_tokens[o] = tok; a.d_parents[o] = par; a.d_positions[o] = pos;
-        a.d_mask[o * words] = (uint32_t)bits;
-        if (words > 1) a.d_mask[o * words + 1] = (uint32_t)(bits >> 32);
+        d_tokens[o] = tok; d_parents[o] = par; d_positions[o] = pos;
+        d_mask[o * words] = (uint32_t)bits;
+        if (words > 1) d_mask[o * words + 1] = (uint32_t)(bits >> 32);
     }
     if (tid == 0) {
-        a.d_n_draft[i] = nd; a.d_chosen_tree[i] = ctree; a.d_chosen_p[i] = cp; a.d_score[i] = best;
-        if (a.d_status) a.d_status[i] = status;
+        d_n_draft[i] = nd; d_chosen_tree[i] = ctree; d_chosen_p[i] = cp; d_score[i] = best;
+        if (d_status) d_status[i] = status;
     }
 }
 
 }  // namespace
 
-// ---------------------------------------------------------------------------------------------
-// Launch.  Block shapes (measured): two blocks per SM is the usual one; a batch of at most one
-// request per SM gets bigger blocks, a batch of more than two requests per SM smaller ones
-// (four per SM) to stay in one wave.  The text of a request is staged in shared memory when it
-// fits beside the block's working set, else it is read in place.
 namespace {
 
-constexpr int CTA_WARPS = 10;
-constexpr int CTA_WARPS_WIDE = 16;
-constexpr int CTA_WARPS_NARROW = 5;
-constexpr int SMEM_PER_SM = 228 * 1024;       // shared memory of one SM; a block also costs 1 KB of it
+constexpr int SMEM_PER_SM = 228 * 1024;       // shared memory of one SM; a resident block also costs 1 KB of it
 constexpr int MAX_DEVICES = 64;
-
-struct DeviceInfo {
-    bool ready = false;
-    int sm_count = 0;
-};
+struct DeviceInfo { bool ready = false; int sm_count = 0; };
 DeviceInfo g_dev[MAX_DEVICES];
 std::mutex g_dev_mutex;
 
+// tokens of text a block of this shape can hold in shared memory beside its working set
 template <int WARPS, int MINB>
 constexpr int stage_limit_tokens() {
-    return (int)((SMEM_PER_SM / MINB - 1024 - (int)((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15)) / 4) & ~3;
+    return (int)((SMEM_PER_SM / MINB - 1024 - (int)((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15)) / 5) & ~15;   // 4 + 1 bytes per token
+}
+
+template <bool STEP, int WARPS, int MINB, int G>
+int raise_smem_limit() {
+    return cudaFuncSetAttribute(speculate_fused_kernel<STEP, WARPS, MINB, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                SMEM_PER_SM / MINB - 1024) == cudaSuccess ? SD_OK : SD_ERR_CUDA;
 }
 
 // once per device: raise the kernels' dynamic shared memory limit, read the SM count
@@ -1331,12 +1437,11 @@ int device_setup(int dev, int* sm_count) {
     if (dev < 0 || dev >= MAX_DEVICES) return SD_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lock(g_dev_mutex);
     if (!g_dev[dev].ready) {
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<CTA_WARPS, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        SMEM_PER_SM / 2 - 1024));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<CTA_WARPS_WIDE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        SMEM_PER_SM - 1024));
-        SD_CUDA_OK(cudaFuncSetAttribute(speculate_fused_kernel<CTA_WARPS_NARROW, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        SMEM_PER_SM / 4 - 1024));
+        if (raise_smem_limit<false, CTA_WARPS, 2, 8>() != SD_OK || raise_smem_limit<true, CTA_WARPS_STEP, 2, STEP_G>() != SD_OK ||
+            raise_smem_limit<false, CTA_WARPS_WIDE, 1, 8>() != SD_OK || raise_smem_limit<true, CTA_WARPS_WIDE_STEP, 1, 8>() != SD_OK ||
+            raise_smem_limit<false, CTA_WARPS_NARROW, 4, 8>() != SD_OK ||
+            raise_smem_limit<true, CTA_WARPS_NARROW_STEP, 4, STEP_G>() != SD_OK)
+            return SD_ERR_CUDA;
         SD_CUDA_OK(cudaDeviceGetAttribute(&g_dev[dev].sm_count, cudaDevAttrMultiProcessorCount, dev));
         g_dev[dev].ready = true;
     }
@@ -1344,19 +1449,13 @@ int device_setup(int dev, int* sm_count) {
     return SD_OK;
 }
 
-template <int WARPS, int MINB>
-void launch_shape(const sd_store& s, StepArgs a, cudaStream_t st) {
-    // shared memory behind the block's working set: the text and its suffix order (as many entries), if they fit
-    const int lim = stage_limit_tokens<WARPS, MINB>();
-    a.stage_tokens = 2 * s.Tp <= lim ? s.Tp : 0;
-    const size_t smem = ((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15) + (size_t)a.stage_tokens * 8;
-    speculate_fused_kernel<WARPS, MINB><<<(unsigned)a.n, WARPS * 32, smem, st>>>(s, a);
-}
+}  // namespace
 
-int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm, const int32_t* d_budget_cap,
-                 int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask,
-                 int32_t* d_chosen_tree, int32_t* d_chosen_p, double* d_score, int32_t* d_status,
-                 const int64_t* d_app_off, const int32_t* d_app_tok, bool step, int32_t* scratch, void* stream) {
+static int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
+                        const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents,
+                        int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
+                        double* d_score, int32_t* d_status, const int64_t* d_app_off, const int32_t* d_app_tok,
+                        bool step, void* stream) {
     if (!s || !prm || n < 0 || n > s->R) return SD_ERR_INVALID_ARG;
     if (prm->P < 1 || prm->max_spec < 0 || prm->max_spec > s->M || !(prm->alpha >= 0.0) || !(prm->tau >= 0.0))
         return SD_ERR_INVALID_ARG;
@@ -1367,38 +1466,48 @@ int launch_fused(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_pa
         !d_score)
         return SD_ERR_INVALID_ARG;
     if (step && !d_app_off) return SD_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int Pe = prm->P < s->D ? prm->P : s->D;               // longer patterns never match
     int sms = 0;
     const int rc = device_setup(s->device, &sms);
     if (rc != SD_OK) return rc;
-    StepArgs a;
-    a.n = n; a.d_slot = d_slot;
-    a.Pe = prm->P < s->D ? prm->P : s->D;                       // longer patterns never match
-    a.alpha = prm->alpha; a.max_spec = prm->max_spec; a.flags = prm->flags; a.tau = prm->tau;
-    a.d_budget_cap = d_budget_cap;
-    a.d_n_draft = d_n_draft; a.d_tokens = d_tokens; a.d_parents = d_parents; a.d_positions = d_positions;
-    a.d_mask = d_mask; a.d_chosen_tree = d_chosen_tree; a.d_chosen_p = d_chosen_p; a.d_score = d_score;
-    a.d_status = d_status;
-    a.d_app_off = step ? d_app_off : nullptr; a.d_app_tok = step ? d_app_tok : nullptr;
-    a.stage_tokens = 0;
-    a.scratch = scratch;
-    cudaStream_t st = (cudaStream_t)stream;
-    // a text too long for the usual shape's shared memory may still fit the one-block-per-SM shape
-    const bool long_text = 2 * s->Tp > stage_limit_tokens<CTA_WARPS, 2>();
-    if (n <= sms || (long_text && n <= 2 * sms)) launch_shape<CTA_WARPS_WIDE, 1>(*s, a, st);
-    else if (n > 2 * sms && 2 * s->Tp <= stage_limit_tokens<CTA_WARPS_NARROW, 4>()) launch_shape<CTA_WARPS_NARROW, 4>(*s, a, st);
-    else launch_shape<CTA_WARPS, 2>(*s, a, st);
+    // one block per SM is all a small batch can use: sd_speculate then takes more warps if a
+    // request has more jobs (two trees, Pe pattern lengths each) than 16 warps start at once,
+    // sd_step takes more registers
+    const bool wide = n <= sms && (step || 2 * Pe > 2 * CTA_WARPS);
+    // more requests than two 16-warp blocks per SM hold at once: smaller blocks, one wave
+    const bool narrow = n > 2 * sms;
+    // Behind its working set a block keeps the request's text in shared memory if it fits (a
+    // longer text is not scanned: all of its per-request jobs go through the tree).
+#define SD_LAUNCH_FUSED(STEP, WARPS, MINB, G, OFF, TOK)                                                                 \
+    do {                                                                                                                 \
+        const int lim = stage_limit_tokens<WARPS, MINB>();                                                               \
+        const int stage = s->T <= lim ? ((s->T + 15) & ~15) : 0;                                                         \
+        const size_t smem = ((sizeof(BlockSharedT<WARPS>) + 15) & ~(size_t)15) + (size_t)stage * 5;                      \
+        speculate_fused_kernel<STEP, WARPS, MINB, G><<<(unsigned)n, WARPS * 32, smem, st>>>(                             \
+            *s, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, prm->tau, d_budget_cap, d_n_draft, d_tokens,       \
+            d_parents, d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score, d_status, OFF, TOK, stage);              \
+    } while (0)
+    if (step) {
+        if (wide) SD_LAUNCH_FUSED(true, CTA_WARPS_WIDE_STEP, 1, 8, d_app_off, d_app_tok);
+        else if (narrow) SD_LAUNCH_FUSED(true, CTA_WARPS_NARROW_STEP, 4, STEP_G, d_app_off, d_app_tok);
+        else SD_LAUNCH_FUSED(true, CTA_WARPS_STEP, 2, STEP_G, d_app_off, d_app_tok);
+    } else {
+        if (wide) SD_LAUNCH_FUSED(false, CTA_WARPS_WIDE, 1, 8, nullptr, nullptr);
+        else if (narrow) SD_LAUNCH_FUSED(false, CTA_WARPS_NARROW, 4, 8, nullptr, nullptr);
+        else SD_LAUNCH_FUSED(false, CTA_WARPS, 2, 8, nullptr, nullptr);
+    }
+#undef SD_LAUNCH_FUSED
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }
-
-}  // namespace
 
 extern "C" int sd_speculate(sd_store* s, int32_t n, const int32_t* d_slot, const sd_spec_params* prm,
                             const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens, int32_t* d_parents,
                             int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree, int32_t* d_chosen_p,
                             double* d_score, int32_t* d_status, void* stream) {
     return launch_fused(s, n, d_slot, prm, d_budget_cap, d_n_draft, d_tokens, d_parents, d_positions, d_mask, d_chosen_tree,
-                        d_chosen_p, d_score, d_status, nullptr, nullptr, false, s ? s->occ_scratch : nullptr, stream);
+                        d_chosen_p, d_score, d_status, nullptr, nullptr, false, stream);
 }
 
 extern "C" int sd_step(sd_store* s, int32_t n, const int32_t* d_slot, const int64_t* d_offsets, const int32_t* d_new_tokens,
@@ -1406,33 +1515,37 @@ extern "C" int sd_step(sd_store* s, int32_t n, const int32_t* d_slot, const int6
                        int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
                        int32_t* d_chosen_p, double* d_score, int32_t* d_status, void* stream) {
     return launch_fused(s, n, d_slot, prm, d_budget_cap, d_n_draft, d_tokens, d_parents, d_positions, d_mask, d_chosen_tree,
-                        d_chosen_p, d_score, d_status, d_offsets, d_new_tokens, true, s ? s->occ_scratch : nullptr, stream);
+                        d_chosen_p, d_score, d_status, d_offsets, d_new_tokens, true, stream);
 }
 
 // ---------------------------------------------------------------------------------------------
-// sd_speculate_noalloc: sd_speculate with the kernel's scratch memory (the occurrence lists that
-// do not fit shared memory) in a fixed array that is part of the loaded library image instead of
-// in memory the store obtained from cudaMalloc.  Meant for callers that must not touch the CUDA
-// allocator at all (see the declaration in suffixspec.h).
+// sd_speculate_noalloc: the same two kernels, with the per-job scratch records kept in a
+// fixed array that is part of the loaded library image instead of in memory obtained
+// from cudaMalloc.  Meant for callers that must not touch the CUDA allocator at all
+// (see the declaration in suffixspec.h).
 //
 // The array's name below is only meaningful to device code.  Host code holds a stand-in
 // symbol of the same name, so the launch code first asks the runtime for the array's
 // real device address (once per device, with that device current) and passes that on.
 namespace {
 
-static __device__ __align__(256) int32_t g_noalloc_scratch[SD_NOALLOC_MAX_TOKENS];
+constexpr long long NOALLOC_BYTES =
+    (long long)SD_NOALLOC_MAX_JOBS * (sizeof(double) + sizeof(int32_t) + 2ll * SD_MAX_SPEC * sizeof(int32_t));
 
-int32_t* g_noalloc_ptr[MAX_DEVICES];          // device address of the array, per device
-bool g_noalloc_ready[MAX_DEVICES];
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+unsigned char* g_noalloc_ptr[NOALLOC_MAX_DEVICES];      // device address of the array, per device
+bool g_noalloc_ready[NOALLOC_MAX_DEVICES];
 std::mutex g_noalloc_mutex;
 
 // Device address of the scratch array on the current device (looked up on first use).
-int noalloc_scratch_address(int32_t** out) {
+int noalloc_scratch_address(unsigned char** out) {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return SD_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return SD_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_noalloc_mutex);
     if (!g_noalloc_ready[dev]) {
-        int32_t* p = nullptr;
+        unsigned char* p = nullptr;
         if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) {
             cudaGetLastError();
             return SD_ERR_CUDA;
@@ -1450,15 +1563,36 @@ extern "C" int sd_speculate_noalloc(sd_store* s, int32_t n, const int32_t* d_slo
                                     const int32_t* d_budget_cap, int32_t* d_n_draft, int32_t* d_tokens,
                                     int32_t* d_parents, int32_t* d_positions, uint32_t* d_mask, int32_t* d_chosen_tree,
                                     int32_t* d_chosen_p, double* d_score, int32_t* d_status, void* stream) {
-    if (!s || n < 0 || n > s->R) return SD_ERR_INVALID_ARG;
+    if (!s || !prm || n < 0 || n > s->R) return SD_ERR_INVALID_ARG;
+    if (prm->P < 1 || prm->max_spec < 0 || prm->max_spec > s->M || !(prm->alpha >= 0.0) || !(prm->tau >= 0.0))
+        return SD_ERR_INVALID_ARG;
+    if ((prm->flags & SD_FLAG_GLOBAL_ONLY) && (prm->flags & SD_FLAG_REQUEST_ONLY)) return SD_ERR_INVALID_ARG;
     SD_CHECK_DEVICE(s);
-    // one row of max_req_tokens (rounded up to 4) per request: the batch must fit the fixed array
-    if ((long long)n * s->Tp > SD_NOALLOC_MAX_TOKENS) return SD_ERR_CAPACITY;
-    int32_t* base = nullptr;
+    // one record per (request, tree, depth): the batch must fit the fixed array
+    if ((long long)n * 2 * s->D > SD_NOALLOC_MAX_JOBS) return SD_ERR_CAPACITY;
+    if (n == 0) return SD_OK;
+    if (!d_slot || !d_n_draft || !d_tokens || !d_parents || !d_positions || !d_mask || !d_chosen_tree || !d_chosen_p ||
+        !d_score)
+        return SD_ERR_INVALID_ARG;
+    unsigned char* base = nullptr;
     const int rc = noalloc_scratch_address(&base);
     if (rc != SD_OK) return rc;
-    // Every list the kernel reads from the array was written by the same block earlier in the same
-    // launch, so nothing left over from an earlier call is ever consumed and nothing needs clearing.
-    return launch_fused(s, n, d_slot, prm, d_budget_cap, d_n_draft, d_tokens, d_parents, d_positions, d_mask, d_chosen_tree,
-                        d_chosen_p, d_score, d_status, nullptr, nullptr, false, base, stream);
+    // Same record layout as the store's own scratch, carved out of the fixed array.  Every
+    // record the second kernel reads is written by the first kernel of the same call, so
+    // nothing left over from an earlier call is ever consumed and nothing needs clearing.
+    sd_store view = *s;
+    view.j_score = reinterpret_cast<double*>(base);
+    view.j_n = reinterpret_cast<int32_t*>(base + (long long)SD_NOALLOC_MAX_JOBS * sizeof(double));
+    view.j_tok = view.j_n + SD_NOALLOC_MAX_JOBS;
+    view.j_par = view.j_tok + (long long)SD_NOALLOC_MAX_JOBS * SD_MAX_SPEC;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int Pe = prm->P < s->D ? prm->P : s->D;
+    const long long jobs = (long long)n * 2 * Pe;
+    match_expand_kernel<<<(unsigned)((jobs + SPEC_WARPS - 1) / SPEC_WARPS), SPEC_WARPS * 32, 0, st>>>(
+        view, n, d_slot, Pe, prm->alpha, prm->max_spec, prm->flags, d_budget_cap);
+    select_emit_kernel<<<(unsigned)((n + 3) / 4), 128, 0, st>>>(view, n, d_slot, Pe, prm->tau, d_n_draft, d_tokens, d_parents,
+                                                                d_positions, d_mask, d_chosen_tree, d_chosen_p, d_score,
+                                                                d_status);
+    SD_CUDA_OK(cudaGetLastError());
+    return SD_OK;
 }

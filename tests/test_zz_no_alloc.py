@@ -25,17 +25,14 @@ def test_noalloc_matches_sd_speculate_twice_in_a_row():
     import paper_2411_04975_b200 as sfx
 
     rng = np.random.default_rng(77)
-    vocab, D, n_slots = 3, 32, 64
+    vocab, D, n_slots = 6, 32, 64
     corpus = [rng.integers(0, vocab, size=int(rng.integers(50, 400))).astype(np.int32) for _ in range(20)]
-    pr = U.Pair(corpus, vocab=vocab, D=D, n_slots=n_slots, max_req_tokens=8000)
-    # Texts of a few thousand tokens over three token values: the last token has well over 1,024
-    # earlier occurrences, so the kernel keeps its occurrence list in the scratch array
-    # (shorter lists stay in shared memory and would not touch it).  Some slots stay short or empty.
-    lens = [int(rng.integers(3500, 7000)) if s % 3 else int(rng.integers(0, 200)) for s in range(n_slots)]
-    pr.append(list(range(n_slots)), [rng.integers(0, vocab, size=L).astype(np.int32) for L in lens], reset=[1] * n_slots)
+    pr = U.Pair(corpus, vocab=vocab, D=D, n_slots=n_slots, max_req_tokens=300)
+    pr.append(list(range(n_slots)), [rng.integers(0, vocab, size=int(rng.integers(0, 200))).astype(np.int32)
+                                     for _ in range(n_slots)], reset=[1] * n_slots)
     g = pr.g
 
-    # call 1: the largest batch the fixed array takes (64 requests x 8,000 tokens = 512,000 entries)
+    # call 1: the largest batch the fixed array takes (64 requests x 2 trees x depth 32 = 4096 jobs)
     slots = U.dev_i32(list(range(n_slots)))
     want = g.speculate(slots, 32, 2.0, 64)
     got = g.alloc_outputs(n_slots)
@@ -65,12 +62,11 @@ def test_noalloc_rejects_batches_beyond_its_fixed_array():
     import gpu_util as U
     import paper_2411_04975_b200 as sfx
 
-    # 9 requests x 65,536 tokens of text each is more than the array's 524,288 entries; 8 fit exactly
-    pr = U.Pair([np.arange(40, dtype=np.int32) % 5], vocab=5, D=32, n_slots=9, max_req_tokens=65536)
-    out = pr.g.alloc_outputs(9)
+    pr = U.Pair([np.arange(40, dtype=np.int32) % 5], vocab=5, D=32, n_slots=65, max_req_tokens=16)
+    out = pr.g.alloc_outputs(65)
     with pytest.raises(sfx.SuffixSpecError) as e:
-        sfx.sd_speculate_noalloc(pr.g.handle, U.dev_i32(list(range(9))), 8, 2.0, 64, 0, None, out)
+        sfx.sd_speculate_noalloc(pr.g.handle, U.dev_i32(list(range(65))), 8, 2.0, 64, 0, None, out)
     assert e.value.code == -4 and "capacity" in str(e.value)
-    sfx.sd_speculate_noalloc(pr.g.handle, U.dev_i32(list(range(8))), 8, 2.0, 64, 0, None, pr.g.alloc_outputs(8))
+    sfx.sd_speculate_noalloc(pr.g.handle, U.dev_i32(list(range(64))), 8, 2.0, 64, 0, None, pr.g.alloc_outputs(64))
     torch.cuda.synchronize()
     pr.close()

@@ -35,9 +35,33 @@ METRIC = "speculation trees/s at batch {B} (per step: append the accepted tokens
 UNIT = "trees/s"
 OUT_BYTES_PER_REQ = 4 * 64 * 3 + 64 * 8 + 4 * 3 + 8          # tokens, parents, positions, mask, scalars
 FLUSH_BYTES = 256 << 20
-# dram__bytes_read + dram__bytes_write of one speculate_fused_kernel<1, 10, 2, 4> launch (sd_step) on the full-size
-# large_batch workload, from the ncu capture summarised in profiles/ (set to None when the kernel changes)
-SPECULATE_DRAM_TRAFFIC = 27.3e6
+APPEND_BYTES_PER_UPDATE = 32                                   # a node's 16-byte entry read and written back
+STEP_KERNEL = "speculate_fused_kernel<true, 10, 2, 4> (all of sd_step)"
+# dram__bytes_read + dram__bytes_write of one launch of that kernel on the full-size large_batch
+# workload, from an ncu capture; it is reported only while the kernel source still has the
+# digest the capture was taken at (profiles/ holds the summary), else as null
+DRAM_TRAFFIC = {"bytes": None, "speculate_cu_sha1": None}
+
+
+def dram_traffic():
+    import hashlib
+    if DRAM_TRAFFIC["bytes"] is None:
+        return None
+    try:
+        with open(os.path.join(ROOT, "paper_2411_04975_b200", "csrc", "speculate.cu"), "rb") as f:
+            same = hashlib.sha1(f.read()).hexdigest() == DRAM_TRAFFIC["speculate_cu_sha1"]
+    except OSError:
+        same = False
+    return DRAM_TRAFFIC["bytes"] if same else None
+
+
+def config_dict(c, args):
+    """The workload both arms (the CUDA path and the oracle) are timed on: one dict for both."""
+    return {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": c.batch,
+            "global_tokens": int(c.n_seqs * c.seq_len), "prompt_len": c.prompt_len, "vocab": c.vocab,
+            "D": c.depth_cap, "P": c.max_pattern, "alpha": c.alpha, "max_spec": c.max_spec, "tau": 0.0,
+            "l2": "GPU arm: flushed between steps (256 MiB write outside the timed events)",
+            "parallelism": f"replica x{args.gpus}, requests sharded" if args.gpus > 1 else "single GPU"}
 
 
 def parse():
@@ -49,7 +73,7 @@ def parse():
     ap.add_argument("--config", default="large_batch")
     ap.add_argument("--no-oracle", action="store_true", help="skip the CPU-oracle leg (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--oracle-samples", type=int, default=4)
+    ap.add_argument("--oracle-samples", type=int, default=25)
     ap.add_argument("--small", action="store_true", help="1/16 corpus, batch 32: quick functional run")
     ap.add_argument("--sweep", action="store_true",
                     help="scalability sweep over the size of the global tree (shape of the paper's appendix table)")
@@ -254,13 +278,6 @@ def run_ours(args):
                     buf[8 * (B + 1) + 4 * B:].view(torch.int32))
 
         s_off, s_slots, s_tok = views(d_in)
-        # the flush is not part of the path: time it alone and take it out
-        torch.cuda.synchronize()
-        t1 = time.perf_counter()
-        for _ in range(Ke):
-            flush.zero_()
-        torch.cuda.synchronize()
-        flush_s = time.perf_counter() - t1
 
         def run_e2e(mode, base):
             h_in, n_tok = [], []
@@ -301,11 +318,13 @@ def run_ours(args):
             moved[0] = moved[1] = 0
             if world > 1:
                 dist.barrier()
-            t0 = time.perf_counter()
+            secs = 0.0
             for k in range(We, E):
                 flush.zero_()
-                one(k)
-            secs = time.perf_counter() - t0 - flush_s
+                torch.cuda.synchronize()                         # the flush is over before the step's clock starts
+                t0 = time.perf_counter()
+                one(k)                                           # ends with a synchronize: the drafts are on the host
+                secs += time.perf_counter() - t0
             secs = sharding.max_over_ranks(secs, dev)
             return {"value": B * world * Ke / secs, "unit": UNIT, "h2d_bytes_per_step": moved[0] // Ke,
                     "d2h_bytes_per_step": moved[1] // Ke, "ms_per_step": secs / Ke * 1e3,
@@ -344,8 +363,9 @@ def run_ours(args):
         ref.global_build(w.corpus(), w.corpus_offsets())
         ref.slot_append_batch(list(range(B)), prompts, n_threads=thr)
         setup_s = time.perf_counter() - t0
-        o_times, desc, adds, ok = [], [], [], True
+        o_times, desc, adds, upd, ok = [], [], [], [], True
         for k in range(max(sample_steps) + 1):
+            u0 = sum(ref.slot_updates(i) for i in range(B)) if k in sample_steps else 0
             t0 = time.perf_counter()
             ref.slot_append_batch(list(range(B)), steps.lists[k], n_threads=thr)
             if k in sample_steps:
@@ -354,6 +374,7 @@ def run_ours(args):
                 o_times.append(time.perf_counter() - t0)
                 desc.append(int(r["visited"][:, 0].sum()))
                 adds.append(int(r["visited"][:, 1].sum()))
+                upd.append(sum(ref.slot_updates(i) for i in range(B)) - u0)
                 g = {n: t.cpu().numpy() for n, t in saved[k].items()}
                 for n in ("n_draft", "tokens", "parents", "positions", "chosen_tree", "chosen_p"):
                     ok = ok and np.array_equal(g[n], r[n])
@@ -364,14 +385,25 @@ def run_ours(args):
                         "sample": f"{len(sample_steps)} of the {K} timed steps (all {B} requests each), "
                                   f"{sum(o_times):.1f} s wall on {thr} threads; setup {setup_s:.0f} s untimed"}
         visits = statistics.mean(d + a for d, a in zip(desc, adds))
-        alg_bytes = statistics.mean(32 * d + 64 * a for d, a in zip(desc, adds)) + B * OUT_BYTES_PER_REQ
+        # necessary bytes of one launch: what the speculation must read and write (a 32-byte
+        # look per node on a match walk, 64 per node added to a draft tree, the outputs) plus
+        # what the append must (every node update reads and writes one 16-byte entry, every
+        # token is written to the text)
+        spec_bytes = statistics.mean(32 * d + 64 * a for d, a in zip(desc, adds)) + B * OUT_BYTES_PER_REQ
+        app_bytes = statistics.mean(upd) * APPEND_BYTES_PER_UPDATE + 4 * float(np.mean([t.size for t in steps.tokens[W:W + K]]))
+        alg_bytes = spec_bytes + app_bytes
         peak, which = measured_peak()
-        spec_s = statistics.mean(tot_ms) / 1e3               # the whole launch: append + speculate
-        achieved = alg_bytes / spec_s / 1e9
+        step_s = statistics.mean(tot_ms) / 1e3                # the whole launch: append + speculate
+        achieved = alg_bytes / step_s / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": SPECULATE_DRAM_TRAFFIC if c.name == "large_batch" and not args.small else None,
-                    "peak_source": which, "kernel": "speculate_fused_kernel<1, 10, 2, 4> (all of sd_step)",
-                    "algorithmic_bytes_per_launch": alg_bytes}
+                    "traffic": dram_traffic() if c.name == "large_batch" and not args.small else None,
+                    "peak_source": which, "kernel": STEP_KERNEL,
+                    "algorithmic_bytes_per_launch": alg_bytes,
+                    "append_bytes_per_launch": app_bytes, "speculate_bytes_per_launch": spec_bytes}
+        if spec_ms:
+            sp = spec_bytes / (statistics.mean(spec_ms) / 1e3) / 1e9
+            roofline["speculate_only"] = {"achieved": sp, "frac": sp / peak,
+                                          "note": "sd_speculate alone (two-call form), its own necessary bytes"}
         extra = {"parity_vs_oracle": "bit-exact" if ok else "MISMATCH", "parity_steps": len(sample_steps),
                  "nodes_visited_per_step": visits,
                  "nodes_visited_per_s": visits * world / (ms_per_step / 1e3)}
@@ -383,11 +415,7 @@ def run_ours(args):
             "metric": METRIC.format(B=B), "value": B * world / (ms_per_step / 1e3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32 trees, f64 scores", "data": "synthetic",
-            "config": {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": B,
-                       "global_tokens": int(c.n_seqs * c.seq_len), "prompt_len": c.prompt_len, "vocab": c.vocab,
-                       "D": c.depth_cap, "P": c.max_pattern, "alpha": c.alpha, "max_spec": c.max_spec,
-                       "l2": "flushed between steps (256 MiB write outside the timed events)",
-                       "parallelism": f"replica x{world}, requests sharded" if world > 1 else "single GPU"},
+            "config": config_dict(c, args),
             "step_us": {"mean": statistics.mean(tot_ms) * 1e3, "p50": statistics.median(tot_ms) * 1e3,
                         "max": max(tot_ms) * 1e3},
             "two_calls": {"steps": K2, "append_us": statistics.mean(app_ms) * 1e3 if app_ms else None,
@@ -666,9 +694,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC.format(B=B), "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
             "warmup": W, "ms_per_step": dt / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int32 trees, f64 scores", "data": "synthetic",
-            "config": {"workload": c.name + (" (small)" if args.small else ""), "batch_per_gpu": B,
-                       "global_tokens": int(c.n_seqs * c.seq_len), "prompt_len": c.prompt_len, "vocab": c.vocab,
-                       "D": c.depth_cap, "P": c.max_pattern, "alpha": c.alpha, "max_spec": c.max_spec},
+            "config": config_dict(c, args),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": thr, "kind": "oracle",
                              "sample": f"{len(sample)} of {B} requests per step, {K} steps"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -676,8 +702,21 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def spawn_ranks(args):
+    """`--gpus N` without a launcher around it: start the N ranks here (one process per GPU)."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 if __name__ == "__main__":
     a = parse()
+    if a.gpus > 1 and "WORLD_SIZE" not in os.environ and a.impl == "ours":
+        sys.exit(spawn_ranks(a))
     if a.impl == "reference":
         run_reference(a)
     elif a.sweep:

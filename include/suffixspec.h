@@ -259,6 +259,22 @@ int sd_query_counts(sd_store* store, int32_t n, const int32_t* d_tree, const int
                     const int32_t* d_paths, int32_t* d_counts, void* stream);
 
 /*
+ * sd_enumerate: every node of a tree as a record (parent record, token, COUNT, depth), for
+ * comparing a whole tree with an independent implementation (the trees of Section 3.1 are
+ * defined by exactly these: which token paths exist and how often each occurred).
+ *   tree: -1 global tree, else a slot.  d_parent, d_token, d_count, d_depth: DEVICE int32[max_nodes],
+ *   caller-owned.  Record i describes one node: d_parent[i] is the record of its parent (-1 for
+ *   a node of depth 1) and always precedes i; d_depth[i] is 1-based.  The order of the records
+ *   is otherwise unspecified and may change from call to call.  h_n: HOST, receives the number of
+ *   nodes of the tree.  If that exceeds max_nodes the call returns SD_ERR_CAPACITY, *h_n still
+ *   holds the number needed and the records are incomplete.
+ * An offline analysis call: allocates temporary device memory (16 bytes per record of room)
+ * and synchronises the stream once per level.
+ */
+int sd_enumerate(sd_store* store, int32_t tree, int64_t max_nodes, int32_t* d_parent, int32_t* d_token,
+                 int32_t* d_count, int32_t* d_depth, int64_t* h_n, void* stream);
+
+/*
  * sd_slot_info: per-slot context length, live node count and status.
  *   d_slot int32[n]; outputs int32[n] each, any may be NULL.
  */

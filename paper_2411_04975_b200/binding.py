@@ -19,7 +19,7 @@ FLAG_GLOBAL_ONLY, FLAG_REQUEST_ONLY, FLAG_LINEAR = 1, 2, 4
 STATUS_BAD_SLOT, STATUS_POOL_FULL, STATUS_GLOBAL_FULL, STATUS_BAD_TOKEN = 1, 2, 4, 8
 
 EXPORTS = ["sd_build", "sd_build_requests", "sd_append", "sd_speculate", "sd_step", "sd_speculate_noalloc", "sd_query_counts",
-           "sd_slot_info", "sd_entropy", "sd_stats", "sd_free", "sd_strerror", "sd_debug_fail_alloc"]
+           "sd_enumerate", "sd_slot_info", "sd_entropy", "sd_stats", "sd_free", "sd_strerror", "sd_debug_fail_alloc"]
 
 
 class SuffixSpecError(RuntimeError):
@@ -72,6 +72,8 @@ def library() -> C.CDLL:
         lib.sd_speculate_noalloc.argtypes = lib.sd_speculate.argtypes
         lib.sd_query_counts.restype = C.c_int
         lib.sd_query_counts.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
+        lib.sd_enumerate.restype = C.c_int
+        lib.sd_enumerate.argtypes = [vp, C.c_int32, C.c_int64, vp, vp, vp, vp, C.POINTER(C.c_int64), vp]
         lib.sd_slot_info.restype = C.c_int
         lib.sd_slot_info.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
         lib.sd_entropy.restype = C.c_int
@@ -318,6 +320,16 @@ class SuffixStore:
         if rc != 0:
             raise SuffixSpecError(rc, "sd_query_counts")
         return counts
+
+    def enumerate(self, tree: int, max_nodes: int) -> Dict[str, torch.Tensor]:
+        """All nodes of `tree` (-1: global) as records parent / token / count / depth (see sd_enumerate)."""
+        o = {k: torch.empty(max(max_nodes, 1), dtype=torch.int32, device=self.device) for k in ("parent", "token", "count", "depth")}
+        n = C.c_int64(0)
+        rc = library().sd_enumerate(self._h, tree, max_nodes, o["parent"].data_ptr(), o["token"].data_ptr(),
+                                    o["count"].data_ptr(), o["depth"].data_ptr(), C.byref(n), _stream())
+        if rc != 0:
+            raise SuffixSpecError(rc, "sd_enumerate")
+        return {k: v[:n.value] for k, v in o.items()}
 
     def slot_info(self, slots: torch.Tensor):
         n = int(slots.numel())

@@ -221,3 +221,88 @@ extern "C" int sd_entropy(sd_store* s, int32_t tree, double* h_entropy, void* st
     *h_entropy = h_w ? h_acc / (double)h_w : 0.0;
     return SD_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// sd_enumerate: every node of a tree, level by level (a node's record comes after its parent's).
+namespace {
+
+// depth 1: the nodes the root table points at
+__global__ void enumerate_root_kernel(const int4* ent, const int32_t* root, int V, long long max_nodes, int32_t* parent,
+                                      int32_t* token, int32_t* count, int32_t* depth, int* next_ent, int* next_rec,
+                                      int* n_next, unsigned long long* n_out) {
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= V || root[v] < 0) return;
+    const int4 e = ent[root[v]];
+    const unsigned long long o = atomicAdd(n_out, 1ull);
+    if ((long long)o < max_nodes) { parent[o] = -1; token[o] = e.x; count[o] = e.y; depth[o] = 1; }
+    if (((unsigned)e.w & RUN_COUNT_MASK) && (long long)o < max_nodes) {
+        const int q = atomicAdd(n_next, 1);
+        next_ent[q] = root[v]; next_rec[q] = (int)o;
+    }
+}
+
+// one thread per node of the current level: a record for each of its children
+__global__ void enumerate_level_kernel(const int4* ent, const int* cur_ent, const int* cur_rec, int n, int level,
+                                       long long max_nodes, int32_t* parent, int32_t* token, int32_t* count, int32_t* depth,
+                                       int* next_ent, int* next_rec, int* n_next, unsigned long long* n_out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int4 e = ent[cur_ent[i]];
+    const int cb = e.z, nc = (int)((unsigned)e.w & RUN_COUNT_MASK);
+    const unsigned long long o0 = atomicAdd(n_out, (unsigned long long)nc);
+    for (int k = 0; k < nc; ++k) {
+        const int4 c = ent[cb + k];
+        const long long o = (long long)o0 + k;
+        if (o >= max_nodes) break;
+        parent[o] = cur_rec[i]; token[o] = c.x; count[o] = c.y; depth[o] = level;
+        if ((unsigned)c.w & RUN_COUNT_MASK) {
+            const int q = atomicAdd(n_next, 1);
+            next_ent[q] = cb + k; next_rec[q] = (int)o;
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" int sd_enumerate(sd_store* s, int32_t tree, int64_t max_nodes, int32_t* d_parent, int32_t* d_token,
+                            int32_t* d_count, int32_t* d_depth, int64_t* h_n, void* stream) {
+    if (!s || !h_n || tree < -1 || tree >= s->R || max_nodes < 0 || max_nodes > 0x7fffffffll) return SD_ERR_INVALID_ARG;
+    if (max_nodes > 0 && (!d_parent || !d_token || !d_count || !d_depth)) return SD_ERR_INVALID_ARG;
+    SD_CHECK_DEVICE(s);
+    cudaStream_t st = (cudaStream_t)stream;
+    const int4* ent = tree < 0 ? s->g_ent : s->s_ent + (long long)tree * s->spn;
+    const int32_t* root = tree < 0 ? s->g_root : s->s_root + (long long)tree * s->V;
+    *h_n = 0;
+    const long long room = max_nodes > 0 ? max_nodes : 1;        // nodes with children among the records written
+    int *fe[2] = {nullptr, nullptr}, *fr[2] = {nullptr, nullptr};
+    unsigned char* small = nullptr;                              // n_out, frontier sizes
+    bool okm = cudaMalloc(&small, 64) == cudaSuccess;
+    for (int b = 0; b < 2 && okm; ++b)
+        okm = cudaMalloc(&fe[b], sizeof(int) * (size_t)room) == cudaSuccess && cudaMalloc(&fr[b], sizeof(int) * (size_t)room) == cudaSuccess;
+    auto release = [&]() { cudaFree(small); for (int b = 0; b < 2; ++b) { cudaFree(fe[b]); cudaFree(fr[b]); } };
+    if (!okm) { cudaGetLastError(); release(); return SD_ERR_NOMEM; }
+    unsigned long long* n_out = (unsigned long long*)small;
+    int* cnt = (int*)(small + 8);                                // cnt[0], cnt[1]: frontier sizes
+    cudaError_t ce = cudaMemsetAsync(small, 0, 64, st);
+    enumerate_root_kernel<<<(s->V + 255) / 256, 256, 0, st>>>(ent, root, s->V, max_nodes, d_parent, d_token, d_count, d_depth,
+                                                             fe[0], fr[0], cnt, n_out);
+    int n = 0, cur = 0;
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&n, cnt, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    for (int level = 2; ce == cudaSuccess && n > 0 && level <= SD_MAX_DEPTH; ++level) {
+        ce = cudaMemsetAsync(cnt + (cur ^ 1), 0, sizeof(int), st);
+        enumerate_level_kernel<<<(n + 255) / 256, 256, 0, st>>>(ent, fe[cur], fr[cur], n, level, max_nodes, d_parent, d_token,
+                                                               d_count, d_depth, fe[cur ^ 1], fr[cur ^ 1], cnt + (cur ^ 1), n_out);
+        if (ce == cudaSuccess) ce = cudaMemcpyAsync(&n, cnt + (cur ^ 1), sizeof(int), cudaMemcpyDeviceToHost, st);
+        if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+        cur ^= 1;
+    }
+    unsigned long long total = 0;
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&total, n_out, sizeof(total), cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    if (ce == cudaSuccess) ce = cudaGetLastError();
+    release();
+    if (ce != cudaSuccess) return SD_ERR_CUDA;
+    *h_n = (int64_t)total;
+    return (long long)total > max_nodes ? SD_ERR_CAPACITY : SD_OK;
+}

@@ -288,7 +288,7 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 //      SCORE (every D <= 1 and D never grows along a path) falls below a score already
 //      reached by another job of the request.
 //   3. select + emit from shared memory; no global scratch.
-constexpr int CTA_WARPS = 16;                  // the usual block
+constexpr int CTA_WARPS = 10;                  // the usual block (96 registers; 16 warps x 64 registers spill: 87 us against 83.5)
 constexpr int CTA_WARPS_STEP = 10;             // the usual block of sd_step: 10 warps with 96 registers each and
 constexpr int STEP_G = 4;                      // an append that moves four entries per round, so that the
                                                // append in front does not spill.  Measured per step: 92.7 us;

@@ -22,6 +22,31 @@ def ragged(seqs):
     return off, flat.astype(np.int32)
 
 
+def path_hashes(parent, token, depth):
+    """A 64-bit hash of every node's root-to-node token path, from records in which a parent
+    precedes its children (level by level: vectorised)."""
+    n = len(token)
+    h = np.zeros(n, dtype=np.uint64)
+    K1, K2 = np.uint64(0x9E3779B97F4A7C15), np.uint64(0xC2B2AE3D27D4EB4F)
+    with np.errstate(over="ignore"):
+        for d in range(1, int(depth.max(initial=0)) + 1):
+            idx = np.nonzero(depth == d)[0]
+            hp = np.where(parent[idx] >= 0, h[np.maximum(parent[idx], 0)], np.uint64(0x1234567))
+            x = (hp ^ (token[idx].astype(np.uint64) + np.uint64(1))) * K1
+            x ^= x >> np.uint64(29)
+            x *= K2
+            x ^= x >> np.uint64(32)
+            h[idx] = x
+    return h
+
+
+def canonical_nodes(parent, token, count, depth):
+    """The tree as a sorted table (path hash, depth, count): equal tables = equal trees."""
+    h = path_hashes(np.asarray(parent), np.asarray(token), np.asarray(depth))
+    t = np.stack([h, np.asarray(depth).astype(np.uint64), np.asarray(count).astype(np.uint64)], axis=1)
+    return t[np.lexsort((t[:, 2], t[:, 1], t[:, 0]))]
+
+
 class Pair:
     """An oracle and a GPU store holding the same trees."""
 
@@ -59,8 +84,8 @@ class Pair:
         self.o.slot_append_batch([slots[i] for i in idx], [token_lists[i] for i in idx], n_threads=oracle_threads)
 
     def check_tree(self, tree):
-        """Every path of the oracle's tree has the same COUNT on the GPU, and the GPU
-        tree has no other node (equal live-node totals)."""
+        """The GPU tree, enumerated on the device, has exactly the oracle's nodes with the oracle's
+        counts; and every path of the oracle's tree, looked up on the GPU, has the same COUNT."""
         depth, parent, tok, cnt = self.o.dump(tree)
         n = len(tok)
         if tree < 0:
@@ -69,6 +94,13 @@ class Pair:
             info = self.g.slot_info(dev_i32([tree]))
             assert int(info["nodes"][0]) == n
             assert int(info["len"][0]) == self.o.slot_len(tree)
+        # the GPU tree enumerated on the device, node by node: the same set of (path, depth, count)
+        rec = {k: v.cpu().numpy() for k, v in self.g.enumerate(tree, n + 8).items()}
+        assert len(rec["token"]) == n
+        if n:
+            assert (rec["parent"] < np.arange(n)).all()
+            assert np.array_equal(canonical_nodes(rec["parent"], rec["token"], rec["count"], rec["depth"]),
+                                  canonical_nodes(parent, tok, cnt, depth)), f"tree {tree}: node sets differ"
         if n == 0:
             return
         off = np.zeros(n + 1, dtype=np.int64)
@@ -87,18 +119,18 @@ class Pair:
         assert bad.size == 0, f"tree {tree}: {bad.size} of {n} counts differ, first path " \
                               f"{flat[off[bad[0]]:off[bad[0] + 1]].tolist()} gpu {got[bad[0]]} oracle {cnt[bad[0]]}"
 
-    def speculate_both(self, slots, P, alpha, max_spec, flags=0, budget_cap=None, oracle_threads=4):
+    def speculate_both(self, slots, P, alpha, max_spec, flags=0, budget_cap=None, oracle_threads=4, tau=0.0):
         bc = None if budget_cap is None else dev_i32(budget_cap)
-        out = self.g.speculate(dev_i32(slots), P, alpha, max_spec, flags, bc)
+        out = self.g.speculate(dev_i32(slots), P, alpha, max_spec, flags, bc, tau=tau)
         torch.cuda.synchronize()
         got = {k: v.cpu().numpy() for k, v in out.items()}
         got["mask"] = got["mask"].view(np.uint32)
         want = self.o.speculate(slots, P, alpha, max_spec, M=self.M, flags=flags, budget_override=budget_cap,
-                                n_threads=oracle_threads)
+                                n_threads=oracle_threads, tau=tau)
         return got, want
 
-    def check_speculate(self, slots, P, alpha, max_spec, flags=0, budget_cap=None):
-        got, want = self.speculate_both(slots, P, alpha, max_spec, flags, budget_cap)
+    def check_speculate(self, slots, P, alpha, max_spec, flags=0, budget_cap=None, tau=0.0):
+        got, want = self.speculate_both(slots, P, alpha, max_spec, flags, budget_cap, tau=tau)
         assert_same_drafts(got, want)
         return got, want
 

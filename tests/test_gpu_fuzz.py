@@ -1,6 +1,6 @@
 """Randomised differential test: small stores with random shapes, vocabularies, depth caps and
 call sequences (batched prompt build or appends, one-launch steps or append + speculate, global
-inserts in between, flags and budget caps), every draft compared bit by bit with the oracle and
+inserts in between, flags, budget caps and score thresholds), every draft compared bit by bit with the oracle and
 the trees compared node by node at the end."""
 import numpy as np
 import pytest
@@ -59,21 +59,22 @@ def _scenario(U, seed):
         flags = int(rng.choice([0, 0, 0, 1, 2, 4, 5, 6]))
         sub = slots if rng.random() < 0.7 else sorted(rng.choice(n_slots, size=max(1, n_slots // 2), replace=False).tolist())
         cap = rng.integers(-1, 40, size=len(sub)).astype(np.int32) if rng.random() < 0.3 else None
+        tau = float(rng.choice([0.0, 0.0, 0.25, 1.0, 1.5, 3.0, 8.0]))   # score threshold of Section 3.2
         lists = _seqs(rng, len(sub), 0, int(rng.choice([1, 4, 12])), vocab, zipf)
         lists = [l[:max(0, maxtok + 60 - pr.o.slot_len(s))] for l, s in zip(lists, sub)]   # stay inside the text buffer
         if rng.random() < 0.5:
             off, flat = U.ragged(lists)
             out = pr.g.step(U.dev_i32(sub), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat) if flat.size else _empty(),
-                            P, alpha, max_spec, flags, None if cap is None else U.dev_i32(cap))
+                            P, alpha, max_spec, flags, None if cap is None else U.dev_i32(cap), tau=tau)
             torch.cuda.synchronize()
             pr.o.slot_append_batch(sub, lists, n_threads=4)
-            want = pr.o.speculate(sub, P, alpha, max_spec, M=64, flags=flags, budget_override=cap, n_threads=4)
+            want = pr.o.speculate(sub, P, alpha, max_spec, M=64, flags=flags, budget_override=cap, n_threads=4, tau=tau)
             got = {k: v.cpu().numpy() for k, v in out.items()}
             got["mask"] = got["mask"].view(np.uint32)
             U.assert_same_drafts(got, want)
         else:
             pr.append(sub, lists)
-            pr.check_speculate(sub, P, alpha, max_spec, flags, cap)
+            pr.check_speculate(sub, P, alpha, max_spec, flags, cap, tau=tau)
         if rng.random() < 0.4:
             finished = _seqs(rng, int(rng.integers(1, 4)), 1, 120, vocab, zipf)
             pr.append([-1] * len(finished), finished)

@@ -654,3 +654,127 @@ def test_step_reports_a_stopped_append(U):
     assert int(out["n_draft"][2]) == int(want["n_draft"][0])
     assert out["tokens"][2].cpu().numpy().tolist() == want["tokens"][0].tolist()
     pr.close()
+
+
+# ---------------------------------------------------------------- score threshold, duplicate slots, allocation failures
+def test_score_threshold_is_strict_on_the_gpu(U):
+    """Section 3.2: the chosen tree is used only if SCORE > tau.  Thresholds just below, at and just
+    above a score that really occurs: sd_speculate, sd_step and sd_speculate_noalloc against the oracle."""
+    import paper_2411_04975_b200 as sfx
+    rng = np.random.default_rng(41)
+    n = 24
+    pr = U.Pair(_rand_seqs(rng, 12, 80, 300, 6), vocab=6, D=16, n_slots=n, max_req_tokens=200)
+    pr.append(list(range(n)), _rand_seqs(rng, n, 20, 120, 6), reset=[1] * n)
+    slots = list(range(n))
+    got0, _ = pr.check_speculate(slots, 16, 2.0, 48)
+    pos = np.sort(got0["score"][got0["score"] > 0])
+    assert pos.size >= 8
+    s = float(pos[pos.size // 2])
+    empty = torch.zeros(0, dtype=torch.int32, device=U.DEV)
+    no_new = torch.zeros(n + 1, dtype=torch.int64, device=U.DEV)
+    for tau in (float(np.nextafter(s, 0.0)), s, float(np.nextafter(s, np.inf)), 1e9):
+        got, want = pr.check_speculate(slots, 16, 2.0, 48, tau=tau)
+        keep = got0["score"] > tau                               # strictly above: kept unchanged
+        assert np.array_equal(got["n_draft"][keep], got0["n_draft"][keep])
+        assert (got["n_draft"][~keep] == 0).all() and (got["chosen_tree"][~keep] == -1).all()
+        assert (got["score"][~keep] == 0).all() and (got["tokens"][~keep] == -1).all()
+        out = pr.g.step(U.dev_i32(slots), no_new, empty, 16, 2.0, 48, tau=tau)
+        alt = pr.g.alloc_outputs(n)
+        sfx.sd_speculate_noalloc(pr.g.handle, U.dev_i32(slots), 16, 2.0, 48, 0, None, alt, tau)
+        torch.cuda.synchronize()
+        for o in (out, alt):
+            g = {k: v.cpu().numpy() for k, v in o.items()}
+            g["mask"] = g["mask"].view(np.uint32)
+            U.assert_same_drafts(g, want)
+    assert (got0["score"] > float(np.nextafter(s, 0.0))).sum() == (got0["score"] > s).sum() + (got0["score"] == s).sum()
+    for bad in (-1.0, float("nan")):
+        with pytest.raises(sfx.SuffixSpecError):
+            pr.g.speculate(U.dev_i32(slots), 16, 2.0, 48, tau=bad)
+    pr.close()
+
+
+def test_a_slot_that_appears_twice_is_refused(U):
+    """Two blocks on one tree would race: every later appearance of a slot gets the bad-slot status
+    and no draft, in sd_speculate and in sd_step (whose extra tokens are not appended either)."""
+    rng = np.random.default_rng(43)
+    pr = U.Pair(_rand_seqs(rng, 8, 50, 200, 5), vocab=5, D=12, n_slots=8, max_req_tokens=300)
+    pr.append(list(range(6)), _rand_seqs(rng, 6, 30, 100, 5), reset=[1] * 6)
+    call = [0, 1, 0, 2, 1, 0, 5]
+    first = [0, 1, 3, 6]                                         # rows that are first appearances
+    out = pr.g.speculate(U.dev_i32(call), 12, 2.0, 40)
+    torch.cuda.synchronize()
+    got = {k: v.cpu().numpy() for k, v in out.items()}
+    got["mask"] = got["mask"].view(np.uint32)
+    assert got["status"].tolist() == [0, 0, 1, 0, 1, 1, 0]
+    assert (got["n_draft"][[2, 4, 5]] == 0).all() and (got["chosen_tree"][[2, 4, 5]] == -1).all()
+    want = pr.o.speculate([call[i] for i in first], 12, 2.0, 40, M=64)
+    U.assert_same_drafts({k: v[first] for k, v in got.items()}, want)
+    # one-launch step: only the first appearance appends
+    lists = _rand_seqs(rng, len(call), 1, 6, 5)
+    off, flat = U.ragged(lists)
+    out = pr.g.step(U.dev_i32(call), torch.as_tensor(off, device=U.DEV), U.dev_i32(flat), 12, 2.0, 40)
+    torch.cuda.synchronize()
+    got = {k: v.cpu().numpy() for k, v in out.items()}
+    got["mask"] = got["mask"].view(np.uint32)
+    assert got["status"].tolist() == [0, 0, 1, 0, 1, 1, 0]
+    pr.o.slot_append_batch([call[i] for i in first], [lists[i] for i in first])
+    want = pr.o.speculate([call[i] for i in first], 12, 2.0, 40, M=64)
+    U.assert_same_drafts({k: v[first] for k, v in got.items()}, want)
+    for s in range(6):
+        pr.check_tree(s)
+    pr.close()
+
+
+def test_device_allocation_failures_are_error_codes(U):
+    """Every device allocation of sd_build and sd_build_requests fails once (test hook of the
+    library): the call returns the out-of-memory code, nothing leaks, and the next call works."""
+    import paper_2411_04975_b200 as sfx
+    rng = np.random.default_rng(47)
+    corpus = _rand_seqs(rng, 6, 40, 120, 7)
+    off, flat = U.ragged(corpus)
+    lib = sfx.library()
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+
+    def build():
+        return sfx.SuffixStore(U.dev_i32(flat), torch.as_tensor(off, device=U.DEV), vocab=7, depth_cap=8,
+                               max_requests=4, max_req_tokens=128, max_spec_cap=32)
+    failed = 0
+    try:
+        for k in range(1, 80):
+            lib.sd_debug_fail_alloc(k)
+            try:
+                store = build()
+            except sfx.SuffixSpecError as e:
+                assert e.code == -3, e
+                failed += 1
+                continue
+            store.free()                                         # the k-th allocation was optional, or there is none
+        assert failed >= 5
+        lib.sd_debug_fail_alloc(0)
+        torch.cuda.synchronize()
+        assert abs(torch.cuda.mem_get_info()[0] - free0) <= (8 << 20)       # nothing left behind
+        # prompts through sd_build_requests with failing workspace allocations, then for real
+        pr = U.Pair(corpus, vocab=7, D=8, n_slots=4, max_req_tokens=128, M=32)
+        prompts = _rand_seqs(rng, 4, 10, 90, 7)
+        poff, pflat = U.ragged(prompts)
+        refused = 0
+        for k in range(1, 40):
+            lib.sd_debug_fail_alloc(k)
+            try:
+                pr.g.build_requests(np.arange(4, dtype=np.int32), poff, U.dev_i32(pflat))
+            except sfx.SuffixSpecError as e:
+                assert e.code == -3, e
+                refused += 1
+        lib.sd_debug_fail_alloc(0)
+        assert refused >= 1
+        pr.g.build_requests(np.arange(4, dtype=np.int32), poff, U.dev_i32(pflat))
+        for s in range(4):
+            pr.o.slot_reset(s)
+        pr.o.slot_append_batch(list(range(4)), prompts)
+        for s in range(4):
+            pr.check_tree(s)
+        pr.check_speculate([0, 1, 2, 3], 8, 2.0, 32)
+        pr.close()
+    finally:
+        lib.sd_debug_fail_alloc(0)

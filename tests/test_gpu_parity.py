@@ -376,20 +376,22 @@ def test_closed_loop_scaled(U):
     pr.close()
 
 
-@pytest.mark.parametrize("one_launch", [False, True])
-def test_large_batch_full_size_sampled_against_oracle(U, one_launch):
-    """The headline workload (large_batch) at full size (4,194,304-token global tree, 256 requests x 4,096-token
-    prompts) in the launch configurations bench.py times: sd_append + sd_speculate, and (one_launch)
-    prompts through sd_build_requests and every decode step as one sd_step.  The oracle holds the
-    full global tree but only a sample of the requests; their rows must be bit-exact, and every
-    row must satisfy the properties that hold for any draft."""
+@pytest.mark.parametrize("name,one_launch", [("large_batch", False), ("large_batch", True), ("agentic", True),
+                                             ("low_repetition", True)])
+def test_full_size_sampled_against_oracle(U, name, one_launch):
+    """The named workloads at full size (large_batch: 4,194,304-token global tree, 256 requests x 4,096-token
+    prompts; agentic: 64 requests x 8,192 tokens, P = 24; low_repetition: 512 requests) in the launch
+    configurations bench.py times: sd_append + sd_speculate, and (one_launch) prompts through
+    sd_build_requests and every decode step as one sd_step.  The oracle holds the full global tree
+    but only a sample of the requests; their rows must be bit-exact, and every row must satisfy the
+    properties that hold for any draft."""
     from workload.generator import accept_schedule, get_workload
     import oracle as oracle_pkg
     import paper_2411_04975_b200 as sfx
-    w = get_workload("large_batch")
+    w = get_workload(name)
     c = w.cfg
     B = c.batch
-    sample = [0, 1, 37, 100, 101, 180, 254, 255]
+    sample = sorted({0, 1, 37 % B, B // 2 - 1, B // 2, (5 * B) // 7, B - 2, B - 1})
     dev = U.DEV
     store = sfx.SuffixStore(torch.as_tensor(w.corpus(), device=dev), torch.as_tensor(w.corpus_offsets(), device=dev),
                             vocab=c.vocab, depth_cap=c.depth_cap, max_requests=B, max_req_tokens=c.prompt_len + 64,
@@ -409,6 +411,7 @@ def test_large_batch_full_size_sampled_against_oracle(U, one_launch):
     cont = [w.continuation(i, prompts[i], length=int(sched[:, i].sum()) + 1) for i in range(B)]
     cur = np.zeros(B, dtype=np.int64)
     pending = None                                             # (offsets, tokens) accepted in the last step
+    drafted = 0
     for step in range(3):
         if one_launch and pending is not None:
             out = store.step(slots, torch.as_tensor(pending[0], device=dev), U.dev_i32(pending[1]), c.max_pattern,
@@ -420,24 +423,8 @@ def test_large_batch_full_size_sampled_against_oracle(U, one_launch):
         got["mask"] = got["mask"].view(np.uint32)
         want = ref.speculate(list(range(len(sample))), c.max_pattern, c.alpha, c.max_spec, n_threads=8)
         U.assert_same_drafts({k: v[sample] for k, v in got.items()}, want)
-        # properties of every row
-        n = got["n_draft"]
-        assert (got["status"] == 0).all() and (n >= 0).all() and (n <= c.max_spec).all()
-        assert ((got["score"] > 0) == (n > 0)).all() and (got["score"] <= n).all()
-        for i in range(B):
-            k = int(n[i])
-            par = got["parents"][i, :k]
-            assert (par < np.arange(k)).all() and (par >= -1).all()
-            depth = np.zeros(k, dtype=np.int64)
-            for j in range(k):
-                depth[j] = 1 if par[j] < 0 else depth[par[j]] + 1
-                row = int(got["mask"][i, j, 0]) | (int(got["mask"][i, j, 1]) << 32)
-                prow = 0 if par[j] < 0 else int(got["mask"][i, par[j], 0]) | (int(got["mask"][i, par[j], 1]) << 32)
-                assert row == prow | (1 << j)
-            t = c.prompt_len + int(cur[i])
-            assert (got["positions"][i, :k] == t + depth - 1).all()
-            assert (got["tokens"][i, k:] == -1).all() and (got["mask"][i, k:] == 0).all()
-            assert k <= max(1, int(c.alpha * got["chosen_p"][i])) and depth.max(initial=0) <= c.depth_cap - got["chosen_p"][i]
+        _check_draft_properties(got, c, c.prompt_len + cur)
+        drafted += int(got["n_draft"].sum())
         # next decode step
         a = sched[step]
         lists = [cont[i][cur[i]:cur[i] + a[i]] for i in range(B)]
@@ -448,21 +435,111 @@ def test_large_batch_full_size_sampled_against_oracle(U, one_launch):
         else:
             store.append(slots, torch.as_tensor(o2, device=dev), U.dev_i32(f2))
         ref.slot_append_batch(list(range(len(sample))), [lists[i] for i in sample], n_threads=8)
-    # the sampled per-request trees, node by node
+    assert drafted > 0
+    # the sampled per-request trees, node by node (enumerated on the device)
     for k, i in enumerate(sample[:3]):
-        depth, parent, tok, cnt = ref.dump(k)
-        nn = len(tok)
-        offp = np.zeros(nn + 1, dtype=np.int64); offp[1:] = np.cumsum(depth)
-        flatp = np.empty(int(offp[-1]), dtype=np.int32)
-        for q in range(nn):
-            b = offp[q]
-            if parent[q] >= 0:
-                pb = offp[parent[q]]
-                flatp[b:b + depth[q] - 1] = flatp[pb:pb + depth[q] - 1]
-            flatp[b + depth[q] - 1] = tok[q]
-        gotc = store.query_counts(U.dev_i32(np.full(nn, i)), torch.as_tensor(offp, device=dev), U.dev_i32(flatp))
-        assert np.array_equal(gotc.cpu().numpy(), cnt)
-        assert int(store.slot_info(U.dev_i32([i]))["nodes"][0]) == nn
+        _same_tree(U, store, i, ref, k)
+    store.free()
+    ref.close()
+
+
+def _check_draft_properties(got, c, t_of):
+    """What holds for every row of any batch: parents precede children, the mask of a node is its
+    parent's plus its own bit, positions follow from the depth, padding is -1 / 0, the budget
+    and the depth cap are respected."""
+    n = got["n_draft"]
+    B = len(n)
+    assert (got["status"] == 0).all() and (n >= 0).all() and (n <= c.max_spec).all()
+    assert ((got["score"] > 0) == (n > 0)).all() and (got["score"] <= n).all()
+    for i in range(B):
+        k = int(n[i])
+        par = got["parents"][i, :k]
+        assert (par < np.arange(k)).all() and (par >= -1).all()
+        depth = np.zeros(k, dtype=np.int64)
+        for j in range(k):
+            depth[j] = 1 if par[j] < 0 else depth[par[j]] + 1
+            row = int(got["mask"][i, j, 0]) | (int(got["mask"][i, j, 1]) << 32)
+            prow = 0 if par[j] < 0 else int(got["mask"][i, par[j], 0]) | (int(got["mask"][i, par[j], 1]) << 32)
+            assert row == prow | (1 << j)
+        assert (got["positions"][i, :k] == int(t_of[i]) + depth - 1).all()
+        assert (got["tokens"][i, k:] == -1).all() and (got["mask"][i, k:] == 0).all()
+        assert k <= max(1, int(c.alpha * got["chosen_p"][i])) and depth.max(initial=0) <= c.depth_cap - got["chosen_p"][i]
+
+
+def _same_tree(U, store, tree, ref, ref_tree):
+    """Tree `tree` of the store, enumerated on the device, against tree `ref_tree` of the oracle."""
+    depth, parent, tok, cnt = ref.dump(ref_tree)
+    nn = len(tok)
+    rec = {k: v.cpu().numpy() for k, v in store.enumerate(tree, nn + 8).items()}
+    assert len(rec["token"]) == nn
+    assert np.array_equal(U.canonical_nodes(rec["parent"], rec["token"], rec["count"], rec["depth"]),
+                          U.canonical_nodes(parent, tok, cnt, depth))
+    if tree >= 0:
+        assert int(store.slot_info(U.dev_i32([tree]))["nodes"][0]) == nn
+
+
+def test_closed_loop_full_size_sampled_against_oracle(U):
+    """The closed-loop workload at full size (256 slots, 4,096-token prompts, 4 M-token global tree), 30 steps:
+    speculate, simulated verification, append; finished outputs go into the global tree and
+    their slots are refilled through sd_build_requests.  Outputs are kept short so that requests
+    do finish within the 30 steps.  The oracle follows the global tree and a sample of the slots."""
+    from workload.generator import get_workload
+    from workload.closed_loop import ClosedLoop
+    import oracle as oracle_pkg
+    import paper_2411_04975_b200 as sfx
+    w = get_workload("closed_loop")
+    c = w.cfg
+    B = c.batch
+    dev = U.DEV
+    sample = [0, 1, 50, 128, 200, 255]
+    pos = {s: k for k, s in enumerate(sample)}
+    store = sfx.SuffixStore(torch.as_tensor(w.corpus(), device=dev), torch.as_tensor(w.corpus_offsets(), device=dev),
+                            vocab=c.vocab, depth_cap=c.depth_cap, max_requests=B, max_req_tokens=c.prompt_len + 128,
+                            max_spec_cap=c.max_spec)
+    ref = oracle_pkg.SuffixOracle(c.depth_cap, len(sample))
+    ref.global_build(w.corpus(), w.corpus_offsets())
+    loop = ClosedLoop(w, B, out_lo=12, out_hi=100)
+
+    def apply(items):
+        sl, lists, reset = items
+        new = [i for i in range(len(sl)) if sl[i] >= 0 and reset[i]]
+        keep = [i for i in range(len(sl)) if not (sl[i] >= 0 and reset[i])]
+        if keep:
+            o, f = U.ragged([lists[i] for i in keep])
+            store.append(U.dev_i32([sl[i] for i in keep]), torch.as_tensor(o, device=dev),
+                         U.dev_i32(f) if f.size else torch.zeros(0, dtype=torch.int32, device=dev))
+        if new:
+            o, f = U.ragged([lists[i] for i in new])
+            store.build_requests(np.asarray([sl[i] for i in new], dtype=np.int32), o, U.dev_i32(f))
+        for i in range(len(sl)):
+            if sl[i] < 0:
+                ref.global_insert(lists[i])
+            elif sl[i] in pos:
+                if reset[i]:
+                    ref.slot_reset(pos[sl[i]])
+                ref.slot_append_batch([pos[sl[i]]], [lists[i]])
+
+    apply(loop.start())
+    slots = torch.arange(B, dtype=torch.int32, device=dev)
+    for step in range(30):
+        out = store.speculate(slots, c.max_pattern, c.alpha, c.max_spec)
+        torch.cuda.synchronize()
+        got = {k: v.cpu().numpy() for k, v in out.items()}
+        got["mask"] = got["mask"].view(np.uint32)
+        want = ref.speculate(list(range(len(sample))), c.max_pattern, c.alpha, c.max_spec, n_threads=6)
+        try:
+            U.assert_same_drafts({k: v[sample] for k, v in got.items()}, want)
+        except AssertionError as e:
+            raise AssertionError(f"step {step}: {e}") from e
+        t_of = store.slot_info(slots)["len"].cpu().numpy()
+        _check_draft_properties(got, c, t_of)
+        apply(loop.advance(got))
+    s = loop.summary()
+    assert s["finished_requests"] >= 20, s
+    st = store.stats()
+    assert st["global_nodes"] == ref.node_count(-1) and st["global_status"] == 0
+    for k in (0, 3):
+        _same_tree(U, store, sample[k], ref, k)
     store.free()
     ref.close()
 

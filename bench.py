@@ -77,6 +77,8 @@ def parse():
     ap.add_argument("--small", action="store_true", help="1/16 corpus, batch 32: quick functional run")
     ap.add_argument("--sweep", action="store_true",
                     help="scalability sweep over the size of the global tree (shape of the paper's appendix table)")
+    ap.add_argument("--sweep-oracle", action="store_true",
+                    help="with --sweep: time the CPU oracle beside every row (one thread, a sample of the requests)")
     ap.add_argument("--closed-loop-oracle", action="store_true",
                     help="closed_loop config: run the CPU oracle in lock-step and compare every step (slow)")
     return ap.parse_args()
@@ -446,7 +448,7 @@ def run_sweep(args):
     dev = torch.device("cuda", 0)
     K, W = min(args.steps, 30), 3
     rows = []
-    for n_seqs in (512, 1024, 2048, 4096, 8192, 16384):
+    for n_seqs in (512, 1024, 2048, 4096, 8192, 16384, 26368):     # the last row: 27.0 M tokens, the paper's first row
         w = get_workload("large_batch", n_seqs=n_seqs)
         c = w.cfg
         B = c.batch
@@ -487,7 +489,8 @@ def run_sweep(args):
                 spec.append(e0.elapsed_time(e1)); app.append(e1.elapsed_time(e2))
                 drafts += int(out["n_draft"].sum().item()); toks += int(d_tok[k].numel())
         n_tok = n_seqs * c.seq_len
-        rows.append({"entries": n_seqs, "tokens": n_tok, "global_nodes": st["global_nodes"],
+        oracle_col = oracle_sweep_row(w, prompts, steps) if args.sweep_oracle else None
+        rows.append({"oracle": oracle_col, "entries": n_seqs, "tokens": n_tok, "global_nodes": st["global_nodes"],
                      "global_tree_MB": st["global_pool_used"] * 16 / 1e6, "bytes_per_token": st["global_pool_used"] * 16 / n_tok,
                      "offline_build_ms": build_ms, "offline_update_us_per_token": build_ms * 1e3 / n_tok,
                      "online_update_us_per_token": sum(app) * 1e3 / toks,
@@ -497,6 +500,38 @@ def run_sweep(args):
         del corpus, offsets, flush
         torch.cuda.empty_cache()
     print(json.dumps({"metric": "scalability sweep (batch 256, 4,096-token prompts, one B200)", "rows": rows}), flush=True)
+
+
+def oracle_sweep_row(w, prompts, steps, n_req=16, n_steps=3):
+    """The CPU oracle on the same corpus, one thread (the paper's table is per-token CPU time):
+    update time per token of the global build, look-up time per speculated token and online
+    update time per token over `n_req` requests and `n_steps` decode steps."""
+    import oracle
+    import psutil
+    c = w.cfg
+    n_tok = c.n_seqs * c.seq_len
+    need = 160 * 10 * n_tok                                       # about 10 nodes per token, 160 B per pointer-trie node
+    if psutil.virtual_memory().available < 1.5 * need:
+        return {"skipped": f"host memory: about {need / 1e9:.0f} GB needed for the pointer trie"}
+    ref = oracle.SuffixOracle(c.depth_cap, n_req)
+    t0 = time.perf_counter()
+    ref.global_build(w.corpus(), w.corpus_offsets())
+    build_s = time.perf_counter() - t0
+    ref.slot_append_batch(list(range(n_req)), prompts[:n_req], n_threads=1)
+    spec_s, app_s, drafts, toks = 0.0, 0.0, 0, 0
+    for k in range(n_steps):
+        t0 = time.perf_counter()
+        r = ref.speculate(list(range(n_req)), c.max_pattern, c.alpha, c.max_spec, n_threads=1)
+        t1 = time.perf_counter()
+        ref.slot_append_batch(list(range(n_req)), steps.lists[k][:n_req], n_threads=1)
+        t2 = time.perf_counter()
+        spec_s += t1 - t0; app_s += t2 - t1
+        drafts += int(r["n_draft"].sum()); toks += sum(len(x) for x in steps.lists[k][:n_req])
+    ref.close()
+    return {"threads": 1, "offline_update_us_per_token": build_s * 1e6 / n_tok,
+            "online_update_us_per_token": app_s * 1e6 / max(toks, 1),
+            "lookup_us_per_speculated_token": spec_s * 1e6 / max(drafts, 1),
+            "sample": f"{n_req} requests x {n_steps} steps"}
 
 
 # --------------------------------------------------------------------------------------------

@@ -275,19 +275,10 @@ __global__ void select_emit_kernel(sd_store sv, int n, const int32_t* __restrict
 
 
 // ---------------------------------------------------------------------------------------------
-// Fused path: one block of W warps per request.  Two blocks per SM is the usual shape: W = 16
-// with 64 registers per thread for sd_speculate, W = 10 with 96 for sd_step, whose append is
-// register hungry.  A batch of at most one request per SM gets bigger blocks (W = 24 / 16), a
-// batch of more than two requests per SM smaller ones (W = 8 / 5, four per SM) to stay in one wave.
-//   1. match: the per-request match nodes are the slot's active nodes; the global match
-//      nodes are advanced from the nodes cached at the previous call by descending only the
-//      tokens appended since (full walks when the cache is stale).  Warp w serves pattern
-//      lengths w + 1, w + 1 + W, ...
-//   2. expand: the (tree, p) jobs that matched go into a queue, costliest first; warps pull
-//      jobs until it is empty.  A job is dropped, exactly, as soon as an upper bound of its
-//      SCORE (every D <= 1 and D never grows along a path) falls below a score already
-//      reached by another job of the request.
-//   3. select + emit from shared memory; no global scratch.
+// Fused path: one block of W warps per request (the kernel itself is described where it is
+// defined).  Two blocks per SM is the usual shape: W = 10 with 96 registers per thread.  A batch
+// of at most one request per SM gets bigger blocks (W = 24 / 16), a batch of more than two
+// requests per SM smaller ones (W = 8 / 5, four per SM) to stay in one wave.
 constexpr int CTA_WARPS = 10;                  // the usual block (96 registers; 16 warps x 64 registers spill: 87 us against 83.5)
 constexpr int CTA_WARPS_STEP = 10;             // the usual block of sd_step: 10 warps with 96 registers each and
 constexpr int STEP_G = 4;                      // an append that moves four entries per round, so that the
@@ -766,16 +757,10 @@ __device__ void expand_job(BlockShared& sh, WarpWork& W, const int4* __restrict_
                 push_children_w(ent, cur_cb, cur_n, load_window(ent, cur_cb, limit, lane), cur_d, cur_idx, W.F, fh, fs, K,
                                 lane);
             } else {
-                // With a full frontier a child only matters if it beats the worst entry.  Counts are
-                // at least 1, so the sibling sum is at least cur_n and D <= cur_d * count / cur_n:
-                // children below the count that needs are skipped without any arithmetic.
-                int cmin = 1;
-                if (fs == K) {
-                    const double need = W.F.d[(fh + fs - 1) & (SD_MAX_SPEC - 1)] / cur_d * (double)cur_n * 0.999999;
-                    cmin = need >= 2.0e9 ? 2000000000 : max(1, (int)need);
-                }
+                // some candidates wait and there is room for more: the K best children by count go
+                // into a list of their own, which is then merged in
                 int ts;
-                scan_run_by_count(ent, cur_cb, cur_n, 0, 1, cur_idx, cmin, W, W.T, 0, ts, K, sum, lane);
+                scan_run_by_count(ent, cur_cb, cur_n, 0, 1, cur_idx, 1, W, W.T, 0, ts, K, sum, lane);
                 counts_to_d(W.T, 0, ts, cur_d, sum, lane);
                 frontier_merge_list(W.F, fh, fs, K, W.T, ts, cur_idx, lane);
             }

@@ -802,6 +802,33 @@ def test_a_slot_that_appears_twice_is_refused(U):
     pr.close()
 
 
+@pytest.mark.parametrize("n_slots", [3, 200, 310])
+def test_text_too_long_for_shared_memory_goes_through_the_tree(U, n_slots):
+    """A store whose text buffer (max_req_tokens) is larger than the shared memory a block can give
+    it: nothing is staged, every per-request job goes through the request's tree and, in sd_step,
+    waits for the append.  One, two and four blocks per SM."""
+    rng = np.random.default_rng(53 + n_slots)
+    pr = U.Pair(_rand_seqs(rng, 10, 60, 300, 7), vocab=7, D=16, n_slots=n_slots, max_req_tokens=40000,
+                slot_pool_nodes=6000)
+    slots = list(range(n_slots))
+    pr.append(slots, _rand_seqs(rng, n_slots, 0, 150, 7), reset=[1] * n_slots)
+    pr.check_speculate(slots, 16, 2.0, 48)
+    for _ in range(3):
+        lists = _rand_seqs(rng, n_slots, 0, 9, 7)
+        off, flat = U.ragged(lists)
+        out = pr.g.step(U.dev_i32(slots), torch.as_tensor(off, device=U.DEV),
+                        U.dev_i32(flat) if flat.size else torch.zeros(0, dtype=torch.int32, device=U.DEV), 16, 2.0, 48)
+        torch.cuda.synchronize()
+        pr.o.slot_append_batch(slots, lists, n_threads=4)
+        want = pr.o.speculate(slots, 16, 2.0, 48, M=64, n_threads=4)
+        got = {k: v.cpu().numpy() for k, v in out.items()}
+        got["mask"] = got["mask"].view(np.uint32)
+        U.assert_same_drafts(got, want)
+    pr.check_tree(0)
+    pr.check_tree(n_slots - 1)
+    pr.close()
+
+
 def test_device_allocation_failures_are_error_codes(U):
     """Every device allocation of sd_build and sd_build_requests fails once (test hook of the
     library): the call returns the out-of-memory code, nothing leaks, and the next call works."""

@@ -3,11 +3,12 @@
 // sd_speculate / sd_step: ONE launch, one thread block per request (speculate_fused_kernel):
 //   - sd_step: warp 0 appends the request's accepted tokens to its tree (exactly what sd_append
 //     does), and nothing but the few jobs that need the tree's wide nodes waits for it;
-//   - the other warps copy the request's text into shared memory and scan it for the earlier
+//   - sd_step: the other warps copy the request's text into shared memory and scan it for the earlier
 //     occurrences of the last token: how many tokens before each one agree with the context says
 //     which patterns it is an occurrence of.  A per-request match node with at most 32
 //     occurrences needs no tree at all: a lane per occurrence, the node's sub-tree is read off
-//     the text behind the occurrences (expand_occ);
+//     the text behind the occurrences (expand_occ).  sd_speculate takes the per-request match
+//     nodes from the slot's active nodes instead (nothing is being appended);
 //   - the global match nodes are advanced from the nodes cached at the previous call by
 //     descending only the tokens appended since;
 //   - the (tree, p) jobs go into a queue, costliest first, a warp per job; a job is dropped,
@@ -1039,7 +1040,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     // the stored text starts its way into shared memory now (asynchronous copies, nothing waits
     // for them here): it arrives while the cached match nodes and the append list are read
     const int32_t* text = ok ? sv.s_text + (long long)slot * sv.T : nullptr;
-    const bool prefetched = ok && gtid >= 0 && t_old <= stage_tokens && !(flags & SD_FLAG_GLOBAL_ONLY);
+    const bool prefetched = STEP && ok && gtid >= 0 && t_old <= stage_tokens && !(flags & SD_FLAG_GLOBAL_ONLY);
     if (prefetched) {
         const unsigned dst0 = (unsigned)__cvta_generic_to_shared(stx);
         for (int q = gtid; q < t_old; q += GT)
@@ -1087,8 +1088,10 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     // all cached nodes read before any is replaced; and: is this a second block for the same slot?
     const bool refused = __syncthreads_or(dup) != 0;
     if (refused) { usable = false; want_g = false; want_r = false; status = SD_STATUS_BAD_SLOT; }
-    // the text can be read off only if it fits the shared memory left for it
-    const bool staged = want_r && t >= 2 && t <= stage_tokens;
+    // The text can be read off only if it fits the shared memory left for it.  sd_speculate does
+    // not read it at all: with no append going on, the slot's active nodes are the per-request
+    // match nodes, at no cost (staging and scanning the text took it 8 us longer than that).
+    const bool staged = STEP && want_r && t >= 2 && t <= stage_tokens;
     const int Lcap = min(Pe, D - 1);                            // a match node at depth D has no children
     if (STEP && wib == 0) {
         if (ok && n_new > 0 && !refused) {
@@ -1216,6 +1219,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
                 c = min(budget_for(alpha, p, cap), 2 * (D - p));
                 if (staged && !(p <= Lcap && sh.r_cum[p] > 0)) c = 0;      // no earlier occurrence: nothing to speculate
                 else if (c > 0 && staged && p >= sh.r_pn) c += 2000;       // read off the text
+                else if (c > 0 && !STEP) c += 1000;                         // nothing to wait for: by cost among the global jobs
             }
             sh.cost[gtid] = c;
         }
@@ -1228,7 +1232,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
                     const int cq = sh.cost[q];
                     rank += (cq > c || (cq == c && q < gtid)) ? 1 : 0;
                 }
-                sh.job[rank] = gtid | (c < 1000 ? 128 : 0);     // bit 7: through the tree, behind the append
+                sh.job[rank] = gtid | ((c < 1000 || (!STEP && gtid >= SD_MAX_DEPTH)) ? 128 : 0);   // bit 7: through the request's tree (sd_step: behind the append)
                 atomicAdd(&sh.njobs, 1);
             }
         }

@@ -365,7 +365,7 @@ def run_ours(args):
         ref.global_build(w.corpus(), w.corpus_offsets())
         ref.slot_append_batch(list(range(B)), prompts, n_threads=thr)
         setup_s = time.perf_counter() - t0
-        o_times, desc, adds, upd, ok = [], [], [], [], True
+        o_times, desc, adds, upd, ctrees, ok = [], [], [], [], [], True
         for k in range(max(sample_steps) + 1):
             u0 = sum(ref.slot_updates(i) for i in range(B)) if k in sample_steps else 0
             t0 = time.perf_counter()
@@ -376,6 +376,7 @@ def run_ours(args):
                 o_times.append(time.perf_counter() - t0)
                 desc.append(int(r["visited"][:, 0].sum()))
                 adds.append(int(r["visited"][:, 1].sum()))
+                ctrees.append(int(r["visited"][:, 2].sum()))
                 upd.append(sum(ref.slot_updates(i) for i in range(B)) - u0)
                 g = {n: t.cpu().numpy() for n, t in saved[k].items()}
                 for n in ("n_draft", "tokens", "parents", "positions", "chosen_tree", "chosen_p"):
@@ -401,12 +402,15 @@ def run_ours(args):
                     "traffic": dram_traffic() if c.name == "large_batch" and not args.small else None,
                     "peak_source": which, "kernel": STEP_KERNEL,
                     "algorithmic_bytes_per_launch": alg_bytes,
-                    "append_bytes_per_launch": app_bytes, "speculate_bytes_per_launch": spec_bytes}
+                    "append_bytes_per_launch": app_bytes, "speculate_bytes_per_launch": spec_bytes,
+                    "frac_of_nominal_8_TBs": achieved / 8000.0}
         if spec_ms:
             sp = spec_bytes / (statistics.mean(spec_ms) / 1e3) / 1e9
             roofline["speculate_only"] = {"achieved": sp, "frac": sp / peak,
                                           "note": "sd_speculate alone (two-call form), its own necessary bytes"}
         extra = {"parity_vs_oracle": "bit-exact" if ok else "MISMATCH", "parity_steps": len(sample_steps),
+                 "candidate_trees_per_step": statistics.mean(ctrees),
+                 "candidate_trees_per_s": statistics.mean(ctrees) * world / (ms_per_step / 1e3),
                  "nodes_visited_per_step": visits,
                  "nodes_visited_per_s": visits * world / (ms_per_step / 1e3)}
         ref.close()

@@ -188,7 +188,7 @@ class SuffixOracle:
             "chosen_tree": np.zeros(n, dtype=np.int32),
             "chosen_p": np.zeros(n, dtype=np.int32),
             "score": np.zeros(n, dtype=np.float64),
-            "visited": np.zeros((n, 2), dtype=np.int64),
+            "visited": np.zeros((n, 3), dtype=np.int64),     # descents, added nodes, candidate trees
         }
         bo = None
         if budget_override is not None:

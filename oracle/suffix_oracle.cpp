@@ -241,7 +241,13 @@ void speculate_one(const Oracle& o, int i, int slot, int P, double alpha, int ca
     const int n = best ? (int)best->drafts.size() : 0;
     r.n_draft[i] = n; r.chosen_tree[i] = best ? best->tree : -1; r.chosen_p[i] = best ? best->p : 0;
     r.score[i] = best_score;
-    if (r.visited) { r.visited[2 * i] = descents; r.visited[2 * i + 1] = adds; }
+    if (r.visited) {
+        // measurement only: descents of all matches, nodes added to all candidate trees, and the
+        // number of candidate trees (matched (tree, p) pairs that got at least one draft node)
+        int64_t trees = 0;
+        for (const TreeCandidate& c : cands) trees += c.drafts.empty() ? 0 : 1;
+        r.visited[3 * i] = descents; r.visited[3 * i + 1] = adds; r.visited[3 * i + 2] = trees;
+    }
     int32_t* tok = r.tokens + (int64_t)i * M; int32_t* par = r.parents + (int64_t)i * M;
     int32_t* pos = r.positions + (int64_t)i * M; uint32_t* msk = r.mask + (int64_t)i * M * words;
     std::vector<int> depth(M, 0);

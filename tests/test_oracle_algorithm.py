@@ -250,10 +250,11 @@ def test_per_request_budget_override(oracle_mod):
 
 @pytest.mark.parametrize("seed", range(8))
 def test_visit_counters_equal_bruteforce(oracle_mod, seed):
-    """The two work counters (they are the numerator of the benchmark's bytes and nodes-visited
+    """The work counters (the numerator of the benchmark's bytes, nodes-visited and candidate-trees
     figures).  descents: for every tree and pattern length, the tokens of the pattern that the walk
     finds before it stops = the longest prefix of the pattern that occurs; adds: draft nodes of
-    every tree that was expanded, whether or not it is chosen.  Both from list scans, no trie."""
+    every tree that was expanded, whether or not it is chosen; candidate trees: the expanded trees
+    that got at least one draft node.  All from list scans, no trie."""
     rng = np.random.default_rng(500 + seed)
     D = int(rng.integers(2, 7))
     vocab = int(rng.integers(2, 5))
@@ -266,7 +267,7 @@ def test_visit_counters_equal_bruteforce(oracle_mod, seed):
         r = o.speculate([0, 1, 2], P, alpha, cap, flags=flags)
         for s in range(3):
             ctx = texts[s]
-            descents = adds = 0
+            descents = adds = trees = 0
             for tree, src in ((0, seqs), (1, [ctx])):
                 if (tree == 0 and flags & 2) or (tree == 1 and flags & 1):
                     continue
@@ -277,8 +278,10 @@ def test_visit_counters_equal_bruteforce(oracle_mod, seed):
                         k += 1
                     descents += k
                     if k == p:
-                        adds += len(greedy_tree(src, pat, D, o.budget(alpha, p, cap), bool(flags & 4))[0])
-            assert r["visited"][s].tolist() == [descents, adds], (s, P, alpha, cap, flags)
+                        size = len(greedy_tree(src, pat, D, o.budget(alpha, p, cap), bool(flags & 4))[0])
+                        adds += size
+                        trees += 1 if size else 0
+            assert r["visited"][s].tolist() == [descents, adds, trees], (s, P, alpha, cap, flags)
 
 
 def test_score_threshold_is_strict(oracle_mod):

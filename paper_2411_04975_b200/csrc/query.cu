@@ -1,5 +1,5 @@
 // Read-only queries on a store: COUNT of token paths (the quantity Eq. 1
-// divides), per-slot and store-wide bookkeeping.
+// divides), every node of a tree as a record, empirical entropy, per-slot and store-wide bookkeeping.
 #include "common.cuh"
 
 namespace {

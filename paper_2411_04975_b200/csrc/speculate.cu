@@ -2,13 +2,13 @@
 //
 // sd_speculate / sd_step: ONE launch, one thread block per request (speculate_fused_kernel):
 //   - sd_step: warp 0 appends the request's accepted tokens to its tree (exactly what sd_append
-//     does), and nothing but the few jobs that need the tree's wide nodes waits for it;
-//   - sd_step: the other warps copy the request's text into shared memory and scan it for the earlier
-//     occurrences of the last token: how many tokens before each one agree with the context says
+//     does) while the other warps match and expand; only jobs through the request's tree wait;
+//   - sd_step, blocks with many tokens to append: the other warps copy the request's text into
+//     shared memory and scan it for the earlier occurrences of the last token: how many tokens before each one agree with the context says
 //     which patterns it is an occurrence of.  A per-request match node with at most 32
 //     occurrences needs no tree at all: a lane per occurrence, the node's sub-tree is read off
-//     the text behind the occurrences (expand_occ).  sd_speculate takes the per-request match
-//     nodes from the slot's active nodes instead (nothing is being appended);
+//     the text behind the occurrences (expand_occ).  Otherwise the per-request match nodes are
+//     the slot's active nodes (sd_step: a job that needs them waits for the append);
 //   - the global match nodes are advanced from the nodes cached at the previous call by
 //     descending only the tokens appended since;
 //   - the (tree, p) jobs go into a queue, costliest first, a warp per job; a job is dropped,
@@ -976,17 +976,19 @@ __device__ void request_tree_job(BlockShared& sh, WarpWork& W, const sd_store& s
 // One block of W warps per request.
 //   1. match.  Global tree: the match nodes are advanced from the nodes cached at the previous
 //      call by descending only the tokens appended since (full walks when the cache is stale).
-//      Per-request tree: the request's text (with the tokens being appended) is copied into
-//      shared memory and scanned for the earlier occurrences of its last token; the number of
-//      tokens before an occurrence that agree with the context says which patterns it belongs to.
+//      Per-request tree: the slot's active nodes are the match nodes (sd_step: once the append
+//      is done).  A block of sd_step that appends many tokens does not wait for that: it copies
+//      the request's text (with the tokens being appended) into shared memory and scans it for the
+//      earlier occurrences of its last token; the number of tokens before an occurrence that
+//      agree with the context says which patterns it belongs to.
 //   2. expand: the (tree, p) jobs that matched go into a queue, costliest first; a warp per job.
 //      Global jobs go through the tree's entries.  Per-request jobs whose match node has at most
-//      32 occurrences are read off the text (expand_occ: a lane per occurrence, no tree); the
-//      others go through the request's tree from the slot's active nodes.  sd_step: warp 0
-//      appends the accepted tokens to the request's tree meanwhile, exactly as sd_append would,
-//      and joins the queue when it is done; the other warps meet at a barrier of their own until
-//      then, and only the jobs that go through the request's tree wait for the append (they
-//      come last in the queue).
+//      32 occurrences in a scanned text are read off the text (expand_occ: a lane per
+//      occurrence, no tree) and come first; the others go through the request's tree from the
+//      slot's active nodes.  sd_step: warp 0 appends the accepted tokens to the request's tree
+//      meanwhile, exactly as sd_append would, and joins the queue when it is done; the other
+//      warps meet at a barrier of their own until then, and only a warp that has taken a job
+//      through the request's tree waits for the append (a bounded wait on a flag).
 //   3. jobs of either tree that start at a wide child run without top block are scanned by all
 //      warps together, behind a block-wide barrier.
 //   4. select + emit from shared memory; no global scratch.
@@ -1009,6 +1011,9 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     constexpr int GW0 = STEP ? 1 : 0, GWARPS = WARPS - GW0, GT = GWARPS * 32;
     BlockShared& sh = *reinterpret_cast<BlockShared*>(smem_raw);
     int* const stx = reinterpret_cast<int*>(smem_raw + ((sizeof(BlockShared) + 15) & ~(size_t)15));
+    // new tokens from which a block reads its text off shared memory: 6 with two blocks per SM
+    // (9 warps scan), 12 with four (4 warps scan); measured, see the staging decision below
+    constexpr int STAGE_MIN_NEW = MINB >= 4 ? 12 : 6;
     const int tid = threadIdx.x, lane = tid & 31, wib = tid >> 5;
     const int gtid = tid - GW0 * 32, gw = wib - GW0;             // index inside that group (negative: warp 0 of sd_step)
     auto group_sync = [&]() {
@@ -1040,7 +1045,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     // the stored text starts its way into shared memory now (asynchronous copies, nothing waits
     // for them here): it arrives while the cached match nodes and the append list are read
     const int32_t* text = ok ? sv.s_text + (long long)slot * sv.T : nullptr;
-    const bool prefetched = STEP && ok && gtid >= 0 && t_old <= stage_tokens && !(flags & SD_FLAG_GLOBAL_ONLY);
+    const bool prefetched = STEP && MINB > 1 && n_new >= STAGE_MIN_NEW && ok && gtid >= 0 && t_old <= stage_tokens && !(flags & SD_FLAG_GLOBAL_ONLY);
     if (prefetched) {
         const unsigned dst0 = (unsigned)__cvta_generic_to_shared(stx);
         for (int q = gtid; q < t_old; q += GT)
@@ -1088,10 +1093,13 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
     // all cached nodes read before any is replaced; and: is this a second block for the same slot?
     const bool refused = __syncthreads_or(dup) != 0;
     if (refused) { usable = false; want_g = false; want_r = false; status = SD_STATUS_BAD_SLOT; }
-    // The text can be read off only if it fits the shared memory left for it.  sd_speculate does
-    // not read it at all: with no append going on, the slot's active nodes are the per-request
-    // match nodes, at no cost (staging and scanning the text took it 8 us longer than that).
-    const bool staged = STEP && want_r && t >= 2 && t <= stage_tokens;
+    // The text can be read off only if it fits the shared memory left for it, and it is only
+    // worth the copy and the scan (about 16 us for 4,096 tokens) where a long append would
+    // otherwise hold the per-request jobs up: from STAGE_MIN_NEW new tokens on.  sd_speculate
+    // does not read it at all: with no append going on, the slot's active nodes are the
+    // per-request match nodes, at no cost.  Nor do blocks that have an SM to themselves (small
+    // batches: measured on 64 requests with 8,192-token texts, 112 us per step without, 141 with).
+    const bool staged = STEP && MINB > 1 && n_new >= STAGE_MIN_NEW && want_r && t >= 2 && t <= stage_tokens;
     const int Lcap = min(Pe, D - 1);                            // a match node at depth D has no children
     if (STEP && wib == 0) {
         if (ok && n_new > 0 && !refused) {
@@ -1219,7 +1227,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
                 c = min(budget_for(alpha, p, cap), 2 * (D - p));
                 if (staged && !(p <= Lcap && sh.r_cum[p] > 0)) c = 0;      // no earlier occurrence: nothing to speculate
                 else if (c > 0 && staged && p >= sh.r_pn) c += 2000;       // read off the text
-                else if (c > 0 && !STEP) c += 1000;                         // nothing to wait for: by cost among the global jobs
+                else if (c > 0) c += 1000;                                  // through the request's tree: by cost among the global jobs
             }
             sh.cost[gtid] = c;
         }
@@ -1232,7 +1240,7 @@ speculate_fused_kernel(sd_store sv, int n, const int32_t* __restrict__ d_slot, i
                     const int cq = sh.cost[q];
                     rank += (cq > c || (cq == c && q < gtid)) ? 1 : 0;
                 }
-                sh.job[rank] = gtid | ((c < 1000 || (!STEP && gtid >= SD_MAX_DEPTH)) ? 128 : 0);   // bit 7: through the request's tree (sd_step: behind the append)
+                sh.job[rank] = gtid | ((c < 2000 && gtid >= SD_MAX_DEPTH) ? 128 : 0);   // bit 7: through the request's tree (sd_step: once the append is done)
                 atomicAdd(&sh.njobs, 1);
             }
         }

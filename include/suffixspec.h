@@ -154,7 +154,12 @@ int sd_append(sd_store* store, int32_t n, const int32_t* d_slot, const int64_t* 
  * A prompt that does not fit the slot's node pool or text buffer leaves the slot empty with
  * SD_STATUS_POOL_FULL.  Unlike the per-step calls this one may allocate device memory: its
  * temporaries (about 100 bytes per prompt token of the largest batch so far) are kept by the
- * store and reused.  It synchronises the stream before it returns.
+ * store and reused.  The host arrays have been read when the call returns (it synchronises the
+ * stream once, after the tokens have been checked); the trees themselves are built
+ * asynchronously on `stream` like any per-step call's work when the prompts hold at most 65,536
+ * tokens in total (a few new requests in the middle of a decode loop), and with further
+ * synchronisations above that.  The workspace is shared by all calls on a store: order calls
+ * made on different streams.
  * Errors: INVALID_ARG (bad slot, slot twice, offsets not ascending, token outside [0, V): nothing
  * is changed), CAPACITY (n * vocab or the token total does not fit 31 bits), NOMEM, CUDA.
  */

@@ -753,9 +753,15 @@ struct Pipeline {
 // room for top blocks in front of long runs.  per_seq_max_len > 0: the sequences are independent
 // (tokens of different sequences never compare equal, sequence k's tokens below sequence k + 1's)
 // and none is longer than that, so each is sorted by a block of its own.
+// no_readback: nothing is read back to the host on the way (no stream synchronisation): the
+// node arrays are sized for the most nodes N tokens can have (N * D) instead of the number
+// counted, and n_nodes / used_entries / n_wide are not filled in.  For small builds without
+// top blocks (a few prompts in the middle of a decode loop), where a round trip to the host
+// costs as much as the kernels between two of them.
 // Returns SD_OK, SD_ERR_NOMEM or SD_ERR_CUDA.
 static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_offsets, int n_seqs, i64 N,
-                        i64 max_token, int D, bool top_blocks, cudaStream_t st, i64 per_seq_max_len = 0) {
+                        i64 max_token, int D, bool top_blocks, cudaStream_t st, i64 per_seq_max_len = 0,
+                        bool no_readback = false) {
     const int T256 = 256;
     P.N = N;
     DeviceArena& tmp = P.tmp;
@@ -834,11 +840,13 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     if (!ok) return SD_ERR_NOMEM;
     exclusive_scan(NewNodes{lcp, len}, N, P.nbase, sb.scan_tmp, st);
     int h_nodes = 0;
-    ce = cudaMemcpyAsync(&h_nodes, P.nbase + N, sizeof(int), cudaMemcpyDeviceToHost, st);
-    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
-    if (ce != cudaSuccess) return SD_ERR_CUDA;
-    const i64 n_nodes = h_nodes;
-    P.n_nodes = n_nodes;
+    if (!no_readback) {
+        ce = cudaMemcpyAsync(&h_nodes, P.nbase + N, sizeof(int), cudaMemcpyDeviceToHost, st);
+        if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+        if (ce != cudaSuccess) return SD_ERR_CUDA;
+    }
+    const i64 n_nodes = no_readback ? N * D : (i64)h_nodes;      // (an upper bound: every suffix opens at most D nodes)
+    P.n_nodes = no_readback ? 0 : n_nodes;
 
     LevelTables& lv = P.lv;
     lv.N = N; lv.D = D;
@@ -858,6 +866,9 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     ms_carry_kernel<<<96, MC_THREADS, 0, st>>>(lv);
     if (small_tiles) ms_apply_kernel<MS_CHUNKS_SMALL><<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, P.nbase, lv);
     else ms_apply_kernel<MS_CHUNKS><<<ms_grid, MS_WARPS * 32, 0, st>>>(lcp, len, P.nbase, lv);
+    // (with the bound, the node ids behind the last real node have no children)
+    if (no_readback) ce = cudaMemsetAsync(P.nchild, 0, sizeof(int) * (size_t)(n_nodes + 1), st);
+    if (ce != cudaSuccess) return SD_ERR_CUDA;
     count_children_kernel<<<grid_for(N, T256), T256, 0, st>>>(lcp, len, P.nbase, lv, P.nchild);
     // child runs (with their top blocks) in node (pre-)order
     exclusive_scan(RunAlloc{P.nchild, top_blocks ? 1 : 0}, n_nodes + 1, P.runstart, P.big_tmp, st);
@@ -865,6 +876,7 @@ static int pipeline_run(Pipeline& P, const int32_t* d_tok, const int64_t* d_seq_
     ce = cudaMemsetAsync(wide_counter, 0, sizeof(int), st);
     if (top_blocks)
         collect_wide_kernel<<<grid_for(n_nodes + 1, T256), T256, 0, st>>>(P.nchild, n_nodes + 1, P.wide_list, wide_counter);
+    if (no_readback) return ce == cudaSuccess ? SD_OK : SD_ERR_CUDA;
     int h_total = 0;
     if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h_total, P.runstart + n_nodes + 1, sizeof(int), cudaMemcpyDeviceToHost, st);
     if (ce == cudaSuccess) ce = cudaMemcpyAsync(&P.n_wide, wide_counter, sizeof(int), cudaMemcpyDeviceToHost, st);
@@ -1163,7 +1175,9 @@ extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, 
     if (N > 0) {
         i64 max_len = 0;
         for (int q = 0; q < n; ++q) max_len = std::max<i64>(max_len, h_offsets[q + 1] - h_offsets[q]);
-        const int rc = pipeline_run(P, mtok, d_off, n, N, (i64)n * s->V, D, false, st, max_len);
+        // a handful of prompts: no round trips to the host on the way
+        const bool small = N <= 65536;
+        const int rc = pipeline_run(P, mtok, d_off, n, N, (i64)n * s->V, D, false, st, max_len, small);
         if (rc != SD_OK) return rc;
         requests_layout_kernel<<<grid_for(n, T256), T256, 0, st>>>(*s, n, d_off, P.nbase, P.runstart, P.lv.E, L);
         emit_nodes_slots_kernel<<<grid_for(N, T256), T256, 0, st>>>(*s, n, d_slot, d_off, mtok, P.sa, P.lcp, P.len, N, P.lv,
@@ -1174,7 +1188,8 @@ extern "C" int sd_build_requests(sd_store* s, int32_t n, const int32_t* h_slot, 
         SD_CUDA_OK(cudaMemsetAsync(L.live, 0, sizeof(int) * n, st));
     }
     requests_finalize_kernel<<<grid_for((i64)n * 32, T256), T256, 0, st>>>(*s, n, d_slot, d_off, L);
-    SD_CUDA_OK(cudaStreamSynchronize(st));                       // the temporaries are released on return
+    // (no synchronisation: the temporaries stay in the store's workspace, and a later call on
+    // another stream must be ordered behind this one by the caller like any other use of the store)
     SD_CUDA_OK(cudaGetLastError());
     return SD_OK;
 }
